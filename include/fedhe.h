@@ -1,0 +1,206 @@
+/*
+ * fedhe.h -- C ABI of the B200 (sm_100a) library for the hot path of FedML-HE
+ * secure aggregation: selective-encryption mask, CKKS packing/encoding,
+ * public-key encryption, server-side weighted ciphertext sum with rescale,
+ * decryption/decoding and merge with the plaintext-averaged remainder.
+ *
+ * The entry points follow the paper's statement of the problem:
+ *   Algorithm 1 ("HE-Based Federated Aggregation"), the aggregation equation
+ *   [W_glob] = sum_i a_i [[M (.) W_i]] + sum_i a_i ((1-M) (.) W_i), "Step 2"
+ *   of Selective Parameter Encryption (mask = ratio p of the most sensitive
+ *   parameters), and the framework API table (key_gen, enc, he_aggregate,
+ *   dec; flatten/reshape stay with the caller).
+ *
+ * Conventions
+ *   - Every call returns an int: HE_OK (0) or a negative HE_ERR_* code; no
+ *     exception crosses this boundary.  he_strerror() names a code.
+ *   - "dev" pointers are device pointers on the context's GPU, owned by the
+ *     caller, never freed by the library; "host" pointers are ordinary host
+ *     memory.  Handles (he_ctx, he_keys, he_mask) are owned by the library
+ *     and released by the matching *_destroy.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls are asynchronous on it unless stated otherwise.  A context keeps
+ *     small library-owned work buffers; calls that share a context must be
+ *     issued on one stream at a time.
+ *   - Kernels never trap or assert.  A numeric anomaly (an encoded
+ *     coefficient of magnitude >= 2^62, or a non-finite input) sets a sticky
+ *     status word read by he_ctx_status().
+ *   - Ring R = Z[X]/(X^N+1), N a power of two, RNS primes q_0..q_{L-1} (all
+ *     of them ciphertext limbs; the rescale drops q_{L-1}); n = N/2 real
+ *     slots per ciphertext; scale Delta = 2^log2_delta.
+ *   - Ciphertext layout: uint64 [T][2][level][N], coefficient domain, natural
+ *     coefficient order, canonical residues in [0, q_j); level = L for fresh
+ *     ciphertexts and L-1 after he_weighted_aggregate.
+ */
+#ifndef FEDHE_H
+#define FEDHE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HE_MAX_LIMBS 16
+#define HE_MAX_CLIENTS 256
+
+enum {
+    HE_OK = 0,
+    HE_ERR_INVALID_ARG = -1, /* null pointer, zero size, k > P, bad handle */
+    HE_ERR_PARAMS = -2,      /* N, L, primes or scale not usable */
+    HE_ERR_ALLOC = -3,       /* device or host allocation failed */
+    HE_ERR_CUDA = -4,        /* a CUDA runtime call failed */
+    HE_ERR_OVERFLOW = -5,    /* status: an encoded coefficient left the range */
+    HE_ERR_LEVEL = -6,       /* operation needs a level the context lacks */
+    HE_ERR_SIZE = -7         /* size beyond what the call supports */
+};
+
+typedef struct he_ctx he_ctx;
+typedef struct he_keys he_keys;
+typedef struct he_mask he_mask;
+
+/* Crypto context = the public configuration every party holds (Algorithm 1,
+ * key generation; the server receives only this). */
+typedef struct he_params {
+    uint32_t N;                  /* ring degree: power of two, 8192..65536 */
+    uint32_t L;                  /* number of RNS primes, 2..HE_MAX_LIMBS */
+    uint64_t q[HE_MAX_LIMBS];    /* distinct primes < 2^62 with q = 1 mod 2N */
+    int32_t log2_delta;          /* scale bits, 1 <= log2_delta, 2^log2_delta < q_0 / 4 */
+} he_params;
+
+const char *he_strerror(int code);
+
+/* Creates a context on the current CUDA device: validates the parameters
+ * (HE_ERR_PARAMS), builds the root/twiddle tables on the host and uploads
+ * them.  Synchronous. */
+int he_ctx_create(const he_params *params, he_ctx **out);
+int he_ctx_destroy(he_ctx *ctx);
+/* Synchronises the device, returns the sticky status (HE_OK or
+ * HE_ERR_OVERFLOW) in *status and clears it. */
+int he_ctx_status(he_ctx *ctx, int *status);
+/* Pre-sizes the library-owned work buffers for encryptions/decryptions of up
+ * to max_k encrypted parameters so that later calls allocate nothing.
+ * Synchronous. */
+int he_ctx_reserve(he_ctx *ctx, size_t max_k);
+
+size_t he_slots(const he_ctx *ctx);                       /* n = N/2 */
+size_t he_num_ct(const he_ctx *ctx, size_t k);            /* T = ceil(k / n): a short vector still costs a ciphertext */
+size_t he_ct_words(const he_ctx *ctx, uint32_t level);    /* 2 * level * N uint64 words per ciphertext */
+
+/* HE.KeyGen (Algorithm 1, first step; API table "key_gen").  s uniform
+ * ternary, a_j uniform mod q_j, e discrete Gaussian (sigma 3.2), all from
+ * Philox4x32-10 streams of `seed`;  pk = (-a s + e, a).  Both keys stay on
+ * the device inside the handle. */
+int he_keygen(he_ctx *ctx, uint64_t seed, he_keys **out, void *stream);
+int he_keys_destroy(he_keys *keys);
+/* Writes the public key (dev uint64 [2][L][N], coefficient domain, canonical)
+ * and/or the secret key (dev int8 [N], values -1,0,1); either may be NULL. */
+int he_keys_export(he_ctx *ctx, const he_keys *keys, uint64_t *pk_dev, int8_t *s_dev, void *stream);
+
+/* Select(., p) of Algorithm 1 / "Step 2": the k parameters with the highest
+ * sensitivity score.  key(score) = its fp32 bit pattern if the sign bit is
+ * clear and it is not NaN, else 0; order by key descending, index ascending;
+ * the first k form the mask.  score: dev float[P], P < 2^32, 0 <= k <= P.
+ * Synchronous (the result sizes are needed on the host). */
+int he_select_mask(he_ctx *ctx, const float *score_dev, size_t P, size_t k, he_mask **out, void *stream);
+/* Variant for the paper's empirical selection recipe (the top-p most
+ * sensitive parameters as well as whole layers, e.g. the first and last):
+ * the mask is the union of the top-k set above and of the half-open index
+ * ranges [ranges[2i], ranges[2i+1]) (host array, at most 64 ranges, each
+ * within [0, P]); its final size is reported by he_mask_indices. */
+int he_select_mask_ranges(he_ctx *ctx, const float *score_dev, size_t P, size_t k,
+                          const uint64_t *ranges_host, size_t num_ranges, he_mask **out, void *stream);
+/* Selected indices, ascending: dev uint32 [k]; pointer owned by the mask. */
+int he_mask_indices(const he_mask *mask, const uint32_t **idx_dev, size_t *k);
+/* Copies the k selected indices into a caller-owned buffer: dev uint32 [k]. */
+int he_mask_copy_indices(const he_mask *mask, uint32_t *out_dev, void *stream);
+int he_mask_destroy(he_mask *mask);
+
+/* Client side of  [W_i] = Enc(pk, M (.) W_i) + (1-M) (.) W_i : gathers the
+ * masked parameters into slot order and compacts the complement.
+ *   x: dev float[P];  sel: dev float[T*n], entries k..T*n-1 are zeroed;
+ *   rest: dev float[P-k] (ascending index order), may be NULL when mask is
+ *   NULL.  mask == NULL means full encryption (k = P). */
+int he_pack(he_ctx *ctx, const he_mask *mask, const float *x_dev, size_t P, float *sel_dev,
+            float *rest_dev, void *stream);
+
+/* CKKS encoding alone (parity hook): m = round(Delta * sigma^{-1}(z)) for the
+ * T = ceil(k/n) slot vectors of sel (dev float[T*n]); m: dev int64 [T][N]. */
+int he_encode(he_ctx *ctx, const float *sel_dev, size_t k, int64_t *m_dev, void *stream);
+
+/* HE.Enc(pk, .) of Algorithm 1 (API table "enc"): encodes and encrypts the T
+ * slot vectors of sel.  Ciphertext t of client `client_id` draws u (ternary),
+ * e0, e1 (Gaussian) from Philox streams of (seed, t, client_id):
+ *   c0 = pk0 u + e0 + m,  c1 = pk1 u + e1  (mod q_j).
+ * ct: dev uint64 [T][2][L][N].  A (seed, client_id, t) triple must not be
+ * reused across rounds. */
+int he_encrypt(he_ctx *ctx, const he_keys *keys, const float *sel_dev, size_t k, uint64_t seed,
+               uint32_t client_id, uint64_t *ct_dev, void *stream);
+
+/* Same for the ciphertext indices t_begin .. t_begin+t_count-1 only (a caller
+ * that streams a large model in chunks): sel points at the slots of
+ * ciphertext t_begin, ct at uint64 [t_count][2][L][N]; the Philox streams are
+ * those of the absolute index, so chunked and whole encryption agree. */
+int he_encrypt_range(he_ctx *ctx, const he_keys *keys, const float *sel_dev, size_t t_begin, size_t t_count,
+                     uint64_t seed, uint32_t client_id, uint64_t *ct_dev, void *stream);
+
+/* Server step  sum_i a_i [[M (.) W_i]]  with plaintext weights and one
+ * multiplicative level (API table "he_aggregate"): W_i = rint(a_i q_{L-1}) as
+ * a constant polynomial, acc = sum_i W_i ct_i mod q_j, then the rescale by
+ * q_{L-1} with rounding, which returns exactly to scale Delta.
+ *   cts: host array of C dev pointers, each uint64 [T][2][L][N];
+ *   alpha: host double[C] (caller normalises: sum = 1), 1 <= C <= HE_MAX_CLIENTS;
+ *   agg: dev uint64 [T][2][L-1][N]. */
+int he_weighted_aggregate(he_ctx *ctx, const uint64_t *const *cts_host, const double *alpha_host,
+                          int C, size_t T, uint64_t *agg_dev, void *stream);
+
+/* Plaintext part  sum_i a_i ((1-M) (.) W_i): out[k] = sum_i alpha_i * rest_i[k]
+ * in fp64, client order, separate multiply and add.
+ *   rests: host array of C dev pointers float[len]; out: dev double[len]. */
+int he_plain_aggregate(he_ctx *ctx, const float *const *rests_host, const double *alpha_host, int C,
+                       size_t len, double *out_dev, void *stream);
+
+/* HE.Dec(sk, .) of Algorithm 1 (API table "dec") on ciphertexts of level L-1:
+ * d = c0 + c1 s mod q_0 centred, decoded to the n slots.
+ *   agg: dev uint64 [T][2][L-1][N];  z: dev double[T*n]. */
+int he_decrypt(he_ctx *ctx, const he_keys *keys, const uint64_t *agg_dev, size_t T, double *z_dev,
+               void *stream);
+/* Same with an explicit level (1..L) so that fresh ciphertexts can be opened. */
+int he_decrypt_level(he_ctx *ctx, const he_keys *keys, const uint64_t *ct_dev, uint32_t level, size_t T,
+                     double *z_dev, void *stream);
+
+/* Client merge  Dec(sk, M (.) [W_glob]) + (1-M) (.) [W_glob]:
+ * w_glob[idx[r]] = z[r], complement positions take rest_avg in order.
+ *   z: dev double[>= k]; rest_avg: dev double[P-k] (NULL if mask NULL);
+ *   w_glob: dev double[P]. */
+int he_unpack(he_ctx *ctx, const he_mask *mask, const double *z_dev, const double *rest_avg_dev,
+              size_t P, double *w_glob_dev, void *stream);
+
+/* Batched negacyclic transforms on raw residues (kernel sweep; no paper
+ * counterpart): polys dev uint64 [B][L][N] in place, canonical residues in,
+ * canonical residues out.  Forward: A[k] = sum_j a_j psi^((2 brev(k)+1) j)
+ * mod q (bit-reversed output order), psi the smallest primitive 2N-th root
+ * of unity mod q; inverse undoes it. */
+int he_ntt_forward(he_ctx *ctx, uint64_t *polys_dev, size_t B, void *stream);
+int he_ntt_inverse(he_ctx *ctx, uint64_t *polys_dev, size_t B, void *stream);
+
+/* One whole round from host memory, the call an application makes when its
+ * updates live on the host: copies every client's update to the device,
+ * runs pack -> encrypt (all clients) -> weighted aggregate + plaintext
+ * remainder -> decrypt -> unpack in chunks of ciphertext indices, and copies
+ * the merged global model back.
+ *   xs: host array of C host pointers float[P]; alpha: host double[C];
+ *   mask: NULL = full encryption; w_glob: host double[P].
+ * Synchronous; allocates its device buffers through the context. */
+int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const float *const *xs_host,
+                  const double *alpha_host, int C, size_t P, uint64_t enc_seed, double *w_glob_host,
+                  void *stream);
+
+/* Number of kernel launches issued by this library since it was loaded. */
+uint64_t he_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FEDHE_H */

@@ -1,0 +1,603 @@
+// C ABI of the library (see include/fedhe.h): argument validation, handle
+// management, host-side table upload and the sequencing of kernel launches.
+#include <math.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "fedhe_host.h"
+#include "fedhe_launch.h"
+
+using namespace fedhe;
+
+namespace {
+
+inline cudaStream_t as_stream(void *s) { return reinterpret_cast<cudaStream_t>(s); }
+inline bool good(const he_ctx *c) { return c && c->magic == CTX_MAGIC; }
+inline bool good(const he_keys *k) { return k && k->magic == KEYS_MAGIC; }
+inline bool good(const he_mask *m) { return m && m->magic == MASK_MAGIC; }
+
+#define CU(expr)                                   \
+    do {                                           \
+        cudaError_t e__ = (expr);                  \
+        if (e__ != cudaSuccess) return e__ == cudaErrorMemoryAllocation ? HE_ERR_ALLOC : HE_ERR_CUDA; \
+    } while (0)
+
+// grows a context-owned device buffer; contents are not preserved
+int ensure(void **buf, size_t *cap, size_t need) {
+    if (need <= *cap) return HE_OK;
+    if (*buf) {
+        CU(cudaFree(*buf));
+        *buf = nullptr;
+        *cap = 0;
+    }
+    CU(cudaMalloc(buf, need));
+    *cap = need;
+    return HE_OK;
+}
+
+template <class T>
+int upload(he_ctx *ctx, const T *host, size_t count, const T **dev) {
+    void *p = nullptr;
+    CU(cudaMalloc(&p, count * sizeof(T)));
+    ctx->owned.push_back(p);
+    CU(cudaMemcpy(p, host, count * sizeof(T), cudaMemcpyHostToDevice));
+    *dev = static_cast<const T *>(p);
+    return HE_OK;
+}
+
+size_t work_bytes(const he_ctx *ctx, size_t T) { return 2 * T * (size_t)ctx->dev.N * sizeof(uint64_t); }
+
+}  // namespace
+
+extern "C" {
+
+const char *he_strerror(int code) {
+    switch (code) {
+    case HE_OK: return "ok";
+    case HE_ERR_INVALID_ARG: return "invalid argument";
+    case HE_ERR_PARAMS: return "unusable crypto parameters";
+    case HE_ERR_ALLOC: return "allocation failed";
+    case HE_ERR_CUDA: return "CUDA runtime error";
+    case HE_ERR_OVERFLOW: return "encoded coefficient out of range";
+    case HE_ERR_LEVEL: return "ciphertext level mismatch";
+    case HE_ERR_SIZE: return "size not supported";
+    default: return "unknown error";
+    }
+}
+
+uint64_t he_launch_count(void) { return launch_count(); }
+
+int he_ctx_create(const he_params *p, he_ctx **out) {
+    if (!p || !out) return HE_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (p->L > HE_MAX_LIMBS) return HE_ERR_PARAMS;
+    if (host_check_params(p->N, p->L, p->q, p->log2_delta)) return HE_ERR_PARAMS;
+    he_ctx *ctx = new (std::nothrow) he_ctx();
+    if (!ctx) return HE_ERR_ALLOC;
+    ctx->magic = CTX_MAGIC;
+    ctx->params = *p;
+    int rc = HE_OK;
+    do {
+        if (cudaGetDevice(&ctx->device) != cudaSuccess) { rc = HE_ERR_CUDA; break; }
+        CtxDev &d = ctx->dev;
+        memset(&d, 0, sizeof(d));
+        d.N = p->N;
+        d.L = p->L;
+        d.log2_delta = p->log2_delta;
+        while ((1u << d.logN) < d.N) d.logN++;
+        d.LOGB = d.logN < 14 ? d.logN : 14;
+        d.A = d.logN - d.LOGB;
+        const uint64_t ql = p->q[p->L - 1];
+        for (uint32_t j = 0; j < p->L && rc == HE_OK; j++) {
+            HostLimb hl;
+            host_build_limb(d.N, p->q[j], hl);
+            LimbDev &ld = d.limb[j];
+            ld.q = hl.q;
+            ld.mu = hl.mu;
+            ld.ninv = tw_t{hl.ninv.w, hl.ninv.wp};
+            ld.wn = tw_t{hl.wn.w, hl.wn.wp};
+            if (j + 1 < p->L) {
+                HostTw qi = host_shoup(host_invmod(ql % hl.q, hl.q), hl.q);
+                ld.qlinv = tw_t{qi.w, qi.wp};
+            }
+            rc = upload(ctx, reinterpret_cast<const tw_t *>(hl.fwd.data()), hl.fwd.size(), &ld.fwd);
+            if (rc == HE_OK) rc = upload(ctx, reinterpret_cast<const tw_t *>(hl.inv.data()), hl.inv.size(), &ld.inv);
+        }
+        if (rc != HE_OK) break;
+        std::vector<double> roots, ftw;
+        host_unit_roots(d.N, roots);
+        host_slot_twiddles(d.N, roots, ftw);
+        rc = upload(ctx, reinterpret_cast<const double2 *>(ftw.data()), ftw.size() / 2, &d.ftw);
+        if (rc != HE_OK) break;
+        void *st = nullptr;
+        if (cudaMalloc(&st, sizeof(int)) != cudaSuccess) { rc = HE_ERR_ALLOC; break; }
+        ctx->owned.push_back(st);
+        if (cudaMemset(st, 0, sizeof(int)) != cudaSuccess) { rc = HE_ERR_CUDA; break; }
+        d.status = static_cast<int *>(st);
+        // pointer and weight tables of the aggregation calls
+        rc = ensure(&ctx->tab, &ctx->tab_bytes,
+                    HE_MAX_CLIENTS * (2 * sizeof(void *) + sizeof(double) + HE_MAX_LIMBS * sizeof(tw_t)));
+    } while (0);
+    if (rc != HE_OK) {
+        he_ctx_destroy(ctx);
+        return rc;
+    }
+    *out = ctx;
+    return HE_OK;
+}
+
+int he_ctx_destroy(he_ctx *ctx) {
+    if (!good(ctx)) return HE_ERR_INVALID_ARG;
+    cudaDeviceSynchronize();
+    for (void *p : ctx->owned) cudaFree(p);
+    if (ctx->ws) cudaFree(ctx->ws);
+    if (ctx->tab) cudaFree(ctx->tab);
+    if (ctx->round_buf) cudaFree(ctx->round_buf);
+    ctx->magic = 0;
+    delete ctx;
+    return HE_OK;
+}
+
+int he_ctx_status(he_ctx *ctx, int *status) {
+    if (!good(ctx) || !status) return HE_ERR_INVALID_ARG;
+    int word = 0;
+    CU(cudaDeviceSynchronize());
+    CU(cudaMemcpy(&word, ctx->dev.status, sizeof(int), cudaMemcpyDeviceToHost));
+    if (word) CU(cudaMemset(ctx->dev.status, 0, sizeof(int)));
+    *status = word ? HE_ERR_OVERFLOW : HE_OK;
+    return HE_OK;
+}
+
+int he_ctx_reserve(he_ctx *ctx, size_t max_k) {
+    if (!good(ctx)) return HE_ERR_INVALID_ARG;
+    return ensure(&ctx->ws, &ctx->ws_bytes, work_bytes(ctx, he_num_ct(ctx, max_k)));
+}
+
+size_t he_slots(const he_ctx *ctx) { return good(ctx) ? ctx->dev.N / 2 : 0; }
+
+size_t he_num_ct(const he_ctx *ctx, size_t k) {
+    if (!good(ctx)) return 0;
+    const size_t n = ctx->dev.N / 2;
+    return (k + n - 1) / n;
+}
+
+size_t he_ct_words(const he_ctx *ctx, uint32_t level) {
+    return good(ctx) ? 2 * (size_t)level * ctx->dev.N : 0;
+}
+
+// ---------------------------------------------------------------------------
+
+int he_keygen(he_ctx *ctx, uint64_t seed, he_keys **out, void *stream) {
+    if (!good(ctx) || !out) return HE_ERR_INVALID_ARG;
+    *out = nullptr;
+    const CtxDev &d = ctx->dev;
+    const size_t LN = (size_t)d.L * d.N;
+    he_keys *k = new (std::nothrow) he_keys();
+    if (!k) return HE_ERR_ALLOC;
+    k->magic = KEYS_MAGIC;
+    k->ctx = ctx;
+    k->storage = nullptr;
+    const size_t bytes = 3 * LN * sizeof(tw_t) + d.N;
+    void *tmp = nullptr;
+    int rc = HE_OK;
+    do {
+        if (cudaMalloc(&k->storage, bytes) != cudaSuccess || cudaMalloc(&tmp, 3 * LN * sizeof(uint64_t)) != cudaSuccess) {
+            rc = HE_ERR_ALLOC;
+            break;
+        }
+        tw_t *base = static_cast<tw_t *>(k->storage);
+        tw_t *pk0 = base, *pk1 = base + LN, *sh = base + 2 * LN;
+        int8_t *s8 = reinterpret_cast<int8_t *>(base + 3 * LN);
+        k->dev = KeysDev{pk0, pk1, sh, s8};
+        cudaStream_t st = as_stream(stream);
+        uint64_t *t64 = static_cast<uint64_t *>(tmp);
+        if (launch_keygen_sample(d, seed, s8, t64, st) != cudaSuccess ||
+            launch_ntt(d, true, t64, 3, LN, 0, d.L, st) != cudaSuccess ||
+            launch_keygen_combine(d, t64, pk0, pk1, sh, st) != cudaSuccess ||
+            cudaStreamSynchronize(st) != cudaSuccess) {
+            rc = HE_ERR_CUDA;
+        }
+    } while (0);
+    if (tmp) cudaFree(tmp);
+    if (rc != HE_OK) {
+        if (k->storage) cudaFree(k->storage);
+        delete k;
+        return rc;
+    }
+    *out = k;
+    return HE_OK;
+}
+
+int he_keys_destroy(he_keys *keys) {
+    if (!good(keys)) return HE_ERR_INVALID_ARG;
+    cudaDeviceSynchronize();
+    cudaFree(keys->storage);
+    keys->magic = 0;
+    delete keys;
+    return HE_OK;
+}
+
+int he_keys_export(he_ctx *ctx, const he_keys *keys, uint64_t *pk_dev, int8_t *s_dev, void *stream) {
+    if (!good(ctx) || !good(keys) || keys->ctx != ctx) return HE_ERR_INVALID_ARG;
+    const CtxDev &d = ctx->dev;
+    const size_t LN = (size_t)d.L * d.N;
+    cudaStream_t st = as_stream(stream);
+    if (pk_dev) {
+        // pk0^ and pk1^ are adjacent in the key storage
+        CU(launch_extract_values(keys->dev.pk0_hat, pk_dev, 2 * LN, st));
+        CU(launch_ntt(d, false, pk_dev, 2, LN, 0, d.L, st));
+    }
+    if (s_dev) CU(cudaMemcpyAsync(s_dev, keys->dev.s, d.N, cudaMemcpyDeviceToDevice, st));
+    return HE_OK;
+}
+
+// ---------------------------------------------------------------------------
+// mask
+// ---------------------------------------------------------------------------
+
+static int build_mask(he_ctx *ctx, const float *score, size_t P, size_t k, const uint64_t *ranges_host,
+                      size_t num_ranges, he_mask **out, void *stream) {
+    if (!good(ctx) || !out || (!score && P) || k > P) return HE_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (P == 0) return HE_ERR_INVALID_ARG;
+    if (P >= (1ull << 32)) return HE_ERR_SIZE;
+    if (num_ranges > 64 || (num_ranges && !ranges_host)) return HE_ERR_INVALID_ARG;
+    for (size_t r = 0; r < num_ranges; r++)
+        if (ranges_host[2 * r] > ranges_host[2 * r + 1] || ranges_host[2 * r + 1] > P) return HE_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    const size_t nblocks = (P + MASK_BLOCK - 1) / MASK_BLOCK, nwords = (P + 31) / 32;
+
+    // scratch: histogram (2048) | totals (2) | blk_a (nblocks) | blk_b (nblocks) | ranges
+    uint32_t *scratch = nullptr;
+    const size_t scratch_words = 2048 + 2 + 2 * nblocks + 4 * 64 + 2;
+    CU(cudaMalloc(reinterpret_cast<void **>(&scratch), scratch_words * sizeof(uint32_t)));
+    uint32_t *hist = scratch, *totals = scratch + 2048, *blk_eq = totals + 2, *blk_sel = blk_eq + nblocks;
+    uint64_t *ranges_dev = reinterpret_cast<uint64_t *>(scratch + ((2048 + 2 + 2 * nblocks + 1) & ~(size_t)1));
+    int rc = HE_OK;
+    he_mask *m = nullptr;
+    uint32_t *bits = nullptr, *wpre = nullptr, *idx = nullptr;
+    do {
+#define MCU(expr) if ((expr) != cudaSuccess) { rc = HE_ERR_CUDA; break; }
+        // radix select of the k-th largest key: 11 + 11 + 10 bits
+        uint32_t prefix = 0, need = (uint32_t)k;   // need = how many keys equal to tau are taken
+        uint32_t tau = 0;
+        if (k == 0) {
+            tau = 0xffffffffu;                       // nothing is above or equal
+            need = 0;
+        } else {
+            static const int digits[3] = {11, 11, 10};
+            int prefix_bits = 0;
+            std::vector<uint32_t> h(2048);
+            bool fail = false;
+            for (int pass = 0; pass < 3; pass++) {
+                const int db = digits[pass];
+                if (cudaMemsetAsync(hist, 0, sizeof(uint32_t) << db, st) != cudaSuccess ||
+                    launch_key_histogram(score, P, prefix, prefix_bits, db, hist, st) != cudaSuccess ||
+                    cudaMemcpyAsync(h.data(), hist, sizeof(uint32_t) << db, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+                    cudaStreamSynchronize(st) != cudaSuccess) {
+                    fail = true;
+                    break;
+                }
+                // walk the digits from the largest down until `need` keys are covered
+                int b = (1 << db) - 1;
+                for (; b > 0; b--) {
+                    if (h[b] >= need) break;
+                    need -= h[b];
+                }
+                prefix = (prefix << db) | (uint32_t)b;
+                prefix_bits += db;
+            }
+            if (fail) { rc = HE_ERR_CUDA; break; }
+            tau = prefix;
+        }
+        MCU(cudaMalloc(reinterpret_cast<void **>(&bits), nwords * sizeof(uint32_t)));
+        MCU(cudaMalloc(reinterpret_cast<void **>(&wpre), nwords * sizeof(uint32_t)));
+        if (num_ranges)
+            MCU(cudaMemcpyAsync(ranges_dev, ranges_host, 2 * num_ranges * sizeof(uint64_t), cudaMemcpyHostToDevice, st));
+        MCU(launch_mask_count_eq(score, P, tau, blk_eq, st));
+        MCU(launch_scan(blk_eq, nblocks, totals, st));
+        MCU(launch_mask_select(score, P, tau, need, ranges_dev, (uint32_t)num_ranges, blk_eq, bits, blk_sel, st));
+        MCU(launch_scan(blk_sel, nblocks, totals + 1, st));
+        uint32_t ksel = 0;
+        MCU(cudaMemcpyAsync(&ksel, totals + 1, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+        MCU(cudaStreamSynchronize(st));
+        if (num_ranges == 0 && ksel != k) { rc = HE_ERR_CUDA; break; }     // cannot happen
+        MCU(cudaMalloc(reinterpret_cast<void **>(&idx), (ksel ? ksel : 1) * sizeof(uint32_t)));
+        MCU(launch_mask_write(P, bits, blk_sel, wpre, idx, st));
+        MCU(cudaStreamSynchronize(st));
+        m = new (std::nothrow) he_mask();
+        if (!m) { rc = HE_ERR_ALLOC; break; }
+        m->magic = MASK_MAGIC;
+        m->P = P;
+        m->k = ksel;
+        m->idx = idx;
+        m->bits = bits;
+        m->wpre = wpre;
+#undef MCU
+    } while (0);
+    cudaFree(scratch);
+    if (rc != HE_OK) {
+        if (bits) cudaFree(bits);
+        if (wpre) cudaFree(wpre);
+        if (idx) cudaFree(idx);
+        return rc;
+    }
+    *out = m;
+    return HE_OK;
+}
+
+int he_select_mask(he_ctx *ctx, const float *score_dev, size_t P, size_t k, he_mask **out, void *stream) {
+    return build_mask(ctx, score_dev, P, k, nullptr, 0, out, stream);
+}
+
+int he_select_mask_ranges(he_ctx *ctx, const float *score_dev, size_t P, size_t k, const uint64_t *ranges_host,
+                          size_t num_ranges, he_mask **out, void *stream) {
+    return build_mask(ctx, score_dev, P, k, ranges_host, num_ranges, out, stream);
+}
+
+int he_mask_indices(const he_mask *mask, const uint32_t **idx_dev, size_t *k) {
+    if (!good(mask)) return HE_ERR_INVALID_ARG;
+    if (idx_dev) *idx_dev = mask->idx;
+    if (k) *k = mask->k;
+    return HE_OK;
+}
+
+int he_mask_copy_indices(const he_mask *mask, uint32_t *out_dev, void *stream) {
+    if (!good(mask) || (!out_dev && mask->k)) return HE_ERR_INVALID_ARG;
+    if (mask->k)
+        CU(cudaMemcpyAsync(out_dev, mask->idx, mask->k * sizeof(uint32_t), cudaMemcpyDeviceToDevice, as_stream(stream)));
+    return HE_OK;
+}
+
+int he_mask_destroy(he_mask *mask) {
+    if (!good(mask)) return HE_ERR_INVALID_ARG;
+    cudaDeviceSynchronize();
+    cudaFree(mask->idx);
+    cudaFree(mask->bits);
+    cudaFree(mask->wpre);
+    mask->magic = 0;
+    delete mask;
+    return HE_OK;
+}
+
+// ---------------------------------------------------------------------------
+// client and server steps
+// ---------------------------------------------------------------------------
+
+int he_pack(he_ctx *ctx, const he_mask *mask, const float *x_dev, size_t P, float *sel_dev, float *rest_dev,
+            void *stream) {
+    if (!good(ctx) || !x_dev || P == 0) return HE_ERR_INVALID_ARG;
+    size_t k = P;
+    if (mask) {
+        if (!good(mask) || mask->P != P) return HE_ERR_INVALID_ARG;
+        k = mask->k;
+        if (k < P && !rest_dev) return HE_ERR_INVALID_ARG;
+    }
+    const size_t padded = he_num_ct(ctx, k) * he_slots(ctx);
+    if (padded && !sel_dev) return HE_ERR_INVALID_ARG;
+    CU(launch_pack(mask, x_dev, P, k, padded, sel_dev, rest_dev, as_stream(stream)));
+    return HE_OK;
+}
+
+int he_encode(he_ctx *ctx, const float *sel_dev, size_t k, int64_t *m_dev, void *stream) {
+    if (!good(ctx) || !sel_dev || !m_dev) return HE_ERR_INVALID_ARG;
+    const size_t T = he_num_ct(ctx, k);
+    if (T == 0) return HE_OK;
+    int rc = ensure(&ctx->ws, &ctx->ws_bytes, work_bytes(ctx, T));
+    if (rc != HE_OK) return rc;
+    CU(launch_encode(ctx->dev, sel_dev, T, static_cast<double2 *>(ctx->ws), m_dev, as_stream(stream)));
+    return HE_OK;
+}
+
+int he_encrypt_range(he_ctx *ctx, const he_keys *keys, const float *sel_dev, size_t t_begin, size_t t_count,
+                     uint64_t seed, uint32_t client_id, uint64_t *ct_dev, void *stream) {
+    if (!good(ctx) || !good(keys) || keys->ctx != ctx) return HE_ERR_INVALID_ARG;
+    if (t_begin + t_count >= (1ull << 32)) return HE_ERR_SIZE;
+    if (t_count == 0) return HE_OK;
+    if (!sel_dev || !ct_dev) return HE_ERR_INVALID_ARG;
+    const CtxDev &d = ctx->dev;
+    int rc = ensure(&ctx->ws, &ctx->ws_bytes, work_bytes(ctx, t_count));
+    if (rc != HE_OK) return rc;
+    int64_t *m = static_cast<int64_t *>(ctx->ws);
+    double2 *cplx = reinterpret_cast<double2 *>(m + t_count * d.N);
+    cudaStream_t st = as_stream(stream);
+    CU(launch_encode(d, sel_dev, t_count, cplx, m, st));
+    CU(launch_encrypt(d, keys->dev, m, (uint32_t)t_begin, t_count, seed, client_id, ct_dev, st));
+    return HE_OK;
+}
+
+int he_encrypt(he_ctx *ctx, const he_keys *keys, const float *sel_dev, size_t k, uint64_t seed,
+               uint32_t client_id, uint64_t *ct_dev, void *stream) {
+    if (!good(ctx)) return HE_ERR_INVALID_ARG;
+    return he_encrypt_range(ctx, keys, sel_dev, 0, he_num_ct(ctx, k), seed, client_id, ct_dev, stream);
+}
+
+int he_weighted_aggregate(he_ctx *ctx, const uint64_t *const *cts_host, const double *alpha_host, int C,
+                          size_t T, uint64_t *agg_dev, void *stream) {
+    if (!good(ctx) || !cts_host || !alpha_host || C < 1) return HE_ERR_INVALID_ARG;
+    if (C > HE_MAX_CLIENTS) return HE_ERR_SIZE;
+    if (T && !agg_dev) return HE_ERR_INVALID_ARG;
+    const CtxDev &d = ctx->dev;
+    const uint32_t L = d.L;
+    // weights as constant polynomials at scale q_{L-1}: W_i = rint(alpha_i * q_{L-1})
+    const double ql = (double)d.limb[L - 1].q;
+    std::vector<unsigned char> host(C * (sizeof(void *) + L * sizeof(tw_t)));
+    const uint64_t **ptrs = reinterpret_cast<const uint64_t **>(host.data());
+    tw_t *wt = reinterpret_cast<tw_t *>(host.data() + C * sizeof(void *));
+    for (int i = 0; i < C; i++) {
+        if (T && !cts_host[i]) return HE_ERR_INVALID_ARG;
+        const double a = alpha_host[i];
+        if (!(a >= 0.0) || !(a <= 1.0)) return HE_ERR_INVALID_ARG;
+        const double prod = a * ql;
+        const uint64_t W = (uint64_t)rint(prod);
+        ptrs[i] = cts_host[i];
+        for (uint32_t j = 0; j < L; j++) {
+            const HostTw w = host_shoup(W % d.limb[j].q, d.limb[j].q);
+            wt[i * L + j] = tw_t{w.w, w.wp};
+        }
+    }
+    if (T == 0) return HE_OK;
+    cudaStream_t st = as_stream(stream);
+    CU(cudaMemcpyAsync(ctx->tab, host.data(), host.size(), cudaMemcpyHostToDevice, st));
+    const uint64_t *const *dptrs = static_cast<const uint64_t *const *>(ctx->tab);
+    const tw_t *dw = reinterpret_cast<const tw_t *>(static_cast<unsigned char *>(ctx->tab) + C * sizeof(void *));
+    CU(launch_aggregate(d, dptrs, dw, C, T, agg_dev, st));
+    return HE_OK;
+}
+
+int he_plain_aggregate(he_ctx *ctx, const float *const *rests_host, const double *alpha_host, int C,
+                       size_t len, double *out_dev, void *stream) {
+    if (!good(ctx) || !rests_host || !alpha_host || C < 1) return HE_ERR_INVALID_ARG;
+    if (C > HE_MAX_CLIENTS) return HE_ERR_SIZE;
+    if (len == 0) return HE_OK;
+    if (!out_dev) return HE_ERR_INVALID_ARG;
+    std::vector<unsigned char> host(C * (sizeof(void *) + sizeof(double)));
+    const float **ptrs = reinterpret_cast<const float **>(host.data());
+    double *al = reinterpret_cast<double *>(host.data() + C * sizeof(void *));
+    for (int i = 0; i < C; i++) {
+        if (!rests_host[i]) return HE_ERR_INVALID_ARG;
+        ptrs[i] = rests_host[i];
+        al[i] = alpha_host[i];
+    }
+    cudaStream_t st = as_stream(stream);
+    // second half of the table buffer, so that it does not collide with a
+    // ciphertext aggregation queued just before
+    unsigned char *base = static_cast<unsigned char *>(ctx->tab) + HE_MAX_CLIENTS * (sizeof(void *) + HE_MAX_LIMBS * sizeof(tw_t));
+    CU(cudaMemcpyAsync(base, host.data(), host.size(), cudaMemcpyHostToDevice, st));
+    CU(launch_plain_aggregate(reinterpret_cast<const float *const *>(base),
+                              reinterpret_cast<const double *>(base + C * sizeof(void *)), C, len, out_dev, st));
+    return HE_OK;
+}
+
+int he_decrypt_level(he_ctx *ctx, const he_keys *keys, const uint64_t *ct_dev, uint32_t level, size_t T,
+                     double *z_dev, void *stream) {
+    if (!good(ctx) || !good(keys) || keys->ctx != ctx) return HE_ERR_INVALID_ARG;
+    if (level < 1 || level > ctx->dev.L) return HE_ERR_LEVEL;
+    if (T == 0) return HE_OK;
+    if (!ct_dev || !z_dev) return HE_ERR_INVALID_ARG;
+    const CtxDev &d = ctx->dev;
+    int rc = ensure(&ctx->ws, &ctx->ws_bytes, work_bytes(ctx, T));
+    if (rc != HE_OK) return rc;
+    uint64_t *scratch = static_cast<uint64_t *>(ctx->ws);
+    double2 *cplx = reinterpret_cast<double2 *>(scratch + T * d.N);
+    cudaStream_t st = as_stream(stream);
+    CU(launch_decrypt(d, keys->dev, ct_dev, level, T, scratch, st));
+    CU(launch_decode(d, reinterpret_cast<const int64_t *>(scratch), T, cplx, z_dev, st));
+    return HE_OK;
+}
+
+int he_decrypt(he_ctx *ctx, const he_keys *keys, const uint64_t *agg_dev, size_t T, double *z_dev, void *stream) {
+    if (!good(ctx)) return HE_ERR_INVALID_ARG;
+    return he_decrypt_level(ctx, keys, agg_dev, ctx->dev.L - 1, T, z_dev, stream);
+}
+
+int he_unpack(he_ctx *ctx, const he_mask *mask, const double *z_dev, const double *rest_avg_dev, size_t P,
+              double *w_glob_dev, void *stream) {
+    if (!good(ctx) || !w_glob_dev || P == 0) return HE_ERR_INVALID_ARG;
+    if (mask) {
+        if (!good(mask) || mask->P != P) return HE_ERR_INVALID_ARG;
+        if (mask->k < P && !rest_avg_dev) return HE_ERR_INVALID_ARG;
+        if (mask->k && !z_dev) return HE_ERR_INVALID_ARG;
+    } else if (!z_dev) {
+        return HE_ERR_INVALID_ARG;
+    }
+    CU(launch_unpack(mask, z_dev, rest_avg_dev, P, w_glob_dev, as_stream(stream)));
+    return HE_OK;
+}
+
+int he_ntt_forward(he_ctx *ctx, uint64_t *polys_dev, size_t B, void *stream) {
+    if (!good(ctx) || !polys_dev) return HE_ERR_INVALID_ARG;
+    const CtxDev &d = ctx->dev;
+    if ((B * d.L) >> (31 - d.A)) return HE_ERR_SIZE;
+    CU(launch_ntt(d, true, polys_dev, B, (size_t)d.L * d.N, 0, d.L, as_stream(stream)));
+    return HE_OK;
+}
+
+int he_ntt_inverse(he_ctx *ctx, uint64_t *polys_dev, size_t B, void *stream) {
+    if (!good(ctx) || !polys_dev) return HE_ERR_INVALID_ARG;
+    const CtxDev &d = ctx->dev;
+    if ((B * d.L) >> (31 - d.A)) return HE_ERR_SIZE;
+    CU(launch_ntt(d, false, polys_dev, B, (size_t)d.L * d.N, 0, d.L, as_stream(stream)));
+    return HE_OK;
+}
+
+// ---------------------------------------------------------------------------
+// whole round from host memory
+// ---------------------------------------------------------------------------
+
+int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const float *const *xs_host,
+                  const double *alpha_host, int C, size_t P, uint64_t enc_seed, double *w_glob_host,
+                  void *stream) {
+    if (!good(ctx) || !good(keys) || keys->ctx != ctx || !xs_host || !alpha_host || !w_glob_host || C < 1 || P == 0)
+        return HE_ERR_INVALID_ARG;
+    if (C > HE_MAX_CLIENTS) return HE_ERR_SIZE;
+    size_t k = P;
+    if (mask) {
+        if (!good(mask) || mask->P != P) return HE_ERR_INVALID_ARG;
+        k = mask->k;
+    }
+    const CtxDev &d = ctx->dev;
+    const size_t n = d.N / 2, T = he_num_ct(ctx, k), padded = T * n, restlen = P - k;
+    const size_t ctw = 2 * (size_t)d.L * d.N, aggw = 2 * (size_t)(d.L - 1) * d.N;
+    // ciphertext indices are processed in chunks that keep all clients'
+    // ciphertexts of a chunk within about 4 GiB
+    size_t Tc = ((size_t)4 << 30) / (C * ctw * sizeof(uint64_t));
+    if (Tc < 1) Tc = 1;
+    if (Tc > T) Tc = T;
+    auto align = [](size_t b) { return (b + 255) & ~(size_t)255; };
+    const size_t b_x = align(P * sizeof(float)), b_sel = align(padded * sizeof(float)),
+                 b_rest = align(restlen * sizeof(float)), b_cts = align(C * Tc * ctw * sizeof(uint64_t)),
+                 b_agg = align(Tc * aggw * sizeof(uint64_t)), b_z = align(padded * sizeof(double)),
+                 b_ravg = align(restlen * sizeof(double)), b_out = align(P * sizeof(double));
+    const size_t total = b_x + C * (b_sel + b_rest) + b_cts + b_agg + b_z + b_ravg + b_out;
+    int rc = ensure(&ctx->round_buf, &ctx->round_bytes, total);
+    if (rc != HE_OK) return rc;
+    rc = ensure(&ctx->ws, &ctx->ws_bytes, work_bytes(ctx, Tc));
+    if (rc != HE_OK) return rc;
+    unsigned char *p = static_cast<unsigned char *>(ctx->round_buf);
+    float *x = reinterpret_cast<float *>(p); p += b_x;
+    std::vector<float *> sel(C), rest(C);
+    for (int i = 0; i < C; i++) { sel[i] = reinterpret_cast<float *>(p); p += b_sel; }
+    for (int i = 0; i < C; i++) { rest[i] = reinterpret_cast<float *>(p); p += b_rest; }
+    uint64_t *cts = reinterpret_cast<uint64_t *>(p); p += b_cts;
+    uint64_t *agg = reinterpret_cast<uint64_t *>(p); p += b_agg;
+    double *z = reinterpret_cast<double *>(p); p += b_z;
+    double *ravg = reinterpret_cast<double *>(p); p += b_ravg;
+    double *out = reinterpret_cast<double *>(p);
+    cudaStream_t st = as_stream(stream);
+
+    for (int i = 0; i < C; i++) {
+        if (!xs_host[i]) return HE_ERR_INVALID_ARG;
+        CU(cudaMemcpyAsync(x, xs_host[i], P * sizeof(float), cudaMemcpyHostToDevice, st));
+        rc = he_pack(ctx, mask, x, P, sel[i], restlen ? rest[i] : nullptr, stream);
+        if (rc != HE_OK) return rc;
+    }
+    std::vector<const uint64_t *> cptr(C);
+    for (size_t t0 = 0; t0 < T; t0 += Tc) {
+        const size_t tc = T - t0 < Tc ? T - t0 : Tc;
+        for (int i = 0; i < C; i++) {
+            uint64_t *ci = cts + (size_t)i * Tc * ctw;
+            rc = he_encrypt_range(ctx, keys, sel[i] + t0 * n, t0, tc, enc_seed, (uint32_t)i, ci, stream);
+            if (rc != HE_OK) return rc;
+            cptr[i] = ci;
+        }
+        rc = he_weighted_aggregate(ctx, cptr.data(), alpha_host, C, tc, agg, stream);
+        if (rc != HE_OK) return rc;
+        rc = he_decrypt(ctx, keys, agg, tc, z + t0 * n, stream);
+        if (rc != HE_OK) return rc;
+    }
+    if (restlen) {
+        std::vector<const float *> rptr(rest.begin(), rest.end());
+        rc = he_plain_aggregate(ctx, rptr.data(), alpha_host, C, restlen, ravg, stream);
+        if (rc != HE_OK) return rc;
+    }
+    rc = he_unpack(ctx, mask, z, restlen ? ravg : nullptr, P, out, stream);
+    if (rc != HE_OK) return rc;
+    CU(cudaMemcpyAsync(w_glob_host, out, P * sizeof(double), cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    return HE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,130 @@
+// Device-side primitives: 64-bit modular arithmetic (Shoup / Barrett, lazy
+// Harvey ranges), Philox4x32-10 and the samplers built on it.
+//
+// Functions marked HD also compile for the host so that the thread-level
+// index arithmetic of the transforms can be exercised without a GPU.
+#pragma once
+
+#include <stdint.h>
+
+#if defined(__CUDACC__)
+#define HD __host__ __device__ __forceinline__
+#else
+#define HD inline
+#endif
+
+namespace fedhe {
+
+// ---------------------------------------------------------------------------
+// 64-bit modular arithmetic
+// ---------------------------------------------------------------------------
+
+HD uint64_t mulhi64(uint64_t a, uint64_t b) {
+#if defined(__CUDA_ARCH__)
+    return __umul64hi(a, b);
+#else
+    return (uint64_t)(((unsigned __int128)a * b) >> 64);
+#endif
+}
+
+// x - m if x >= m
+HD uint64_t csub(uint64_t x, uint64_t m) { return x >= m ? x - m : x; }
+
+// Shoup product with a fixed operand w < q and wp = floor(w 2^64 / q):
+// returns x w mod q up to one extra q, i.e. a value in [0, 2q), for any x.
+HD uint64_t shoup_lazy(uint64_t x, uint64_t w, uint64_t wp, uint64_t q) {
+    uint64_t hi = mulhi64(x, wp);
+    return x * w - hi * q;
+}
+
+HD uint64_t shoup(uint64_t x, uint64_t w, uint64_t wp, uint64_t q) {
+    return csub(shoup_lazy(x, w, wp, q), q);
+}
+
+// Barrett reduction of any 64-bit x with mu = floor(2^64 / q): result in [0, q)
+HD uint64_t barrett64(uint64_t x, uint64_t q, uint64_t mu) {
+    uint64_t t = mulhi64(x, mu);
+    uint64_t r = x - t * q;           // in [0, 3q)
+    r = csub(r, 2 * q);
+    return csub(r, q);
+}
+
+// residue in [0, q) of a signed 64-bit integer
+HD uint64_t signed_residue(int64_t v, uint64_t q, uint64_t mu) {
+    uint64_t a = v < 0 ? (uint64_t)0 - (uint64_t)v : (uint64_t)v;
+    uint64_t r = barrett64(a, q, mu);
+    return (v < 0 && r != 0) ? q - r : r;
+}
+
+// residue of a small signed value |v| < q
+HD uint64_t small_residue(int v, uint64_t q) { return v < 0 ? q - (uint64_t)(-v) : (uint64_t)v; }
+
+// Harvey butterflies.  Forward (Cooley-Tukey): inputs and outputs in [0, 4q).
+HD void ct_butterfly(uint64_t &x, uint64_t &y, uint64_t w, uint64_t wp, uint64_t q, uint64_t q2) {
+    uint64_t u = csub(x, q2);
+    uint64_t v = shoup_lazy(y, w, wp, q);
+    x = u + v;
+    y = u - v + q2;
+}
+
+// Inverse (Gentleman-Sande): inputs and outputs in [0, 2q).
+HD void gs_butterfly(uint64_t &x, uint64_t &y, uint64_t w, uint64_t wp, uint64_t q, uint64_t q2) {
+    uint64_t u = x, v = y;
+    x = csub(u + v, q2);
+    y = shoup_lazy(u - v + q2, w, wp, q);
+}
+
+// ---------------------------------------------------------------------------
+// Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11)
+// ---------------------------------------------------------------------------
+
+struct u32x4 { uint32_t x, y, z, w; };
+
+HD void mulhilo32(uint32_t a, uint32_t b, uint32_t &hi, uint32_t &lo) {
+#if defined(__CUDA_ARCH__)
+    lo = a * b;
+    hi = __umulhi(a, b);
+#else
+    uint64_t p = (uint64_t)a * b;
+    lo = (uint32_t)p;
+    hi = (uint32_t)(p >> 32);
+#endif
+}
+
+HD u32x4 philox4x32_10(u32x4 c, uint32_t k0, uint32_t k1) {
+#pragma unroll
+    for (int r = 0; r < 10; r++) {
+        uint32_t h0, l0, h1, l1;
+        mulhilo32(0xD2511F53u, c.x, h0, l0);
+        mulhilo32(0xCD9E8D57u, c.z, h1, l1);
+        u32x4 n;
+        n.x = h1 ^ c.y ^ k0;
+        n.y = l1;
+        n.z = h0 ^ c.w ^ k1;
+        n.w = l0;
+        c = n;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return c;
+}
+
+// Stream coordinates: counter = (block, ciphertext index, client, tag | limb << 8),
+// key = the two halves of the seed.
+enum : uint32_t { TAG_SK = 1, TAG_PK_A = 2, TAG_PK_E = 3, TAG_ENC_U = 4, TAG_ENC_E0 = 5, TAG_ENC_E1 = 6 };
+
+HD u32x4 stream_block(uint64_t seed, uint32_t block, uint32_t t, uint32_t client, uint32_t tag_limb) {
+    u32x4 c = {block, t, client, tag_limb};
+    return philox4x32_10(c, (uint32_t)seed, (uint32_t)(seed >> 32));
+}
+
+// uniform ternary value from one 32-bit word: floor(3 w / 2^32) - 1
+HD int ternary_from_word(uint32_t w) {
+#if defined(__CUDA_ARCH__)
+    return (int)__umulhi(w, 3u) - 1;
+#else
+    return (int)(((uint64_t)w * 3u) >> 32) - 1;
+#endif
+}
+
+}  // namespace fedhe

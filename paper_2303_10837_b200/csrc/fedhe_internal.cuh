@@ -1,0 +1,75 @@
+// Internal types shared by the kernels and the C ABI of the CUDA library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/fedhe.h"
+#include "fedhe_ntt.cuh"
+
+namespace fedhe {
+
+// Per-prime constants and table pointers, passed to kernels by value.
+struct LimbDev {
+    uint64_t q;          // the prime
+    uint64_t mu;         // floor(2^64 / q), Barrett
+    tw_t ninv;           // 1/N
+    tw_t wn;             // (inverse twiddle of stage 0) / N
+    tw_t qlinv;          // 1 / q_{L-1} mod q (unused for the last prime)
+    const tw_t *fwd;     // psi^brev(i)
+    const tw_t *inv;     // psi^-brev(i)
+};
+
+struct CtxDev {
+    uint32_t N, logN, L;
+    uint32_t LOGB, A;    // a length-N transform = 2^A blocks of 2^LOGB
+    int32_t log2_delta;
+    LimbDev limb[HE_MAX_LIMBS];
+    const double2 *ftw;  // slot-transform twiddles, entry [len/2 + j]
+    int *status;         // sticky anomaly word
+};
+
+struct KeysDev {
+    const tw_t *pk0_hat; // [L][N] transform-domain public key with Shoup companions
+    const tw_t *pk1_hat;
+    const tw_t *s_hat;   // [L][N] transform-domain secret key
+    const int8_t *s;     // [N]
+};
+
+}  // namespace fedhe
+
+struct he_ctx {
+    uint32_t magic;
+    int device;
+    fedhe::CtxDev dev;
+    he_params params;
+    std::vector<void *> owned;     // device allocations freed with the context
+    // growable work buffers (device)
+    void *ws = nullptr;            // encode output / decrypt scratch
+    size_t ws_bytes = 0;
+    void *tab = nullptr;           // per-call pointer and weight tables
+    size_t tab_bytes = 0;
+    void *round_buf = nullptr;     // buffers of he_round_host
+    size_t round_bytes = 0;
+};
+
+struct he_keys {
+    uint32_t magic;
+    he_ctx *ctx;
+    fedhe::KeysDev dev;
+    void *storage;
+};
+
+struct he_mask {
+    uint32_t magic;
+    size_t P, k;
+    uint32_t *idx;       // [k] ascending
+    uint32_t *bits;      // [ceil(P/32)] bit i of word i/32 set if parameter i is encrypted
+    uint32_t *wpre;      // [ceil(P/32)] number of encrypted parameters before the word
+};
+
+namespace fedhe {
+constexpr uint32_t CTX_MAGIC = 0x48454358u, KEYS_MAGIC = 0x48454b59u, MASK_MAGIC = 0x48454d4bu;
+}

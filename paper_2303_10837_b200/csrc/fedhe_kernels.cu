@@ -1,0 +1,1101 @@
+// CUDA kernels (sm_100a) of the FedML-HE secure-aggregation hot path and their
+// launch wrappers.  Nothing here is a dense floating-point contraction, so no
+// tensor-core path exists: the transforms are bound by 64-bit integer
+// multiply throughput, the pointwise passes by HBM bandwidth.
+#include "fedhe_launch.h"
+
+#include <atomic>
+
+namespace fedhe {
+
+static std::atomic<uint64_t> g_launches{0};
+uint64_t launch_count() { return g_launches.load(); }
+
+#define FEDHE_LAUNCHED() (g_launches.fetch_add(1), cudaGetLastError())
+
+static inline unsigned blocks_for(size_t count, unsigned per_block) {
+    return (unsigned)((count + per_block - 1) / per_block);
+}
+
+// ---------------------------------------------------------------------------
+// discrete Gaussian, sigma = 3.2 on [-19, 19]: thresholds floor(2^64 Pr[X <= x])
+// for x = -19 .. 18; a 64-bit uniform r maps to -19 + #{x : r >= T[x]}
+// ---------------------------------------------------------------------------
+__constant__ uint64_t c_gauss_cdf[38] = {
+    0x0000000bd798c7acull, 0x00000053f5e234f7ull, 0x000001e24b89625aull, 0x000009adbc7900e1ull,
+    0x00002d17ca1e3a82ull, 0x0000bf05ff772ee2ull, 0x0002e06843bbf95dull, 0x000a19062dceb033ull,
+    0x00204c0ded173b17ull, 0x005e3163ffc656a8ull, 0x00fab6a7e614dfaeull, 0x0261b16e99bc14f8ull,
+    0x054c69348bbc9867ull, 0x0acd276539458231ull, 0x143796b3c337f00bull, 0x22d43df09de40e7aull,
+    0x37651d96aa4fb429ull, 0x51a5da2b40f1bff1ull, 0x700ad4bf5a6e80e2ull, 0x8ff52b40a5917f1dull,
+    0xae5a25d4bf0e400eull, 0xc89ae26955b04bd6ull, 0xdd2bc20f621bf185ull, 0xebc8694c3cc80ff4ull,
+    0xf532d89ac6ba7dceull, 0xfab396cb74436798ull, 0xfd9e4e916643eb07ull, 0xff05495819eb2051ull,
+    0xffa1ce9c0039a957ull, 0xffdfb3f212e8c4e8ull, 0xfff5e6f9d2314fccull, 0xfffd1f97bc4406a2ull,
+    0xffff40fa0088d11dull, 0xffffd2e835e1c57dull, 0xfffff6524386ff1eull, 0xfffffe1db4769da5ull,
+    0xffffffac0a1dcb08ull, 0xfffffff428673853ull};
+
+__device__ __forceinline__ int gauss_from_u64(uint64_t r) {
+    int v = -19;
+#pragma unroll
+    for (int x = 0; x < 38; x++) v += (r >= c_gauss_cdf[x]) ? 1 : 0;
+    return v;
+}
+
+__device__ __forceinline__ uint64_t addmod(uint64_t a, uint64_t b, uint64_t q) { return csub(a + b, q); }
+__device__ __forceinline__ uint64_t submod(uint64_t a, uint64_t b, uint64_t q) { return a >= b ? a - b : a + q - b; }
+
+// slow exact helpers, used only at key generation
+__device__ uint64_t mod_u128(uint64_t hi, uint64_t lo, uint64_t q) {
+    uint64_t r = 0;
+    for (int i = 63; i >= 0; i--) { r = (r << 1) | ((hi >> i) & 1); r = csub(r, q); }
+    for (int i = 63; i >= 0; i--) { r = (r << 1) | ((lo >> i) & 1); r = csub(r, q); }
+    return r;
+}
+__device__ uint64_t mulmod_slow(uint64_t a, uint64_t b, uint64_t q) {
+    return mod_u128(__umul64hi(a, b), a * b, q);
+}
+__device__ uint64_t shoup_companion(uint64_t w, uint64_t q) {   // floor(w 2^64 / q), w < q
+    uint64_t rem = w, quo = 0;
+    for (int i = 0; i < 64; i++) {
+        rem <<= 1; quo <<= 1;
+        if (rem >= q) { rem -= q; quo |= 1; }
+    }
+    return quo;
+}
+
+// ===========================================================================
+// batched negacyclic NTT
+// ===========================================================================
+
+template <class L, bool FWD, bool SCALED>
+__global__ void __launch_bounds__(L::NT, 1)
+ntt_block_kernel(const __grid_constant__ CtxDev c, uint64_t *data, size_t poly_stride, uint32_t limb0,
+                 uint32_t nlimbs) {
+    extern __shared__ __align__(16) uint64_t sm[];
+    const uint32_t tid = threadIdx.x;
+    uint32_t b = blockIdx.x;
+    const uint32_t blk = b & ((1u << c.A) - 1u);
+    b >>= c.A;
+    const uint32_t limb = b % nlimbs;
+    const size_t poly = b / nlimbs;
+    const LimbDev &lb = c.limb[limb0 + limb];
+    const uint64_t q = lb.q, q2 = 2 * q;
+    uint64_t *p = data + poly * poly_stride + (size_t)limb * c.N + ((size_t)blk << L::LOGB);
+    uint64_t x[L::E];
+    constexpr int LAST = L::NPH - 1;
+    if constexpr (FWD) {
+#pragma unroll
+        for (int r = 0; r < L::E; r++) x[r] = p[L::template idx<0>(tid, r)];
+        NttArgs a = {lb.fwd, q, q2, c.A, blk};
+        block_ntt_forward<L>(x, sm, tid, a);
+#pragma unroll
+        for (int r = 0; r < L::E; r += 2) {          // registers r, r+1 are neighbours in memory
+            ulonglong2 v;
+            v.x = csub(csub(x[r], q2), q);
+            v.y = csub(csub(x[r + 1], q2), q);
+            *reinterpret_cast<ulonglong2 *>(p + L::template idx<LAST>(tid, r)) = v;
+        }
+    } else {
+#pragma unroll
+        for (int r = 0; r < L::E; r += 2) {
+            ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(p + L::template idx<LAST>(tid, r));
+            x[r] = v.x;
+            x[r + 1] = v.y;
+        }
+        NttArgs a = {lb.inv, q, q2, c.A, blk};
+        block_ntt_inverse<L, SCALED>(x, sm, tid, a, lb.ninv, lb.wn);
+#pragma unroll
+        for (int r = 0; r < L::E; r++)
+            p[L::template idx<0>(tid, r)] = SCALED ? csub(x[r], q) : x[r];
+    }
+}
+
+// The A = logN - LOGB outer stages of a long transform: every thread owns two
+// neighbouring columns of the 2^A x B matrix view and does the A stages that
+// pair rows, reading and writing whole 16-byte words.
+template <bool FWD>
+__global__ void __launch_bounds__(256)
+ntt_outer_kernel(const __grid_constant__ CtxDev c, uint64_t *data, size_t poly_stride, uint32_t limb0,
+                 uint32_t nlimbs, size_t total) {
+    size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t B = 1u << c.LOGB, half = B >> 1;
+    const uint32_t col = (uint32_t)(g % half) * 2;
+    g /= half;
+    const uint32_t limb = (uint32_t)(g % nlimbs);
+    const size_t poly = g / nlimbs;
+    const LimbDev &lb = c.limb[limb0 + limb];
+    const uint64_t q = lb.q, q2 = 2 * q;
+    uint64_t *p = data + poly * poly_stride + (size_t)limb * c.N + col;
+    const uint32_t A = c.A, rows = 1u << A;      // A is 1 or 2
+    u64x2 x[4];
+    for (uint32_t a = 0; a < rows; a++) x[a] = *reinterpret_cast<const u64x2 *>(p + (size_t)a * B);
+    if (FWD) {
+        for (uint32_t s = 0; s < A; s++) {
+            const uint32_t bit = 1u << (A - 1 - s);
+            for (uint32_t a = 0; a < rows; a++) {
+                if (a & bit) continue;
+                tw_t w = load_tw(lb.fwd + (1u << s) + (a >> (A - s)));
+                ct_butterfly(x[a].x, x[a | bit].x, w.w, w.wp, q, q2);
+                ct_butterfly(x[a].y, x[a | bit].y, w.w, w.wp, q, q2);
+            }
+        }
+    } else {
+        for (int s = (int)A - 1; s >= 1; s--) {
+            const uint32_t bit = 1u << (A - 1 - s);
+            for (uint32_t a = 0; a < rows; a++) {
+                if (a & bit) continue;
+                tw_t w = load_tw(lb.inv + (1u << s) + (a >> (A - s)));
+                gs_butterfly(x[a].x, x[a | bit].x, w.w, w.wp, q, q2);
+                gs_butterfly(x[a].y, x[a | bit].y, w.w, w.wp, q, q2);
+            }
+        }
+        const uint32_t bit = 1u << (A - 1);      // stage 0 with 1/N folded in
+        for (uint32_t a = 0; a < rows; a++) {
+            if (a & bit) continue;
+            uint64_t u0 = x[a].x, v0 = x[a | bit].x, u1 = x[a].y, v1 = x[a | bit].y;
+            x[a].x = shoup(u0 + v0, lb.ninv.w, lb.ninv.wp, q);
+            x[a | bit].x = shoup(u0 - v0 + q2, lb.wn.w, lb.wn.wp, q);
+            x[a].y = shoup(u1 + v1, lb.ninv.w, lb.ninv.wp, q);
+            x[a | bit].y = shoup(u1 - v1 + q2, lb.wn.w, lb.wn.wp, q);
+        }
+    }
+    for (uint32_t a = 0; a < rows; a++) *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = x[a];
+}
+
+template <class L>
+static cudaError_t launch_ntt_blocks(const CtxDev &c, bool forward, uint64_t *data, size_t npoly,
+                                     size_t poly_stride, uint32_t limb0, uint32_t nlimbs, cudaStream_t s) {
+    const size_t smem = sizeof(uint64_t) << L::LOGB;
+    const unsigned grid = (unsigned)((npoly * nlimbs) << c.A);
+    cudaError_t e;
+    if (forward) {
+        auto k = ntt_block_kernel<L, true, false>;
+        if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+        k<<<grid, L::NT, smem, s>>>(c, data, poly_stride, limb0, nlimbs);
+    } else if (c.A == 0) {
+        auto k = ntt_block_kernel<L, false, true>;
+        if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+        k<<<grid, L::NT, smem, s>>>(c, data, poly_stride, limb0, nlimbs);
+    } else {
+        auto k = ntt_block_kernel<L, false, false>;
+        if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+        k<<<grid, L::NT, smem, s>>>(c, data, poly_stride, limb0, nlimbs);
+    }
+    return FEDHE_LAUNCHED();
+}
+
+cudaError_t launch_ntt(const CtxDev &c, bool forward, uint64_t *data, size_t npoly, size_t poly_stride,
+                       uint32_t limb0, uint32_t nlimbs, cudaStream_t s) {
+    if (npoly == 0 || nlimbs == 0) return cudaSuccess;
+    cudaError_t e;
+    const size_t outer_threads = npoly * nlimbs * ((size_t)1 << (c.LOGB - 1));
+    if (forward && c.A > 0) {
+        ntt_outer_kernel<true><<<blocks_for(outer_threads, 256), 256, 0, s>>>(c, data, poly_stride, limb0,
+                                                                              nlimbs, outer_threads);
+        if ((e = FEDHE_LAUNCHED())) return e;
+    }
+    if (c.LOGB == 13) e = launch_ntt_blocks<Lay<13, 4>>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
+    else e = launch_ntt_blocks<Lay<14, 4>>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
+    if (e) return e;
+    if (!forward && c.A > 0) {
+        ntt_outer_kernel<false><<<blocks_for(outer_threads, 256), 256, 0, s>>>(c, data, poly_stride, limb0,
+                                                                               nlimbs, outer_threads);
+        if ((e = FEDHE_LAUNCHED())) return e;
+    }
+    return cudaSuccess;
+}
+
+// ===========================================================================
+// key generation
+// ===========================================================================
+
+// tmp[0] = s, tmp[1] = a, tmp[2] = e as residues, each [L][N]
+__global__ void __launch_bounds__(256)
+keygen_sample_kernel(const __grid_constant__ CtxDev c, uint64_t seed, int8_t *s8, uint64_t *tmp) {
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= c.N) return;
+    u32x4 ws = stream_block(seed, i >> 2, 0, 0, TAG_SK);
+    const uint32_t wsel = (i & 3) == 0 ? ws.x : (i & 3) == 1 ? ws.y : (i & 3) == 2 ? ws.z : ws.w;
+    const int sv = ternary_from_word(wsel);
+    u32x4 we = stream_block(seed, i >> 1, 0, 0, TAG_PK_E);
+    const uint64_t r = (i & 1) ? ((uint64_t)we.z | ((uint64_t)we.w << 32)) : ((uint64_t)we.x | ((uint64_t)we.y << 32));
+    const int ev = gauss_from_u64(r);
+    s8[i] = (int8_t)sv;
+    const size_t LN = (size_t)c.L * c.N;
+    for (uint32_t j = 0; j < c.L; j++) {
+        const uint64_t q = c.limb[j].q;
+        u32x4 wa = stream_block(seed, i, 0, 0, TAG_PK_A | (j << 8));
+        const uint64_t lo = (uint64_t)wa.x | ((uint64_t)wa.y << 32), hi = (uint64_t)wa.z | ((uint64_t)wa.w << 32);
+        tmp[0 * LN + (size_t)j * c.N + i] = small_residue(sv, q);
+        tmp[1 * LN + (size_t)j * c.N + i] = mod_u128(hi, lo, q);
+        tmp[2 * LN + (size_t)j * c.N + i] = small_residue(ev, q);
+    }
+}
+
+// transform-domain keys with Shoup companions: pk1^ = a^, pk0^ = e^ - a^ s^
+__global__ void __launch_bounds__(256)
+keygen_combine_kernel(const __grid_constant__ CtxDev c, const uint64_t *tmp, tw_t *pk0_hat, tw_t *pk1_hat,
+                      tw_t *s_hat) {
+    const size_t LN = (size_t)c.L * c.N;
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= LN) return;
+    const uint64_t q = c.limb[g / c.N].q;
+    const uint64_t S = tmp[g], A = tmp[LN + g], E = tmp[2 * LN + g];
+    const uint64_t p0 = submod(E, mulmod_slow(A, S, q), q);
+    pk0_hat[g] = tw_t{p0, shoup_companion(p0, q)};
+    pk1_hat[g] = tw_t{A, shoup_companion(A, q)};
+    s_hat[g] = tw_t{S, shoup_companion(S, q)};
+}
+
+__global__ void __launch_bounds__(256) extract_values_kernel(const tw_t *src, uint64_t *dst, size_t count) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g < count) dst[g] = src[g].w;
+}
+
+cudaError_t launch_keygen_sample(const CtxDev &c, uint64_t seed, int8_t *s8, uint64_t *tmp, cudaStream_t s) {
+    keygen_sample_kernel<<<blocks_for(c.N, 256), 256, 0, s>>>(c, seed, s8, tmp);
+    return FEDHE_LAUNCHED();
+}
+cudaError_t launch_keygen_combine(const CtxDev &c, const uint64_t *tmp, tw_t *pk0_hat, tw_t *pk1_hat,
+                                  tw_t *s_hat, cudaStream_t s) {
+    keygen_combine_kernel<<<blocks_for((size_t)c.L * c.N, 256), 256, 0, s>>>(c, tmp, pk0_hat, pk1_hat, s_hat);
+    return FEDHE_LAUNCHED();
+}
+cudaError_t launch_extract_values(const tw_t *src, uint64_t *dst, size_t count, cudaStream_t s) {
+    extract_values_kernel<<<blocks_for(count, 256), 256, 0, s>>>(src, dst, count);
+    return FEDHE_LAUNCHED();
+}
+
+// ===========================================================================
+// CKKS slot transform (fp64).  Encoding must reproduce one fixed radix-2
+// network operation by operation (separate IEEE multiply and add, no fused
+// multiply-add), because the rounded integers are compared bit for bit.
+// ===========================================================================
+
+struct cpx { double re, im; };
+
+__device__ __forceinline__ cpx cadd_rn(cpx a, cpx b) { return cpx{__dadd_rn(a.re, b.re), __dadd_rn(a.im, b.im)}; }
+__device__ __forceinline__ cpx csub_rn(cpx a, cpx b) { return cpx{__dsub_rn(a.re, b.re), __dsub_rn(a.im, b.im)}; }
+// (a + bi)(c + di) = (ac - bd) + (ad + bc) i, data operand first
+__device__ __forceinline__ cpx cmul_rn(cpx x, cpx w) {
+    cpx r;
+    r.re = __dsub_rn(__dmul_rn(x.re, w.re), __dmul_rn(x.im, w.im));
+    r.im = __dadd_rn(__dmul_rn(x.re, w.im), __dmul_rn(x.im, w.re));
+    return r;
+}
+__device__ __forceinline__ cpx load_ftw(const double2 *ftw, uint32_t i) {
+    double2 v = __ldg(ftw + i);
+    return cpx{v.x, v.y};
+}
+
+// decimation-in-frequency stage of the inverse (encoding) network
+template <class L, int P, int I>
+__device__ __forceinline__ void dif_stage(cpx (&x)[L::E], uint32_t tid, const double2 *ftw) {
+    constexpr int s = P * L::LE + I;
+    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
+    constexpr int bit = nst - 1 - I;
+    constexpr uint32_t half = 1u << (L::LOGB - 1 - s);
+#pragma unroll
+    for (int r = 0; r < L::E; r++) {
+        if (r & (1 << bit)) continue;
+        const uint32_t j = L::template idx<P>(tid, r) & (half - 1u);
+        cpx w = load_ftw(ftw, half + j);
+        w.im = -w.im;
+        const cpx U = x[r], V = x[r | (1 << bit)];
+        x[r] = cadd_rn(U, V);
+        x[r | (1 << bit)] = cmul_rn(csub_rn(U, V), w);
+    }
+}
+
+// decimation-in-time stage of the forward (decoding) network
+template <class L, int P, int I>
+__device__ __forceinline__ void dit_stage(cpx (&x)[L::E], uint32_t tid, const double2 *ftw) {
+    constexpr int s = P * L::LE + I;
+    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
+    constexpr int bit = nst - 1 - I;
+    constexpr uint32_t half = 1u << (L::LOGB - 1 - s);
+#pragma unroll
+    for (int r = 0; r < L::E; r++) {
+        if (r & (1 << bit)) continue;
+        const uint32_t j = L::template idx<P>(tid, r) & (half - 1u);
+        const cpx w = load_ftw(ftw, half + j);
+        const cpx U = x[r], V = cmul_rn(x[r | (1 << bit)], w);
+        x[r] = cadd_rn(U, V);
+        x[r | (1 << bit)] = csub_rn(U, V);
+    }
+}
+
+template <class L, int P, int I = 0>
+__device__ __forceinline__ void dif_phase(cpx (&x)[L::E], uint32_t tid, const double2 *ftw) {
+    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
+    if constexpr (I < nst) {
+        dif_stage<L, P, I>(x, tid, ftw);
+        dif_phase<L, P, I + 1>(x, tid, ftw);
+    }
+}
+template <class L, int P, int I>
+__device__ __forceinline__ void dit_phase_from(cpx (&x)[L::E], uint32_t tid, const double2 *ftw) {
+    if constexpr (I >= 0) {
+        dit_stage<L, P, I>(x, tid, ftw);
+        dit_phase_from<L, P, I - 1>(x, tid, ftw);
+    }
+}
+
+template <class L, int PF, int PT>
+__device__ __forceinline__ void cpx_exchange(cpx (&x)[L::E], cpx *sm, uint32_t tid) {
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < L::E; r++) sm[swz(L::template idx<PF>(tid, r))] = x[r];
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < L::E; r++) x[r] = sm[swz(L::template idx<PT>(tid, r))];
+}
+
+template <class L, int P = 0>
+__device__ __forceinline__ void block_dif(cpx (&x)[L::E], cpx *sm, uint32_t tid, const double2 *ftw) {
+    dif_phase<L, P>(x, tid, ftw);
+    if constexpr (P + 1 < L::NPH) {
+        cpx_exchange<L, P, P + 1>(x, sm, tid);
+        block_dif<L, P + 1>(x, sm, tid, ftw);
+    }
+}
+template <class L, int P = L::NPH - 1>
+__device__ __forceinline__ void block_dit(cpx (&x)[L::E], cpx *sm, uint32_t tid, const double2 *ftw) {
+    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
+    dit_phase_from<L, P, nst - 1>(x, tid, ftw);
+    if constexpr (P > 0) {
+        cpx_exchange<L, P, P - 1>(x, sm, tid);
+        block_dit<L, P - 1>(x, sm, tid, ftw);
+    }
+}
+
+__device__ __forceinline__ uint32_t bitrev(uint32_t v, int bits) { return __brev(v) >> (32 - bits); }
+
+// Block part of the encoder: the last LOGB stages on one block of 2^LOGB
+// slots, the bit-reversal, the scaling by Delta/n and the rounding.
+// FROM_CPLX: the block's input comes from the outer stages (n > block).
+template <class L, bool FROM_CPLX>
+__global__ void __launch_bounds__(L::NT)
+encode_block_kernel(const __grid_constant__ CtxDev c, const float *sel, const double2 *cplx, int64_t *m) {
+    extern __shared__ __align__(16) unsigned char smraw[];
+    cpx *sm = reinterpret_cast<cpx *>(smraw);
+    const uint32_t tid = threadIdx.x;
+    const uint32_t n = c.N >> 1, logn = c.logN - 1;
+    const uint32_t nblk = n >> L::LOGB;
+    const uint32_t blk = blockIdx.x % nblk;
+    const size_t t = blockIdx.x / nblk;
+    const size_t base = t * n + ((size_t)blk << L::LOGB);
+    cpx x[L::E];
+#pragma unroll
+    for (int r = 0; r < L::E; r++) {
+        const uint32_t i = L::template idx<0>(tid, r);
+        if constexpr (FROM_CPLX) {
+            double2 v = cplx[base + i];
+            x[r] = cpx{v.x, v.y};
+        } else {
+            x[r] = cpx{(double)sel[base + i], 0.0};
+        }
+    }
+    block_dif<L>(x, sm, tid, c.ftw);
+    // Delta / n is a power of two: one exact multiplication
+    const double scale = __longlong_as_double((long long)(1023 + c.log2_delta - (int)logn) << 52);
+    const double lim = 4611686018427387904.0;   // 2^62
+    int64_t *mt = m + t * c.N;
+    bool bad = false;
+#pragma unroll
+    for (int r = 0; r < L::E; r++) {
+        const uint32_t p = (blk << L::LOGB) | L::template idx<L::NPH - 1>(tid, r);
+        const uint32_t k = bitrev(p, logn);
+        double re = __dmul_rn(x[r].re, scale), im = __dmul_rn(x[r].im, scale);
+        if (!(fabs(re) < lim) || !(fabs(im) < lim)) { bad = true; re = 0.0; im = 0.0; }
+        mt[k] = __double2ll_rn(re);
+        mt[k + n] = __double2ll_rn(im);
+    }
+    if (bad) atomicOr(c.status, 1);
+}
+
+// Outer stages of the encoder for n > block: each thread owns one column of
+// the (n / block) x block view and does the first log2(n / block) stages.
+template <int LOGB>
+__global__ void __launch_bounds__(256)
+encode_outer_kernel(const __grid_constant__ CtxDev c, const float *sel, double2 *cplx, size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t n = c.N >> 1, B = 1u << LOGB;
+    const uint32_t A = (c.logN - 1) - LOGB, rows = 1u << A;   // 1 or 2
+    const uint32_t col = (uint32_t)(g % B);
+    const size_t t = g / B;
+    cpx x[4];
+    for (uint32_t a = 0; a < rows; a++) x[a] = cpx{(double)sel[t * n + (size_t)a * B + col], 0.0};
+    for (uint32_t s = 0; s < A; s++) {
+        const uint32_t bit = 1u << (A - 1 - s), half = n >> (s + 1);
+        for (uint32_t a = 0; a < rows; a++) {
+            if (a & bit) continue;
+            const uint32_t j = (a * B + col) & (half - 1u);
+            cpx w = load_ftw(c.ftw, half + j);
+            w.im = -w.im;
+            const cpx U = x[a], V = x[a | bit];
+            x[a] = cadd_rn(U, V);
+            x[a | bit] = cmul_rn(csub_rn(U, V), w);
+        }
+    }
+    for (uint32_t a = 0; a < rows; a++) cplx[t * n + (size_t)a * B + col] = make_double2(x[a].re, x[a].im);
+}
+
+// Block part of the decoder: bit-reversed load of (d_k + i d_{k+n}) / Delta,
+// the first LOGB stages.  TO_CPLX: more stages follow in decode_outer_kernel.
+template <class L, bool TO_CPLX>
+__global__ void __launch_bounds__(L::NT)
+decode_block_kernel(const __grid_constant__ CtxDev c, const int64_t *d, double2 *cplx, double *z) {
+    extern __shared__ __align__(16) unsigned char smraw[];
+    cpx *sm = reinterpret_cast<cpx *>(smraw);
+    const uint32_t tid = threadIdx.x;
+    const uint32_t n = c.N >> 1, logn = c.logN - 1;
+    const uint32_t nblk = n >> L::LOGB;
+    const uint32_t blk = blockIdx.x % nblk;
+    const size_t t = blockIdx.x / nblk;
+    const int64_t *dt = d + t * c.N;
+    const double inv_delta = __longlong_as_double((long long)(1023 - c.log2_delta) << 52);
+    cpx x[L::E];
+#pragma unroll
+    for (int r = 0; r < L::E; r++) {
+        const uint32_t p = (blk << L::LOGB) | L::template idx<L::NPH - 1>(tid, r);
+        const uint32_t k = bitrev(p, logn);
+        x[r] = cpx{(double)dt[k] * inv_delta, (double)dt[k + n] * inv_delta};
+    }
+    block_dit<L>(x, sm, tid, c.ftw);
+    const size_t base = t * n + ((size_t)blk << L::LOGB);
+#pragma unroll
+    for (int r = 0; r < L::E; r++) {
+        const uint32_t i = L::template idx<0>(tid, r);
+        if constexpr (TO_CPLX) cplx[base + i] = make_double2(x[r].re, x[r].im);
+        else z[base + i] = x[r].re;
+    }
+}
+
+template <int LOGB>
+__global__ void __launch_bounds__(256)
+decode_outer_kernel(const __grid_constant__ CtxDev c, const double2 *cplx, double *z, size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t n = c.N >> 1, B = 1u << LOGB;
+    const uint32_t A = (c.logN - 1) - LOGB, rows = 1u << A;
+    const uint32_t col = (uint32_t)(g % B);
+    const size_t t = g / B;
+    cpx x[4];
+    for (uint32_t a = 0; a < rows; a++) {
+        double2 v = cplx[t * n + (size_t)a * B + col];
+        x[a] = cpx{v.x, v.y};
+    }
+    for (int s = (int)A - 1; s >= 0; s--) {
+        const uint32_t bit = 1u << (A - 1 - s), half = n >> (s + 1);
+        for (uint32_t a = 0; a < rows; a++) {
+            if (a & bit) continue;
+            const uint32_t j = (a * B + col) & (half - 1u);
+            const cpx w = load_ftw(c.ftw, half + j);
+            const cpx U = x[a], V = cmul_rn(x[a | bit], w);
+            x[a] = cadd_rn(U, V);
+            x[a | bit] = csub_rn(U, V);
+        }
+    }
+    for (uint32_t a = 0; a < rows; a++) z[t * n + (size_t)a * B + col] = x[a].re;
+}
+
+template <class L>
+static cudaError_t launch_encode_t(const CtxDev &c, const float *sel, size_t T, double2 *cplx, int64_t *m,
+                                   cudaStream_t s) {
+    const uint32_t n = c.N >> 1;
+    const size_t smem = sizeof(cpx) << L::LOGB;
+    const unsigned grid = (unsigned)(T * (n >> L::LOGB));
+    cudaError_t e;
+    if ((n >> L::LOGB) > 1) {
+        const size_t total = T << L::LOGB;
+        encode_outer_kernel<L::LOGB><<<blocks_for(total, 256), 256, 0, s>>>(c, sel, cplx, total);
+        if ((e = FEDHE_LAUNCHED())) return e;
+        auto k = encode_block_kernel<L, true>;
+        if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+        k<<<grid, L::NT, smem, s>>>(c, sel, cplx, m);
+    } else {
+        auto k = encode_block_kernel<L, false>;
+        if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+        k<<<grid, L::NT, smem, s>>>(c, sel, cplx, m);
+    }
+    return FEDHE_LAUNCHED();
+}
+
+cudaError_t launch_encode(const CtxDev &c, const float *sel, size_t T, double2 *cplx, int64_t *m,
+                          cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    if (c.logN == 13) return launch_encode_t<Lay<12, 4>>(c, sel, T, cplx, m, s);
+    return launch_encode_t<Lay<13, 4>>(c, sel, T, cplx, m, s);
+}
+
+template <class L>
+static cudaError_t launch_decode_t(const CtxDev &c, const int64_t *d, size_t T, double2 *cplx, double *z,
+                                   cudaStream_t s) {
+    const uint32_t n = c.N >> 1;
+    const size_t smem = sizeof(cpx) << L::LOGB;
+    const unsigned grid = (unsigned)(T * (n >> L::LOGB));
+    cudaError_t e;
+    if ((n >> L::LOGB) > 1) {
+        auto k = decode_block_kernel<L, true>;
+        if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+        k<<<grid, L::NT, smem, s>>>(c, d, cplx, z);
+        if ((e = FEDHE_LAUNCHED())) return e;
+        const size_t total = T << L::LOGB;
+        decode_outer_kernel<L::LOGB><<<blocks_for(total, 256), 256, 0, s>>>(c, cplx, z, total);
+    } else {
+        auto k = decode_block_kernel<L, false>;
+        if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+        k<<<grid, L::NT, smem, s>>>(c, d, cplx, z);
+    }
+    return FEDHE_LAUNCHED();
+}
+
+cudaError_t launch_decode(const CtxDev &c, const int64_t *d, size_t T, double2 *cplx, double *z,
+                          cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    if (c.logN == 13) return launch_decode_t<Lay<12, 4>>(c, d, T, cplx, z, s);
+    return launch_decode_t<Lay<13, 4>>(c, d, T, cplx, z, s);
+}
+
+// ===========================================================================
+// encryption:  c0 = pk0 u + e0 + m,  c1 = pk1 u + e1   (mod every q_j)
+// ===========================================================================
+
+// Fused path for N <= 2^14 (one block holds a whole limb): one thread block
+// per ciphertext draws u, e0, e1 once into shared memory, then for every limb
+// transforms u, multiplies by both halves of the public key, transforms back
+// and adds the error (and message) terms.  Only the ciphertext itself is
+// written to global memory; the second product waits, in transform order, in
+// the c1 slot it will finally occupy.
+template <class L>
+__global__ void __launch_bounds__(L::NT, 1)
+encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const int64_t *m, uint32_t t0,
+                     uint64_t seed, uint32_t client, uint64_t *ct) {
+    extern __shared__ __align__(16) uint64_t sm[];
+    constexpr uint32_t B = 1u << L::LOGB;
+    constexpr int LAST = L::NPH - 1;
+    int8_t *su = reinterpret_cast<int8_t *>(sm + B);
+    int8_t *se0 = su + B, *se1 = se0 + B;
+    const uint32_t tid = threadIdx.x;
+    const size_t tl = blockIdx.x;            // ciphertext within this call
+    const uint32_t t = t0 + (uint32_t)tl;    // stream coordinate
+
+    for (uint32_t b = tid; b < B / 4; b += L::NT) {
+        u32x4 w = stream_block(seed, b, t, client, TAG_ENC_U);
+        char4 v = make_char4((signed char)ternary_from_word(w.x), (signed char)ternary_from_word(w.y),
+                             (signed char)ternary_from_word(w.z), (signed char)ternary_from_word(w.w));
+        reinterpret_cast<char4 *>(su)[b] = v;
+    }
+    for (uint32_t b = tid; b < B / 2; b += L::NT) {
+        u32x4 w0 = stream_block(seed, b, t, client, TAG_ENC_E0);
+        u32x4 w1 = stream_block(seed, b, t, client, TAG_ENC_E1);
+        char2 a = make_char2((signed char)gauss_from_u64((uint64_t)w0.x | ((uint64_t)w0.y << 32)),
+                             (signed char)gauss_from_u64((uint64_t)w0.z | ((uint64_t)w0.w << 32)));
+        char2 e = make_char2((signed char)gauss_from_u64((uint64_t)w1.x | ((uint64_t)w1.y << 32)),
+                             (signed char)gauss_from_u64((uint64_t)w1.z | ((uint64_t)w1.w << 32)));
+        reinterpret_cast<char2 *>(se0)[b] = a;
+        reinterpret_cast<char2 *>(se1)[b] = e;
+    }
+    __syncthreads();
+
+    const int64_t *mt = m + tl * B;
+    uint64_t x[L::E];
+    for (uint32_t j = 0; j < c.L; j++) {
+        const LimbDev &lb = c.limb[j];
+        const uint64_t q = lb.q, q2 = 2 * q;
+        uint64_t *c0 = ct + ((tl * 2 + 0) * c.L + j) * B;
+        uint64_t *c1 = ct + ((tl * 2 + 1) * c.L + j) * B;
+        const tw_t *p0 = k.pk0_hat + (size_t)j * B, *p1 = k.pk1_hat + (size_t)j * B;
+#pragma unroll
+        for (int r = 0; r < L::E; r++) x[r] = small_residue(su[L::template idx<0>(tid, r)], q);
+        NttArgs fa = {lb.fwd, q, q2, 0, 0};
+        block_ntt_forward<L>(x, sm, tid, fa);
+#pragma unroll
+        for (int r = 0; r < L::E; r += 2) {
+            const uint32_t p = L::template idx<LAST>(tid, r);
+            tw_t a0 = load_tw(p1 + p), a1 = load_tw(p1 + p + 1);
+            ulonglong2 v;
+            v.x = shoup_lazy(x[r], a0.w, a0.wp, q);
+            v.y = shoup_lazy(x[r + 1], a1.w, a1.wp, q);
+            *reinterpret_cast<ulonglong2 *>(c1 + p) = v;
+            tw_t b0 = load_tw(p0 + p), b1 = load_tw(p0 + p + 1);
+            x[r] = shoup_lazy(x[r], b0.w, b0.wp, q);
+            x[r + 1] = shoup_lazy(x[r + 1], b1.w, b1.wp, q);
+        }
+        NttArgs ia = {lb.inv, q, q2, 0, 0};
+        block_ntt_inverse<L, true>(x, sm, tid, ia, lb.ninv, lb.wn);
+#pragma unroll
+        for (int r = 0; r < L::E; r++) {
+            const uint32_t i = L::template idx<0>(tid, r);
+            const uint64_t add = signed_residue(mt[i] + (int64_t)se0[i], q, lb.mu);
+            c0[i] = addmod(csub(x[r], q), add, q);
+        }
+#pragma unroll
+        for (int r = 0; r < L::E; r += 2) {
+            ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(c1 + L::template idx<LAST>(tid, r));
+            x[r] = v.x;
+            x[r + 1] = v.y;
+        }
+        block_ntt_inverse<L, true>(x, sm, tid, ia, lb.ninv, lb.wn);
+#pragma unroll
+        for (int r = 0; r < L::E; r++) {
+            const uint32_t i = L::template idx<0>(tid, r);
+            c1[i] = addmod(csub(x[r], q), small_residue(se1[i], q), q);
+        }
+    }
+}
+
+// General path (any N): three elementwise kernels around the batched
+// transforms, with the ciphertext buffer itself as the only work space.
+
+// u as residues into the c1 slots of every limb
+__global__ void __launch_bounds__(256)
+enc_sample_u_kernel(const __grid_constant__ CtxDev c, uint32_t t0, uint64_t seed, uint32_t client,
+                    uint64_t *ct, size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t quads = c.N >> 2;
+    const uint32_t b = (uint32_t)(g % quads);
+    const size_t tl = g / quads;
+    u32x4 w = stream_block(seed, b, t0 + (uint32_t)tl, client, TAG_ENC_U);
+    const int u0 = ternary_from_word(w.x), u1 = ternary_from_word(w.y), u2 = ternary_from_word(w.z),
+              u3 = ternary_from_word(w.w);
+    for (uint32_t j = 0; j < c.L; j++) {
+        const uint64_t q = c.limb[j].q;
+        uint64_t *c1 = ct + ((tl * 2 + 1) * c.L + j) * c.N + 4 * (size_t)b;
+        reinterpret_cast<ulonglong2 *>(c1)[0] = make_ulonglong2(small_residue(u0, q), small_residue(u1, q));
+        reinterpret_cast<ulonglong2 *>(c1)[1] = make_ulonglong2(small_residue(u2, q), small_residue(u3, q));
+    }
+}
+
+// c0 = u^ pk0^, c1 = u^ pk1^ in the transform domain
+__global__ void __launch_bounds__(256)
+enc_pointwise_kernel(const __grid_constant__ CtxDev c, const KeysDev k, uint64_t *ct, size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t i = (uint32_t)(g % c.N);
+    const uint32_t j = (uint32_t)((g / c.N) % c.L);
+    const size_t tl = g / ((size_t)c.N * c.L);
+    const uint64_t q = c.limb[j].q;
+    uint64_t *c0 = ct + ((tl * 2 + 0) * c.L + j) * c.N + i;
+    uint64_t *c1 = ct + ((tl * 2 + 1) * c.L + j) * c.N + i;
+    const uint64_t u = *c1;
+    const tw_t a = load_tw(k.pk0_hat + (size_t)j * c.N + i), b = load_tw(k.pk1_hat + (size_t)j * c.N + i);
+    *c0 = shoup_lazy(u, a.w, a.wp, q);
+    *c1 = shoup_lazy(u, b.w, b.wp, q);
+}
+
+// c0 += e0 + m, c1 += e1: one thread per pair of coefficients, all limbs
+__global__ void __launch_bounds__(256)
+enc_add_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint32_t t0, uint64_t seed,
+               uint32_t client, uint64_t *ct, size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t pairs = c.N >> 1;
+    const uint32_t b = (uint32_t)(g % pairs);
+    const size_t tl = g / pairs;
+    const uint32_t t = t0 + (uint32_t)tl;
+    u32x4 w0 = stream_block(seed, b, t, client, TAG_ENC_E0);
+    u32x4 w1 = stream_block(seed, b, t, client, TAG_ENC_E1);
+    const int e0a = gauss_from_u64((uint64_t)w0.x | ((uint64_t)w0.y << 32));
+    const int e0b = gauss_from_u64((uint64_t)w0.z | ((uint64_t)w0.w << 32));
+    const int e1a = gauss_from_u64((uint64_t)w1.x | ((uint64_t)w1.y << 32));
+    const int e1b = gauss_from_u64((uint64_t)w1.z | ((uint64_t)w1.w << 32));
+    const longlong2 mm = *reinterpret_cast<const longlong2 *>(m + tl * c.N + 2 * (size_t)b);
+    for (uint32_t j = 0; j < c.L; j++) {
+        const LimbDev &lb = c.limb[j];
+        const uint64_t q = lb.q;
+        ulonglong2 *c0 = reinterpret_cast<ulonglong2 *>(ct + ((tl * 2 + 0) * c.L + j) * c.N + 2 * (size_t)b);
+        ulonglong2 *c1 = reinterpret_cast<ulonglong2 *>(ct + ((tl * 2 + 1) * c.L + j) * c.N + 2 * (size_t)b);
+        ulonglong2 v0 = *c0, v1 = *c1;
+        v0.x = addmod(v0.x, signed_residue(mm.x + e0a, q, lb.mu), q);
+        v0.y = addmod(v0.y, signed_residue(mm.y + e0b, q, lb.mu), q);
+        v1.x = addmod(v1.x, small_residue(e1a, q), q);
+        v1.y = addmod(v1.y, small_residue(e1b, q), q);
+        *c0 = v0;
+        *c1 = v1;
+    }
+}
+
+template <class L>
+static cudaError_t launch_encrypt_fused(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0,
+                                        size_t T, uint64_t seed, uint32_t client, uint64_t *ct,
+                                        cudaStream_t s) {
+    const size_t smem = (sizeof(uint64_t) << L::LOGB) + (3u << L::LOGB);
+    auto kern = encrypt_fused_kernel<L>;
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+    kern<<<(unsigned)T, L::NT, smem, s>>>(c, k, m, t0, seed, client, ct);
+    return FEDHE_LAUNCHED();
+}
+
+cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0, size_t T,
+                           uint64_t seed, uint32_t client, uint64_t *ct, cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    if (c.A == 0) {
+        if (c.LOGB == 13) return launch_encrypt_fused<Lay<13, 4>>(c, k, m, t0, T, seed, client, ct, s);
+        return launch_encrypt_fused<Lay<14, 4>>(c, k, m, t0, T, seed, client, ct, s);
+    }
+    cudaError_t e;
+    const size_t ctw = 2 * (size_t)c.L * c.N;
+    size_t total = T * (c.N >> 2);
+    enc_sample_u_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, t0, seed, client, ct, total);
+    if ((e = FEDHE_LAUNCHED())) return e;
+    if ((e = launch_ntt(c, true, ct + (size_t)c.L * c.N, T, ctw, 0, c.L, s))) return e;   // the c1 halves
+    total = T * (size_t)c.L * c.N;
+    enc_pointwise_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, k, ct, total);
+    if ((e = FEDHE_LAUNCHED())) return e;
+    if ((e = launch_ntt(c, false, ct, 2 * T, (size_t)c.L * c.N, 0, c.L, s))) return e;
+    total = T * (c.N >> 1);
+    enc_add_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, m, t0, seed, client, ct, total);
+    return FEDHE_LAUNCHED();
+}
+
+// ===========================================================================
+// server: weighted ciphertext sum over all clients fused with the rescale
+// ===========================================================================
+
+// One thread per pair of neighbouring coefficients of one (ciphertext,
+// component).  The last limb is accumulated first: its centred value is the
+// rounding term of every other limb.
+__global__ void __launch_bounds__(256)
+aggregate_rescale_kernel(const __grid_constant__ CtxDev c, const uint64_t *const *ptrs, const tw_t *wtab,
+                         int C, uint64_t *out, size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t pairs = c.N >> 1;
+    const uint32_t i = (uint32_t)(g % pairs) * 2;
+    const size_t tc = g / pairs;                 // t * 2 + component
+    const uint32_t L = c.L;
+    const uint64_t ql = c.limb[L - 1].q;
+    uint64_t rx, ry;
+    {
+        const uint64_t q2 = 2 * ql;
+        const size_t off = (tc * L + (L - 1)) * c.N + i;
+        uint64_t ax = 0, ay = 0;
+        for (int cl = 0; cl < C; cl++) {
+            const ulonglong2 v = __ldg(reinterpret_cast<const ulonglong2 *>(ptrs[cl] + off));
+            const tw_t w = wtab[cl * L + (L - 1)];
+            ax = csub(ax + shoup_lazy(v.x, w.w, w.wp, ql), q2);
+            ay = csub(ay + shoup_lazy(v.y, w.w, w.wp, ql), q2);
+        }
+        rx = csub(ax, ql);
+        ry = csub(ay, ql);
+    }
+    const bool negx = rx > ql / 2, negy = ry > ql / 2;
+    const uint64_t mx = negx ? ql - rx : rx, my = negy ? ql - ry : ry;   // |centred remainder|
+    for (uint32_t j = 0; j + 1 < L; j++) {
+        const LimbDev &lb = c.limb[j];
+        const uint64_t q = lb.q, q2 = 2 * q;
+        const size_t off = (tc * L + j) * c.N + i;
+        uint64_t ax = 0, ay = 0;
+        for (int cl = 0; cl < C; cl++) {
+            const ulonglong2 v = __ldg(reinterpret_cast<const ulonglong2 *>(ptrs[cl] + off));
+            const tw_t w = wtab[cl * L + j];
+            ax = csub(ax + shoup_lazy(v.x, w.w, w.wp, q), q2);
+            ay = csub(ay + shoup_lazy(v.y, w.w, w.wp, q), q2);
+        }
+        ax = csub(ax, q);
+        ay = csub(ay, q);
+        uint64_t sx = barrett64(mx, q, lb.mu), sy = barrett64(my, q, lb.mu);
+        // acc - r: subtracting a negative remainder adds its magnitude
+        const uint64_t dx = negx ? addmod(ax, sx, q) : submod(ax, sx, q);
+        const uint64_t dy = negy ? addmod(ay, sy, q) : submod(ay, sy, q);
+        ulonglong2 o;
+        o.x = shoup(dx, lb.qlinv.w, lb.qlinv.wp, q);
+        o.y = shoup(dy, lb.qlinv.w, lb.qlinv.wp, q);
+        *reinterpret_cast<ulonglong2 *>(out + (tc * (L - 1) + j) * c.N + i) = o;
+    }
+}
+
+cudaError_t launch_aggregate(const CtxDev &c, const uint64_t *const *ptrs, const tw_t *wtab, int C,
+                             size_t T, uint64_t *out, cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    const size_t total = T * 2 * (c.N >> 1);
+    aggregate_rescale_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, ptrs, wtab, C, out, total);
+    return FEDHE_LAUNCHED();
+}
+
+// plaintext remainder: out = sum_i alpha_i * (double) rest_i, client order,
+// separate multiply and add
+__global__ void __launch_bounds__(256)
+plain_aggregate_kernel(const float *const *ptrs, const double *alpha, int C, size_t len, double *out) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= len) return;
+    double a = 0.0;
+    for (int cl = 0; cl < C; cl++) a = __dadd_rn(a, __dmul_rn(alpha[cl], (double)__ldg(ptrs[cl] + g)));
+    out[g] = a;
+}
+
+cudaError_t launch_plain_aggregate(const float *const *ptrs, const double *alpha, int C, size_t len,
+                                   double *out, cudaStream_t s) {
+    if (len == 0) return cudaSuccess;
+    plain_aggregate_kernel<<<blocks_for(len, 256), 256, 0, s>>>(ptrs, alpha, C, len, out);
+    return FEDHE_LAUNCHED();
+}
+
+// ===========================================================================
+// decryption: d = c0 + c1 s on limb 0, centred
+// ===========================================================================
+
+__global__ void __launch_bounds__(256)
+dec_gather_kernel(const __grid_constant__ CtxDev c, const uint64_t *ct, uint32_t level, uint64_t *scratch,
+                  size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t i = (uint32_t)(g % c.N);
+    const size_t t = g / c.N;
+    scratch[g] = ct[((t * 2 + 1) * level + 0) * c.N + i];
+}
+
+__global__ void __launch_bounds__(256)
+dec_pointwise_kernel(const __grid_constant__ CtxDev c, const KeysDev k, uint64_t *scratch, size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t i = (uint32_t)(g % c.N);
+    const tw_t s = load_tw(k.s_hat + i);
+    scratch[g] = shoup_lazy(scratch[g], s.w, s.wp, c.limb[0].q);
+}
+
+__global__ void __launch_bounds__(256)
+dec_finish_kernel(const __grid_constant__ CtxDev c, const uint64_t *ct, uint32_t level, uint64_t *scratch,
+                  size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t i = (uint32_t)(g % c.N);
+    const size_t t = g / c.N;
+    const uint64_t q = c.limb[0].q;
+    const uint64_t r = addmod(scratch[g], ct[((t * 2 + 0) * level + 0) * c.N + i], q);
+    const int64_t d = r > q / 2 ? -(int64_t)(q - r) : (int64_t)r;
+    reinterpret_cast<int64_t *>(scratch)[g] = d;
+}
+
+cudaError_t launch_decrypt(const CtxDev &c, const KeysDev &k, const uint64_t *ct, uint32_t level,
+                           size_t T, uint64_t *scratch, cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    cudaError_t e;
+    const size_t total = T * c.N;
+    dec_gather_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, ct, level, scratch, total);
+    if ((e = FEDHE_LAUNCHED())) return e;
+    if ((e = launch_ntt(c, true, scratch, T, c.N, 0, 1, s))) return e;
+    dec_pointwise_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, k, scratch, total);
+    if ((e = FEDHE_LAUNCHED())) return e;
+    if ((e = launch_ntt(c, false, scratch, T, c.N, 0, 1, s))) return e;
+    dec_finish_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, ct, level, scratch, total);
+    return FEDHE_LAUNCHED();
+}
+
+// ===========================================================================
+// selective-encryption mask
+// ===========================================================================
+
+// ordering key of a sensitivity score: its bit pattern when it is a
+// non-negative number, 0 for negatives, -0 and NaN
+__device__ __forceinline__ uint32_t score_key(float s) {
+    const uint32_t b = __float_as_uint(s);
+    return ((b & 0x80000000u) || b > 0x7f800000u) ? 0u : b;
+}
+
+// histogram of the next `digit_bits` key bits among the keys whose leading
+// `prefix_bits` bits equal `prefix`
+__global__ void __launch_bounds__(512)
+key_histogram_kernel(const float *score, size_t P, uint32_t prefix, int prefix_bits, int digit_bits,
+                     uint32_t *hist) {
+    extern __shared__ uint32_t sh[];
+    const uint32_t bins = 1u << digit_bits;
+    for (uint32_t b = threadIdx.x; b < bins; b += blockDim.x) sh[b] = 0;
+    __syncthreads();
+    const int shift = 32 - prefix_bits - digit_bits;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < P; i += (size_t)gridDim.x * blockDim.x) {
+        const uint32_t key = score_key(__ldg(score + i));
+        if (prefix_bits == 0 || (key >> (32 - prefix_bits)) == prefix)
+            atomicAdd(&sh[(key >> shift) & (bins - 1u)], 1u);
+    }
+    __syncthreads();
+    for (uint32_t b = threadIdx.x; b < bins; b += blockDim.x)
+        if (sh[b]) atomicAdd(&hist[b], sh[b]);
+}
+
+cudaError_t launch_key_histogram(const float *score, size_t P, uint32_t prefix, int prefix_bits,
+                                 int digit_bits, uint32_t *hist, cudaStream_t s) {
+    unsigned grid = blocks_for(P, 512);
+    if (grid > 148 * 8) grid = 148 * 8;
+    if (grid == 0) grid = 1;
+    key_histogram_kernel<<<grid, 512, sizeof(uint32_t) << digit_bits, s>>>(score, P, prefix, prefix_bits,
+                                                                          digit_bits, hist);
+    return FEDHE_LAUNCHED();
+}
+
+// number of keys equal to tau in every block of MASK_BLOCK parameters
+__global__ void __launch_bounds__(MASK_BLOCK)
+mask_count_eq_kernel(const float *score, size_t P, uint32_t tau, uint32_t *blk_eq) {
+    const size_t i = (size_t)blockIdx.x * MASK_BLOCK + threadIdx.x;
+    const bool eq = i < P && score_key(__ldg(score + i)) == tau;
+    const int n = __syncthreads_count(eq);
+    if (threadIdx.x == 0) blk_eq[blockIdx.x] = (uint32_t)n;
+}
+
+cudaError_t launch_mask_count_eq(const float *score, size_t P, uint32_t tau, uint32_t *blk_eq,
+                                 cudaStream_t s) {
+    mask_count_eq_kernel<<<blocks_for(P, MASK_BLOCK), MASK_BLOCK, 0, s>>>(score, P, tau, blk_eq);
+    return FEDHE_LAUNCHED();
+}
+
+// exclusive prefix sum inside a block of 1024 threads; returns the block total
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t *warp_sums, uint32_t &total) {
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t o = __shfl_up_sync(0xffffffffu, inc, d);
+        if (lane >= (uint32_t)d) inc += o;
+    }
+    if (lane == 31) warp_sums[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t w = warp_sums[lane], winc = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t o = __shfl_up_sync(0xffffffffu, winc, d);
+            if (lane >= (uint32_t)d) winc += o;
+        }
+        warp_sums[lane] = winc - w;          // exclusive warp offsets
+        if (lane == 31) warp_sums[32] = winc;
+    }
+    __syncthreads();
+    const uint32_t res = warp_sums[warp] + inc - v;
+    total = warp_sums[32];
+    __syncthreads();
+    return res;
+}
+
+// single-block exclusive scan of an array (block totals: at most a few
+// hundred thousand entries)
+__global__ void __launch_bounds__(1024) scan_kernel(uint32_t *a, size_t count, uint32_t *total_out) {
+    __shared__ uint32_t warp_sums[33];
+    uint32_t carry = 0;
+    for (size_t base = 0; base < count; base += 1024) {
+        const size_t i = base + threadIdx.x;
+        const uint32_t v = i < count ? a[i] : 0u;
+        uint32_t tot;
+        const uint32_t ex = block_exclusive_scan(v, warp_sums, tot);
+        if (i < count) a[i] = carry + ex;
+        carry += tot;
+    }
+    if (threadIdx.x == 0) *total_out = carry;
+}
+
+cudaError_t launch_scan(uint32_t *a, size_t count, uint32_t *total, cudaStream_t s) {
+    scan_kernel<<<1, 1024, 0, s>>>(a, count, total);
+    return FEDHE_LAUNCHED();
+}
+
+// membership bits: key > tau, or key == tau and fewer than `need` equal keys
+// at lower indices, or inside a forced index range
+__global__ void __launch_bounds__(MASK_BLOCK)
+mask_select_kernel(const float *score, size_t P, uint32_t tau, uint32_t need, const uint64_t *ranges,
+                   uint32_t nranges, const uint32_t *blk_eq_prefix, uint32_t *bits, uint32_t *blk_sel) {
+    __shared__ uint32_t warp_sums[33];
+    const size_t i = (size_t)blockIdx.x * MASK_BLOCK + threadIdx.x;
+    const uint32_t key = i < P ? score_key(__ldg(score + i)) : 0u;
+    const bool eq = i < P && key == tau;
+    uint32_t tot;
+    const uint32_t eq_before = blk_eq_prefix[blockIdx.x] + block_exclusive_scan(eq ? 1u : 0u, warp_sums, tot);
+    bool sel = i < P && (key > tau || (eq && eq_before < need));
+    if (i < P && !sel) {
+        for (uint32_t r = 0; r < nranges; r++)
+            if (i >= ranges[2 * r] && i < ranges[2 * r + 1]) sel = true;
+    }
+    const uint32_t word = __ballot_sync(0xffffffffu, sel);
+    if ((threadIdx.x & 31) == 0 && i < P) bits[i >> 5] = word;
+    const int n = __syncthreads_count(sel);
+    if (threadIdx.x == 0) blk_sel[blockIdx.x] = (uint32_t)n;
+}
+
+cudaError_t launch_mask_select(const float *score, size_t P, uint32_t tau, uint32_t need,
+                               const uint64_t *ranges, uint32_t nranges, const uint32_t *blk_eq_prefix,
+                               uint32_t *bits, uint32_t *blk_sel, cudaStream_t s) {
+    mask_select_kernel<<<blocks_for(P, MASK_BLOCK), MASK_BLOCK, 0, s>>>(score, P, tau, need, ranges, nranges,
+                                                                        blk_eq_prefix, bits, blk_sel);
+    return FEDHE_LAUNCHED();
+}
+
+// per-word prefix counts and the ascending index list
+__global__ void __launch_bounds__(MASK_BLOCK)
+mask_write_kernel(size_t P, const uint32_t *bits, const uint32_t *blk_sel_prefix, uint32_t *wpre,
+                  uint32_t *idx) {
+    __shared__ uint32_t warp_sums[33];
+    const size_t i = (size_t)blockIdx.x * MASK_BLOCK + threadIdx.x;
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t word = i < P ? bits[i >> 5] : 0u;      // same for the whole warp
+    const bool sel = i < P && ((word >> lane) & 1u);
+    uint32_t tot;
+    const uint32_t before = blk_sel_prefix[blockIdx.x] + block_exclusive_scan(sel ? 1u : 0u, warp_sums, tot);
+    if (lane == 0 && i < P) wpre[i >> 5] = before;
+    if (sel) idx[before] = (uint32_t)i;
+}
+
+cudaError_t launch_mask_write(size_t P, const uint32_t *bits, const uint32_t *blk_sel_prefix,
+                              uint32_t *wpre, uint32_t *idx, cudaStream_t s) {
+    mask_write_kernel<<<blocks_for(P, MASK_BLOCK), MASK_BLOCK, 0, s>>>(P, bits, blk_sel_prefix, wpre, idx);
+    return FEDHE_LAUNCHED();
+}
+
+// ===========================================================================
+// packing and merging
+// ===========================================================================
+
+// one pass over the update: masked parameters go to their slot, the others to
+// the compacted remainder; the tail of the last ciphertext is zeroed
+__global__ void __launch_bounds__(256)
+pack_kernel(const uint32_t *bits, const uint32_t *wpre, const float *x, size_t P, size_t k, size_t padded,
+            float *sel, float *rest) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < P) {
+        const float v = __ldg(x + i);
+        if (bits == nullptr) {
+            sel[i] = v;
+        } else {
+            const uint32_t w = bits[i >> 5], lane = (uint32_t)(i & 31);
+            const size_t before = (size_t)wpre[i >> 5] + __popc(w & ((1u << lane) - 1u));
+            if ((w >> lane) & 1u) sel[before] = v;
+            else rest[i - before] = v;
+        }
+    }
+    if (i < padded - k) sel[k + i] = 0.0f;
+}
+
+cudaError_t launch_pack(const he_mask *mask, const float *x, size_t P, size_t k, size_t padded,
+                        float *sel, float *rest, cudaStream_t s) {
+    size_t threads = P > padded - k ? P : padded - k;
+    if (threads == 0) return cudaSuccess;
+    pack_kernel<<<blocks_for(threads, 256), 256, 0, s>>>(mask ? mask->bits : nullptr, mask ? mask->wpre : nullptr,
+                                                          x, P, k, padded, sel, rest);
+    return FEDHE_LAUNCHED();
+}
+
+__global__ void __launch_bounds__(256)
+unpack_kernel(const uint32_t *bits, const uint32_t *wpre, const double *z, const double *rest_avg, size_t P,
+              double *w_glob) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= P) return;
+    if (bits == nullptr) {
+        w_glob[i] = z[i];
+        return;
+    }
+    const uint32_t w = bits[i >> 5], lane = (uint32_t)(i & 31);
+    const size_t before = (size_t)wpre[i >> 5] + __popc(w & ((1u << lane) - 1u));
+    w_glob[i] = ((w >> lane) & 1u) ? z[before] : rest_avg[i - before];
+}
+
+cudaError_t launch_unpack(const he_mask *mask, const double *z, const double *rest_avg, size_t P,
+                          double *w_glob, cudaStream_t s) {
+    if (P == 0) return cudaSuccess;
+    unpack_kernel<<<blocks_for(P, 256), 256, 0, s>>>(mask ? mask->bits : nullptr, mask ? mask->wpre : nullptr, z,
+                                                     rest_avg, P, w_glob);
+    return FEDHE_LAUNCHED();
+}
+
+}  // namespace fedhe

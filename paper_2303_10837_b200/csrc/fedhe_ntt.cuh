@@ -1,0 +1,210 @@
+// Register-tiled negacyclic NTT of one block of B = 2^LOGB residues held by
+// one thread block: every thread keeps E = 2^LE residues in registers, does
+// LE butterfly stages on them, and the block re-distributes the residues
+// through shared memory between such phases.
+//
+// Index conventions (forward transform, natural order in, bit-reversed out):
+// stage s (0-based) of a length-N transform pairs the elements whose indices
+// differ in bit logN-1-s and uses the twiddle  tw[2^s + (index >> (logN - s))],
+// tw[i] = psi^brev(i).  The inverse transform runs the stages backwards with
+// the inverse table.  A block may be one of 2^A consecutive pieces of a
+// longer transform (N = 2^A B) whose first A stages were done elsewhere; then
+// the local stage s' is the global stage A + s' and the block index enters
+// the twiddle index.
+//
+// Phase p < NPH-1 keeps in registers the elements that differ in index bits
+// [lo, lo+LE), lo = LOGB - (p+1) LE; the last phase holds the remaining R low
+// bits plus the LE-R top bits (so that a thread owns runs of 2^R consecutive
+// elements and a warp covers whole 128-byte lines).
+#pragma once
+
+#include "fedhe_device.cuh"
+
+namespace fedhe {
+
+struct tw_t { uint64_t w, wp; };   // twiddle and its Shoup companion floor(w 2^64 / q)
+
+#if defined(__CUDACC__)
+// 16-byte read-only load of a table entry
+__device__ __forceinline__ tw_t load_tw(const tw_t *p) {
+    ulonglong2 v = __ldg(reinterpret_cast<const ulonglong2 *>(p));
+    tw_t t = {v.x, v.y};
+    return t;
+}
+#endif
+#if defined(__CUDA_ARCH__)
+#define FEDHE_LD_TW(p) load_tw(p)
+#else
+#define FEDHE_LD_TW(p) (*(p))
+#endif
+
+struct alignas(16) u64x2 { uint64_t x, y; };   // two neighbouring residues
+
+// shared-memory index swizzle: makes all phase layouts free of bank conflicts
+// for 8-byte accesses (xor the low nibble with the next one)
+HD uint32_t swz(uint32_t i) { return i ^ ((i >> 4) & 15u); }
+
+template <int LOGB_, int LE_>
+struct Lay {
+    static constexpr int LOGB = LOGB_, LE = LE_;
+    static constexpr int E = 1 << LE;
+    static constexpr int NT = 1 << (LOGB - LE);
+    static constexpr int NPH = (LOGB + LE - 1) / LE;
+    static constexpr int R = LOGB - (NPH - 1) * LE;   // stages of the last phase, 1..LE
+    static constexpr int HB = LE - R;                 // top bits held in the last phase
+
+    // element index held in register r of thread tid during phase P
+    template <int P>
+    static HD uint32_t idx(uint32_t tid, int r) {
+        if constexpr (P < NPH - 1) {
+            constexpr int lo = LOGB - (P + 1) * LE;
+            return ((tid >> lo) << (lo + LE)) | ((uint32_t)r << lo) | (tid & ((1u << lo) - 1u));
+        } else {
+            uint32_t rl = (uint32_t)r & ((1u << R) - 1u), rh = (uint32_t)r >> R;
+            return (rh << (LOGB - HB)) | (tid << R) | rl;
+        }
+    }
+
+    // index >> (LOGB - s) for the butterflies of local stage s = P LE + i whose
+    // lower register has the given group number g (the register bits above the
+    // pair bit)
+    template <int P, int I>
+    static HD uint32_t top(uint32_t tid, int r) {
+        constexpr int s = P * LE + I;
+        return idx<P>(tid, r) >> (LOGB - s);
+    }
+};
+
+// ---- phases ----------------------------------------------------------------
+
+struct NttArgs {
+    const tw_t *tw;      // table of this limb and direction, indexed by the global twiddle index
+    uint64_t q, q2;      // modulus and twice the modulus
+    uint32_t A;          // log2 of the number of blocks the whole transform is cut into
+    uint32_t blk;        // which block this is
+};
+
+template <class L, int P, int I>
+HD void fwd_stage(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
+    constexpr int s = P * L::LE + I;
+    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
+    constexpr int bit = nst - 1 - I;              // register bit of the pair
+    const uint32_t base = (1u << (a.A + s)) + (a.blk << s);
+#pragma unroll
+    for (int r = 0; r < L::E; r++) {
+        if (r & (1 << bit)) continue;
+        // all registers that agree above the pair bit share one twiddle; the
+        // compiler merges the equal loads of an unrolled group
+        const tw_t *pw = a.tw + base + L::template top<P, I>(tid, r);
+        tw_t w = FEDHE_LD_TW(pw);
+        ct_butterfly(x[r], x[r | (1 << bit)], w.w, w.wp, a.q, a.q2);
+    }
+}
+
+template <class L, int P, int I>
+HD void inv_stage(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
+    constexpr int s = P * L::LE + I;
+    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
+    constexpr int bit = nst - 1 - I;
+    const uint32_t base = (1u << (a.A + s)) + (a.blk << s);
+#pragma unroll
+    for (int r = 0; r < L::E; r++) {
+        if (r & (1 << bit)) continue;
+        const tw_t *pw = a.tw + base + L::template top<P, I>(tid, r);
+        tw_t w = FEDHE_LD_TW(pw);
+        gs_butterfly(x[r], x[r | (1 << bit)], w.w, w.wp, a.q, a.q2);
+    }
+}
+
+// last inverse stage of a whole transform (global stage 0) with the factor
+// 1/N folded in: x <- (x + y)/N, y <- (x - y) w /N.  ninv = 1/N, wn = w/N.
+template <class L>
+HD void inv_stage0_scaled(uint64_t (&x)[L::E], tw_t ninv, tw_t wn, uint64_t q, uint64_t q2) {
+    constexpr int bit = L::LE - 1;
+#pragma unroll
+    for (int r = 0; r < L::E; r++) {
+        if (r & (1 << bit)) continue;
+        uint64_t u = x[r], v = x[r | (1 << bit)];
+        x[r] = shoup_lazy(u + v, ninv.w, ninv.wp, q);
+        x[r | (1 << bit)] = shoup_lazy(u - v + q2, wn.w, wn.wp, q);
+    }
+}
+
+template <class L, int P, int I = 0>
+HD void fwd_phase(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
+    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
+    if constexpr (I < nst) {
+        fwd_stage<L, P, I>(x, tid, a);
+        fwd_phase<L, P, I + 1>(x, tid, a);
+    }
+}
+
+// inverse phase: stages nst-1 down to STOP (STOP = 1 leaves stage 0 of the
+// phase to the caller)
+template <class L, int P, int STOP, int I>
+HD void inv_phase_from(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
+    if constexpr (I >= STOP) {
+        inv_stage<L, P, I>(x, tid, a);
+        inv_phase_from<L, P, STOP, I - 1>(x, tid, a);
+    }
+}
+
+template <class L, int P, int STOP = 0>
+HD void inv_phase(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
+    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
+    inv_phase_from<L, P, STOP, nst - 1>(x, tid, a);
+}
+
+// ---- exchange through shared memory ---------------------------------------
+
+template <class L, int P>
+HD void xchg_write(const uint64_t (&x)[L::E], uint64_t *sm, uint32_t tid) {
+#pragma unroll
+    for (int r = 0; r < L::E; r++) sm[swz(L::template idx<P>(tid, r))] = x[r];
+}
+
+template <class L, int P>
+HD void xchg_read(uint64_t (&x)[L::E], const uint64_t *sm, uint32_t tid) {
+#pragma unroll
+    for (int r = 0; r < L::E; r++) x[r] = sm[swz(L::template idx<P>(tid, r))];
+}
+
+#if defined(__CUDACC__)
+// Whole-block transforms.  sm: B words of shared memory.  The residues enter
+// in the layout of phase 0 (forward) or of the last phase (inverse) and leave
+// in the other one.
+
+template <class L, int P = 0>
+__device__ __forceinline__ void block_ntt_forward(uint64_t (&x)[L::E], uint64_t *sm, uint32_t tid,
+                                                  const NttArgs &a) {
+    fwd_phase<L, P>(x, tid, a);
+    if constexpr (P + 1 < L::NPH) {
+        __syncthreads();                       // earlier readers of sm are done
+        xchg_write<L, P>(x, sm, tid);
+        __syncthreads();
+        xchg_read<L, P + 1>(x, sm, tid);
+        block_ntt_forward<L, P + 1>(x, sm, tid, a);
+    }
+}
+
+// SCALED: fold 1/N into global stage 0 (only valid when A == 0)
+template <class L, bool SCALED, int P = L::NPH - 1>
+__device__ __forceinline__ void block_ntt_inverse(uint64_t (&x)[L::E], uint64_t *sm, uint32_t tid,
+                                                  const NttArgs &a, tw_t ninv, tw_t wn) {
+    if constexpr (P == 0 && SCALED) {
+        inv_phase<L, 0, 1>(x, tid, a);
+        inv_stage0_scaled<L>(x, ninv, wn, a.q, a.q2);
+    } else {
+        inv_phase<L, P>(x, tid, a);
+    }
+    if constexpr (P > 0) {
+        __syncthreads();
+        xchg_write<L, P>(x, sm, tid);
+        __syncthreads();
+        xchg_read<L, P - 1>(x, sm, tid);
+        block_ntt_inverse<L, SCALED, P - 1>(x, sm, tid, a, ninv, wn);
+    }
+}
+#endif
+
+}  // namespace fedhe

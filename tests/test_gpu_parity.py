@@ -1,0 +1,331 @@
+"""GPU parity: every step of the CUDA path, called through the C ABI, against the
+CPU oracle on the same seeded inputs.  Integer outputs (transforms, keys,
+encoded polynomials, ciphertexts, aggregates, masks, packing) must be
+bit-exact; decoded fp64 values within 1e-9 of the oracle's decode and within
+1e-6 of plaintext FedAvg."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synthetic_inputs as si
+from gpu_common import dev_f32, to_dev_u64, to_host_u64
+
+pytestmark = pytest.mark.gpu
+
+DECODE_TOL = 1e-9     # GPU decode vs oracle decode (same integers in, fp64 transform order differs)
+FEDAVG_TOL = 1e-6     # homomorphic result vs plaintext weighted average
+
+
+@pytest.fixture(scope="module")
+def he():
+    import paper_2303_10837_b200 as he
+    assert torch.cuda.is_available()
+    return he
+
+
+def contexts(he, N, primes, ld):
+    return he.he_ctx_create(N, list(primes), ld), oracle.Context(N, primes, ld)
+
+
+# --------------------------------------------------------------------------- transforms
+
+@pytest.mark.parametrize("N,L,B", [(8192, 2, 5), (16384, 4, 3), (32768, 2, 3), (65536, 4, 2), (16384, 12, 1)])
+def test_ntt_forward_inverse_bit_exact(he, N, L, B):
+    primes = si.PRIMES_SWEEP[:L]
+    g, o = contexts(he, N, primes, 40)
+    a = si.random_residues(N + L, (B, L, N), primes)
+    a[0, 0, :] = 0
+    a[0, 0, 1] = 1                                   # impulse: output = odd powers of psi
+    a[B - 1, L - 1, :] = primes[L - 1] - 1           # all-maximal residues
+    d = to_dev_u64(a)
+    he.he_ntt_forward(g, d)
+    f = to_host_u64(d)
+    for b in range(B):
+        for j in range(L):
+            assert np.array_equal(f[b, j], o.ntt_forward(j, a[b, j])), (b, j)
+    he.he_ntt_inverse(g, d)
+    assert np.array_equal(to_host_u64(d), a)
+    # inverse alone on arbitrary data
+    d2 = to_dev_u64(a)
+    he.he_ntt_inverse(g, d2)
+    i2 = to_host_u64(d2)
+    for j in range(L):
+        assert np.array_equal(i2[0, j], o.ntt_inverse(j, a[0, j]))
+
+
+@pytest.mark.parametrize("N,primes", [(8192, si.PRIMES_N8192), (16384, si.PRIMES_N16384),
+                                      (32768, si.PRIMES_N32768), (65536, si.PRIMES_SWEEP[:3])])
+def test_keygen_bit_exact(he, N, primes):
+    g, o = contexts(he, N, primes, 40)
+    keys = he.he_keygen(g, 0xABCDEF0123)
+    pk, s = he.he_keys_export(g, keys)
+    s_o, pk_o = o.keygen(0xABCDEF0123)
+    assert np.array_equal(s.cpu().numpy(), s_o)
+    assert np.array_equal(to_host_u64(pk), pk_o)
+
+
+# --------------------------------------------------------------------------- encode / encrypt
+
+def workload_cases():
+    return [
+        si.scaled(si.TINY, 2 * 4096 + 101, name="tiny-ragged"),               # N=8192, 3 cts, ragged tail
+        si.scaled(si.RESNET18, 3 * 8192 - 7, clients=3, name="r18-ragged"),    # N=16384, L=4
+        si.scaled(si.bert(1.0), 16384 + 33, clients=2, name="bert-ragged"),    # N=32768, L=6, Delta=2^45
+    ]
+
+
+@pytest.mark.parametrize("w", workload_cases(), ids=lambda w: w.name)
+def test_encode_bit_exact(he, w):
+    g, o = contexts(he, w.N, w.primes, w.log2_delta)
+    x = si.client_update(w, 0)
+    sel_o, _ = o.pack(None, w.P, x)
+    sel, _ = he.he_pack(g, None, dev_f32(x))
+    assert np.array_equal(sel.cpu().numpy(), sel_o)
+    m = he.he_encode(g, sel).cpu().numpy()
+    for t in range(w.T):
+        m_o, ov = o.encode(sel_o[t * w.n:(t + 1) * w.n])
+        assert not ov
+        assert np.array_equal(m[t], m_o), t
+    assert he.he_ctx_status(g) == he.HE_OK
+
+
+def test_encode_special_values_and_overflow_flag(he):
+    w = si.TINY
+    g, o = contexts(he, w.N, w.primes, w.log2_delta)
+    z = np.zeros(2 * w.n, np.float32)
+    z[: w.n] = 0.25                              # constant slots -> constant polynomial
+    z[w.n + 5] = -1.5
+    m = he.he_encode(g, dev_f32(z)).cpu().numpy()
+    assert m[0, 0] == 2**38 and not m[0, 1:].any()
+    assert np.array_equal(m[1], o.encode(z[w.n:])[0])
+    assert he.he_ctx_status(g) == he.HE_OK
+    z[3] = 3e38                                   # |coefficient| >= 2^62: flagged, not trapped
+    m = he.he_encode(g, dev_f32(z)).cpu().numpy()
+    assert he.he_ctx_status(g) == he.HE_ERR_OVERFLOW
+    assert he.he_ctx_status(g) == he.HE_OK        # sticky word is cleared by the read
+    m_o, ov = o.encode(z[: w.n])
+    assert ov and np.array_equal(m[0], m_o)
+
+
+@pytest.mark.parametrize("w", workload_cases(), ids=lambda w: w.name)
+def test_encrypt_aggregate_decrypt_bit_exact(he, w):
+    g, o = contexts(he, w.N, w.primes, w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    s_o, pk_o = o.keygen(w.key_seed)
+    xs = si.client_updates(w)
+    alpha = si.client_weights(w)
+    cts, cts_o = [], []
+    for i, x in enumerate(xs):
+        sel, _ = he.he_pack(g, None, dev_f32(x))
+        ct = he.he_encrypt(g, keys, sel, w.enc_seed, i)
+        ct_o, bad = o.encrypt(pk_o, o.pack(None, w.P, x)[0], w.enc_seed, i)
+        assert bad == 0
+        assert np.array_equal(to_host_u64(ct), ct_o), "ciphertext of client %d" % i
+        cts.append(ct)
+        cts_o.append(ct_o)
+    # chunked encryption uses the absolute ciphertext index
+    sel, _ = he.he_pack(g, None, dev_f32(xs[0]))
+    part = torch.empty((w.T - 1, 2, w.L, w.N), dtype=torch.int64, device="cuda")
+    he.he_encrypt_range(g, keys, sel[w.n:], 1, w.T - 1, w.enc_seed, 0, part)
+    assert torch.equal(part, cts[0][1:])
+    # server
+    agg = he.he_weighted_aggregate(g, cts, alpha)
+    agg_o = o.rescale(o.weighted_sum(cts_o, o.weights(alpha)))
+    assert np.array_equal(to_host_u64(agg), agg_o)
+    # client
+    z = he.he_decrypt(g, keys, agg).cpu().numpy()
+    z_o = o.decode(o.decrypt(s_o, agg_o, w.L - 1)).reshape(-1)
+    assert np.abs(z - z_o).max() <= DECODE_TOL
+    want = sum(a * x.astype(np.float64) for a, x in zip(alpha, xs))
+    assert np.abs(z[: w.P] - want).max() <= FEDAVG_TOL
+    out = he.he_unpack(g, None, torch.from_numpy(z).cuda(), None, w.P).cpu().numpy()
+    assert np.array_equal(out, z[: w.P])
+    # a fresh ciphertext opens to its own message
+    z0 = he.he_decrypt_level(g, keys, cts[0], w.L).cpu().numpy()
+    assert np.abs(z0[: w.P] - xs[0].astype(np.float64)).max() <= FEDAVG_TOL
+    assert he.he_ctx_status(g) == he.HE_OK
+
+
+def test_dropout_subset_of_clients(he):
+    """Aggregating any subset with renormalised weights needs no new keys."""
+    w = si.scaled(si.RESNET18, 8192 + 11, clients=4, name="r18-dropout")
+    g, o = contexts(he, w.N, w.primes, w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    xs, alpha = si.client_updates(w), si.client_weights(w)
+    cts = [he.he_encrypt(g, keys, he.he_pack(g, None, dev_f32(x))[0], w.enc_seed, i) for i, x in enumerate(xs)]
+    keep = [0, 2, 3]
+    sub = alpha[keep] / alpha[keep].sum()
+    z = he.he_decrypt(g, keys, he.he_weighted_aggregate(g, [cts[i] for i in keep], sub)).cpu().numpy()
+    want = sum(a * xs[i].astype(np.float64) for a, i in zip(sub, keep))
+    assert np.abs(z[: w.P] - want).max() <= FEDAVG_TOL
+    # one client with weight 1 is a plain re-scaling
+    z1 = he.he_decrypt(g, keys, he.he_weighted_aggregate(g, [cts[1]], [1.0])).cpu().numpy()
+    assert np.abs(z1[: w.P] - xs[1].astype(np.float64)).max() <= FEDAVG_TOL
+
+
+# --------------------------------------------------------------------------- mask and packing
+
+def test_select_mask_bit_exact(he):
+    g, _ = contexts(he, 8192, si.PRIMES_N8192, 40)
+    w = si.scaled(si.RESNET50_TOP10, 100_003)
+    score = si.sensitivity_scores(w)
+    d = dev_f32(score)
+    for k in (0, 1, 1000, w.k, 99_999, w.P):
+        mask = he.he_select_mask(g, d, k)
+        assert mask.k == k
+        got = he.he_mask_indices(mask).cpu().numpy().view(np.uint32)
+        assert np.array_equal(got, oracle.select_mask(score, k)), k
+
+
+def test_select_mask_ties_and_special_values(he):
+    g, _ = contexts(he, 8192, si.PRIMES_N8192, 40)
+    rng = np.random.default_rng(5)
+    score = rng.integers(0, 4, size=5000).astype(np.float32)        # heavy ties
+    score[17] = np.nan
+    score[18] = -1.0
+    score[19] = -0.0
+    score[20] = np.inf
+    d = dev_f32(score)
+    for k in (1, 2, 100, 1234, 2500, 4999, 5000):
+        got = he.he_mask_indices(he.he_select_mask(g, d, k)).cpu().numpy().view(np.uint32)
+        assert np.array_equal(got, oracle.select_mask(score, k)), k
+    same = np.full(4097, 0.125, np.float32)
+    got = he.he_mask_indices(he.he_select_mask(g, dev_f32(same), 33)).cpu().numpy()
+    assert list(got) == list(range(33))
+
+
+def test_mask_with_forced_ranges(he):
+    """Top-k plus whole index ranges (first and last layers)."""
+    g, _ = contexts(he, 8192, si.PRIMES_N8192, 40)
+    w = si.scaled(si.RESNET50_TOP10, 50_000)
+    score = si.sensitivity_scores(w)
+    ranges = [(0, 700), (49_000, 50_000)]
+    mask = he.he_select_mask_ranges(g, dev_f32(score), w.k, ranges)
+    got = he.he_mask_indices(mask).cpu().numpy().view(np.uint32)
+    top = oracle.select_mask(score, w.k)
+    want = np.union1d(top, np.concatenate([np.arange(a, b) for a, b in ranges])).astype(np.uint32)
+    assert np.array_equal(got, want) and mask.k == want.size
+
+
+def test_pack_unpack_plain_aggregate_bit_exact(he):
+    w = si.scaled(si.RESNET50_TOP10, 70_001, clients=4)
+    g, o = contexts(he, w.N, w.primes, w.log2_delta)
+    score = si.sensitivity_scores(w)
+    mask = he.he_select_mask(g, dev_f32(score), w.k)
+    idx = oracle.select_mask(score, w.k)
+    xs, alpha = si.client_updates(w), si.client_weights(w)
+    rests = []
+    for x in xs:
+        sel, rest = he.he_pack(g, mask, dev_f32(x))
+        sel_o, rest_o = o.pack(idx, w.k, x)
+        assert np.array_equal(sel.cpu().numpy(), sel_o)
+        assert np.array_equal(rest.cpu().numpy(), rest_o)
+        rests.append(rest)
+    avg = he.he_plain_aggregate(g, rests, alpha)
+    avg_o = oracle.plain_aggregate([r.cpu().numpy() for r in rests], alpha)
+    assert np.array_equal(avg.cpu().numpy(), avg_o)
+    z = np.random.default_rng(1).standard_normal(he.he_num_ct(g, w.k) * w.n)
+    out = he.he_unpack(g, mask, torch.from_numpy(z).cuda(), avg, w.P).cpu().numpy()
+    assert np.array_equal(out, oracle.unpack(idx, w.k, z, avg_o, w.P))
+
+
+# --------------------------------------------------------------------------- whole rounds
+
+def run_round_gpu(he, g, keys, mask, xs, alpha, w):
+    cts, rests = [], []
+    for i, x in enumerate(xs):
+        sel, rest = he.he_pack(g, mask, dev_f32(x))
+        cts.append(he.he_encrypt(g, keys, sel, w.enc_seed, i))
+        rests.append(rest)
+    z = he.he_decrypt(g, keys, he.he_weighted_aggregate(g, cts, alpha))
+    avg = he.he_plain_aggregate(g, rests, alpha) if mask is not None else None
+    return he.he_unpack(g, mask, z, avg, w.P).cpu().numpy()
+
+
+def test_tiny_config_whole_round(he):
+    """Config 1 in full: N=8192, 60/40/60-bit primes, 3 clients, 100,000 parameters."""
+    w = si.TINY
+    g, o = contexts(he, w.N, w.primes, w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    xs, alpha = si.client_updates(w), si.client_weights(w)
+    out = run_round_gpu(he, g, keys, None, xs, alpha, w)
+    out_o = o.round(xs, alpha, None, w.P, w.key_seed, w.enc_seed)
+    assert np.abs(out - out_o).max() <= DECODE_TOL
+    want = sum(a * x.astype(np.float64) for a, x in zip(alpha, xs))
+    assert np.abs(out - want).max() <= FEDAVG_TOL
+    # the same through the host-buffer entry point
+    host = torch.empty(w.P, dtype=torch.float64)
+    he.he_round_host(g, keys, None, [torch.from_numpy(x) for x in xs], alpha, w.enc_seed, host)
+    assert np.array_equal(host.numpy(), out)
+
+
+def test_selective_round_with_mask(he):
+    """Config 3 shape at reduced size: top-10 % encrypted, the rest averaged in plaintext."""
+    w = si.scaled(si.RESNET50_TOP10, 300_000, clients=4)
+    g, o = contexts(he, w.N, w.primes, w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    xs, alpha = si.client_updates(w), si.client_weights(w)
+    score = si.sensitivity_scores(w)
+    mask = he.he_select_mask(g, dev_f32(score), w.k)
+    idx = oracle.select_mask(score, w.k)
+    assert np.array_equal(he.he_mask_indices(mask).cpu().numpy().view(np.uint32), idx)
+    out = run_round_gpu(he, g, keys, mask, xs, alpha, w)
+    out_o = o.round(xs, alpha, idx, w.k, w.key_seed, w.enc_seed)
+    comp = np.setdiff1d(np.arange(w.P), idx)
+    assert np.array_equal(out[comp], out_o[comp])                   # plaintext part: bit-exact
+    assert np.abs(out[idx] - out_o[idx]).max() <= DECODE_TOL
+    want = sum(a * x.astype(np.float64) for a, x in zip(alpha, xs))
+    assert np.abs(out - want).max() <= FEDAVG_TOL
+    host = torch.empty(w.P, dtype=torch.float64)
+    he.he_round_host(g, keys, mask, [torch.from_numpy(x) for x in xs], alpha, w.enc_seed, host)
+    assert np.array_equal(host.numpy(), out)
+
+
+def test_empty_and_degenerate_inputs(he):
+    w = si.TINY
+    g, o = contexts(he, w.N, w.primes, w.log2_delta)
+    keys = he.he_keygen(g, 1)
+    # P = 1: one slot used, one whole ciphertext
+    x = np.array([0.5], np.float32)
+    sel, _ = he.he_pack(g, None, dev_f32(x))
+    assert sel.numel() == w.n and float(sel[0]) == 0.5 and not sel[1:].any()
+    ct = he.he_encrypt(g, keys, sel, 3, 0)
+    assert ct.shape == (1, 2, w.L, w.N)
+    z = he.he_decrypt(g, keys, he.he_weighted_aggregate(g, [ct], [1.0])).cpu().numpy()
+    assert abs(z[0] - 0.5) <= FEDAVG_TOL and np.abs(z[1:]).max() <= FEDAVG_TOL
+    # k = 0: nothing is encrypted, everything is averaged in plaintext
+    score = dev_f32(np.arange(1000, dtype=np.float32))
+    mask = he.he_select_mask(g, score, 0)
+    xs = [np.full(1000, 1.0, np.float32), np.full(1000, 3.0, np.float32)]
+    sel, rest = he.he_pack(g, mask, dev_f32(xs[0]))
+    assert sel.numel() == 0 and rest.numel() == 1000
+    out = run_round_gpu(he, g, keys, mask, xs, [0.25, 0.75], si.scaled(w, 1000, clients=2))
+    assert np.array_equal(out, np.full(1000, 2.5))
+    # invalid arguments come back as error codes
+    with pytest.raises(he.HeError) as ei:
+        he.he_select_mask(g, score, 1001)
+    assert ei.value.code == he.HE_ERR_INVALID_ARG
+    with pytest.raises(he.HeError) as ei:
+        he.he_weighted_aggregate(g, [ct], [1.5])
+    assert ei.value.code == he.HE_ERR_INVALID_ARG
+    with pytest.raises(he.HeError) as ei:
+        he.he_decrypt_level(g, keys, ct, w.L + 1)
+    assert ei.value.code == he.HE_ERR_LEVEL
+    other = he.he_ctx_create(w.N, list(w.primes), w.log2_delta)
+    with pytest.raises(he.HeError) as ei:
+        he.he_encrypt(other, keys, sel if sel.numel() else dev_f32(np.zeros(w.n, np.float32)), 1, 0)
+    assert ei.value.code == he.HE_ERR_INVALID_ARG
+
+
+def test_runs_are_deterministic(he):
+    """Bit-identical outputs on repeated runs (a race would show up here)."""
+    w = si.scaled(si.RESNET18, 5 * 8192, clients=2)
+    g, _ = contexts(he, w.N, w.primes, w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    sel, _ = he.he_pack(g, None, dev_f32(si.client_update(w, 0)))
+    a = he.he_encrypt(g, keys, sel, 5, 1)
+    b = he.he_encrypt(g, keys, sel, 5, 1)
+    assert torch.equal(a, b)
+    c = he.he_encrypt(g, keys, sel, 6, 1)
+    assert not torch.equal(a, c)
