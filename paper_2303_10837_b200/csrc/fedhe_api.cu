@@ -111,6 +111,8 @@ int he_ctx_create(const he_params *p, he_ctx **out) {
         host_slot_twiddles(d.N, roots, ftw);
         rc = upload(ctx, reinterpret_cast<const double2 *>(ftw.data()), ftw.size() / 2, &d.ftw);
         if (rc != HE_OK) break;
+        rc = upload(ctx, d.limb, HE_MAX_LIMBS, &d.limb_dev);
+        if (rc != HE_OK) break;
         void *st = nullptr;
         if (cudaMalloc(&st, sizeof(int)) != cudaSuccess) { rc = HE_ERR_ALLOC; break; }
         ctx->owned.push_back(st);

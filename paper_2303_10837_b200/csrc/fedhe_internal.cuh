@@ -27,6 +27,7 @@ struct CtxDev {
     uint32_t LOGB, A;    // a length-N transform = 2^A blocks of 2^LOGB
     int32_t log2_delta;
     LimbDev limb[HE_MAX_LIMBS];
+    const LimbDev *limb_dev;   // the same table in device memory, for kernels that loop over limbs
     const double2 *ftw;  // slot-transform twiddles, entry [len/2 + j]
     int *status;         // sticky anomaly word
 };

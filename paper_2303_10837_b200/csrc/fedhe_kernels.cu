@@ -5,6 +5,7 @@
 #include "fedhe_launch.h"
 
 #include <atomic>
+#include <cstdlib>
 
 namespace fedhe {
 
@@ -38,6 +39,38 @@ __device__ __forceinline__ int gauss_from_u64(uint64_t r) {
 #pragma unroll
     for (int x = 0; x < 38; x++) v += (r >= c_gauss_cdf[x]) ? 1 : 0;
     return v;
+}
+
+// The same map through shared-memory tables: the top byte of r selects the
+// thresholds that are certainly below r (`base`) and the few that share its
+// byte (`nb`, compared one by one).
+struct GaussTables {
+    uint64_t cdf[38];
+    uint8_t base[256];
+    uint8_t nb[256];
+};
+
+__device__ __forceinline__ void gauss_tables_init(GaussTables &g, uint32_t tid) {
+    if (tid < 38) g.cdf[tid] = c_gauss_cdf[tid];
+    if (tid < 256) {
+        const uint64_t lo = (uint64_t)tid << 56, hi = lo | 0x00ffffffffffffffull;
+        int base = 0, nb = 0;
+        for (int x = 0; x < 38; x++) {
+            const uint64_t t = c_gauss_cdf[x];
+            if (t <= lo) base++;
+            else if (t <= hi) nb++;
+        }
+        g.base[tid] = (uint8_t)base;
+        g.nb[tid] = (uint8_t)nb;
+    }
+}
+
+__device__ __forceinline__ int gauss_from_u64(const GaussTables &g, uint64_t r) {
+    const uint32_t b = (uint32_t)(r >> 56);
+    const int base = g.base[b], nb = g.nb[b];
+    int v = base;
+    for (int i = 0; i < nb; i++) v += (r >= g.cdf[base + i]) ? 1 : 0;
+    return v - 19;
 }
 
 __device__ __forceinline__ uint64_t addmod(uint64_t a, uint64_t b, uint64_t q) { return csub(a + b, q); }
@@ -195,7 +228,8 @@ cudaError_t launch_ntt(const CtxDev &c, bool forward, uint64_t *data, size_t npo
         if ((e = FEDHE_LAUNCHED())) return e;
     }
     if (c.LOGB == 13) e = launch_ntt_blocks<Lay<13, 4>>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
-    else e = launch_ntt_blocks<Lay<14, 4>>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
+    else if (getenv("FEDHE_LE4")) e = launch_ntt_blocks<Lay<14, 4>>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
+    else e = launch_ntt_blocks<Lay<14, 5>>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
     if (e) return e;
     if (!forward && c.A > 0) {
         ntt_outer_kernel<false><<<blocks_for(outer_threads, 256), 256, 0, s>>>(c, data, poly_stride, limb0,
@@ -569,80 +603,84 @@ cudaError_t launch_decode(const CtxDev &c, const int64_t *d, size_t T, double2 *
 // and adds the error (and message) terms.  Only the ciphertext itself is
 // written to global memory; the second product waits, in transform order, in
 // the c1 slot it will finally occupy.
-template <class L>
-__global__ void __launch_bounds__(L::NT, 1)
+template <class L, int V>
+__global__ void __launch_bounds__(L::NT / V, 1)
 encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const int64_t *m, uint32_t t0,
                      uint64_t seed, uint32_t client, uint64_t *ct) {
     extern __shared__ __align__(16) uint64_t sm[];
-    constexpr uint32_t B = 1u << L::LOGB;
-    constexpr int LAST = L::NPH - 1;
+    constexpr uint32_t B = 1u << L::LOGB, RT = L::NT / V;
     int8_t *su = reinterpret_cast<int8_t *>(sm + B);
     int8_t *se0 = su + B, *se1 = se0 + B;
     const uint32_t tid = threadIdx.x;
     const size_t tl = blockIdx.x;            // ciphertext within this call
     const uint32_t t = t0 + (uint32_t)tl;    // stream coordinate
+    __shared__ GaussTables gt;
+    gauss_tables_init(gt, tid);
+    __syncthreads();
 
-    for (uint32_t b = tid; b < B / 4; b += L::NT) {
+    for (uint32_t b = tid; b < B / 4; b += RT) {
         u32x4 w = stream_block(seed, b, t, client, TAG_ENC_U);
         char4 v = make_char4((signed char)ternary_from_word(w.x), (signed char)ternary_from_word(w.y),
                              (signed char)ternary_from_word(w.z), (signed char)ternary_from_word(w.w));
         reinterpret_cast<char4 *>(su)[b] = v;
     }
-    for (uint32_t b = tid; b < B / 2; b += L::NT) {
+    for (uint32_t b = tid; b < B / 2; b += RT) {
         u32x4 w0 = stream_block(seed, b, t, client, TAG_ENC_E0);
         u32x4 w1 = stream_block(seed, b, t, client, TAG_ENC_E1);
-        char2 a = make_char2((signed char)gauss_from_u64((uint64_t)w0.x | ((uint64_t)w0.y << 32)),
-                             (signed char)gauss_from_u64((uint64_t)w0.z | ((uint64_t)w0.w << 32)));
-        char2 e = make_char2((signed char)gauss_from_u64((uint64_t)w1.x | ((uint64_t)w1.y << 32)),
-                             (signed char)gauss_from_u64((uint64_t)w1.z | ((uint64_t)w1.w << 32)));
+        char2 a = make_char2((signed char)gauss_from_u64(gt, (uint64_t)w0.x | ((uint64_t)w0.y << 32)),
+                             (signed char)gauss_from_u64(gt, (uint64_t)w0.z | ((uint64_t)w0.w << 32)));
+        char2 e = make_char2((signed char)gauss_from_u64(gt, (uint64_t)w1.x | ((uint64_t)w1.y << 32)),
+                             (signed char)gauss_from_u64(gt, (uint64_t)w1.z | ((uint64_t)w1.w << 32)));
         reinterpret_cast<char2 *>(se0)[b] = a;
         reinterpret_cast<char2 *>(se1)[b] = e;
     }
     __syncthreads();
 
     const int64_t *mt = m + tl * B;
-    uint64_t x[L::E];
+    const size_t cstride = (size_t)c.L * B;          // from c0 to c1 of the same limb
     for (uint32_t j = 0; j < c.L; j++) {
         const LimbDev &lb = c.limb[j];
         const uint64_t q = lb.q, q2 = 2 * q;
-        uint64_t *c0 = ct + ((tl * 2 + 0) * c.L + j) * B;
-        uint64_t *c1 = ct + ((tl * 2 + 1) * c.L + j) * B;
-        const tw_t *p0 = k.pk0_hat + (size_t)j * B, *p1 = k.pk1_hat + (size_t)j * B;
-#pragma unroll
-        for (int r = 0; r < L::E; r++) x[r] = small_residue(su[L::template idx<0>(tid, r)], q);
-        NttArgs fa = {lb.fwd, q, q2, 0, 0};
-        block_ntt_forward<L>(x, sm, tid, fa);
-#pragma unroll
-        for (int r = 0; r < L::E; r += 2) {
-            const uint32_t p = L::template idx<LAST>(tid, r);
-            tw_t a0 = load_tw(p1 + p), a1 = load_tw(p1 + p + 1);
-            ulonglong2 v;
-            v.x = shoup_lazy(x[r], a0.w, a0.wp, q);
-            v.y = shoup_lazy(x[r + 1], a1.w, a1.wp, q);
-            *reinterpret_cast<ulonglong2 *>(c1 + p) = v;
-            tw_t b0 = load_tw(p0 + p), b1 = load_tw(p0 + p + 1);
-            x[r] = shoup_lazy(x[r], b0.w, b0.wp, q);
-            x[r + 1] = shoup_lazy(x[r + 1], b1.w, b1.wp, q);
+        uint64_t *cbase = ct + ((tl * 2 + 0) * c.L + j) * B;
+        {
+            const tw_t *p0 = k.pk0_hat + (size_t)j * B, *p1 = k.pk1_hat + (size_t)j * B;
+            uint64_t *c1 = cbase + cstride;
+            const NttArgs fa = {lb.fwd, q, q2, 0, 0};
+            smem_ntt_forward<L, V>(
+                sm, tid, fa, [&](uint32_t i) { return small_residue(su[i], q); },
+                [&](uint32_t p, uint64_t a, uint64_t b) {
+                    // u^ pk1^ is parked in its final c1 slot until the second pass
+                    // below; u^ pk0^ stays in shared memory for the first pass
+                    const tw_t a0 = load_tw(p1 + p), a1 = load_tw(p1 + p + 1);
+                    u64x2 v;
+                    v.x = shoup_lazy(a, a0.w, a0.wp, q);
+                    v.y = shoup_lazy(b, a1.w, a1.wp, q);
+                    *reinterpret_cast<u64x2 *>(c1 + p) = v;
+                    const tw_t b0 = load_tw(p0 + p), b1 = load_tw(p0 + p + 1);
+                    sm[swz(p)] = shoup_lazy(a, b0.w, b0.wp, q);
+                    sm[swz(p + 1)] = shoup_lazy(b, b1.w, b1.wp, q);
+                });
         }
-        NttArgs ia = {lb.inv, q, q2, 0, 0};
-        block_ntt_inverse<L, true>(x, sm, tid, ia, lb.ninv, lb.wn);
-#pragma unroll
-        for (int r = 0; r < L::E; r++) {
-            const uint32_t i = L::template idx<0>(tid, r);
-            const uint64_t add = signed_residue(mt[i] + (int64_t)se0[i], q, lb.mu);
-            c0[i] = addmod(csub(x[r], q), add, q);
-        }
-#pragma unroll
-        for (int r = 0; r < L::E; r += 2) {
-            ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(c1 + L::template idx<LAST>(tid, r));
-            x[r] = v.x;
-            x[r + 1] = v.y;
-        }
-        block_ntt_inverse<L, true>(x, sm, tid, ia, lb.ninv, lb.wn);
-#pragma unroll
-        for (int r = 0; r < L::E; r++) {
-            const uint32_t i = L::template idx<0>(tid, r);
-            c1[i] = addmod(csub(x[r], q), small_residue(se1[i], q), q);
+        // two passes over one copy of the inverse-transform code: h = 0 gives
+        // c0 = pk0 u + e0 + m from shared memory, h = 1 reloads the parked
+        // product and gives c1 = pk1 u + e1
+#pragma unroll 1
+        for (int h = 0; h < 2; h++) {
+            uint64_t *cc = cbase + h * cstride;
+            const int8_t *se = se0 + h * B;
+            const NttArgs ia = {lb.inv, q, q2, 0, 0};
+            smem_ntt_inverse<L, V, true>(
+                sm, tid, ia, lb.ninv, lb.wn,
+                [&](uint32_t p) {
+                    if (h == 0) return u64x2{sm[swz(p)], sm[swz(p + 1)]};
+                    return *reinterpret_cast<const u64x2 *>(cc + p);
+                },
+                [&](uint32_t i, uint64_t v) {
+                    int64_t add = (int64_t)se[i];
+                    if (h == 0) add += mt[i];
+                    cc[i] = addmod(csub(v, q), signed_residue(add, q, lb.mu), q);
+                });
+            __syncthreads();   // phase-0 readers are done before the next transform writes
         }
     }
 }
@@ -719,15 +757,15 @@ enc_add_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint32_t t0, 
     }
 }
 
-template <class L>
+template <class L, int V>
 static cudaError_t launch_encrypt_fused(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0,
                                         size_t T, uint64_t seed, uint32_t client, uint64_t *ct,
                                         cudaStream_t s) {
     const size_t smem = (sizeof(uint64_t) << L::LOGB) + (3u << L::LOGB);
-    auto kern = encrypt_fused_kernel<L>;
+    auto kern = encrypt_fused_kernel<L, V>;
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-    kern<<<(unsigned)T, L::NT, smem, s>>>(c, k, m, t0, seed, client, ct);
+    kern<<<(unsigned)T, L::NT / V, smem, s>>>(c, k, m, t0, seed, client, ct);
     return FEDHE_LAUNCHED();
 }
 
@@ -735,8 +773,9 @@ cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const int64_t *m, 
                            uint64_t seed, uint32_t client, uint64_t *ct, cudaStream_t s) {
     if (T == 0) return cudaSuccess;
     if (c.A == 0) {
-        if (c.LOGB == 13) return launch_encrypt_fused<Lay<13, 4>>(c, k, m, t0, T, seed, client, ct, s);
-        return launch_encrypt_fused<Lay<14, 4>>(c, k, m, t0, T, seed, client, ct, s);
+        if (c.LOGB == 13) return launch_encrypt_fused<Lay<13, 3>, 2>(c, k, m, t0, T, seed, client, ct, s);
+        if (getenv("FEDHE_LE4")) return launch_encrypt_fused<Lay<14, 4>, 1>(c, k, m, t0, T, seed, client, ct, s);
+        return launch_encrypt_fused<Lay<14, 3>, 2>(c, k, m, t0, T, seed, client, ct, s);
     }
     cudaError_t e;
     const size_t ctw = 2 * (size_t)c.L * c.N;

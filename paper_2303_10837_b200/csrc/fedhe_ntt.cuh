@@ -207,4 +207,87 @@ __device__ __forceinline__ void block_ntt_inverse(uint64_t (&x)[L::E], uint64_t 
 }
 #endif
 
+#if defined(__CUDACC__)
+// ---------------------------------------------------------------------------
+// In-place variant: the block's residues stay in shared memory (swizzled) and
+// every thread plays V "virtual threads" per phase, each of which loads its
+// E residues, does the phase's butterflies in registers and stores them back
+// to the same places, so that only E residues are live per thread at a time
+// and no separate exchange buffer is needed.  The first phase takes its input
+// from `src`, the last hands its output to `dst`:
+//   forward:  src(i) -> residue i;            dst(i, a, b): residues i, i+1
+//   inverse:  src(i) -> residues i, i+1;      dst(i, a): residue i
+// (pairs always start at an even index and are neighbours in memory).
+// ---------------------------------------------------------------------------
+
+template <class L, int V, class Src, class Dst, int P = 0>
+__device__ __forceinline__ void smem_ntt_forward(uint64_t *sm, uint32_t tid, const NttArgs &a, const Src &src,
+                                                 const Dst &dst) {
+    constexpr int RT = L::NT / V, LAST = L::NPH - 1;
+#pragma unroll 1
+    for (int v = 0; v < V; v++) {
+        const uint32_t vt = tid + v * RT;
+        uint64_t x[L::E];
+#pragma unroll
+        for (int r = 0; r < L::E; r++) {
+            const uint32_t i = L::template idx<P>(vt, r);
+            if constexpr (P == 0) x[r] = src(i);
+            else x[r] = sm[swz(i)];
+        }
+        fwd_phase<L, P>(x, vt, a);
+        if constexpr (P == LAST) {
+#pragma unroll
+            for (int r = 0; r < L::E; r += 2) dst(L::template idx<P>(vt, r), x[r], x[r + 1]);
+        } else {
+#pragma unroll
+            for (int r = 0; r < L::E; r++) sm[swz(L::template idx<P>(vt, r))] = x[r];
+        }
+    }
+    if constexpr (P < LAST) {
+        __syncthreads();
+        smem_ntt_forward<L, V, Src, Dst, P + 1>(sm, tid, a, src, dst);
+    }
+}
+
+template <class L, int V, bool SCALED, class Src, class Dst, int P = L::NPH - 1>
+__device__ __forceinline__ void smem_ntt_inverse(uint64_t *sm, uint32_t tid, const NttArgs &a, tw_t ninv,
+                                                 tw_t wn, const Src &src, const Dst &dst) {
+    constexpr int RT = L::NT / V, LAST = L::NPH - 1;
+#pragma unroll 1
+    for (int v = 0; v < V; v++) {
+        const uint32_t vt = tid + v * RT;
+        uint64_t x[L::E];
+        if constexpr (P == LAST) {
+#pragma unroll
+            for (int r = 0; r < L::E; r += 2) {
+                const u64x2 t = src(L::template idx<P>(vt, r));
+                x[r] = t.x;
+                x[r + 1] = t.y;
+            }
+        } else {
+#pragma unroll
+            for (int r = 0; r < L::E; r++) x[r] = sm[swz(L::template idx<P>(vt, r))];
+        }
+        if constexpr (P == 0 && SCALED) {
+            inv_phase<L, 0, 1>(x, vt, a);
+            inv_stage0_scaled<L>(x, ninv, wn, a.q, a.q2);
+        } else {
+            inv_phase<L, P>(x, vt, a);
+        }
+        if constexpr (P == 0) {
+#pragma unroll
+            for (int r = 0; r < L::E; r++) dst(L::template idx<0>(vt, r), x[r]);
+        } else {
+#pragma unroll
+            for (int r = 0; r < L::E; r++) sm[swz(L::template idx<P>(vt, r))] = x[r];
+        }
+    }
+    if constexpr (P > 0) {
+        __syncthreads();
+        smem_ntt_inverse<L, V, SCALED, Src, Dst, P - 1>(sm, tid, a, ninv, wn, src, dst);
+    }
+}
+#endif
+
+
 }  // namespace fedhe
