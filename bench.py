@@ -37,16 +37,16 @@ import synthetic_inputs as si
 METRIC = "HE-agg params/s (encrypt+weighted sum+decrypt); NTT % of HBM roofline"
 UNIT = "params/s"
 
-# 32-bit integer operations that one 64-bit Harvey/Shoup butterfly needs at
-# least on a machine with 32-bit multipliers: 4 products for the high half of
-# x*w', 3 + 3 for the low halves of x*w and hi*q, and 12 add/sub/compare ops
-# (two-word subtract, conditional 2q correction, two-word add and sub).
-INT_OPS_PER_BUTTERFLY = 22
-# Integer issue ceiling: 4 schedulers x 32 lanes per SM and clock; on B200 a
-# 32-bit multiply-add issues at half that rate (measured, see profiles/), so
-# the ceiling for this mix (10 of 22 ops are multiplies) is 128 / (12/22 + 2*10/22).
-INT_LANES_PER_SM_CLK = 128.0
-IMAD_RATE = 0.5
+# Integer roofline of the transforms.  On B200 every integer multiply goes
+# through one pipe that retires 64 32-bit multiply-adds per SM and clock
+# (measured: 63.8), and a 32x32->64 multiply-add costs 2.5 of those slots
+# (measured: 25.5 per SM and clock); see profiles/int_pipe_microbenchmark.md.
+# A 64-bit Shoup butterfly needs at least the high half of x*w' (4 wide
+# products) and the low halves of x*w and hi*q (1 wide + 2 narrow each):
+# 6 wide + 4 narrow = 19 multiply slots.  Additions go to another pipe.
+IMAD_PER_SM_CLK = 64.0
+WIDE_COST = 2.5
+MUL_SLOTS_PER_BUTTERFLY = 6 * WIDE_COST + 4
 
 
 def fallback_peaks():
@@ -162,7 +162,7 @@ def run_reference(args, w):
     rank, world, _ = dist_env()
     if rank != 0:
         return
-    n_ct = 24
+    n_ct = 256
     for _ in range(args.warmup):
         oracle_sample(w, 2)
     units, secs, cores = 0, 0.0, 1
@@ -326,30 +326,33 @@ def run_ours(args, w):
             dist.destroy_process_group()
         return
 
-    # roofline of the dominant kernel (integer-bound): butterflies per launch
+    # roofline of the dominant kernel (bound by the integer-multiply pipe)
     logN = w.N.bit_length() - 1
-    butterflies = 3 * w.L * (w.N // 2) * logN * T
-    achieved = butterflies * INT_OPS_PER_BUTTERFLY / (kern_ms * 1e-3) / 1e12
+    butterflies = 3 * w.L * (w.N // 2) * logN * T           # per launch: 3 limb transforms per limb
+    achieved = butterflies * MUL_SLOTS_PER_BUTTERFLY / (kern_ms * 1e-3) / 1e12
     n_sm = torch.cuda.get_device_properties(local).multi_processor_count
-    mul_share = 10.0 / INT_OPS_PER_BUTTERFLY
-    mix_rate = INT_LANES_PER_SM_CLK / ((1 - mul_share) + mul_share / IMAD_RATE)
-    peak = n_sm * mix_rate * peaks["sm_max_mhz"] * 1e6 / 1e12
+    peak = n_sm * IMAD_PER_SM_CLK * peaks["sm_max_mhz"] * 1e6 / 1e12
     alg_bytes = (16.0 + 32.0 * w.L) * n * T          # read m, write the ciphertext
     roofline = {
         "kernel": "encrypt_fused_kernel" if w.N <= 16384 else "ntt_block_kernel (inside he_encrypt)",
-        "bound": "alu", "achieved": achieved, "peak": peak, "unit": "Tiop/s (32-bit integer ops)",
+        "bound": "alu", "achieved": achieved, "peak": peak,
+        "unit": "T multiply-slots/s (32-bit integer multiply pipe)",
         "frac": achieved / peak, "traffic": None,
-        "ms_per_launch": kern_ms, "launches_per_step": w.clients,
+        "ms_per_launch": kern_ms, "launches_per_step": w.clients, "butterflies_per_launch": butterflies,
         "hbm_gbs_of_kernel": alg_bytes / (kern_ms * 1e-3) / 1e9,
         "hbm_frac_of_kernel": alg_bytes / (kern_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
         "ntt_standalone": {"gbs": ntt_gbs, "hbm_frac": ntt_gbs / peaks["hbm_gbs"], "ms": ntt_ms,
-                           "batch_polys": B, "bytes_per_launch": pass_bytes},
-        "peak_source": peaks["source"] + " hbm_gbs; integer ceiling derived from SM count, lanes and max clock",
+                           "batch_polys": B, "bytes_per_launch": pass_bytes,
+                           "mul_pipe_frac": (B * w.L * (w.N // 2) * logN * MUL_SLOTS_PER_BUTTERFLY
+                                             / (ntt_ms * 1e-3) / 1e12) / peak},
+        "peak_source": "integer-multiply pipe: SM count x 64 per clock (microbenchmark) x max SM clock; "
+                       + peaks["source"] + " hbm_gbs for the HBM fractions",
     }
 
-    cpu_p, cpu_dt, cores = oracle_sample(w, 24)
+    cpu_ct = min(w.T, 768)
+    cpu_p, cpu_dt, cores = oracle_sample(w, cpu_ct)
     cpu = {"value": cpu_p / cpu_dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-           "sample": "first 24 of %d ciphertext indices (%d params), all %d clients, %.1f s" % (w.T, cpu_p, w.clients, cpu_dt)}
+           "sample": "first %d of %d ciphertext indices (%d params), all %d clients, %.1f s" % (cpu_ct, w.T, cpu_p, w.clients, cpu_dt)}
 
     line = {
         "metric": METRIC, "value": units / job_secs, "unit": UNIT, "n_gpus": world, "steps": args.steps,

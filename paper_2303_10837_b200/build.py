@@ -66,6 +66,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
         tmp = OUT + ".tmp.%d" % os.getpid()
         subprocess.run([_nvcc(), "-shared", "-o", tmp] + objs + ["-lquadmath"], check=True)
         os.replace(tmp, OUT)
+    tool_src = os.path.join(CSRC, "int_pipe_bench.cu")
+    tool = os.path.join(HERE, "int_pipe_bench")
+    if force or _stale(tool, [tool_src]):
+        subprocess.run([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-o", tool, tool_src],
+                       check=True, capture_output=True)
     return OUT
 
 

@@ -1,0 +1,40 @@
+// Integer issue-rate microbenchmark for the roofline of the transforms: eight
+// independent chains per thread of one instruction kind each, 2 x 1024
+// threads per SM, reported per SM and clock at the nominal maximum clock.
+// Standalone program (built by build.py as `int_pipe_bench`); not part of the library.
+#include <cstdio>
+#include <cstdint>
+#include <cuda_runtime.h>
+#define CHK(x) do{cudaError_t e=(x); if(e){printf("err %s line %d\n", cudaGetErrorString(e), __LINE__); return 1;}}while(0)
+template<int MODE> __global__ void k(uint64_t* out, int iters, uint32_t seed) {
+  uint32_t a[8]; uint64_t b[8];
+  for (int i=0;i<8;i++){ a[i]=threadIdx.x*7+i+seed; b[i]=((uint64_t)a[i]<<32)|(a[i]*2654435761u); }
+  uint32_t m = seed|1; uint64_t m64 = ((uint64_t)seed<<33)|0x9E3779B97F4A7C15ull;
+  for (int it=0; it<iters; it++) {
+    #pragma unroll
+    for (int i=0;i<8;i++) {
+      if (MODE==0) a[i] = a[i]*m + 12345u;                 // IMAD lo 32
+      if (MODE==1) b[i] = (uint64_t)(uint32_t)b[i]*m + b[i];   // IMAD.WIDE
+      if (MODE==2) b[i] = __umul64hi(b[i], m64) + 1;       // 64-bit mulhi
+      if (MODE==3) b[i] = b[i]*m64 + 1;                    // 64-bit mullo
+      if (MODE==4) a[i] = (a[i] + m) ^ (a[i]>>3);          // IADD/LOP/SHF
+      if (MODE==5) { uint64_t hi=__umul64hi(b[i], m64); b[i] = b[i]*0x1234567ull - hi*0xffffffffffc0001ull; } // shoup
+    }
+  }
+  uint64_t s=0; for (int i=0;i<8;i++) s += a[i] + b[i];
+  out[blockIdx.x*blockDim.x+threadIdx.x]=s;
+}
+template<int MODE> int run(const char* name, double ops_per_iter) {
+  int sms; cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, 0);
+  int blocks = sms*2, threads=1024, iters=20000;
+  uint64_t* out; CHK(cudaMalloc(&out, (size_t)blocks*threads*8));
+  cudaEvent_t e0,e1; cudaEventCreate(&e0); cudaEventCreate(&e1);
+  k<MODE><<<blocks,threads>>>(out, 1000, 3); CHK(cudaDeviceSynchronize());
+  float best=1e30f;
+  for (int r=0;r<3;r++){ cudaEventRecord(e0); k<MODE><<<blocks,threads>>>(out, iters, 3+r); cudaEventRecord(e1); CHK(cudaEventSynchronize(e1)); float ms; cudaEventElapsedTime(&ms,e0,e1); if(ms<best)best=ms; }
+  double total = (double)blocks*threads*iters*8*ops_per_iter;
+  printf("%-22s %8.3f ms  %10.3f Gop/s  per SM per clk @1.965GHz: %6.1f\n", name, best, total/best/1e6, total/(best*1e-3)/sms/1.965e9);
+  cudaFree(out); return 0;
+}
+int main(){ int sms; cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, 0); int clk; cudaDeviceGetAttribute(&clk, cudaDevAttrClockRate, 0); printf("SMs %d clock attr %d kHz\n", sms, clk);
+  run<0>("imad.lo32",1); run<1>("imad.wide",1); run<2>("umul64hi",1); run<3>("mul.lo.u64",1); run<4>("iadd+lop+shf (3 ops)",3); run<5>("shoup lazy modmul",1); return 0; }

@@ -329,3 +329,36 @@ def test_runs_are_deterministic(he):
     assert torch.equal(a, b)
     c = he.he_encrypt(g, keys, sel, 6, 1)
     assert not torch.equal(a, c)
+
+
+def test_sensitivity_map_round(he):
+    """Stage 2 of Algorithm 1: the clients' sensitivity maps go through the same fully encrypted
+    path, the aggregated map is decrypted and the mask is selected from it."""
+    w = si.scaled(si.RESNET18, 60_000, clients=3, name="sens-map")
+    g, o = contexts(he, w.N, w.primes, w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    s_o, pk_o = o.keygen(w.key_seed)
+    rng = np.random.default_rng(17)
+    # non-negative, heavy-tailed maps (means of absolute values in the paper)
+    maps = [np.abs(rng.standard_cauchy(w.P)).clip(0, 50).astype(np.float32) * np.float32(0.01) for _ in range(w.clients)]
+    alpha = si.client_weights(w)
+    cts, cts_o = [], []
+    for i, s_map in enumerate(maps):
+        sel, _ = he.he_pack(g, None, dev_f32(s_map))
+        cts.append(he.he_encrypt(g, keys, sel, 99, i))
+        cts_o.append(o.encrypt(pk_o, o.pack(None, w.P, s_map)[0], 99, i)[0])
+        assert np.array_equal(to_host_u64(cts[-1]), cts_o[-1])
+    agg = he.he_weighted_aggregate(g, cts, alpha)
+    z = he.he_decrypt(g, keys, agg)[: w.P]
+    z_o = o.decode(o.decrypt(s_o, o.rescale(o.weighted_sum(cts_o, o.weights(alpha))), w.L - 1)).reshape(-1)[: w.P]
+    assert np.abs(z.cpu().numpy() - z_o).max() <= DECODE_TOL
+    want = sum(a * m.astype(np.float64) for a, m in zip(alpha, maps))
+    assert np.abs(z.cpu().numpy() - want).max() <= FEDAVG_TOL
+    score = z.float().contiguous()
+    k = int(round(0.3 * w.P))
+    mask = he.he_select_mask(g, score, k)
+    got = he.he_mask_indices(mask).cpu().numpy().view(np.uint32)
+    assert np.array_equal(got, oracle.select_mask(score.cpu().numpy(), k))
+    # the mask agrees with the one a plaintext aggregation would give, except at the noise-level boundary
+    plain = oracle.select_mask(want.astype(np.float32), k)
+    assert np.intersect1d(got, plain).size >= 0.999 * k
