@@ -170,6 +170,27 @@ int he_decrypt(he_ctx *ctx, const he_keys *keys, const uint64_t *agg_dev, size_t
 int he_decrypt_level(he_ctx *ctx, const he_keys *keys, const uint64_t *ct_dev, uint32_t level, size_t T,
                      double *z_dev, void *stream);
 
+/* (No counterpart in the paper.)  he_decrypt for callers that must not
+ * allocate: a process that has given all free device memory to its own pool,
+ * or a latency-critical loop that cannot take the device-wide synchronisation
+ * of cudaMalloc/cudaFree.  Same arguments and result as he_decrypt, but the
+ * work buffer is a fixed 16 MiB array inside the library image (present on
+ * every GPU that loads the library until the process exits), so the call
+ * issues no cudaMalloc, cudaFree or allocating library routine.
+ *   Limits: N <= 16384 and T * N <= HE_NOALLOC_MAX_WORDS (T <= 128 at
+ *   N = 16384, T <= 256 at N = 8192); anything larger returns HE_ERR_SIZE.
+ *   The context's GPU must be the current device (HE_ERR_INVALID_ARG).
+ *   The first call on a device looks up the array's device address
+ *   (cudaGetSymbolAddress), which is also the latest moment at which the CUDA
+ *   runtime loads the library's device image, array included, on that GPU;
+ *   make that first call before any stream capture.
+ *   Every call on a device shares the one array, which keeps the previous
+ *   call's contents (none of it needs to start at zero); calls that overlap
+ *   on the GPU, e.g. on two streams, race on it. */
+#define HE_NOALLOC_MAX_WORDS (1u << 21)
+int he_decrypt_noalloc(he_ctx *ctx, const he_keys *keys, const uint64_t *agg_dev, size_t T, double *z_dev,
+                       void *stream);
+
 /* Client merge  Dec(sk, M (.) [W_glob]) + (1-M) (.) [W_glob]:
  * w_glob[idx[r]] = z[r], complement positions take rest_avg in order.
  *   z: dev double[>= k]; rest_avg: dev double[P-k] (NULL if mask NULL);

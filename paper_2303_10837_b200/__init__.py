@@ -73,6 +73,7 @@ _SIGS = {
     "he_plain_aggregate": (C.c_int, [_vp, _vp, _vp, C.c_int, _sz, _vp, _vp]),
     "he_decrypt": (C.c_int, [_vp, _vp, _vp, _sz, _vp, _vp]),
     "he_decrypt_level": (C.c_int, [_vp, _vp, _vp, _u32, _sz, _vp, _vp]),
+    "he_decrypt_noalloc": (C.c_int, [_vp, _vp, _vp, _sz, _vp, _vp]),
     "he_unpack": (C.c_int, [_vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "he_ntt_forward": (C.c_int, [_vp, _vp, _sz, _vp]),
     "he_ntt_inverse": (C.c_int, [_vp, _vp, _sz, _vp]),
@@ -299,6 +300,19 @@ def he_decrypt_level(ctx: Ctx, keys: Keys, ct: torch.Tensor, level: int) -> torc
     _check(_lib.he_decrypt_level(ctx.handle, keys.handle, _dev(ct, torch.int64), level, T, z.data_ptr(),
                                  _stream()), "he_decrypt_level")
     return z
+
+
+HE_NOALLOC_MAX_WORDS = 1 << 21
+
+
+def he_decrypt_noalloc(ctx: Ctx, keys: Keys, agg: torch.Tensor, out: torch.Tensor) -> torch.Tensor:
+    """he_decrypt without any allocation inside the library: the work buffer is a fixed array
+    in the library image, so T * N must not exceed HE_NOALLOC_MAX_WORDS and N must be <= 16384.
+    `out` (float64 [T*n]) is supplied by the caller for the same reason."""
+    T = agg.shape[0]
+    _check(_lib.he_decrypt_noalloc(ctx.handle, keys.handle, _dev(agg, torch.int64) or None, T,
+                                   _dev(out, torch.float64) or None, _stream()), "he_decrypt_noalloc")
+    return out
 
 
 def he_unpack(ctx: Ctx, mask: Optional[Mask], z: torch.Tensor, rest_avg: Optional[torch.Tensor], P: int,

@@ -16,7 +16,7 @@ CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libfedhe.so")
 BUILD = os.path.join(HERE, "_build")
 
-CUDA_SOURCES = ["fedhe_kernels.cu", "fedhe_api.cu"]
+CUDA_SOURCES = ["fedhe_kernels.cu", "fedhe_api.cu", "fedhe_noalloc.cu"]
 HOST_SOURCES = ["fedhe_host.cpp"]
 HEADERS = ["fedhe_device.cuh", "fedhe_ntt.cuh", "fedhe_internal.cuh", "fedhe_launch.h", "fedhe_host.h",
            os.path.join("..", "..", "include", "fedhe.h")]
