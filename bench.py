@@ -378,9 +378,11 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=["resnet18", "tiny", "resnet50-top10"], default="resnet18")
+    ap.add_argument("--workload", choices=["resnet18", "tiny", "resnet50-top10", "bert-1", "bert-10"],
+                    default="resnet18")
     args = ap.parse_args()
-    w = {"resnet18": si.RESNET18, "tiny": si.TINY, "resnet50-top10": si.RESNET50_TOP10}[args.workload]
+    w = {"resnet18": si.RESNET18, "tiny": si.TINY, "resnet50-top10": si.RESNET50_TOP10,
+         "bert-1": si.bert(0.01), "bert-10": si.bert(0.10)}[args.workload]
     if args.impl == "reference":
         run_reference(args, w)
     else:
