@@ -5,7 +5,6 @@
 #include "fedhe_launch.h"
 
 #include <atomic>
-#include <cstdlib>
 
 namespace fedhe {
 
@@ -99,10 +98,13 @@ __device__ uint64_t shoup_companion(uint64_t w, uint64_t q) {   // floor(w 2^64 
 // batched negacyclic NTT
 // ===========================================================================
 
-template <class L, bool FWD, bool SCALED>
-__global__ void __launch_bounds__(L::NT, 1)
+// One block of B = 2^LOGB residues per thread block (a whole limb for
+// N <= 2^14), transformed in place in shared memory; every thread plays V
+// virtual threads per phase with E residues in registers at a time.
+template <class L, int V, bool FWD, bool SCALED>
+__global__ void __launch_bounds__(L::NT / V, 1)
 ntt_block_kernel(const __grid_constant__ CtxDev c, uint64_t *data, size_t poly_stride, uint32_t limb0,
-                 uint32_t nlimbs) {
+                         uint32_t nlimbs) {
     extern __shared__ __align__(16) uint64_t sm[];
     const uint32_t tid = threadIdx.x;
     uint32_t b = blockIdx.x;
@@ -113,32 +115,21 @@ ntt_block_kernel(const __grid_constant__ CtxDev c, uint64_t *data, size_t poly_s
     const LimbDev &lb = c.limb[limb0 + limb];
     const uint64_t q = lb.q, q2 = 2 * q;
     uint64_t *p = data + poly * poly_stride + (size_t)limb * c.N + ((size_t)blk << L::LOGB);
-    uint64_t x[L::E];
-    constexpr int LAST = L::NPH - 1;
     if constexpr (FWD) {
-#pragma unroll
-        for (int r = 0; r < L::E; r++) x[r] = p[L::template idx<0>(tid, r)];
-        NttArgs a = {lb.fwd, q, q2, c.A, blk};
-        block_ntt_forward<L>(x, sm, tid, a);
-#pragma unroll
-        for (int r = 0; r < L::E; r += 2) {          // registers r, r+1 are neighbours in memory
-            ulonglong2 v;
-            v.x = csub(csub(x[r], q2), q);
-            v.y = csub(csub(x[r + 1], q2), q);
-            *reinterpret_cast<ulonglong2 *>(p + L::template idx<LAST>(tid, r)) = v;
-        }
+        const NttArgs a = {lb.fwd, q, q2, c.A, blk};
+        smem_ntt_forward<L, V>(
+            sm, tid, a, [&](uint32_t i) { return p[i]; },
+            [&](uint32_t i, uint64_t u, uint64_t v) {
+                u64x2 o;
+                o.x = csub(csub(u, q2), q);
+                o.y = csub(csub(v, q2), q);
+                *reinterpret_cast<u64x2 *>(p + i) = o;
+            });
     } else {
-#pragma unroll
-        for (int r = 0; r < L::E; r += 2) {
-            ulonglong2 v = *reinterpret_cast<const ulonglong2 *>(p + L::template idx<LAST>(tid, r));
-            x[r] = v.x;
-            x[r + 1] = v.y;
-        }
-        NttArgs a = {lb.inv, q, q2, c.A, blk};
-        block_ntt_inverse<L, SCALED>(x, sm, tid, a, lb.ninv, lb.wn);
-#pragma unroll
-        for (int r = 0; r < L::E; r++)
-            p[L::template idx<0>(tid, r)] = SCALED ? csub(x[r], q) : x[r];
+        const NttArgs a = {lb.inv, q, q2, c.A, blk};
+        smem_ntt_inverse<L, V, SCALED>(
+            sm, tid, a, lb.ninv, lb.wn, [&](uint32_t i) { return *reinterpret_cast<const u64x2 *>(p + i); },
+            [&](uint32_t i, uint64_t v) { p[i] = SCALED ? csub(v, q) : v; });
     }
 }
 
@@ -195,24 +186,25 @@ ntt_outer_kernel(const __grid_constant__ CtxDev c, uint64_t *data, size_t poly_s
     for (uint32_t a = 0; a < rows; a++) *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = x[a];
 }
 
-template <class L>
+template <class L, int V>
 static cudaError_t launch_ntt_blocks(const CtxDev &c, bool forward, uint64_t *data, size_t npoly,
-                                     size_t poly_stride, uint32_t limb0, uint32_t nlimbs, cudaStream_t s) {
+                                             size_t poly_stride, uint32_t limb0, uint32_t nlimbs,
+                                             cudaStream_t s) {
     const size_t smem = sizeof(uint64_t) << L::LOGB;
     const unsigned grid = (unsigned)((npoly * nlimbs) << c.A);
     cudaError_t e;
     if (forward) {
-        auto k = ntt_block_kernel<L, true, false>;
+        auto k = ntt_block_kernel<L, V, true, false>;
         if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-        k<<<grid, L::NT, smem, s>>>(c, data, poly_stride, limb0, nlimbs);
+        k<<<grid, L::NT / V, smem, s>>>(c, data, poly_stride, limb0, nlimbs);
     } else if (c.A == 0) {
-        auto k = ntt_block_kernel<L, false, true>;
+        auto k = ntt_block_kernel<L, V, false, true>;
         if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-        k<<<grid, L::NT, smem, s>>>(c, data, poly_stride, limb0, nlimbs);
+        k<<<grid, L::NT / V, smem, s>>>(c, data, poly_stride, limb0, nlimbs);
     } else {
-        auto k = ntt_block_kernel<L, false, false>;
+        auto k = ntt_block_kernel<L, V, false, false>;
         if ((e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-        k<<<grid, L::NT, smem, s>>>(c, data, poly_stride, limb0, nlimbs);
+        k<<<grid, L::NT / V, smem, s>>>(c, data, poly_stride, limb0, nlimbs);
     }
     return FEDHE_LAUNCHED();
 }
@@ -227,9 +219,8 @@ cudaError_t launch_ntt(const CtxDev &c, bool forward, uint64_t *data, size_t npo
                                                                               nlimbs, outer_threads);
         if ((e = FEDHE_LAUNCHED())) return e;
     }
-    if (c.LOGB == 13) e = launch_ntt_blocks<Lay<13, 4>>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
-    else if (getenv("FEDHE_LE4")) e = launch_ntt_blocks<Lay<14, 4>>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
-    else e = launch_ntt_blocks<Lay<14, 5>>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
+    if (c.LOGB == 13) e = launch_ntt_blocks<Lay<13, 3>, 2>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
+    else e = launch_ntt_blocks<Lay<14, 3>, 2>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
     if (e) return e;
     if (!forward && c.A > 0) {
         ntt_outer_kernel<false><<<blocks_for(outer_threads, 256), 256, 0, s>>>(c, data, poly_stride, limb0,
@@ -774,7 +765,6 @@ cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const int64_t *m, 
     if (T == 0) return cudaSuccess;
     if (c.A == 0) {
         if (c.LOGB == 13) return launch_encrypt_fused<Lay<13, 3>, 2>(c, k, m, t0, T, seed, client, ct, s);
-        if (getenv("FEDHE_LE4")) return launch_encrypt_fused<Lay<14, 4>, 1>(c, k, m, t0, T, seed, client, ct, s);
         return launch_encrypt_fused<Lay<14, 3>, 2>(c, k, m, t0, T, seed, client, ct, s);
     }
     cudaError_t e;
@@ -798,47 +788,64 @@ cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const int64_t *m, 
 
 // One thread per pair of neighbouring coefficients of one (ciphertext,
 // component).  The last limb is accumulated first: its centred value is the
-// rounding term of every other limb.
+// rounding term of every other limb.  The pass is bound by HBM reads
+// (32 L C bytes per parameter), so the client pointers and weights are
+// staged in shared memory once per block and the loads of four clients are
+// issued before their multiply-adds to keep enough bytes in flight.
+__device__ __forceinline__ void weighted_sum_pair(const uint64_t *const *sp, const tw_t *sw, int C, uint32_t L,
+                                                  uint32_t j, size_t off, uint64_t q, uint64_t &ax,
+                                                  uint64_t &ay) {
+    const uint64_t q2 = 2 * q;
+    ax = 0;
+    ay = 0;
+    int cl = 0;
+    for (; cl + 4 <= C; cl += 4) {
+        ulonglong2 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; u++) v[u] = __ldg(reinterpret_cast<const ulonglong2 *>(sp[cl + u] + off));
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+            const tw_t w = sw[(cl + u) * L + j];
+            ax = csub(ax + shoup_lazy(v[u].x, w.w, w.wp, q), q2);
+            ay = csub(ay + shoup_lazy(v[u].y, w.w, w.wp, q), q2);
+        }
+    }
+    for (; cl < C; cl++) {
+        const ulonglong2 v = __ldg(reinterpret_cast<const ulonglong2 *>(sp[cl] + off));
+        const tw_t w = sw[cl * L + j];
+        ax = csub(ax + shoup_lazy(v.x, w.w, w.wp, q), q2);
+        ay = csub(ay + shoup_lazy(v.y, w.w, w.wp, q), q2);
+    }
+    ax = csub(ax, q);
+    ay = csub(ay, q);
+}
+
 __global__ void __launch_bounds__(256)
 aggregate_rescale_kernel(const __grid_constant__ CtxDev c, const uint64_t *const *ptrs, const tw_t *wtab,
                          int C, uint64_t *out, size_t total) {
+    extern __shared__ __align__(16) unsigned char agg_sm[];
+    const uint32_t L = c.L;
+    tw_t *sw = reinterpret_cast<tw_t *>(agg_sm);                                    // [C][L]
+    const uint64_t **sp = reinterpret_cast<const uint64_t **>(sw + (size_t)C * L);  // [C]
+    for (int e = threadIdx.x; e < C * (int)L; e += blockDim.x) sw[e] = wtab[e];
+    for (int e = threadIdx.x; e < C; e += blockDim.x) sp[e] = ptrs[e];
+    __syncthreads();
     const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= total) return;
     const uint32_t pairs = c.N >> 1;
     const uint32_t i = (uint32_t)(g % pairs) * 2;
     const size_t tc = g / pairs;                 // t * 2 + component
-    const uint32_t L = c.L;
     const uint64_t ql = c.limb[L - 1].q;
     uint64_t rx, ry;
-    {
-        const uint64_t q2 = 2 * ql;
-        const size_t off = (tc * L + (L - 1)) * c.N + i;
-        uint64_t ax = 0, ay = 0;
-        for (int cl = 0; cl < C; cl++) {
-            const ulonglong2 v = __ldg(reinterpret_cast<const ulonglong2 *>(ptrs[cl] + off));
-            const tw_t w = wtab[cl * L + (L - 1)];
-            ax = csub(ax + shoup_lazy(v.x, w.w, w.wp, ql), q2);
-            ay = csub(ay + shoup_lazy(v.y, w.w, w.wp, ql), q2);
-        }
-        rx = csub(ax, ql);
-        ry = csub(ay, ql);
-    }
+    weighted_sum_pair(sp, sw, C, L, L - 1, (tc * L + (L - 1)) * c.N + i, ql, rx, ry);
     const bool negx = rx > ql / 2, negy = ry > ql / 2;
     const uint64_t mx = negx ? ql - rx : rx, my = negy ? ql - ry : ry;   // |centred remainder|
     for (uint32_t j = 0; j + 1 < L; j++) {
         const LimbDev &lb = c.limb[j];
-        const uint64_t q = lb.q, q2 = 2 * q;
-        const size_t off = (tc * L + j) * c.N + i;
-        uint64_t ax = 0, ay = 0;
-        for (int cl = 0; cl < C; cl++) {
-            const ulonglong2 v = __ldg(reinterpret_cast<const ulonglong2 *>(ptrs[cl] + off));
-            const tw_t w = wtab[cl * L + j];
-            ax = csub(ax + shoup_lazy(v.x, w.w, w.wp, q), q2);
-            ay = csub(ay + shoup_lazy(v.y, w.w, w.wp, q), q2);
-        }
-        ax = csub(ax, q);
-        ay = csub(ay, q);
-        uint64_t sx = barrett64(mx, q, lb.mu), sy = barrett64(my, q, lb.mu);
+        const uint64_t q = lb.q;
+        uint64_t ax, ay;
+        weighted_sum_pair(sp, sw, C, L, j, (tc * L + j) * c.N + i, q, ax, ay);
+        const uint64_t sx = barrett64(mx, q, lb.mu), sy = barrett64(my, q, lb.mu);
         // acc - r: subtracting a negative remainder adds its magnitude
         const uint64_t dx = negx ? addmod(ax, sx, q) : submod(ax, sx, q);
         const uint64_t dy = negy ? addmod(ay, sy, q) : submod(ay, sy, q);
@@ -853,7 +860,12 @@ cudaError_t launch_aggregate(const CtxDev &c, const uint64_t *const *ptrs, const
                              size_t T, uint64_t *out, cudaStream_t s) {
     if (T == 0) return cudaSuccess;
     const size_t total = T * 2 * (c.N >> 1);
-    aggregate_rescale_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, ptrs, wtab, C, out, total);
+    const size_t smem = (size_t)C * c.L * sizeof(tw_t) + (size_t)C * sizeof(void *);
+    cudaError_t e;
+    if (smem > 48 * 1024 &&
+        (e = cudaFuncSetAttribute(aggregate_rescale_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)))
+        return e;
+    aggregate_rescale_kernel<<<blocks_for(total, 256), 256, smem, s>>>(c, ptrs, wtab, C, out, total);
     return FEDHE_LAUNCHED();
 }
 

@@ -1,7 +1,7 @@
 // Register-tiled negacyclic NTT of one block of B = 2^LOGB residues held by
-// one thread block: every thread keeps E = 2^LE residues in registers, does
-// LE butterfly stages on them, and the block re-distributes the residues
-// through shared memory between such phases.
+// one thread block in shared memory: a thread takes E = 2^LE residues into
+// registers, does LE butterfly stages on them and puts them back; between
+// such phases the index bits are re-dealt among the threads.
 //
 // Index conventions (forward transform, natural order in, bit-reversed out):
 // stage s (0-based) of a length-N transform pairs the elements whose indices
@@ -155,65 +155,14 @@ HD void inv_phase(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
     inv_phase_from<L, P, STOP, nst - 1>(x, tid, a);
 }
 
-// ---- exchange through shared memory ---------------------------------------
-
-template <class L, int P>
-HD void xchg_write(const uint64_t (&x)[L::E], uint64_t *sm, uint32_t tid) {
-#pragma unroll
-    for (int r = 0; r < L::E; r++) sm[swz(L::template idx<P>(tid, r))] = x[r];
-}
-
-template <class L, int P>
-HD void xchg_read(uint64_t (&x)[L::E], const uint64_t *sm, uint32_t tid) {
-#pragma unroll
-    for (int r = 0; r < L::E; r++) x[r] = sm[swz(L::template idx<P>(tid, r))];
-}
-
-#if defined(__CUDACC__)
-// Whole-block transforms.  sm: B words of shared memory.  The residues enter
-// in the layout of phase 0 (forward) or of the last phase (inverse) and leave
-// in the other one.
-
-template <class L, int P = 0>
-__device__ __forceinline__ void block_ntt_forward(uint64_t (&x)[L::E], uint64_t *sm, uint32_t tid,
-                                                  const NttArgs &a) {
-    fwd_phase<L, P>(x, tid, a);
-    if constexpr (P + 1 < L::NPH) {
-        __syncthreads();                       // earlier readers of sm are done
-        xchg_write<L, P>(x, sm, tid);
-        __syncthreads();
-        xchg_read<L, P + 1>(x, sm, tid);
-        block_ntt_forward<L, P + 1>(x, sm, tid, a);
-    }
-}
-
-// SCALED: fold 1/N into global stage 0 (only valid when A == 0)
-template <class L, bool SCALED, int P = L::NPH - 1>
-__device__ __forceinline__ void block_ntt_inverse(uint64_t (&x)[L::E], uint64_t *sm, uint32_t tid,
-                                                  const NttArgs &a, tw_t ninv, tw_t wn) {
-    if constexpr (P == 0 && SCALED) {
-        inv_phase<L, 0, 1>(x, tid, a);
-        inv_stage0_scaled<L>(x, ninv, wn, a.q, a.q2);
-    } else {
-        inv_phase<L, P>(x, tid, a);
-    }
-    if constexpr (P > 0) {
-        __syncthreads();
-        xchg_write<L, P>(x, sm, tid);
-        __syncthreads();
-        xchg_read<L, P - 1>(x, sm, tid);
-        block_ntt_inverse<L, SCALED, P - 1>(x, sm, tid, a, ninv, wn);
-    }
-}
-#endif
-
 #if defined(__CUDACC__)
 // ---------------------------------------------------------------------------
-// In-place variant: the block's residues stay in shared memory (swizzled) and
-// every thread plays V "virtual threads" per phase, each of which loads its
-// E residues, does the phase's butterflies in registers and stores them back
-// to the same places, so that only E residues are live per thread at a time
-// and no separate exchange buffer is needed.  The first phase takes its input
+// Whole-block transforms.  The block's residues stay in shared memory
+// (swizzled) and every thread plays V "virtual threads" per phase, each of
+// which loads its E residues, does the phase's butterflies in registers and
+// stores them back to the same places, so that only E residues are live per
+// thread at a time (E = 8 keeps a 1024-thread block within 64 registers with
+// no spills) and no separate exchange buffer is needed.  The first phase takes its input
 // from `src`, the last hands its output to `dst`:
 //   forward:  src(i) -> residue i;            dst(i, a, b): residues i, i+1
 //   inverse:  src(i) -> residues i, i+1;      dst(i, a): residue i
