@@ -81,6 +81,11 @@ int he_ctx_create(const he_params *p, he_ctx **out) {
     int rc = HE_OK;
     do {
         if (cudaGetDevice(&ctx->device) != cudaSuccess) { rc = HE_ERR_CUDA; break; }
+        if (cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device) != cudaSuccess ||
+            ctx->sm_count < 1) {
+            rc = HE_ERR_CUDA;
+            break;
+        }
         CtxDev &d = ctx->dev;
         memset(&d, 0, sizeof(d));
         d.N = p->N;
@@ -137,6 +142,11 @@ int he_ctx_destroy(he_ctx *ctx) {
     if (ctx->ws) cudaFree(ctx->ws);
     if (ctx->tab) cudaFree(ctx->tab);
     if (ctx->round_buf) cudaFree(ctx->round_buf);
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+    for (int i = 0; i < 2; i++) {
+        if (ctx->ev_ready[i]) cudaEventDestroy(ctx->ev_ready[i]);
+        if (ctx->ev_free[i]) cudaEventDestroy(ctx->ev_free[i]);
+    }
     ctx->magic = 0;
     delete ctx;
     return HE_OK;
@@ -544,8 +554,10 @@ int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const f
     const size_t n = d.N / 2, T = he_num_ct(ctx, k), padded = T * n, restlen = P - k;
     const size_t ctw = 2 * (size_t)d.L * d.N, aggw = 2 * (size_t)(d.L - 1) * d.N;
     // ciphertext indices are processed in chunks that keep all clients'
-    // ciphertexts of a chunk within about 4 GiB
-    size_t Tc = ((size_t)4 << 30) / (C * ctw * sizeof(uint64_t));
+    // ciphertexts of a chunk within about 8 GiB; a chunk is a whole number of
+    // waves of one thread block per SM
+    size_t Tc = ((size_t)8 << 30) / (C * ctw * sizeof(uint64_t));
+    if (Tc > (size_t)ctx->sm_count) Tc -= Tc % ctx->sm_count;
     if (Tc < 1) Tc = 1;
     if (Tc > T) Tc = T;
     auto align = [](size_t b) { return (b + 255) & ~(size_t)255; };
@@ -553,13 +565,15 @@ int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const f
                  b_rest = align(restlen * sizeof(float)), b_cts = align(C * Tc * ctw * sizeof(uint64_t)),
                  b_agg = align(Tc * aggw * sizeof(uint64_t)), b_z = align(padded * sizeof(double)),
                  b_ravg = align(restlen * sizeof(double)), b_out = align(P * sizeof(double));
-    const size_t total = b_x + C * (b_sel + b_rest) + b_cts + b_agg + b_z + b_ravg + b_out;
+    const size_t total = 2 * b_x + C * (b_sel + b_rest) + b_cts + b_agg + b_z + b_ravg + b_out;
     int rc = ensure(&ctx->round_buf, &ctx->round_bytes, total);
     if (rc != HE_OK) return rc;
     rc = ensure(&ctx->ws, &ctx->ws_bytes, work_bytes(ctx, Tc));
     if (rc != HE_OK) return rc;
     unsigned char *p = static_cast<unsigned char *>(ctx->round_buf);
-    float *x = reinterpret_cast<float *>(p); p += b_x;
+    float *x[2];
+    x[0] = reinterpret_cast<float *>(p); p += b_x;
+    x[1] = reinterpret_cast<float *>(p); p += b_x;
     std::vector<float *> sel(C), rest(C);
     for (int i = 0; i < C; i++) { sel[i] = reinterpret_cast<float *>(p); p += b_sel; }
     for (int i = 0; i < C; i++) { rest[i] = reinterpret_cast<float *>(p); p += b_rest; }
@@ -570,21 +584,40 @@ int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const f
     double *out = reinterpret_cast<double *>(p);
     cudaStream_t st = as_stream(stream);
 
-    for (int i = 0; i < C; i++) {
-        if (!xs_host[i]) return HE_ERR_INVALID_ARG;
-        CU(cudaMemcpyAsync(x, xs_host[i], P * sizeof(float), cudaMemcpyHostToDevice, st));
-        rc = he_pack(ctx, mask, x, P, sel[i], restlen ? rest[i] : nullptr, stream);
-        if (rc != HE_OK) return rc;
+    if (!ctx->copy_stream) {
+        CU(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+        for (int i = 0; i < 2; i++) {
+            CU(cudaEventCreateWithFlags(&ctx->ev_ready[i], cudaEventDisableTiming));
+            CU(cudaEventCreateWithFlags(&ctx->ev_free[i], cudaEventDisableTiming));
+        }
     }
+    for (int i = 0; i < C; i++)
+        if (!xs_host[i]) return HE_ERR_INVALID_ARG;
+    // The upload of client i+1 (copy stream, two staging buffers) overlaps
+    // the packing of client i and the encryption of its first chunk.
+    CU(cudaEventRecord(ctx->ev_free[0], st));       // earlier work on `st` may still use the buffers
+    CU(cudaEventRecord(ctx->ev_free[1], st));
     std::vector<const uint64_t *> cptr(C);
-    for (size_t t0 = 0; t0 < T; t0 += Tc) {
+    for (size_t t0 = 0; t0 < T || t0 == 0; t0 += Tc) {
         const size_t tc = T - t0 < Tc ? T - t0 : Tc;
         for (int i = 0; i < C; i++) {
+            if (t0 == 0) {
+                const int b = i & 1;
+                CU(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_free[b], 0));
+                CU(cudaMemcpyAsync(x[b], xs_host[i], P * sizeof(float), cudaMemcpyHostToDevice, ctx->copy_stream));
+                CU(cudaEventRecord(ctx->ev_ready[b], ctx->copy_stream));
+                CU(cudaStreamWaitEvent(st, ctx->ev_ready[b], 0));
+                rc = he_pack(ctx, mask, x[b], P, sel[i], restlen ? rest[i] : nullptr, stream);
+                if (rc != HE_OK) return rc;
+                CU(cudaEventRecord(ctx->ev_free[b], st));
+            }
+            if (tc == 0) continue;
             uint64_t *ci = cts + (size_t)i * Tc * ctw;
             rc = he_encrypt_range(ctx, keys, sel[i] + t0 * n, t0, tc, enc_seed, (uint32_t)i, ci, stream);
             if (rc != HE_OK) return rc;
             cptr[i] = ci;
         }
+        if (tc == 0) break;
         rc = he_weighted_aggregate(ctx, cptr.data(), alpha_host, C, tc, agg, stream);
         if (rc != HE_OK) return rc;
         rc = he_decrypt(ctx, keys, agg, tc, z + t0 * n, stream);

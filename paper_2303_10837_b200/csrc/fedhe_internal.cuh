@@ -54,6 +54,9 @@ struct he_ctx {
     size_t tab_bytes = 0;
     void *round_buf = nullptr;     // buffers of he_round_host
     size_t round_bytes = 0;
+    int sm_count = 0;
+    cudaStream_t copy_stream = nullptr;   // uploads of he_round_host, overlapped with compute
+    cudaEvent_t ev_ready[2] = {nullptr, nullptr}, ev_free[2] = {nullptr, nullptr};
 };
 
 struct he_keys {
