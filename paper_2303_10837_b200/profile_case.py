@@ -3,6 +3,7 @@
     python paper_2303_10837_b200/profile_case.py encrypt [--cts 296] [--reps 2]
     python paper_2303_10837_b200/profile_case.py ntt [--polys 256]
     python paper_2303_10837_b200/profile_case.py aggregate [--cts 64]
+    python paper_2303_10837_b200/profile_case.py sweep            # kernel sweep table (no profiler)
 
 Each case touches more memory than the L2 holds so that DRAM counters mean something,
 launches the kernel of interest a handful of times and exits.
@@ -24,14 +25,75 @@ import paper_2303_10837_b200 as he
 import synthetic_inputs as si
 
 
+def read_hbm_peak():
+    import json
+    try:
+        return float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def timed(fn, reps):
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    fn()
+    torch.cuda.synchronize()
+    ev0.record()
+    for _ in range(reps):
+        fn()
+    ev1.record()
+    torch.cuda.synchronize()
+    return ev0.elapsed_time(ev1) / reps
+
+
+def sweep():
+    """Batched forward+inverse NTT and encode+encrypt over ring degrees, limb counts and batch
+    sizes; GB/s counts 16 N bytes per limb transform (32 N for N > 2^14: two passes) and the
+    ciphertext bytes written per encryption."""
+    peak, src = read_hbm_peak()
+    print("HBM peak %.1f GB/s (%s)" % (peak, src))
+    print("%6s %3s %6s | %10s %9s %7s | %10s %9s %7s" % ("N", "L", "batch", "ntt us", "GB/s", "%HBM", "encrypt us", "GB/s", "%HBM"))
+    for logn in (13, 14, 15, 16):
+        N = 1 << logn
+        for L in (2, 4, 8, 12):
+            primes = si.PRIMES_SWEEP[:L]
+            g = he.he_ctx_create(N, list(primes), 40)
+            keys = he.he_keygen(g, 5)
+            for B in (1, 4, 16, 64, 256, 1024, 4096):
+                words = B * L * N
+                if words * 8 > 8 << 30 or 2 * words * 8 > 12 << 30:
+                    continue
+                polys = torch.randint(0, 1 << 59, (B, L, N), dtype=torch.int64, device="cuda")
+                reps = 3 if words > (1 << 26) else 10
+
+                def both():
+                    he.he_ntt_forward(g, polys)
+                    he.he_ntt_inverse(g, polys)
+                t_ntt = timed(both, reps) / 2
+                passes = 1 if logn <= 14 else 2
+                gbs_ntt = 16.0 * N * L * B * passes / (t_ntt * 1e-3) / 1e9
+                del polys
+                sel = torch.randn(B * (N // 2), dtype=torch.float32, device="cuda") * 0.01
+                ct = torch.empty((B, 2, L, N), dtype=torch.int64, device="cuda")
+                t_enc = timed(lambda: he.he_encrypt(g, keys, sel, 3, 0, out=ct), reps)
+                gbs_enc = (16.0 * N * L + 2.0 * N) * B / (t_enc * 1e-3) / 1e9
+                del sel, ct
+                print("%6d %3d %6d | %10.1f %9.1f %6.1f%% | %10.1f %9.1f %6.1f%%"
+                      % (N, L, B, t_ntt * 1e3, gbs_ntt, 100 * gbs_ntt / peak, t_enc * 1e3, gbs_enc,
+                         100 * gbs_enc / peak), flush=True)
+            del keys, g
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["encrypt", "ntt", "aggregate", "decrypt"])
+    ap.add_argument("case", choices=["encrypt", "ntt", "aggregate", "decrypt", "sweep"])
     ap.add_argument("--cts", type=int, default=296)
     ap.add_argument("--polys", type=int, default=256)
     ap.add_argument("--reps", type=int, default=2)
     ap.add_argument("--workload", choices=["resnet18", "tiny", "bert"], default="resnet18")
     a = ap.parse_args()
+    if a.case == "sweep":
+        sweep()
+        return
     base = {"resnet18": si.RESNET18, "tiny": si.TINY, "bert": si.bert(1.0)}[a.workload]
     w = si.scaled(base, a.cts * base.n, clients=base.clients)
     g = he.he_ctx_create(w.N, list(w.primes), w.log2_delta)
