@@ -44,6 +44,10 @@ UNIT = "params/s"
 # A 64-bit Shoup butterfly needs at least the high half of x*w' (4 wide
 # products) and the low halves of x*w and hi*q (1 wide + 2 narrow each):
 # 6 wide + 4 narrow = 19 multiply slots.  Additions go to another pipe.
+# DRAM bytes (read + write) per ciphertext of encrypt_fused_kernel at N = 16384,
+# L = 4, from the ncu capture in profiles/encrypt_fused_kernel_resnet18_296cts.md
+# (480.1 MB for 296 ciphertexts; traffic grows in proportion to the count).
+ENCRYPT_DRAM_BYTES_PER_CT_N16384_L4 = 480.087552e6 / 296
 IMAD_PER_SM_CLK = 64.0
 WIDE_COST = 2.5
 MUL_SLOTS_PER_BUTTERFLY = 6 * WIDE_COST + 4
@@ -337,7 +341,9 @@ def run_ours(args, w):
         "kernel": "encrypt_fused_kernel" if w.N <= 16384 else "ntt_block_kernel (inside he_encrypt)",
         "bound": "alu", "achieved": achieved, "peak": peak,
         "unit": "T multiply-slots/s (32-bit integer multiply pipe)",
-        "frac": achieved / peak, "traffic": None,
+        "frac": achieved / peak,
+        "traffic": ENCRYPT_DRAM_BYTES_PER_CT_N16384_L4 * T if (w.N == 16384 and w.L == 4) else None,
+        "algorithmic_bytes": alg_bytes,
         "ms_per_launch": kern_ms, "launches_per_step": w.clients, "butterflies_per_launch": butterflies,
         "hbm_gbs_of_kernel": alg_bytes / (kern_ms * 1e-3) / 1e9,
         "hbm_frac_of_kernel": alg_bytes / (kern_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
