@@ -80,6 +80,10 @@ _plain = _sig("orc_plain_aggregate", None, _vp, _vp, _u32, _sz, _vp)
 _dec_limb = _sig("orc_decrypt_limb", None, _vp, _vp, _vp, _u32, _u32, _vp)
 _decrypt = _sig("orc_decrypt", None, _vp, _vp, _vp, _u32, _sz, _vp)
 _decode = _sig("orc_decode", None, _vp, _vp, _vp)
+_th_split = _sig("orc_threshold_split", None, _vp, _vp, _u64, _vp, _vp)
+_smudge = _sig("orc_sample_smudge", None, _u64, _u32, _u32, _u32, _u32, _vp)
+_th_partial = _sig("orc_partial_decrypt", None, _vp, _vp, _u32, _vp, _u32, _u64, _u32, _u32, _vp)
+_th_combine = _sig("orc_threshold_combine", None, _vp, _vp, _u32, _vp, _u32, _vp)
 _select = _sig("orc_select_mask", None, _vp, _sz, _sz, _vp)
 _pack = _sig("orc_pack", None, _vp, _vp, _sz, _vp, _sz, _vp, _vp)
 _unpack = _sig("orc_unpack", None, _vp, _sz, _vp, _vp, _sz, _vp)
@@ -150,6 +154,12 @@ def sample_gauss(seed, t, client, tag, N):
 def sample_uniform(seed, t, client, tag, limb, q, N):
     out = np.empty(N, np.uint64)
     _s_unif(seed, t, client, tag, limb, q, N, _p(out))
+    return out
+
+
+def sample_smudge(seed, t, party, bits, N):
+    out = np.empty(N, np.int64)
+    _smudge(seed, t, party, bits, N, _p(out))
     return out
 
 
@@ -312,6 +322,27 @@ class Context:
         for t in range(d.shape[0]):
             _decode(self._h, d[t].ctypes.data_as(_vp), z[t].ctypes.data_as(_vp))
         return z
+
+    def threshold_split(self, s, seed):
+        s = _arr(s, np.int8)
+        a = np.empty((self.L, self.N), np.uint64)
+        b = np.empty((self.L, self.N), np.uint64)
+        _th_split(self._h, _p(s), seed, _p(a), _p(b))
+        return a, b
+
+    def partial_decrypt(self, share, party, ct, level, seed, t, bits):
+        share = _arr(share, np.uint64)
+        ct = _arr(ct, np.uint64)
+        out = np.empty(self.N, np.uint64)
+        _th_partial(self._h, _p(share), party, _p(ct), level, seed, t, bits, _p(out))
+        return out
+
+    def threshold_combine(self, ct, level, parts):
+        ct = _arr(ct, np.uint64)
+        parts = [_arr(x, np.uint64) for x in parts]
+        d = np.empty(self.N, np.int64)
+        _th_combine(self._h, _p(ct), level, _ptr_array(parts), len(parts), _p(d))
+        return d
 
     def pack(self, idx, k, x):
         x = _arr(x, np.float32)

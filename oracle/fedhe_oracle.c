@@ -614,6 +614,59 @@ void orc_decrypt(const orc_ctx *c, const int8_t *s, const uint64_t *ct, uint32_t
 }
 
 /* ------------------------------------------------------------------------- */
+/* two-party threshold decryption: each party decrypts partially with its    */
+/* share of the key and the partial results are merged (paper, appendix      */
+/* "Key Management And Threshold HE").  The interactive key agreement is     */
+/* replaced by a dealer that splits an existing secret additively.           */
+/* ------------------------------------------------------------------------- */
+
+void orc_threshold_split(const orc_ctx *c, const int8_t *s, uint64_t seed, uint64_t *share0,
+                         uint64_t *share1) {
+    uint32_t N = c->N;
+    for (uint32_t j = 0; j < c->L; j++) {
+        uint64_t q = c->q[j];
+        uint64_t *a = share0 + (size_t)j * N, *b = share1 + (size_t)j * N;
+        orc_sample_uniform(seed, 0, 0, 7, j, q, N, a);
+        for (uint32_t i = 0; i < N; i++) b[i] = submod(from_signed(s[i], q), a[i], q);
+    }
+}
+
+/* coefficient j: the 64-bit r of words 2(j&1), 2(j&1)+1 of block j>>1;
+ * value = (r >> (63 - bits)) - 2^bits */
+void orc_sample_smudge(uint64_t seed, uint32_t t, uint32_t party, uint32_t bits, uint32_t N, int64_t *out) {
+    for (uint32_t j = 0; j < N; j++) {
+        uint32_t w[4];
+        stream_block(seed, j >> 1, t, party, 8, 0, w);
+        uint64_t r = (uint64_t)w[2 * (j & 1)] | ((uint64_t)w[2 * (j & 1) + 1] << 32);
+        out[j] = (int64_t)(r >> (63 - bits)) - ((int64_t)1 << bits);
+    }
+}
+
+void orc_partial_decrypt(const orc_ctx *c, const uint64_t *share, uint32_t party, const uint64_t *ct,
+                         uint32_t level, uint64_t seed, uint32_t t, uint32_t bits, uint64_t *out) {
+    uint32_t N = c->N;
+    uint64_t q = c->q[0];
+    const uint64_t *c1 = ct + (size_t)(1 * level + 0) * N;
+    int64_t *e = (int64_t *)malloc(sizeof(int64_t) * N);
+    orc_sample_smudge(seed, t, party, bits, N, e);
+    orc_negacyclic_mul_ntt(c, 0, c1, share, out);             /* limb 0 of the share */
+    for (uint32_t i = 0; i < N; i++) out[i] = addmod(out[i], from_signed(e[i], q), q);
+    free(e);
+}
+
+void orc_threshold_combine(const orc_ctx *c, const uint64_t *ct, uint32_t level,
+                           const uint64_t *const *parts, uint32_t nparts, int64_t *d) {
+    uint32_t N = c->N;
+    uint64_t q = c->q[0];
+    const uint64_t *c0 = ct + (size_t)(0 * level + 0) * N;
+    for (uint32_t i = 0; i < N; i++) {
+        uint64_t r = c0[i];
+        for (uint32_t p = 0; p < nparts; p++) r = addmod(r, parts[p][i], q);
+        d[i] = r > q / 2 ? -(int64_t)(q - r) : (int64_t)r;
+    }
+}
+
+/* ------------------------------------------------------------------------- */
 /* selective-encryption mask ("Step 2"), packing, merge                       */
 /* ------------------------------------------------------------------------- */
 

@@ -98,6 +98,22 @@ void orc_decrypt(const orc_ctx *c, const int8_t *s, const uint64_t *ct, uint32_t
                  size_t T, int64_t *d);
 void orc_decode(const orc_ctx *c, const int64_t *d, double *z);
 
+/* ---- two-party threshold decryption (appendix "Key Management And Threshold HE") ---- */
+/* dealer split of the secret: share0[L][N] uniform mod q_j (stream tag 7),
+ * share1 = s - share0 (mod q_j) */
+void orc_threshold_split(const orc_ctx *c, const int8_t *s, uint64_t seed, uint64_t *share0,
+                         uint64_t *share1);
+/* smudging noise of `party` for ciphertext index t: uniform integers in
+ * [-2^bits, 2^bits) from stream tag 8 */
+void orc_sample_smudge(uint64_t seed, uint32_t t, uint32_t party, uint32_t bits, uint32_t N, int64_t *out);
+/* partial decryption of one ciphertext on limb 0: c1 share + E (mod q_0);
+ * share points at the party's [L][N] residues */
+void orc_partial_decrypt(const orc_ctx *c, const uint64_t *share, uint32_t party, const uint64_t *ct,
+                         uint32_t level, uint64_t seed, uint32_t t, uint32_t bits, uint64_t *out);
+/* d = c0 + sum of the parts (mod q_0), centred */
+void orc_threshold_combine(const orc_ctx *c, const uint64_t *ct, uint32_t level,
+                           const uint64_t *const *parts, uint32_t nparts, int64_t *d);
+
 /* ---- selective-encryption mask, packing ---------------------------------- */
 /* indices of the k largest keys (ties: lower index first), ascending */
 void orc_select_mask(const float *score, size_t P, size_t k, uint32_t *idx);
