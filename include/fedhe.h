@@ -198,6 +198,27 @@ int he_decrypt_noalloc(he_ctx *ctx, const he_keys *keys, const uint64_t *agg_dev
 int he_unpack(he_ctx *ctx, const he_mask *mask, const double *z_dev, const double *rest_avg_dev,
               size_t P, double *w_glob_dev, void *stream);
 
+/* Two-party threshold decryption (paper appendix "Key Management And
+ * Threshold HE": every party holds a share of the secret key, decrypts the
+ * final ciphertext partially, and the partial results are merged).  The
+ * interactive key agreement is out of scope: a dealer splits an existing
+ * secret additively, share0 uniform mod q_j (Philox stream of `seed`),
+ * share1 = s - share0.  The share handles are released with he_keys_destroy
+ * and are accepted only by he_partial_decrypt.  Synchronous. */
+int he_threshold_split(he_ctx *ctx, const he_keys *keys, uint64_t seed, he_keys **share0, he_keys **share1,
+                       void *stream);
+/* Party `party`'s partial decryption of T ciphertexts of `level` limbs:
+ * part = c1 * share + E (mod q_0), E uniform in [-2^smudge_bits, 2^smudge_bits)
+ * per coefficient from the Philox stream of (seed, t, party); smudge_bits <= 40.
+ *   ct: dev uint64 [T][2][level][N]; part: dev uint64 [T][N], canonical residues. */
+int he_partial_decrypt(he_ctx *ctx, const he_keys *share, uint32_t party, const uint64_t *ct_dev, uint32_t level,
+                       size_t T, uint64_t seed, uint32_t smudge_bits, uint64_t *part_dev, void *stream);
+/* Merge: d = c0 + sum of the parts (mod q_0), centred and decoded like
+ * he_decrypt.  parts: host array of nparts (<= 8) dev pointers uint64 [T][N];
+ * z: dev double[T*n]. */
+int he_threshold_combine(he_ctx *ctx, const uint64_t *ct_dev, uint32_t level, const uint64_t *const *parts_host,
+                         int nparts, size_t T, double *z_dev, void *stream);
+
 /* Batched negacyclic transforms on raw residues (kernel sweep; no paper
  * counterpart): polys dev uint64 [B][L][N] in place, canonical residues in,
  * canonical residues out.  Forward: A[k] = sum_j a_j psi^((2 brev(k)+1) j)

@@ -74,6 +74,9 @@ _SIGS = {
     "he_decrypt": (C.c_int, [_vp, _vp, _vp, _sz, _vp, _vp]),
     "he_decrypt_level": (C.c_int, [_vp, _vp, _vp, _u32, _sz, _vp, _vp]),
     "he_decrypt_noalloc": (C.c_int, [_vp, _vp, _vp, _sz, _vp, _vp]),
+    "he_threshold_split": (C.c_int, [_vp, _vp, _u64, C.POINTER(_vp), C.POINTER(_vp), _vp]),
+    "he_partial_decrypt": (C.c_int, [_vp, _vp, _u32, _vp, _u32, _sz, _u64, _u32, _vp, _vp]),
+    "he_threshold_combine": (C.c_int, [_vp, _vp, _u32, _vp, C.c_int, _sz, _vp, _vp]),
     "he_unpack": (C.c_int, [_vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "he_ntt_forward": (C.c_int, [_vp, _vp, _sz, _vp]),
     "he_ntt_inverse": (C.c_int, [_vp, _vp, _sz, _vp]),
@@ -299,6 +302,33 @@ def he_decrypt_level(ctx: Ctx, keys: Keys, ct: torch.Tensor, level: int) -> torc
     z = torch.empty(T * ctx.n, dtype=torch.float64, device="cuda")
     _check(_lib.he_decrypt_level(ctx.handle, keys.handle, _dev(ct, torch.int64), level, T, z.data_ptr(),
                                  _stream()), "he_decrypt_level")
+    return z
+
+
+def he_threshold_split(ctx: Ctx, keys: Keys, seed: int):
+    """Two additive shares of the secret key (handles accepted by he_partial_decrypt only)."""
+    a, b = _vp(), _vp()
+    _check(_lib.he_threshold_split(ctx.handle, keys.handle, seed, C.byref(a), C.byref(b), _stream()),
+           "he_threshold_split")
+    return Keys(a.value, ctx), Keys(b.value, ctx)
+
+
+def he_partial_decrypt(ctx: Ctx, share: Keys, party: int, ct: torch.Tensor, level: int, seed: int,
+                       smudge_bits: int) -> torch.Tensor:
+    """Residues mod q_0, uint64-as-int64 [T][N]."""
+    T = ct.shape[0]
+    part = torch.empty((T, ctx.N), dtype=torch.int64, device="cuda")
+    _check(_lib.he_partial_decrypt(ctx.handle, share.handle, party, _dev(ct, torch.int64) or None, level, T,
+                                   seed, smudge_bits, part.data_ptr() or None, _stream()), "he_partial_decrypt")
+    return part
+
+
+def he_threshold_combine(ctx: Ctx, ct: torch.Tensor, level: int, parts: List[torch.Tensor]) -> torch.Tensor:
+    T = ct.shape[0]
+    ptrs = (_vp * len(parts))(*[_dev(p, torch.int64) for p in parts])
+    z = torch.empty(T * ctx.n, dtype=torch.float64, device="cuda")
+    _check(_lib.he_threshold_combine(ctx.handle, _dev(ct, torch.int64) or None, level, C.cast(ptrs, _vp),
+                                     len(parts), T, z.data_ptr() or None, _stream()), "he_threshold_combine")
     return z
 
 

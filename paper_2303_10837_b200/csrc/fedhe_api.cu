@@ -51,6 +51,14 @@ size_t work_bytes(const he_ctx *ctx, size_t T) { return 2 * T * (size_t)ctx->dev
 
 }  // namespace
 
+namespace fedhe {
+int ctx_workspace(he_ctx *ctx, size_t T, void **out) {
+    const int rc = ensure(&ctx->ws, &ctx->ws_bytes, work_bytes(ctx, T));
+    *out = ctx->ws;
+    return rc;
+}
+}  // namespace fedhe
+
 extern "C" {
 
 const char *he_strerror(int code) {
@@ -232,7 +240,7 @@ int he_keys_destroy(he_keys *keys) {
 }
 
 int he_keys_export(he_ctx *ctx, const he_keys *keys, uint64_t *pk_dev, int8_t *s_dev, void *stream) {
-    if (!good(ctx) || !good(keys) || keys->ctx != ctx) return HE_ERR_INVALID_ARG;
+    if (!good(ctx) || !good(keys) || keys->ctx != ctx || keys->is_share) return HE_ERR_INVALID_ARG;
     const CtxDev &d = ctx->dev;
     const size_t LN = (size_t)d.L * d.N;
     cudaStream_t st = as_stream(stream);
@@ -405,7 +413,7 @@ int he_encode(he_ctx *ctx, const float *sel_dev, size_t k, int64_t *m_dev, void 
 
 int he_encrypt_range(he_ctx *ctx, const he_keys *keys, const float *sel_dev, size_t t_begin, size_t t_count,
                      uint64_t seed, uint32_t client_id, uint64_t *ct_dev, void *stream) {
-    if (!good(ctx) || !good(keys) || keys->ctx != ctx) return HE_ERR_INVALID_ARG;
+    if (!good(ctx) || !good(keys) || keys->ctx != ctx || keys->is_share) return HE_ERR_INVALID_ARG;
     if (t_begin + t_count >= (1ull << 32)) return HE_ERR_SIZE;
     if (t_count == 0) return HE_OK;
     if (!sel_dev || !ct_dev) return HE_ERR_INVALID_ARG;
@@ -485,7 +493,7 @@ int he_plain_aggregate(he_ctx *ctx, const float *const *rests_host, const double
 
 int he_decrypt_level(he_ctx *ctx, const he_keys *keys, const uint64_t *ct_dev, uint32_t level, size_t T,
                      double *z_dev, void *stream) {
-    if (!good(ctx) || !good(keys) || keys->ctx != ctx) return HE_ERR_INVALID_ARG;
+    if (!good(ctx) || !good(keys) || keys->ctx != ctx || keys->is_share) return HE_ERR_INVALID_ARG;
     if (level < 1 || level > ctx->dev.L) return HE_ERR_LEVEL;
     if (T == 0) return HE_OK;
     if (!ct_dev || !z_dev) return HE_ERR_INVALID_ARG;
@@ -536,13 +544,99 @@ int he_ntt_inverse(he_ctx *ctx, uint64_t *polys_dev, size_t B, void *stream) {
 }
 
 // ---------------------------------------------------------------------------
+// two-party threshold decryption
+// ---------------------------------------------------------------------------
+
+int he_threshold_split(he_ctx *ctx, const he_keys *keys, uint64_t seed, he_keys **share0, he_keys **share1,
+                       void *stream) {
+    if (!good(ctx) || !good(keys) || keys->ctx != ctx || keys->is_share || !share0 || !share1)
+        return HE_ERR_INVALID_ARG;
+    *share0 = *share1 = nullptr;
+    const CtxDev &d = ctx->dev;
+    const size_t LN = (size_t)d.L * d.N;
+    cudaStream_t st = as_stream(stream);
+    void *tmp = nullptr;
+    he_keys *sh[2] = {nullptr, nullptr};
+    int rc = HE_OK;
+    do {
+        if (cudaMalloc(&tmp, 2 * LN * sizeof(uint64_t)) != cudaSuccess) { rc = HE_ERR_ALLOC; break; }
+        uint64_t *t64 = static_cast<uint64_t *>(tmp);
+        if (launch_threshold_split(d, keys->dev.s, seed, t64, st) != cudaSuccess ||
+            launch_ntt(d, true, t64, 2, LN, 0, d.L, st) != cudaSuccess) {
+            rc = HE_ERR_CUDA;
+            break;
+        }
+        for (int p = 0; p < 2 && rc == HE_OK; p++) {
+            sh[p] = new (std::nothrow) he_keys();
+            if (!sh[p]) { rc = HE_ERR_ALLOC; break; }
+            sh[p]->magic = KEYS_MAGIC;
+            sh[p]->ctx = ctx;
+            sh[p]->is_share = true;
+            sh[p]->storage = nullptr;
+            if (cudaMalloc(&sh[p]->storage, LN * sizeof(tw_t)) != cudaSuccess) { rc = HE_ERR_ALLOC; break; }
+            tw_t *tab = static_cast<tw_t *>(sh[p]->storage);
+            sh[p]->dev = KeysDev{nullptr, nullptr, tab, nullptr};
+            if (launch_share_tables(d, t64 + p * LN, tab, st) != cudaSuccess) rc = HE_ERR_CUDA;
+        }
+        if (rc == HE_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = HE_ERR_CUDA;
+    } while (0);
+    if (tmp) cudaFree(tmp);
+    if (rc != HE_OK) {
+        for (int p = 0; p < 2; p++)
+            if (sh[p]) {
+                if (sh[p]->storage) cudaFree(sh[p]->storage);
+                delete sh[p];
+            }
+        return rc;
+    }
+    *share0 = sh[0];
+    *share1 = sh[1];
+    return HE_OK;
+}
+
+int he_partial_decrypt(he_ctx *ctx, const he_keys *share, uint32_t party, const uint64_t *ct_dev, uint32_t level,
+                       size_t T, uint64_t seed, uint32_t smudge_bits, uint64_t *part_dev, void *stream) {
+    if (!good(ctx) || !good(share) || share->ctx != ctx || !share->is_share) return HE_ERR_INVALID_ARG;
+    if (level < 1 || level > ctx->dev.L) return HE_ERR_LEVEL;
+    if (smudge_bits > 40 || T >= (1ull << 32)) return HE_ERR_SIZE;
+    if (T == 0) return HE_OK;
+    if (!ct_dev || !part_dev) return HE_ERR_INVALID_ARG;
+    CU(launch_partial_decrypt(ctx->dev, share->dev, party, ct_dev, level, T, seed, smudge_bits, part_dev,
+                              as_stream(stream)));
+    return HE_OK;
+}
+
+int he_threshold_combine(he_ctx *ctx, const uint64_t *ct_dev, uint32_t level, const uint64_t *const *parts_host,
+                         int nparts, size_t T, double *z_dev, void *stream) {
+    if (!good(ctx) || !parts_host || nparts < 1) return HE_ERR_INVALID_ARG;
+    if (nparts > 8) return HE_ERR_SIZE;
+    if (level < 1 || level > ctx->dev.L) return HE_ERR_LEVEL;
+    if (T == 0) return HE_OK;
+    if (!ct_dev || !z_dev) return HE_ERR_INVALID_ARG;
+    PartPtrs pp = {};
+    for (int p = 0; p < nparts; p++) {
+        if (!parts_host[p]) return HE_ERR_INVALID_ARG;
+        pp.p[p] = parts_host[p];
+    }
+    void *ws = nullptr;
+    const int rc = ctx_workspace(ctx, T, &ws);
+    if (rc != HE_OK) return rc;
+    int64_t *d = static_cast<int64_t *>(ws);
+    double2 *cplx = reinterpret_cast<double2 *>(d + T * ctx->dev.N);
+    cudaStream_t st = as_stream(stream);
+    CU(launch_threshold_combine(ctx->dev, ct_dev, level, pp, nparts, T, d, st));
+    CU(launch_decode(ctx->dev, d, T, cplx, z_dev, st));
+    return HE_OK;
+}
+
+// ---------------------------------------------------------------------------
 // whole round from host memory
 // ---------------------------------------------------------------------------
 
 int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const float *const *xs_host,
                   const double *alpha_host, int C, size_t P, uint64_t enc_seed, double *w_glob_host,
                   void *stream) {
-    if (!good(ctx) || !good(keys) || keys->ctx != ctx || !xs_host || !alpha_host || !w_glob_host || C < 1 || P == 0)
+    if (!good(ctx) || !good(keys) || keys->ctx != ctx || keys->is_share || !xs_host || !alpha_host || !w_glob_host || C < 1 || P == 0)
         return HE_ERR_INVALID_ARG;
     if (C > HE_MAX_CLIENTS) return HE_ERR_SIZE;
     size_t k = P;

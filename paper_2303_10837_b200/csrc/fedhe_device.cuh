@@ -111,7 +111,10 @@ HD u32x4 philox4x32_10(u32x4 c, uint32_t k0, uint32_t k1) {
 
 // Stream coordinates: counter = (block, ciphertext index, client, tag | limb << 8),
 // key = the two halves of the seed.
-enum : uint32_t { TAG_SK = 1, TAG_PK_A = 2, TAG_PK_E = 3, TAG_ENC_U = 4, TAG_ENC_E0 = 5, TAG_ENC_E1 = 6 };
+enum : uint32_t {
+    TAG_SK = 1, TAG_PK_A = 2, TAG_PK_E = 3, TAG_ENC_U = 4, TAG_ENC_E0 = 5, TAG_ENC_E1 = 6,
+    TAG_SHARE = 7, TAG_SMUDGE = 8
+};
 
 HD u32x4 stream_block(uint64_t seed, uint32_t block, uint32_t t, uint32_t client, uint32_t tag_limb) {
     u32x4 c = {block, t, client, tag_limb};

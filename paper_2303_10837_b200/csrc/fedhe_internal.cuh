@@ -64,6 +64,7 @@ struct he_keys {
     he_ctx *ctx;
     fedhe::KeysDev dev;
     void *storage;
+    bool is_share = false;   // a party's share of the secret (no public key, no small secret)
 };
 
 struct he_mask {

@@ -939,6 +939,106 @@ cudaError_t launch_decrypt(const CtxDev &c, const KeysDev &k, const uint64_t *ct
 }
 
 // ===========================================================================
+// two-party threshold decryption: dealer split of the secret, partial
+// decryption with smudging noise, merge
+// ===========================================================================
+
+// tmp[0] = uniform share, tmp[1] = s - share, as residues [L][N]
+__global__ void __launch_bounds__(256)
+threshold_split_kernel(const __grid_constant__ CtxDev c, const int8_t *s8, uint64_t seed, uint64_t *tmp) {
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= c.N) return;
+    const int sv = s8[i];
+    const size_t LN = (size_t)c.L * c.N;
+    for (uint32_t j = 0; j < c.L; j++) {
+        const uint64_t q = c.limb[j].q;
+        u32x4 wa = stream_block(seed, i, 0, 0, TAG_SHARE | (j << 8));
+        const uint64_t lo = (uint64_t)wa.x | ((uint64_t)wa.y << 32), hi = (uint64_t)wa.z | ((uint64_t)wa.w << 32);
+        const uint64_t a = mod_u128(hi, lo, q);
+        tmp[(size_t)j * c.N + i] = a;
+        tmp[LN + (size_t)j * c.N + i] = submod(small_residue(sv, q), a, q);
+    }
+}
+
+__global__ void __launch_bounds__(256)
+share_tables_kernel(const __grid_constant__ CtxDev c, const uint64_t *share_hat, tw_t *s_hat) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= (size_t)c.L * c.N) return;
+    const uint64_t v = share_hat[g];
+    s_hat[g] = tw_t{v, shoup_companion(v, c.limb[g / c.N].q)};
+}
+
+// part += E (mod q_0), E uniform in [-2^bits, 2^bits): one thread per pair of coefficients
+__global__ void __launch_bounds__(256)
+partial_finish_kernel(const __grid_constant__ CtxDev c, uint32_t party, uint64_t seed, uint32_t bits,
+                      uint64_t *part, size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t pairs = c.N >> 1;
+    const uint32_t b = (uint32_t)(g % pairs);
+    const size_t t = g / pairs;
+    const uint64_t q = c.limb[0].q, mu = c.limb[0].mu;
+    u32x4 w = stream_block(seed, b, (uint32_t)t, party, TAG_SMUDGE);
+    const uint64_t r0 = (uint64_t)w.x | ((uint64_t)w.y << 32), r1 = (uint64_t)w.z | ((uint64_t)w.w << 32);
+    const int64_t e0 = (int64_t)(r0 >> (63 - bits)) - ((int64_t)1 << bits);
+    const int64_t e1 = (int64_t)(r1 >> (63 - bits)) - ((int64_t)1 << bits);
+    u64x2 *p = reinterpret_cast<u64x2 *>(part + t * c.N + 2 * (size_t)b);
+    u64x2 v = *p;
+    v.x = addmod(csub(v.x, q), signed_residue(e0, q, mu), q);
+    v.y = addmod(csub(v.y, q), signed_residue(e1, q, mu), q);
+    *p = v;
+}
+
+__global__ void __launch_bounds__(256)
+threshold_combine_kernel(const __grid_constant__ CtxDev c, const uint64_t *ct, uint32_t level,
+                         const PartPtrs parts, int nparts, int64_t *d, size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t i = (uint32_t)(g % c.N);
+    const size_t t = g / c.N;
+    const uint64_t q = c.limb[0].q;
+    uint64_t r = ct[((t * 2 + 0) * level + 0) * c.N + i];
+    for (int p = 0; p < nparts; p++) r = addmod(r, parts.p[p][g], q);
+    d[g] = r > q / 2 ? -(int64_t)(q - r) : (int64_t)r;
+}
+
+cudaError_t launch_threshold_split(const CtxDev &c, const int8_t *s8, uint64_t seed, uint64_t *tmp,
+                                   cudaStream_t s) {
+    threshold_split_kernel<<<blocks_for(c.N, 256), 256, 0, s>>>(c, s8, seed, tmp);
+    return FEDHE_LAUNCHED();
+}
+
+cudaError_t launch_share_tables(const CtxDev &c, const uint64_t *share_hat, tw_t *s_hat, cudaStream_t s) {
+    share_tables_kernel<<<blocks_for((size_t)c.L * c.N, 256), 256, 0, s>>>(c, share_hat, s_hat);
+    return FEDHE_LAUNCHED();
+}
+
+cudaError_t launch_partial_decrypt(const CtxDev &c, const KeysDev &share, uint32_t party, const uint64_t *ct,
+                                   uint32_t level, size_t T, uint64_t seed, uint32_t bits, uint64_t *part,
+                                   cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    cudaError_t e;
+    const size_t total = T * c.N;
+    dec_gather_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, ct, level, part, total);
+    if ((e = FEDHE_LAUNCHED())) return e;
+    if ((e = launch_ntt(c, true, part, T, c.N, 0, 1, s))) return e;
+    dec_pointwise_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, share, part, total);
+    if ((e = FEDHE_LAUNCHED())) return e;
+    if ((e = launch_ntt(c, false, part, T, c.N, 0, 1, s))) return e;
+    const size_t pairs = T * (c.N >> 1);
+    partial_finish_kernel<<<blocks_for(pairs, 256), 256, 0, s>>>(c, party, seed, bits, part, pairs);
+    return FEDHE_LAUNCHED();
+}
+
+cudaError_t launch_threshold_combine(const CtxDev &c, const uint64_t *ct, uint32_t level, const PartPtrs &parts,
+                                     int nparts, size_t T, int64_t *d, cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    const size_t total = T * c.N;
+    threshold_combine_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, ct, level, parts, nparts, d, total);
+    return FEDHE_LAUNCHED();
+}
+
+// ===========================================================================
 // selective-encryption mask
 // ===========================================================================
 

@@ -42,6 +42,21 @@ cudaError_t launch_plain_aggregate(const float *const *ptrs, const double *alpha
 cudaError_t launch_decrypt(const CtxDev &c, const KeysDev &k, const uint64_t *ct, uint32_t level,
                            size_t T, uint64_t *scratch, cudaStream_t s);
 
+// two-party threshold decryption.  tmp: uint64 [2][L][N] (shares as residues)
+cudaError_t launch_threshold_split(const CtxDev &c, const int8_t *s8, uint64_t seed, uint64_t *tmp,
+                                   cudaStream_t s);
+cudaError_t launch_share_tables(const CtxDev &c, const uint64_t *share_hat, tw_t *s_hat, cudaStream_t s);
+// part: uint64 [T][N], work space and result (canonical residues mod q_0)
+cudaError_t launch_partial_decrypt(const CtxDev &c, const KeysDev &share, uint32_t party, const uint64_t *ct,
+                                   uint32_t level, size_t T, uint64_t seed, uint32_t bits, uint64_t *part,
+                                   cudaStream_t s);
+struct PartPtrs { const uint64_t *p[8]; };
+cudaError_t launch_threshold_combine(const CtxDev &c, const uint64_t *ct, uint32_t level, const PartPtrs &parts,
+                                     int nparts, size_t T, int64_t *d, cudaStream_t s);
+
+// context-owned work space for T ciphertexts (2 * T * N words); implemented in fedhe_api.cu
+int ctx_workspace(he_ctx *ctx, size_t T, void **out);
+
 // mask construction (blocks of MASK_BLOCK consecutive parameters)
 constexpr uint32_t MASK_BLOCK = 1024;
 cudaError_t launch_key_histogram(const float *score, size_t P, uint32_t prefix, int prefix_bits,

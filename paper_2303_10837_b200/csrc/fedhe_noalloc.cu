@@ -49,7 +49,8 @@ int scratch_for_current_device(uint64_t **out) {
 
 extern "C" int he_decrypt_noalloc(he_ctx *ctx, const he_keys *keys, const uint64_t *agg_dev, size_t T,
                                   double *z_dev, void *stream) {
-    if (!ctx || ctx->magic != CTX_MAGIC || !keys || keys->magic != KEYS_MAGIC || keys->ctx != ctx)
+    if (!ctx || ctx->magic != CTX_MAGIC || !keys || keys->magic != KEYS_MAGIC || keys->ctx != ctx ||
+        keys->is_share)
         return HE_ERR_INVALID_ARG;
     const CtxDev &d = ctx->dev;
     int dev = -1;

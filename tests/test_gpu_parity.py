@@ -362,3 +362,39 @@ def test_sensitivity_map_round(he):
     # the mask agrees with the one a plaintext aggregation would give, except at the noise-level boundary
     plain = oracle.select_mask(want.astype(np.float32), k)
     assert np.intersect1d(got, plain).size >= 0.999 * k
+
+
+@pytest.mark.parametrize("w", [si.scaled(si.TINY, 4096 + 50, name="thr-tiny"),
+                               si.scaled(si.bert(1.0), 16384 + 9, clients=2, name="thr-bert")],
+                         ids=lambda w: w.name)
+def test_threshold_decryption_bit_exact(he, w):
+    """Two-party threshold decryption: partial results bit-exact against the oracle, merged result
+    within the decode tolerance, and close to FedAvg up to the smudging noise."""
+    g, o = contexts(he, w.N, w.primes, w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    s_o, pk_o = o.keygen(w.key_seed)
+    xs, alpha = si.client_updates(w), si.client_weights(w)
+    cts = [he.he_encrypt(g, keys, he.he_pack(g, None, dev_f32(x))[0], w.enc_seed, i) for i, x in enumerate(xs)]
+    agg = he.he_weighted_aggregate(g, cts, alpha)
+    agg_o = to_host_u64(agg)
+    level, bits, seed = w.L - 1, 10, 777
+    shares = he.he_threshold_split(g, keys, 31)
+    shares_o = o.threshold_split(s_o, 31)
+    parts = [he.he_partial_decrypt(g, shares[p], p, agg, level, seed, bits) for p in range(2)]
+    T = agg.shape[0]
+    d_o = np.empty((T, w.N), np.int64)
+    for t in range(T):
+        po = [o.partial_decrypt(shares_o[p], p, agg_o[t], level, seed, t, bits) for p in range(2)]
+        for p in range(2):
+            assert np.array_equal(to_host_u64(parts[p][t]), po[p]), (t, p)
+        d_o[t] = o.threshold_combine(agg_o[t], level, po)
+    z = he.he_threshold_combine(g, agg, level, parts).cpu().numpy()
+    assert np.abs(z - o.decode(d_o).reshape(-1)).max() <= DECODE_TOL
+    want = sum(a * x.astype(np.float64) for a, x in zip(alpha, xs))
+    assert np.abs(z[: w.P] - want).max() <= 1e-5           # 2^10 of smudging per coefficient and party
+    # shares are not keys: the single-key entry points refuse them
+    for bad in (lambda: he.he_decrypt(g, shares[0], agg), lambda: he.he_keys_export(g, shares[0]),
+                lambda: he.he_partial_decrypt(g, keys, 0, agg, level, seed, bits)):
+        with pytest.raises(he.HeError) as ei:
+            bad()
+        assert ei.value.code == he.HE_ERR_INVALID_ARG
