@@ -588,51 +588,61 @@ cudaError_t launch_decode(const CtxDev &c, const int64_t *d, size_t T, double2 *
 // encryption:  c0 = pk0 u + e0 + m,  c1 = pk1 u + e1   (mod every q_j)
 // ===========================================================================
 
-// Fused path for N <= 2^14 (one block holds a whole limb): one thread block
-// per ciphertext draws u, e0, e1 once into shared memory, then for every limb
-// transforms u, multiplies by both halves of the public key, transforms back
-// and adds the error (and message) terms.  Only the ciphertext itself is
-// written to global memory; the second product waits, in transform order, in
-// the c1 slot it will finally occupy.
+// Fused path for N <= 2^14 (one block holds a whole limb): a thread block
+// draws u, e0, e1 of a ciphertext once into shared memory, then for every
+// limb of it transforms u, multiplies by both halves of the public key,
+// transforms back and adds the error (and message) terms.  Only the
+// ciphertext itself is written to global memory; the second product waits,
+// in transform order, in the c1 slot it will finally occupy.
 template <class L, int V>
 __global__ void __launch_bounds__(L::NT / V, 1)
 encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const int64_t *m, uint32_t t0,
-                     uint64_t seed, uint32_t client, uint64_t *ct) {
+                     uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
     extern __shared__ __align__(16) uint64_t sm[];
     constexpr uint32_t B = 1u << L::LOGB, RT = L::NT / V;
     int8_t *su = reinterpret_cast<int8_t *>(sm + B);
     int8_t *se0 = su + B, *se1 = se0 + B;
     const uint32_t tid = threadIdx.x;
-    const size_t tl = blockIdx.x;            // ciphertext within this call
-    const uint32_t t = t0 + (uint32_t)tl;    // stream coordinate
     __shared__ GaussTables gt;
     gauss_tables_init(gt, tid);
-    __syncthreads();
 
-    for (uint32_t b = tid; b < B / 4; b += RT) {
-        u32x4 w = stream_block(seed, b, t, client, TAG_ENC_U);
-        char4 v = make_char4((signed char)ternary_from_word(w.x), (signed char)ternary_from_word(w.y),
-                             (signed char)ternary_from_word(w.z), (signed char)ternary_from_word(w.w));
-        reinterpret_cast<char4 *>(su)[b] = v;
-    }
-    for (uint32_t b = tid; b < B / 2; b += RT) {
-        u32x4 w0 = stream_block(seed, b, t, client, TAG_ENC_E0);
-        u32x4 w1 = stream_block(seed, b, t, client, TAG_ENC_E1);
-        char2 a = make_char2((signed char)gauss_from_u64(gt, (uint64_t)w0.x | ((uint64_t)w0.y << 32)),
-                             (signed char)gauss_from_u64(gt, (uint64_t)w0.z | ((uint64_t)w0.w << 32)));
-        char2 e = make_char2((signed char)gauss_from_u64(gt, (uint64_t)w1.x | ((uint64_t)w1.y << 32)),
-                             (signed char)gauss_from_u64(gt, (uint64_t)w1.z | ((uint64_t)w1.w << 32)));
-        reinterpret_cast<char2 *>(se0)[b] = a;
-        reinterpret_cast<char2 *>(se1)[b] = e;
-    }
-    __syncthreads();
-
-    const int64_t *mt = m + tl * B;
+    // Work units are (ciphertext, limb) pairs in ciphertext-major order, dealt
+    // evenly to the blocks of the grid (one block per SM), so that the last
+    // wave is as full as the others; a block re-draws u, e0, e1 whenever its
+    // range moves on to the next ciphertext.
+    const uint64_t units = (uint64_t)T * c.L;
+    const uint32_t u_begin = (uint32_t)(units * blockIdx.x / gridDim.x);
+    const uint32_t u_end = (uint32_t)(units * (blockIdx.x + 1) / gridDim.x);
     const size_t cstride = (size_t)c.L * B;          // from c0 to c1 of the same limb
-    for (uint32_t j = 0; j < c.L; j++) {
+    uint32_t sampled = 0xffffffffu;
+    for (uint32_t unit = u_begin; unit < u_end; unit++) {
+        const uint32_t tl = unit / c.L, j = unit % c.L;   // ciphertext within this call, limb
+        if (tl != sampled) {
+            sampled = tl;
+            const uint32_t t = t0 + tl;                   // stream coordinate
+            __syncthreads();                              // tables ready / previous samples no longer read
+            for (uint32_t b = tid; b < B / 4; b += RT) {
+                u32x4 w = stream_block(seed, b, t, client, TAG_ENC_U);
+                char4 v = make_char4((signed char)ternary_from_word(w.x), (signed char)ternary_from_word(w.y),
+                                     (signed char)ternary_from_word(w.z), (signed char)ternary_from_word(w.w));
+                reinterpret_cast<char4 *>(su)[b] = v;
+            }
+            for (uint32_t b = tid; b < B / 2; b += RT) {
+                u32x4 w0 = stream_block(seed, b, t, client, TAG_ENC_E0);
+                u32x4 w1 = stream_block(seed, b, t, client, TAG_ENC_E1);
+                char2 a = make_char2((signed char)gauss_from_u64(gt, (uint64_t)w0.x | ((uint64_t)w0.y << 32)),
+                                     (signed char)gauss_from_u64(gt, (uint64_t)w0.z | ((uint64_t)w0.w << 32)));
+                char2 e = make_char2((signed char)gauss_from_u64(gt, (uint64_t)w1.x | ((uint64_t)w1.y << 32)),
+                                     (signed char)gauss_from_u64(gt, (uint64_t)w1.z | ((uint64_t)w1.w << 32)));
+                reinterpret_cast<char2 *>(se0)[b] = a;
+                reinterpret_cast<char2 *>(se1)[b] = e;
+            }
+            __syncthreads();
+        }
+        const int64_t *mt = m + (size_t)tl * B;
         const LimbDev &lb = c.limb[j];
         const uint64_t q = lb.q, q2 = 2 * q;
-        uint64_t *cbase = ct + ((tl * 2 + 0) * c.L + j) * B;
+        uint64_t *cbase = ct + (((size_t)tl * 2 + 0) * c.L + j) * B;
         {
             const tw_t *p0 = k.pk0_hat + (size_t)j * B, *p1 = k.pk1_hat + (size_t)j * B;
             uint64_t *c1 = cbase + cstride;
@@ -756,7 +766,13 @@ static cudaError_t launch_encrypt_fused(const CtxDev &c, const KeysDev &k, const
     auto kern = encrypt_fused_kernel<L, V>;
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-    kern<<<(unsigned)T, L::NT / V, smem, s>>>(c, k, m, t0, seed, client, ct);
+    // one block per SM (the kernel's shared memory allows no more), fewer if there is less work
+    int dev = 0, n_sm = 0;
+    if ((e = cudaGetDevice(&dev)) || (e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev))) return e;
+    const size_t per_sm = (size_t)(227 * 1024) / smem;               // blocks that fit one SM
+    size_t grid = (size_t)n_sm * (per_sm ? per_sm : 1);
+    if (grid > T * c.L) grid = T * c.L;
+    kern<<<(unsigned)grid, L::NT / V, smem, s>>>(c, k, m, t0, seed, client, ct, (uint32_t)T);
     return FEDHE_LAUNCHED();
 }
 
