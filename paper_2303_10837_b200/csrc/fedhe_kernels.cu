@@ -677,9 +677,10 @@ encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const in
                     return *reinterpret_cast<const u64x2 *>(cc + p);
                 },
                 [&](uint32_t i, uint64_t v) {
-                    int64_t add = (int64_t)se[i];
-                    if (h == 0) add += mt[i];
-                    cc[i] = addmod(csub(v, q), signed_residue(add, q, lb.mu), q);
+                    // e1 is a small value; e0 + m needs a full reduction
+                    const uint64_t add = h == 0 ? signed_residue(mt[i] + (int64_t)se[i], q, lb.mu)
+                                                : small_residue(se[i], q);
+                    cc[i] = addmod(csub(v, q), add, q);
                 });
             __syncthreads();   // phase-0 readers are done before the next transform writes
         }
