@@ -102,7 +102,7 @@ __device__ uint64_t shoup_companion(uint64_t w, uint64_t q) {   // floor(w 2^64 
 // N <= 2^14), transformed in place in shared memory; every thread plays V
 // virtual threads per phase with E residues in registers at a time.
 template <class L, int V, bool FWD, bool SCALED>
-__global__ void __launch_bounds__(L::NT / V, 1)
+__global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
 ntt_block_kernel(const __grid_constant__ CtxDev c, uint64_t *data, size_t poly_stride, uint32_t limb0,
                          uint32_t nlimbs) {
     extern __shared__ __align__(16) uint64_t sm[];
@@ -687,6 +687,122 @@ encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const in
     }
 }
 
+// The same for N = 2 * 2^LOGB (N = 2^14 with LOGB = 13): the thread block is
+// two groups of threads, each of which transforms one half of the limb as a
+// sub-block of the long transform on its own schedule (named barriers), so
+// that one group's barrier and memory waits overlap the other's arithmetic.
+// The stage that pairs the two halves is done where both are at hand: on the
+// way in for the forward transform (u is ternary, so the twiddle product is
+// 0, w or q-w, computed by both groups from the shared samples) and by the
+// whole block after the two inverse sub-transforms, fused with the epilogue.
+template <class L, int V>
+__global__ void __launch_bounds__(2 * L::NT / V, 1)
+encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const int64_t *m, uint32_t t0,
+                      uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
+    extern __shared__ __align__(16) uint64_t sm[];
+    constexpr uint32_t H = 1u << L::LOGB, B = 2 * H;       // half and whole limb
+    constexpr uint32_t GT = L::NT / V, RT = 2 * GT;        // threads per group, per block
+    int8_t *su = reinterpret_cast<int8_t *>(sm + B);
+    int8_t *se0 = su + B, *se1 = se0 + B;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t grp = tid / GT, gt = tid % GT;
+    uint64_t *smg = sm + grp * H;                          // this group's half
+    const GroupSync gsync = {1 + grp, GT};
+    __shared__ GaussTables gt_tab;
+    gauss_tables_init(gt_tab, tid);
+
+    const uint64_t units = (uint64_t)T * c.L;
+    const uint32_t u_begin = (uint32_t)(units * blockIdx.x / gridDim.x);
+    const uint32_t u_end = (uint32_t)(units * (blockIdx.x + 1) / gridDim.x);
+    const size_t cstride = (size_t)c.L * B;
+    uint32_t sampled = 0xffffffffu;
+    for (uint32_t unit = u_begin; unit < u_end; unit++) {
+        const uint32_t tl = unit / c.L, j = unit % c.L;
+        if (tl != sampled) {
+            sampled = tl;
+            const uint32_t t = t0 + tl;
+            __syncthreads();
+            for (uint32_t b = tid; b < B / 4; b += RT) {
+                u32x4 w = stream_block(seed, b, t, client, TAG_ENC_U);
+                char4 v = make_char4((signed char)ternary_from_word(w.x), (signed char)ternary_from_word(w.y),
+                                     (signed char)ternary_from_word(w.z), (signed char)ternary_from_word(w.w));
+                reinterpret_cast<char4 *>(su)[b] = v;
+            }
+            for (uint32_t b = tid; b < B / 2; b += RT) {
+                u32x4 w0 = stream_block(seed, b, t, client, TAG_ENC_E0);
+                u32x4 w1 = stream_block(seed, b, t, client, TAG_ENC_E1);
+                char2 a = make_char2((signed char)gauss_from_u64(gt_tab, (uint64_t)w0.x | ((uint64_t)w0.y << 32)),
+                                     (signed char)gauss_from_u64(gt_tab, (uint64_t)w0.z | ((uint64_t)w0.w << 32)));
+                char2 e = make_char2((signed char)gauss_from_u64(gt_tab, (uint64_t)w1.x | ((uint64_t)w1.y << 32)),
+                                     (signed char)gauss_from_u64(gt_tab, (uint64_t)w1.z | ((uint64_t)w1.w << 32)));
+                reinterpret_cast<char2 *>(se0)[b] = a;
+                reinterpret_cast<char2 *>(se1)[b] = e;
+            }
+            __syncthreads();
+        }
+        const int64_t *mt = m + (size_t)tl * B;
+        const LimbDev &lb = c.limb[j];
+        const uint64_t q = lb.q, q2 = 2 * q;
+        uint64_t *cbase = ct + (((size_t)tl * 2 + 0) * c.L + j) * B;
+        {
+            const tw_t *p0 = k.pk0_hat + (size_t)j * B + grp * H, *p1 = k.pk1_hat + (size_t)j * B + grp * H;
+            uint64_t *c1 = cbase + cstride + grp * H;
+            const uint64_t w0 = load_tw(lb.fwd + 1).w;     // twiddle of the stage that pairs the halves
+            const NttArgs fa = {lb.fwd, q, q2, 1, grp};
+            smem_ntt_forward<L, V>(
+                smg, gt, fa,
+                [&](uint32_t i) {
+                    const int b = su[i + H];
+                    const uint64_t u = small_residue(su[i], q);
+                    const uint64_t v = b == 0 ? 0 : (b > 0 ? w0 : q - w0);
+                    return grp == 0 ? u + v : u - v + q2;
+                },
+                [&](uint32_t p, uint64_t a, uint64_t b) {
+                    const tw_t a0 = load_tw(p1 + p), a1 = load_tw(p1 + p + 1);
+                    u64x2 v;
+                    v.x = shoup_lazy(a, a0.w, a0.wp, q);
+                    v.y = shoup_lazy(b, a1.w, a1.wp, q);
+                    *reinterpret_cast<u64x2 *>(c1 + p) = v;      // parked until the second pass
+                    const tw_t b0 = load_tw(p0 + p), b1 = load_tw(p0 + p + 1);
+                    smg[swz(p)] = shoup_lazy(a, b0.w, b0.wp, q);
+                    smg[swz(p + 1)] = shoup_lazy(b, b1.w, b1.wp, q);
+                },
+                gsync);
+        }
+#pragma unroll 1
+        for (int h = 0; h < 2; h++) {
+            uint64_t *cc = cbase + h * cstride;
+            const int8_t *se = se0 + h * B;
+            const NttArgs ia = {lb.inv, q, q2, 1, grp};
+            smem_ntt_inverse<L, V, false>(
+                smg, gt, ia, lb.ninv, lb.wn,
+                [&](uint32_t p) {
+                    if (h == 0) return u64x2{smg[swz(p)], smg[swz(p + 1)]};
+                    return *reinterpret_cast<const u64x2 *>(cc + grp * H + p);
+                },
+                [&](uint32_t i, uint64_t v) { smg[swz(i)] = v; }, gsync);
+            __syncthreads();
+            // last stage across the halves with 1/N folded in, then the error / message terms
+            for (uint32_t e = tid; e < H; e += RT) {
+                const uint64_t a = sm[swz(e)], b = sm[H + swz(e)];
+                const uint64_t lo = shoup(a + b, lb.ninv.w, lb.ninv.wp, q);
+                const uint64_t hi = shoup(a - b + q2, lb.wn.w, lb.wn.wp, q);
+                uint64_t add_lo, add_hi;
+                if (h == 0) {
+                    add_lo = signed_residue(mt[e] + (int64_t)se[e], q, lb.mu);
+                    add_hi = signed_residue(mt[e + H] + (int64_t)se[e + H], q, lb.mu);
+                } else {
+                    add_lo = small_residue(se[e], q);
+                    add_hi = small_residue(se[e + H], q);
+                }
+                cc[e] = addmod(lo, add_lo, q);
+                cc[e + H] = addmod(hi, add_hi, q);
+            }
+            __syncthreads();
+        }
+    }
+}
+
 // General path (any N): three elementwise kernels around the batched
 // transforms, with the ciphertext buffer itself as the only work space.
 
@@ -759,12 +875,12 @@ enc_add_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint32_t t0, 
     }
 }
 
-template <class L, int V>
+template <class L, int V, bool TWO_GROUPS>
 static cudaError_t launch_encrypt_fused(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0,
                                         size_t T, uint64_t seed, uint32_t client, uint64_t *ct,
                                         cudaStream_t s) {
-    const size_t smem = (sizeof(uint64_t) << L::LOGB) + (3u << L::LOGB);
-    auto kern = encrypt_fused_kernel<L, V>;
+    const size_t smem = ((sizeof(uint64_t) << L::LOGB) + (3u << L::LOGB)) * (TWO_GROUPS ? 2 : 1);
+    auto kern = TWO_GROUPS ? encrypt_fused2_kernel<L, V> : encrypt_fused_kernel<L, V>;
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
     // one block per SM (the kernel's shared memory allows no more), fewer if there is less work
@@ -773,7 +889,7 @@ static cudaError_t launch_encrypt_fused(const CtxDev &c, const KeysDev &k, const
     const size_t per_sm = (size_t)(227 * 1024) / smem;               // blocks that fit one SM
     size_t grid = (size_t)n_sm * (per_sm ? per_sm : 1);
     if (grid > T * c.L) grid = T * c.L;
-    kern<<<(unsigned)grid, L::NT / V, smem, s>>>(c, k, m, t0, seed, client, ct, (uint32_t)T);
+    kern<<<(unsigned)grid, (TWO_GROUPS ? 2 : 1) * L::NT / V, smem, s>>>(c, k, m, t0, seed, client, ct, (uint32_t)T);
     return FEDHE_LAUNCHED();
 }
 
@@ -781,8 +897,8 @@ cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const int64_t *m, 
                            uint64_t seed, uint32_t client, uint64_t *ct, cudaStream_t s) {
     if (T == 0) return cudaSuccess;
     if (c.A == 0) {
-        if (c.LOGB == 13) return launch_encrypt_fused<Lay<13, 3>, 2>(c, k, m, t0, T, seed, client, ct, s);
-        return launch_encrypt_fused<Lay<14, 3>, 2>(c, k, m, t0, T, seed, client, ct, s);
+        if (c.LOGB == 13) return launch_encrypt_fused<Lay<13, 3>, 2, false>(c, k, m, t0, T, seed, client, ct, s);
+        return launch_encrypt_fused<Lay<13, 3>, 2, true>(c, k, m, t0, T, seed, client, ct, s);
     }
     cudaError_t e;
     const size_t ctw = 2 * (size_t)c.L * c.N;

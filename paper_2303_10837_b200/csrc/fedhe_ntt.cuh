@@ -169,9 +169,22 @@ HD void inv_phase(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
 // (pairs always start at an even index and are neighbours in memory).
 // ---------------------------------------------------------------------------
 
-template <class L, int V, class Src, class Dst, int P = 0>
+// Barrier over the whole thread block, or over one of its halves / quarters
+// when several groups of threads transform separate sub-blocks on their own
+// schedules (named barrier 1 + group; every thread of the group must call it).
+struct BlockSync {
+    __device__ __forceinline__ void operator()() const { __syncthreads(); }
+};
+struct GroupSync {
+    uint32_t id, nthreads;
+    __device__ __forceinline__ void operator()() const {
+        asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+    }
+};
+
+template <class L, int V, class Src, class Dst, class Sync = BlockSync, int P = 0>
 __device__ __forceinline__ void smem_ntt_forward(uint64_t *sm, uint32_t tid, const NttArgs &a, const Src &src,
-                                                 const Dst &dst) {
+                                                 const Dst &dst, const Sync &sync = Sync()) {
     constexpr int RT = L::NT / V, LAST = L::NPH - 1;
 #pragma unroll 1
     for (int v = 0; v < V; v++) {
@@ -193,14 +206,15 @@ __device__ __forceinline__ void smem_ntt_forward(uint64_t *sm, uint32_t tid, con
         }
     }
     if constexpr (P < LAST) {
-        __syncthreads();
-        smem_ntt_forward<L, V, Src, Dst, P + 1>(sm, tid, a, src, dst);
+        sync();
+        smem_ntt_forward<L, V, Src, Dst, Sync, P + 1>(sm, tid, a, src, dst, sync);
     }
 }
 
-template <class L, int V, bool SCALED, class Src, class Dst, int P = L::NPH - 1>
+template <class L, int V, bool SCALED, class Src, class Dst, class Sync = BlockSync, int P = L::NPH - 1>
 __device__ __forceinline__ void smem_ntt_inverse(uint64_t *sm, uint32_t tid, const NttArgs &a, tw_t ninv,
-                                                 tw_t wn, const Src &src, const Dst &dst) {
+                                                 tw_t wn, const Src &src, const Dst &dst,
+                                                 const Sync &sync = Sync()) {
     constexpr int RT = L::NT / V, LAST = L::NPH - 1;
 #pragma unroll 1
     for (int v = 0; v < V; v++) {
@@ -232,8 +246,8 @@ __device__ __forceinline__ void smem_ntt_inverse(uint64_t *sm, uint32_t tid, con
         }
     }
     if constexpr (P > 0) {
-        __syncthreads();
-        smem_ntt_inverse<L, V, SCALED, Src, Dst, P - 1>(sm, tid, a, ninv, wn, src, dst);
+        sync();
+        smem_ntt_inverse<L, V, SCALED, Src, Dst, Sync, P - 1>(sm, tid, a, ninv, wn, src, dst, sync);
     }
 }
 #endif
