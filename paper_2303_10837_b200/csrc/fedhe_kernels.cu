@@ -595,7 +595,7 @@ cudaError_t launch_decode(const CtxDev &c, const int64_t *d, size_t T, double2 *
 // ciphertext itself is written to global memory; the second product waits,
 // in transform order, in the c1 slot it will finally occupy.
 template <class L, int V>
-__global__ void __launch_bounds__(L::NT / V, 1)
+__global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
 encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const int64_t *m, uint32_t t0,
                      uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
     extern __shared__ __align__(16) uint64_t sm[];
