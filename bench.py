@@ -46,8 +46,8 @@ UNIT = "params/s"
 # 6 wide + 4 narrow = 19 multiply slots.  Additions go to another pipe.
 # DRAM bytes (read + write) per ciphertext of encrypt_fused_kernel at N = 16384,
 # L = 4, from the ncu capture in profiles/encrypt_fused_kernel_resnet18_296cts.md
-# (480.1 MB for 296 ciphertexts; traffic grows in proportion to the count).
-ENCRYPT_DRAM_BYTES_PER_CT_N16384_L4 = 480.087552e6 / 296
+# (363.6 MB for 296 ciphertexts; traffic grows in proportion to the count).
+ENCRYPT_DRAM_BYTES_PER_CT_N16384_L4 = 363.57248e6 / 296
 IMAD_PER_SM_CLK = 64.0
 WIDE_COST = 2.5
 MUL_SLOTS_PER_BUTTERFLY = 6 * WIDE_COST + 4
