@@ -427,14 +427,27 @@ encode_block_kernel(const __grid_constant__ CtxDev c, const float *sel, const do
     const double lim = 4611686018427387904.0;   // 2^62
     int64_t *mt = m + t * c.N;
     bool bad = false;
+    // The bit-reversed order would scatter 8-byte writes over the whole
+    // polynomial: the rounded integers go through shared memory (real parts
+    // in the first half, imaginary parts in the second) and leave in order.
+    int64_t *stage = reinterpret_cast<int64_t *>(smraw);
+    constexpr uint32_t NB = 1u << L::LOGB;
+    __syncthreads();                                   // the exchange buffer is free again
 #pragma unroll
     for (int r = 0; r < L::E; r++) {
-        const uint32_t p = (blk << L::LOGB) | L::template idx<L::NPH - 1>(tid, r);
-        const uint32_t k = bitrev(p, logn);
+        const uint32_t kk = bitrev(L::template idx<L::NPH - 1>(tid, r), L::LOGB);
         double re = __dmul_rn(x[r].re, scale), im = __dmul_rn(x[r].im, scale);
         if (!(fabs(re) < lim) || !(fabs(im) < lim)) { bad = true; re = 0.0; im = 0.0; }
-        mt[k] = __double2ll_rn(re);
-        mt[k + n] = __double2ll_rn(im);
+        stage[kk] = __double2ll_rn(re);
+        stage[NB + kk] = __double2ll_rn(im);
+    }
+    __syncthreads();
+    // slot k of the whole transform = (local bit-reversed index, bit-reversed block number)
+    const uint32_t A = logn - L::LOGB, rb = A ? bitrev(blk, A) : 0u;
+    for (uint32_t kk = tid; kk < NB; kk += L::NT) {
+        const uint32_t k = (kk << A) | rb;
+        mt[k] = stage[kk];
+        mt[k + n] = stage[NB + kk];
     }
     if (bad) atomicOr(c.status, 1);
 }
