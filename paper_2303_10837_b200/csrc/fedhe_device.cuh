@@ -27,14 +27,53 @@ HD uint64_t mulhi64(uint64_t a, uint64_t b) {
 #endif
 }
 
-// x - m if x >= m
-HD uint64_t csub(uint64_t x, uint64_t m) { return x >= m ? x - m : x; }
+// 64-bit add / subtract / conditional subtract.  On the device they are
+// written as 32-bit carry chains: left to itself the compiler puts the high
+// halves of 64-bit additions on the integer multiply-add pipe, which is the
+// pipe the transforms saturate; carry chains stay on the plain ALU pipe
+// (measured: +9 % butterflies per clock).
+HD uint64_t add64(uint64_t a, uint64_t b) {
+#if defined(__CUDA_ARCH__)
+    uint32_t rl, rh;
+    asm("add.cc.u32 %0, %2, %4; addc.u32 %1, %3, %5;"
+        : "=r"(rl), "=r"(rh)
+        : "r"((uint32_t)a), "r"((uint32_t)(a >> 32)), "r"((uint32_t)b), "r"((uint32_t)(b >> 32)));
+    return ((uint64_t)rh << 32) | rl;
+#else
+    return a + b;
+#endif
+}
+
+HD uint64_t sub64(uint64_t a, uint64_t b) {
+#if defined(__CUDA_ARCH__)
+    uint32_t rl, rh;
+    asm("sub.cc.u32 %0, %2, %4; subc.u32 %1, %3, %5;"
+        : "=r"(rl), "=r"(rh)
+        : "r"((uint32_t)a), "r"((uint32_t)(a >> 32)), "r"((uint32_t)b), "r"((uint32_t)(b >> 32)));
+    return ((uint64_t)rh << 32) | rl;
+#else
+    return a - b;
+#endif
+}
+
+// x - m if x >= m (the borrow of x - m decides)
+HD uint64_t csub(uint64_t x, uint64_t m) {
+#if defined(__CUDA_ARCH__)
+    uint32_t rl, rh, borrow;
+    asm("sub.cc.u32 %0, %3, %5; subc.cc.u32 %1, %4, %6; subc.u32 %2, 0, 0;"
+        : "=r"(rl), "=r"(rh), "=r"(borrow)
+        : "r"((uint32_t)x), "r"((uint32_t)(x >> 32)), "r"((uint32_t)m), "r"((uint32_t)(m >> 32)));
+    return borrow ? x : (((uint64_t)rh << 32) | rl);
+#else
+    return x >= m ? x - m : x;
+#endif
+}
 
 // Shoup product with a fixed operand w < q and wp = floor(w 2^64 / q):
 // returns x w mod q up to one extra q, i.e. a value in [0, 2q), for any x.
 HD uint64_t shoup_lazy(uint64_t x, uint64_t w, uint64_t wp, uint64_t q) {
     uint64_t hi = mulhi64(x, wp);
-    return x * w - hi * q;
+    return sub64(x * w, hi * q);
 }
 
 HD uint64_t shoup(uint64_t x, uint64_t w, uint64_t wp, uint64_t q) {
@@ -63,15 +102,15 @@ HD uint64_t small_residue(int v, uint64_t q) { return v < 0 ? q - (uint64_t)(-v)
 HD void ct_butterfly(uint64_t &x, uint64_t &y, uint64_t w, uint64_t wp, uint64_t q, uint64_t q2) {
     uint64_t u = csub(x, q2);
     uint64_t v = shoup_lazy(y, w, wp, q);
-    x = u + v;
-    y = u - v + q2;
+    x = add64(u, v);
+    y = add64(sub64(u, v), q2);
 }
 
 // Inverse (Gentleman-Sande): inputs and outputs in [0, 2q).
 HD void gs_butterfly(uint64_t &x, uint64_t &y, uint64_t w, uint64_t wp, uint64_t q, uint64_t q2) {
     uint64_t u = x, v = y;
-    x = csub(u + v, q2);
-    y = shoup_lazy(u - v + q2, w, wp, q);
+    x = csub(add64(u, v), q2);
+    y = shoup_lazy(add64(sub64(u, v), q2), w, wp, q);
 }
 
 // ---------------------------------------------------------------------------
