@@ -100,7 +100,7 @@ int he_ctx_create(const he_params *p, he_ctx **out) {
         d.L = p->L;
         d.log2_delta = p->log2_delta;
         while ((1u << d.logN) < d.N) d.logN++;
-        d.LOGB = d.logN < 14 ? d.logN : 14;
+        d.LOGB = d.logN <= 14 ? d.logN : 13;   // longer transforms: 2^13 blocks, two per SM
         d.A = d.logN - d.LOGB;
         const uint64_t ql = p->q[p->L - 1];
         for (uint32_t j = 0; j < p->L && rc == HE_OK; j++) {

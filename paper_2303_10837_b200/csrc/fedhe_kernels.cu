@@ -150,8 +150,8 @@ ntt_outer_kernel(const __grid_constant__ CtxDev c, uint64_t *data, size_t poly_s
     const LimbDev &lb = c.limb[limb0 + limb];
     const uint64_t q = lb.q, q2 = 2 * q;
     uint64_t *p = data + poly * poly_stride + (size_t)limb * c.N + col;
-    const uint32_t A = c.A, rows = 1u << A;      // A is 1 or 2
-    u64x2 x[4];
+    const uint32_t A = c.A, rows = 1u << A;      // A is 1, 2 or 3
+    u64x2 x[8];
     for (uint32_t a = 0; a < rows; a++) x[a] = *reinterpret_cast<const u64x2 *>(p + (size_t)a * B);
     if (FWD) {
         for (uint32_t s = 0; s < A; s++) {
