@@ -395,6 +395,10 @@ __device__ __forceinline__ void block_dit(cpx (&x)[L::E], cpx *sm, uint32_t tid,
 }
 
 __device__ __forceinline__ uint32_t bitrev(uint32_t v, int bits) { return __brev(v) >> (32 - bits); }
+// index swizzle of the encoder's output staging buffer: bit-reversed writes of
+// a warp differ only in high index bits; folding them into the low nibble
+// spreads them over the banks (checked exhaustively for both block sizes)
+__device__ __forceinline__ uint32_t stage_swz(uint32_t k) { return k ^ (((k >> 8) ^ (k >> 4)) & 15u); }
 
 // Block part of the encoder: the last LOGB stages on one block of 2^LOGB
 // slots, the bit-reversal, the scaling by Delta/n and the rounding.
@@ -438,16 +442,16 @@ encode_block_kernel(const __grid_constant__ CtxDev c, const float *sel, const do
         const uint32_t kk = bitrev(L::template idx<L::NPH - 1>(tid, r), L::LOGB);
         double re = __dmul_rn(x[r].re, scale), im = __dmul_rn(x[r].im, scale);
         if (!(fabs(re) < lim) || !(fabs(im) < lim)) { bad = true; re = 0.0; im = 0.0; }
-        stage[kk] = __double2ll_rn(re);
-        stage[NB + kk] = __double2ll_rn(im);
+        stage[stage_swz(kk)] = __double2ll_rn(re);
+        stage[NB + stage_swz(kk)] = __double2ll_rn(im);
     }
     __syncthreads();
     // slot k of the whole transform = (local bit-reversed index, bit-reversed block number)
     const uint32_t A = logn - L::LOGB, rb = A ? bitrev(blk, A) : 0u;
     for (uint32_t kk = tid; kk < NB; kk += L::NT) {
         const uint32_t k = (kk << A) | rb;
-        mt[k] = stage[kk];
-        mt[k + n] = stage[NB + kk];
+        mt[k] = stage[stage_swz(kk)];
+        mt[k + n] = stage[NB + stage_swz(kk)];
     }
     if (bad) atomicOr(c.status, 1);
 }
