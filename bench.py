@@ -40,12 +40,12 @@ UNIT = "params/s"
 # Integer roofline of the transforms.  On B200 every integer multiply goes
 # through one pipe that retires 64 32-bit multiply-adds per SM and clock
 # (measured: 63.8), and a 32x32->64 multiply-add costs 2.5 of those slots
-# (measured: 25.5 per SM and clock); see profiles/int_pipe_microbenchmark.md.
+# (measured: 25.5 per SM and clock) with the int_pipe_bench tool of the package.
 # A 64-bit Shoup butterfly needs at least the high half of x*w' (4 wide
 # products) and the low halves of x*w and hi*q (1 wide + 2 narrow each):
 # 6 wide + 4 narrow = 19 multiply slots.  Additions go to another pipe.
 # DRAM bytes (read + write) per ciphertext of encrypt_fused_kernel at N = 16384,
-# L = 4, from the ncu capture in profiles/encrypt_fused_kernel_resnet18_296cts.md
+# L = 4, from an ncu capture of the profile_case.py encrypt case (summary under profiles/)
 # (363.6 MB for 296 ciphertexts; traffic grows in proportion to the count).
 ENCRYPT_DRAM_BYTES_PER_CT_N16384_L4 = 363.57248e6 / 296
 IMAD_PER_SM_CLK = 64.0

@@ -121,7 +121,7 @@ class Ctx:
         self.n = N // 2
 
     def __del__(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and _lib is not None:     # _lib is gone at interpreter exit
             _lib.he_ctx_destroy(self.handle)
             self.handle = None
 
@@ -131,7 +131,7 @@ class Keys:
         self.handle, self.ctx = handle, ctx
 
     def __del__(self):
-        if getattr(self, "handle", None) and getattr(self.ctx, "handle", None):
+        if getattr(self, "handle", None) and getattr(self.ctx, "handle", None) and _lib is not None:
             _lib.he_keys_destroy(self.handle)
             self.handle = None
 
@@ -141,7 +141,7 @@ class Mask:
         self.handle, self.P, self.k, self.idx_ptr = handle, P, k, idx_ptr
 
     def __del__(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and _lib is not None:
             _lib.he_mask_destroy(self.handle)
             self.handle = None
 
