@@ -498,6 +498,10 @@ int he_decrypt_level(he_ctx *ctx, const he_keys *keys, const uint64_t *ct_dev, u
     if (T == 0) return HE_OK;
     if (!ct_dev || !z_dev) return HE_ERR_INVALID_ARG;
     const CtxDev &d = ctx->dev;
+    if (d.logN <= 14) {                 // one fused kernel, no work buffer
+        CU(launch_decrypt_fused(d, keys->dev, ct_dev, level, T, z_dev, as_stream(stream)));
+        return HE_OK;
+    }
     int rc = ensure(&ctx->ws, &ctx->ws_bytes, work_bytes(ctx, T));
     if (rc != HE_OK) return rc;
     uint64_t *scratch = static_cast<uint64_t *>(ctx->ws);

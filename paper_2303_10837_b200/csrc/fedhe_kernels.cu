@@ -1088,6 +1088,77 @@ cudaError_t launch_decrypt(const CtxDev &c, const KeysDev &k, const uint64_t *ct
     return FEDHE_LAUNCHED();
 }
 
+// Fused path for N <= 2^14: one thread block per ciphertext transforms c1
+// (limb 0), multiplies by the secret key, transforms back, adds c0, centres,
+// and runs the slot transform on the result without leaving the SM; only the
+// two limb-0 polynomials are read and the n decoded values written.
+// L: layout of the length-N integer transform (played by L::NT / V threads),
+// LF: layout of the length-n complex transform with LF::NT == L::NT / V.
+template <class L, int V, class LF>
+__global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
+decrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const uint64_t *ct, uint32_t level,
+                     double *z) {
+    static_assert(LF::NT == L::NT / V && LF::LOGB + 1 == L::LOGB, "thread counts and sizes must match");
+    extern __shared__ __align__(16) uint64_t sm[];
+    constexpr uint32_t B = 1u << L::LOGB, n = B >> 1;
+    const uint32_t tid = threadIdx.x;
+    const size_t t = blockIdx.x;
+    const LimbDev &lb = c.limb[0];
+    const uint64_t q = lb.q, q2 = 2 * q;
+    const uint64_t *c0 = ct + ((t * 2 + 0) * level) * B, *c1 = ct + ((t * 2 + 1) * level) * B;
+    {
+        const NttArgs fa = {lb.fwd, q, q2, 0, 0};
+        smem_ntt_forward<L, V>(
+            sm, tid, fa, [&](uint32_t i) { return c1[i]; },
+            [&](uint32_t p, uint64_t a, uint64_t b) {
+                const tw_t s0 = load_tw(k.s_hat + p), s1 = load_tw(k.s_hat + p + 1);
+                sm[swz(p)] = shoup_lazy(a, s0.w, s0.wp, q);
+                sm[swz(p + 1)] = shoup_lazy(b, s1.w, s1.wp, q);
+            });
+    }
+    int64_t *d = reinterpret_cast<int64_t *>(sm);
+    {
+        const NttArgs ia = {lb.inv, q, q2, 0, 0};
+        smem_ntt_inverse<L, V, true>(
+            sm, tid, ia, lb.ninv, lb.wn, [&](uint32_t p) { return u64x2{sm[swz(p)], sm[swz(p + 1)]}; },
+            [&](uint32_t i, uint64_t v) {
+                const uint64_t r = addmod(csub(v, q), c0[i], q);
+                d[swz(i)] = r > q / 2 ? -(int64_t)(q - r) : (int64_t)r;
+            });
+    }
+    __syncthreads();
+    // slot transform: bit-reversed load of (d_k + i d_{k+n}) / Delta from shared memory
+    const double inv_delta = __longlong_as_double((long long)(1023 - c.log2_delta) << 52);
+    cpx x[LF::E];
+#pragma unroll
+    for (int r = 0; r < LF::E; r++) {
+        const uint32_t kk = bitrev(LF::template idx<LF::NPH - 1>(tid, r), LF::LOGB);
+        x[r] = cpx{(double)d[swz(kk)] * inv_delta, (double)d[swz(kk + n)] * inv_delta};
+    }
+    __syncthreads();                      // all inputs are in registers: the buffer becomes the exchange buffer
+    block_dit<LF>(x, reinterpret_cast<cpx *>(sm), tid, c.ftw);
+#pragma unroll
+    for (int r = 0; r < LF::E; r++) z[t * n + LF::template idx<0>(tid, r)] = x[r].re;
+}
+
+template <class L, int V, class LF>
+static cudaError_t launch_decrypt_fused_t(const CtxDev &c, const KeysDev &k, const uint64_t *ct, uint32_t level,
+                                          size_t T, double *z, cudaStream_t s) {
+    const size_t smem = sizeof(uint64_t) << L::LOGB;
+    auto kern = decrypt_fused_kernel<L, V, LF>;
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+    kern<<<(unsigned)T, L::NT / V, smem, s>>>(c, k, ct, level, z);
+    return FEDHE_LAUNCHED();
+}
+
+cudaError_t launch_decrypt_fused(const CtxDev &c, const KeysDev &k, const uint64_t *ct, uint32_t level,
+                                 size_t T, double *z, cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    if (c.logN == 13) return launch_decrypt_fused_t<Lay<13, 3>, 2, Lay<12, 3>>(c, k, ct, level, T, z, s);
+    return launch_decrypt_fused_t<Lay<14, 3>, 2, Lay<13, 3>>(c, k, ct, level, T, z, s);
+}
+
 // ===========================================================================
 // two-party threshold decryption: dealer split of the secret, partial
 // decryption with smudging noise, merge

@@ -42,6 +42,10 @@ cudaError_t launch_plain_aggregate(const float *const *ptrs, const double *alpha
 cudaError_t launch_decrypt(const CtxDev &c, const KeysDev &k, const uint64_t *ct, uint32_t level,
                            size_t T, uint64_t *scratch, cudaStream_t s);
 
+// fused decrypt + decode for N <= 2^14 (no scratch): z double [T][n]
+cudaError_t launch_decrypt_fused(const CtxDev &c, const KeysDev &k, const uint64_t *ct, uint32_t level,
+                                 size_t T, double *z, cudaStream_t s);
+
 // two-party threshold decryption.  tmp: uint64 [2][L][N] (shares as residues)
 cudaError_t launch_threshold_split(const CtxDev &c, const int8_t *s8, uint64_t seed, uint64_t *tmp,
                                    cudaStream_t s);
