@@ -106,6 +106,21 @@ HD void ct_butterfly(uint64_t &x, uint64_t &y, uint64_t w, uint64_t wp, uint64_t
     y = add64(sub64(u, v), q2);
 }
 
+// The same butterflies without any conditional subtraction, for primes small
+// enough that the values may simply grow: forward, every stage adds at most
+// 2q to the bound; inverse, the sum doubles it, and the difference is kept
+// non-negative by adding `bound`, a multiple of q not below the inputs.
+HD void ct_butterfly_grow(uint64_t &x, uint64_t &y, uint64_t w, uint64_t wp, uint64_t q, uint64_t q2) {
+    const uint64_t u = x, v = shoup_lazy(y, w, wp, q);
+    x = add64(u, v);
+    y = add64(sub64(u, v), q2);
+}
+HD void gs_butterfly_grow(uint64_t &x, uint64_t &y, uint64_t w, uint64_t wp, uint64_t q, uint64_t bound) {
+    const uint64_t u = x, v = y;
+    x = add64(u, v);
+    y = shoup_lazy(add64(sub64(u, v), bound), w, wp, q);
+}
+
 // Inverse (Gentleman-Sande): inputs and outputs in [0, 2q).
 HD void gs_butterfly(uint64_t &x, uint64_t &y, uint64_t w, uint64_t wp, uint64_t q, uint64_t q2) {
     uint64_t u = x, v = y;

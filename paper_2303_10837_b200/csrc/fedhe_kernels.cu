@@ -760,50 +760,53 @@ encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const i
         const int64_t *mt = m + (size_t)tl * B;
         const LimbDev &lb = c.limb[j];
         const uint64_t q = lb.q, q2 = 2 * q;
+        // primes below 2^45 run the transforms without conditional subtractions:
+        // 13 growing stages keep every value below 2^14 q < 2^59
+        const bool small_q = q < (1ull << 45);
+        const uint64_t diff_bound = small_q ? q << L::LOGB + 1 : q2;
         uint64_t *cbase = ct + (((size_t)tl * 2 + 0) * c.L + j) * B;
         {
             const tw_t *p0 = k.pk0_hat + (size_t)j * B + grp * H, *p1 = k.pk1_hat + (size_t)j * B + grp * H;
             uint64_t *c1 = cbase + cstride + grp * H;
             const uint64_t w0 = load_tw(lb.fwd + 1).w;     // twiddle of the stage that pairs the halves
             const NttArgs fa = {lb.fwd, q, q2, 1, grp};
-            smem_ntt_forward<L, V>(
-                smg, gt, fa,
-                [&](uint32_t i) {
-                    const int b = su[i + H];
-                    const uint64_t u = small_residue(su[i], q);
-                    const uint64_t v = b == 0 ? 0 : (b > 0 ? w0 : q - w0);
-                    return grp == 0 ? u + v : u - v + q2;
-                },
-                [&](uint32_t p, uint64_t a, uint64_t b) {
-                    const tw_t a0 = load_tw(p1 + p), a1 = load_tw(p1 + p + 1);
-                    u64x2 v;
-                    v.x = shoup_lazy(a, a0.w, a0.wp, q);
-                    v.y = shoup_lazy(b, a1.w, a1.wp, q);
-                    *reinterpret_cast<u64x2 *>(c1 + p) = v;      // parked until the second pass
-                    const tw_t b0 = load_tw(p0 + p), b1 = load_tw(p0 + p + 1);
-                    smg[swz(p)] = shoup_lazy(a, b0.w, b0.wp, q);
-                    smg[swz(p + 1)] = shoup_lazy(b, b1.w, b1.wp, q);
-                },
-                gsync);
+            auto src = [&](uint32_t i) {
+                const int b = su[i + H];
+                const uint64_t u = small_residue(su[i], q);
+                const uint64_t v = b == 0 ? 0 : (b > 0 ? w0 : q - w0);
+                return grp == 0 ? u + v : u - v + q2;
+            };
+            auto dst = [&](uint32_t p, uint64_t a, uint64_t b) {
+                const tw_t a0 = load_tw(p1 + p), a1 = load_tw(p1 + p + 1);
+                u64x2 v;
+                v.x = shoup_lazy(a, a0.w, a0.wp, q);
+                v.y = shoup_lazy(b, a1.w, a1.wp, q);
+                *reinterpret_cast<u64x2 *>(c1 + p) = v;      // parked until the second pass
+                const tw_t b0 = load_tw(p0 + p), b1 = load_tw(p0 + p + 1);
+                smg[swz(p)] = shoup_lazy(a, b0.w, b0.wp, q);
+                smg[swz(p + 1)] = shoup_lazy(b, b1.w, b1.wp, q);
+            };
+            if (small_q) smem_ntt_forward<L, V, true>(smg, gt, fa, src, dst, gsync);
+            else smem_ntt_forward<L, V, false>(smg, gt, fa, src, dst, gsync);
         }
 #pragma unroll 1
         for (int h = 0; h < 2; h++) {
             uint64_t *cc = cbase + h * cstride;
             const int8_t *se = se0 + h * B;
             const NttArgs ia = {lb.inv, q, q2, 1, grp};
-            smem_ntt_inverse<L, V, false>(
-                smg, gt, ia, lb.ninv, lb.wn,
-                [&](uint32_t p) {
-                    if (h == 0) return u64x2{smg[swz(p)], smg[swz(p + 1)]};
-                    return *reinterpret_cast<const u64x2 *>(cc + grp * H + p);
-                },
-                [&](uint32_t i, uint64_t v) { smg[swz(i)] = v; }, gsync);
+            auto isrc = [&](uint32_t p) {
+                if (h == 0) return u64x2{smg[swz(p)], smg[swz(p + 1)]};
+                return *reinterpret_cast<const u64x2 *>(cc + grp * H + p);
+            };
+            auto idst = [&](uint32_t i, uint64_t v) { smg[swz(i)] = v; };
+            if (small_q) smem_ntt_inverse<L, V, false, true>(smg, gt, ia, lb.ninv, lb.wn, isrc, idst, gsync);
+            else smem_ntt_inverse<L, V, false, false>(smg, gt, ia, lb.ninv, lb.wn, isrc, idst, gsync);
             __syncthreads();
             // last stage across the halves with 1/N folded in, then the error / message terms
             for (uint32_t e = tid; e < H; e += RT) {
                 const uint64_t a = sm[swz(e)], b = sm[H + swz(e)];
                 const uint64_t lo = shoup(a + b, lb.ninv.w, lb.ninv.wp, q);
-                const uint64_t hi = shoup(a - b + q2, lb.wn.w, lb.wn.wp, q);
+                const uint64_t hi = shoup(a - b + diff_bound, lb.wn.w, lb.wn.wp, q);
                 uint64_t add_lo, add_hi;
                 if (h == 0) {
                     add_lo = signed_residue(mt[e] + (int64_t)se[e], q, lb.mu);

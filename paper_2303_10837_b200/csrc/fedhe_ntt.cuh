@@ -84,7 +84,10 @@ struct NttArgs {
     uint32_t blk;        // which block this is
 };
 
-template <class L, int P, int I>
+// GROW: no conditional subtractions (small primes only, see the *_grow
+// butterflies): a sub-block's inverse input must lie below 2q, and after k
+// inverse stages the values lie below 2^(k+1) q.
+template <class L, int P, int I, bool GROW = false>
 HD void fwd_stage(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
     constexpr int s = P * L::LE + I;
     constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
@@ -97,11 +100,12 @@ HD void fwd_stage(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
         // compiler merges the equal loads of an unrolled group
         const tw_t *pw = a.tw + base + L::template top<P, I>(tid, r);
         tw_t w = FEDHE_LD_TW(pw);
-        ct_butterfly(x[r], x[r | (1 << bit)], w.w, w.wp, a.q, a.q2);
+        if constexpr (GROW) ct_butterfly_grow(x[r], x[r | (1 << bit)], w.w, w.wp, a.q, a.q2);
+        else ct_butterfly(x[r], x[r | (1 << bit)], w.w, w.wp, a.q, a.q2);
     }
 }
 
-template <class L, int P, int I>
+template <class L, int P, int I, bool GROW = false>
 HD void inv_stage(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
     constexpr int s = P * L::LE + I;
     constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
@@ -112,7 +116,9 @@ HD void inv_stage(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
         if (r & (1 << bit)) continue;
         const tw_t *pw = a.tw + base + L::template top<P, I>(tid, r);
         tw_t w = FEDHE_LD_TW(pw);
-        gs_butterfly(x[r], x[r | (1 << bit)], w.w, w.wp, a.q, a.q2);
+        // local stage s is the (LOGB - 1 - s)-th to run: inputs lie below 2^(LOGB - s) q
+        if constexpr (GROW) gs_butterfly_grow(x[r], x[r | (1 << bit)], w.w, w.wp, a.q, a.q << (L::LOGB - s));
+        else gs_butterfly(x[r], x[r | (1 << bit)], w.w, w.wp, a.q, a.q2);
     }
 }
 
@@ -130,29 +136,29 @@ HD void inv_stage0_scaled(uint64_t (&x)[L::E], tw_t ninv, tw_t wn, uint64_t q, u
     }
 }
 
-template <class L, int P, int I = 0>
+template <class L, int P, int I = 0, bool GROW = false>
 HD void fwd_phase(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
     constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
     if constexpr (I < nst) {
-        fwd_stage<L, P, I>(x, tid, a);
-        fwd_phase<L, P, I + 1>(x, tid, a);
+        fwd_stage<L, P, I, GROW>(x, tid, a);
+        fwd_phase<L, P, I + 1, GROW>(x, tid, a);
     }
 }
 
 // inverse phase: stages nst-1 down to STOP (STOP = 1 leaves stage 0 of the
 // phase to the caller)
-template <class L, int P, int STOP, int I>
+template <class L, int P, int STOP, int I, bool GROW = false>
 HD void inv_phase_from(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
     if constexpr (I >= STOP) {
-        inv_stage<L, P, I>(x, tid, a);
-        inv_phase_from<L, P, STOP, I - 1>(x, tid, a);
+        inv_stage<L, P, I, GROW>(x, tid, a);
+        inv_phase_from<L, P, STOP, I - 1, GROW>(x, tid, a);
     }
 }
 
-template <class L, int P, int STOP = 0>
+template <class L, int P, int STOP = 0, bool GROW = false>
 HD void inv_phase(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
     constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
-    inv_phase_from<L, P, STOP, nst - 1>(x, tid, a);
+    inv_phase_from<L, P, STOP, nst - 1, GROW>(x, tid, a);
 }
 
 #if defined(__CUDACC__)
@@ -182,7 +188,7 @@ struct GroupSync {
     }
 };
 
-template <class L, int V, class Src, class Dst, class Sync = BlockSync, int P = 0>
+template <class L, int V, bool GROW = false, class Src, class Dst, class Sync = BlockSync, int P = 0>
 __device__ __forceinline__ void smem_ntt_forward(uint64_t *sm, uint32_t tid, const NttArgs &a, const Src &src,
                                                  const Dst &dst, const Sync &sync = Sync()) {
     constexpr int RT = L::NT / V, LAST = L::NPH - 1;
@@ -196,7 +202,7 @@ __device__ __forceinline__ void smem_ntt_forward(uint64_t *sm, uint32_t tid, con
             if constexpr (P == 0) x[r] = src(i);
             else x[r] = sm[swz(i)];
         }
-        fwd_phase<L, P>(x, vt, a);
+        fwd_phase<L, P, 0, GROW>(x, vt, a);
         if constexpr (P == LAST) {
 #pragma unroll
             for (int r = 0; r < L::E; r += 2) dst(L::template idx<P>(vt, r), x[r], x[r + 1]);
@@ -207,11 +213,12 @@ __device__ __forceinline__ void smem_ntt_forward(uint64_t *sm, uint32_t tid, con
     }
     if constexpr (P < LAST) {
         sync();
-        smem_ntt_forward<L, V, Src, Dst, Sync, P + 1>(sm, tid, a, src, dst, sync);
+        smem_ntt_forward<L, V, GROW, Src, Dst, Sync, P + 1>(sm, tid, a, src, dst, sync);
     }
 }
 
-template <class L, int V, bool SCALED, class Src, class Dst, class Sync = BlockSync, int P = L::NPH - 1>
+template <class L, int V, bool SCALED, bool GROW = false, class Src, class Dst, class Sync = BlockSync,
+          int P = L::NPH - 1>
 __device__ __forceinline__ void smem_ntt_inverse(uint64_t *sm, uint32_t tid, const NttArgs &a, tw_t ninv,
                                                  tw_t wn, const Src &src, const Dst &dst,
                                                  const Sync &sync = Sync()) {
@@ -231,11 +238,12 @@ __device__ __forceinline__ void smem_ntt_inverse(uint64_t *sm, uint32_t tid, con
 #pragma unroll
             for (int r = 0; r < L::E; r++) x[r] = sm[swz(L::template idx<P>(vt, r))];
         }
+        static_assert(!(SCALED && GROW), "the scaled last stage expects inputs below 2q");
         if constexpr (P == 0 && SCALED) {
             inv_phase<L, 0, 1>(x, vt, a);
             inv_stage0_scaled<L>(x, ninv, wn, a.q, a.q2);
         } else {
-            inv_phase<L, P>(x, vt, a);
+            inv_phase<L, P, 0, GROW>(x, vt, a);
         }
         if constexpr (P == 0) {
 #pragma unroll
@@ -247,7 +255,7 @@ __device__ __forceinline__ void smem_ntt_inverse(uint64_t *sm, uint32_t tid, con
     }
     if constexpr (P > 0) {
         sync();
-        smem_ntt_inverse<L, V, SCALED, Src, Dst, Sync, P - 1>(sm, tid, a, ninv, wn, src, dst, sync);
+        smem_ntt_inverse<L, V, SCALED, GROW, Src, Dst, Sync, P - 1>(sm, tid, a, ninv, wn, src, dst, sync);
     }
 }
 #endif
