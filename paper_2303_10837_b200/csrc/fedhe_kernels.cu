@@ -133,10 +133,56 @@ ntt_block_kernel(const __grid_constant__ CtxDev c, uint64_t *data, size_t poly_s
     }
 }
 
-// The A = logN - LOGB outer stages of a long transform: every thread owns two
-// neighbouring columns of the 2^A x B matrix view and does the A stages that
-// pair rows, reading and writing whole 16-byte words.
-template <bool FWD>
+// The A = logN - LOGB outer stages of a long transform on two neighbouring
+// columns of the 2^A x B matrix view (x[a] = row a): forward in [0, 4q) out,
+// inverse [0, 2q) in and canonical out with 1/N folded into stage 0.
+template <uint32_t A>
+__device__ __forceinline__ void outer_forward(u64x2 (&x)[1u << A], const LimbDev &lb) {
+    const uint64_t q = lb.q, q2 = 2 * q;
+    constexpr uint32_t rows = 1u << A;
+#pragma unroll
+    for (uint32_t s = 0; s < A; s++) {
+        const uint32_t bit = 1u << (A - 1 - s);
+#pragma unroll
+        for (uint32_t a = 0; a < rows; a++) {
+            if (a & bit) continue;
+            tw_t w = load_tw(lb.fwd + (1u << s) + (a >> (A - s)));
+            ct_butterfly(x[a].x, x[a | bit].x, w.w, w.wp, q, q2);
+            ct_butterfly(x[a].y, x[a | bit].y, w.w, w.wp, q, q2);
+        }
+    }
+}
+
+template <uint32_t A>
+__device__ __forceinline__ void outer_inverse(u64x2 (&x)[1u << A], const LimbDev &lb) {
+    const uint64_t q = lb.q, q2 = 2 * q;
+    constexpr uint32_t rows = 1u << A;
+#pragma unroll
+    for (int s = (int)A - 1; s >= 1; s--) {
+        const uint32_t bit = 1u << (A - 1 - s);
+#pragma unroll
+        for (uint32_t a = 0; a < rows; a++) {
+            if (a & bit) continue;
+            tw_t w = load_tw(lb.inv + (1u << s) + (a >> (A - s)));
+            gs_butterfly(x[a].x, x[a | bit].x, w.w, w.wp, q, q2);
+            gs_butterfly(x[a].y, x[a | bit].y, w.w, w.wp, q, q2);
+        }
+    }
+    const uint32_t bit = 1u << (A - 1);      // stage 0 with 1/N folded in
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++) {
+        if (a & bit) continue;
+        const uint64_t u0 = x[a].x, v0 = x[a | bit].x, u1 = x[a].y, v1 = x[a | bit].y;
+        x[a].x = shoup(u0 + v0, lb.ninv.w, lb.ninv.wp, q);
+        x[a | bit].x = shoup(u0 - v0 + q2, lb.wn.w, lb.wn.wp, q);
+        x[a].y = shoup(u1 + v1, lb.ninv.w, lb.ninv.wp, q);
+        x[a | bit].y = shoup(u1 - v1 + q2, lb.wn.w, lb.wn.wp, q);
+    }
+}
+
+// The outer stages as an elementwise pass over HBM: every thread owns two
+// neighbouring columns and reads and writes whole 16-byte words.
+template <bool FWD, uint32_t A>
 __global__ void __launch_bounds__(256)
 ntt_outer_kernel(const __grid_constant__ CtxDev c, uint64_t *data, size_t poly_stride, uint32_t limb0,
                  uint32_t nlimbs, size_t total) {
@@ -150,41 +196,23 @@ ntt_outer_kernel(const __grid_constant__ CtxDev c, uint64_t *data, size_t poly_s
     const LimbDev &lb = c.limb[limb0 + limb];
     const uint64_t q = lb.q, q2 = 2 * q;
     uint64_t *p = data + poly * poly_stride + (size_t)limb * c.N + col;
-    const uint32_t A = c.A, rows = 1u << A;      // A is 1, 2 or 3
-    u64x2 x[8];
+    constexpr uint32_t rows = 1u << A;
+    u64x2 x[rows];
+#pragma unroll
     for (uint32_t a = 0; a < rows; a++) x[a] = *reinterpret_cast<const u64x2 *>(p + (size_t)a * B);
-    if (FWD) {
-        for (uint32_t s = 0; s < A; s++) {
-            const uint32_t bit = 1u << (A - 1 - s);
-            for (uint32_t a = 0; a < rows; a++) {
-                if (a & bit) continue;
-                tw_t w = load_tw(lb.fwd + (1u << s) + (a >> (A - s)));
-                ct_butterfly(x[a].x, x[a | bit].x, w.w, w.wp, q, q2);
-                ct_butterfly(x[a].y, x[a | bit].y, w.w, w.wp, q, q2);
-            }
-        }
-    } else {
-        for (int s = (int)A - 1; s >= 1; s--) {
-            const uint32_t bit = 1u << (A - 1 - s);
-            for (uint32_t a = 0; a < rows; a++) {
-                if (a & bit) continue;
-                tw_t w = load_tw(lb.inv + (1u << s) + (a >> (A - s)));
-                gs_butterfly(x[a].x, x[a | bit].x, w.w, w.wp, q, q2);
-                gs_butterfly(x[a].y, x[a | bit].y, w.w, w.wp, q, q2);
-            }
-        }
-        const uint32_t bit = 1u << (A - 1);      // stage 0 with 1/N folded in
-        for (uint32_t a = 0; a < rows; a++) {
-            if (a & bit) continue;
-            uint64_t u0 = x[a].x, v0 = x[a | bit].x, u1 = x[a].y, v1 = x[a | bit].y;
-            x[a].x = shoup(u0 + v0, lb.ninv.w, lb.ninv.wp, q);
-            x[a | bit].x = shoup(u0 - v0 + q2, lb.wn.w, lb.wn.wp, q);
-            x[a].y = shoup(u1 + v1, lb.ninv.w, lb.ninv.wp, q);
-            x[a | bit].y = shoup(u1 - v1 + q2, lb.wn.w, lb.wn.wp, q);
-        }
-    }
+    if (FWD) outer_forward<A>(x, lb);
+    else outer_inverse<A>(x, lb);
+#pragma unroll
     for (uint32_t a = 0; a < rows; a++) *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = x[a];
 }
+
+// launches kern<A> for the context's A (1, 2 or 3)
+#define FEDHE_FOR_A(c, CALL)                 \
+    switch ((c).A) {                         \
+    case 1: { constexpr uint32_t A_ = 1; CALL; } break; \
+    case 2: { constexpr uint32_t A_ = 2; CALL; } break; \
+    default: { constexpr uint32_t A_ = 3; CALL; } break; \
+    }
 
 template <class L, int V>
 static cudaError_t launch_ntt_blocks(const CtxDev &c, bool forward, uint64_t *data, size_t npoly,
@@ -209,22 +237,27 @@ static cudaError_t launch_ntt_blocks(const CtxDev &c, bool forward, uint64_t *da
     return FEDHE_LAUNCHED();
 }
 
+// the block (inner) stages only
+static cudaError_t launch_ntt_inner(const CtxDev &c, bool forward, uint64_t *data, size_t npoly,
+                                    size_t poly_stride, uint32_t limb0, uint32_t nlimbs, cudaStream_t s) {
+    if (c.LOGB == 13) return launch_ntt_blocks<Lay<13, 3>, 2>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
+    return launch_ntt_blocks<Lay<14, 3>, 2>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
+}
+
 cudaError_t launch_ntt(const CtxDev &c, bool forward, uint64_t *data, size_t npoly, size_t poly_stride,
                        uint32_t limb0, uint32_t nlimbs, cudaStream_t s) {
     if (npoly == 0 || nlimbs == 0) return cudaSuccess;
     cudaError_t e;
     const size_t outer_threads = npoly * nlimbs * ((size_t)1 << (c.LOGB - 1));
     if (forward && c.A > 0) {
-        ntt_outer_kernel<true><<<blocks_for(outer_threads, 256), 256, 0, s>>>(c, data, poly_stride, limb0,
-                                                                              nlimbs, outer_threads);
+        FEDHE_FOR_A(c, (ntt_outer_kernel<true, A_><<<blocks_for(outer_threads, 256), 256, 0, s>>>(
+                           c, data, poly_stride, limb0, nlimbs, outer_threads)));
         if ((e = FEDHE_LAUNCHED())) return e;
     }
-    if (c.LOGB == 13) e = launch_ntt_blocks<Lay<13, 3>, 2>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
-    else e = launch_ntt_blocks<Lay<14, 3>, 2>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
-    if (e) return e;
+    if ((e = launch_ntt_inner(c, forward, data, npoly, poly_stride, limb0, nlimbs, s))) return e;
     if (!forward && c.A > 0) {
-        ntt_outer_kernel<false><<<blocks_for(outer_threads, 256), 256, 0, s>>>(c, data, poly_stride, limb0,
-                                                                               nlimbs, outer_threads);
+        FEDHE_FOR_A(c, (ntt_outer_kernel<false, A_><<<blocks_for(outer_threads, 256), 256, 0, s>>>(
+                           c, data, poly_stride, limb0, nlimbs, outer_threads)));
         if ((e = FEDHE_LAUNCHED())) return e;
     }
     return cudaSuccess;
@@ -823,75 +856,128 @@ encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const i
     }
 }
 
-// General path (any N): three elementwise kernels around the batched
-// transforms, with the ciphertext buffer itself as the only work space.
+// Long rings (N = 2^15, 2^16), where a limb does not fit one SM: the ciphertext
+// buffer itself is the only work space and every pass over it does as much as
+// it can.  (1) draw u and run the outer forward stages into the c1 slots;
+// (2) block transforms of the c1 slots whose last phase writes both products
+// u^ pk0^ -> c0 and u^ pk1^ -> c1; (3) inverse block transforms of all slots;
+// (4) outer inverse stages fused with the error and message terms.
 
-// u as residues into the c1 slots of every limb
+// (1) one thread per pair of neighbouring columns of one ciphertext, all limbs
+template <uint32_t A>
 __global__ void __launch_bounds__(256)
-enc_sample_u_kernel(const __grid_constant__ CtxDev c, uint32_t t0, uint64_t seed, uint32_t client,
-                    uint64_t *ct, size_t total) {
-    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+enc_outer_sample_kernel(const __grid_constant__ CtxDev c, uint32_t t0, uint64_t seed, uint32_t client,
+                        uint64_t *ct, size_t total) {
+    size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= total) return;
-    const uint32_t quads = c.N >> 2;
-    const uint32_t b = (uint32_t)(g % quads);
-    const size_t tl = g / quads;
-    u32x4 w = stream_block(seed, b, t0 + (uint32_t)tl, client, TAG_ENC_U);
-    const int u0 = ternary_from_word(w.x), u1 = ternary_from_word(w.y), u2 = ternary_from_word(w.z),
-              u3 = ternary_from_word(w.w);
+    const uint32_t B = 1u << c.LOGB, half = B >> 1;
+    constexpr uint32_t rows = 1u << A;
+    const uint32_t col = (uint32_t)(g % half) * 2;
+    const size_t tl = g / half;
+    int u[rows][2];
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++) {
+        const uint32_t i = a * B + col;               // even: both columns share a Philox block
+        const u32x4 w = stream_block(seed, i >> 2, t0 + (uint32_t)tl, client, TAG_ENC_U);
+        u[a][0] = ternary_from_word((i & 2) ? w.z : w.x);
+        u[a][1] = ternary_from_word((i & 2) ? w.w : w.y);
+    }
+#pragma unroll 1
     for (uint32_t j = 0; j < c.L; j++) {
-        const uint64_t q = c.limb[j].q;
-        uint64_t *c1 = ct + ((tl * 2 + 1) * c.L + j) * c.N + 4 * (size_t)b;
-        reinterpret_cast<ulonglong2 *>(c1)[0] = make_ulonglong2(small_residue(u0, q), small_residue(u1, q));
-        reinterpret_cast<ulonglong2 *>(c1)[1] = make_ulonglong2(small_residue(u2, q), small_residue(u3, q));
+        const LimbDev &lb = c.limb[j];
+        u64x2 x[rows];
+#pragma unroll
+        for (uint32_t a = 0; a < rows; a++) x[a] = u64x2{small_residue(u[a][0], lb.q), small_residue(u[a][1], lb.q)};
+        outer_forward<A>(x, lb);
+        uint64_t *p = ct + ((tl * 2 + 1) * c.L + j) * c.N + col;
+#pragma unroll
+        for (uint32_t a = 0; a < rows; a++) *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = x[a];
     }
 }
 
-// c0 = u^ pk0^, c1 = u^ pk1^ in the transform domain
-__global__ void __launch_bounds__(256)
-enc_pointwise_kernel(const __grid_constant__ CtxDev c, const KeysDev k, uint64_t *ct, size_t total) {
-    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (g >= total) return;
-    const uint32_t i = (uint32_t)(g % c.N);
-    const uint32_t j = (uint32_t)((g / c.N) % c.L);
-    const size_t tl = g / ((size_t)c.N * c.L);
-    const uint64_t q = c.limb[j].q;
-    uint64_t *c0 = ct + ((tl * 2 + 0) * c.L + j) * c.N + i;
-    uint64_t *c1 = ct + ((tl * 2 + 1) * c.L + j) * c.N + i;
-    const uint64_t u = *c1;
-    const tw_t a = load_tw(k.pk0_hat + (size_t)j * c.N + i), b = load_tw(k.pk1_hat + (size_t)j * c.N + i);
-    *c0 = shoup_lazy(u, a.w, a.wp, q);
-    *c1 = shoup_lazy(u, b.w, b.wp, q);
+// (2) one thread block per (ciphertext, limb, block): forward block transform of
+// the c1 slot, products with both halves of the public key on the way out
+template <class L, int V>
+__global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
+enc_block_forward_kernel(const __grid_constant__ CtxDev c, const KeysDev k, uint64_t *ct) {
+    extern __shared__ __align__(16) uint64_t sm[];
+    const uint32_t tid = threadIdx.x;
+    uint32_t b = blockIdx.x;
+    const uint32_t blk = b & ((1u << c.A) - 1u);
+    b >>= c.A;
+    const uint32_t j = b % c.L;
+    const size_t tl = b / c.L;
+    const LimbDev &lb = c.limb[j];
+    const uint64_t q = lb.q, q2 = 2 * q;
+    const size_t off = ((size_t)blk << L::LOGB);
+    uint64_t *c0 = ct + ((tl * 2 + 0) * c.L + j) * c.N + off;
+    uint64_t *c1 = ct + ((tl * 2 + 1) * c.L + j) * c.N + off;
+    const tw_t *p0 = k.pk0_hat + (size_t)j * c.N + off, *p1 = k.pk1_hat + (size_t)j * c.N + off;
+    const NttArgs a = {lb.fwd, q, q2, c.A, blk};
+    smem_ntt_forward<L, V>(
+        sm, tid, a, [&](uint32_t i) { return c1[i]; },
+        [&](uint32_t p, uint64_t x, uint64_t y) {
+            const tw_t a0 = load_tw(p0 + p), a1 = load_tw(p0 + p + 1), b0 = load_tw(p1 + p), b1 = load_tw(p1 + p + 1);
+            u64x2 v0, v1;
+            v0.x = shoup_lazy(x, a0.w, a0.wp, q);
+            v0.y = shoup_lazy(y, a1.w, a1.wp, q);
+            v1.x = shoup_lazy(x, b0.w, b0.wp, q);
+            v1.y = shoup_lazy(y, b1.w, b1.wp, q);
+            *reinterpret_cast<u64x2 *>(c0 + p) = v0;
+            *reinterpret_cast<u64x2 *>(c1 + p) = v1;
+        });
 }
 
-// c0 += e0 + m, c1 += e1: one thread per pair of coefficients, all limbs
-__global__ void __launch_bounds__(256)
-enc_add_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint32_t t0, uint64_t seed,
-               uint32_t client, uint64_t *ct, size_t total) {
-    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+// (4) one thread per pair of neighbouring columns of one ciphertext: draws the
+// errors once, then for every limb finishes both components
+template <uint32_t A>
+__global__ void __launch_bounds__(256, 2)
+enc_outer_inverse_add_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint32_t t0, uint64_t seed,
+                             uint32_t client, uint64_t *ct, size_t total) {
+    size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= total) return;
-    const uint32_t pairs = c.N >> 1;
-    const uint32_t b = (uint32_t)(g % pairs);
-    const size_t tl = g / pairs;
+    const uint32_t B = 1u << c.LOGB, half = B >> 1;
+    constexpr uint32_t rows = 1u << A;
+    const uint32_t col = (uint32_t)(g % half) * 2;
+    const size_t tl = g / half;
     const uint32_t t = t0 + (uint32_t)tl;
-    u32x4 w0 = stream_block(seed, b, t, client, TAG_ENC_E0);
-    u32x4 w1 = stream_block(seed, b, t, client, TAG_ENC_E1);
-    const int e0a = gauss_from_u64((uint64_t)w0.x | ((uint64_t)w0.y << 32));
-    const int e0b = gauss_from_u64((uint64_t)w0.z | ((uint64_t)w0.w << 32));
-    const int e1a = gauss_from_u64((uint64_t)w1.x | ((uint64_t)w1.y << 32));
-    const int e1b = gauss_from_u64((uint64_t)w1.z | ((uint64_t)w1.w << 32));
-    const longlong2 mm = *reinterpret_cast<const longlong2 *>(m + tl * c.N + 2 * (size_t)b);
+    int e1[rows][2];
+    int64_t me0[rows][2];                              // m + e0
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++) {
+        const uint32_t i = a * B + col;               // one Philox block per pair of coefficients
+        const u32x4 w0 = stream_block(seed, i >> 1, t, client, TAG_ENC_E0);
+        const u32x4 w1 = stream_block(seed, i >> 1, t, client, TAG_ENC_E1);
+        const longlong2 mm = *reinterpret_cast<const longlong2 *>(m + tl * c.N + i);
+        me0[a][0] = mm.x + gauss_from_u64((uint64_t)w0.x | ((uint64_t)w0.y << 32));
+        me0[a][1] = mm.y + gauss_from_u64((uint64_t)w0.z | ((uint64_t)w0.w << 32));
+        e1[a][0] = gauss_from_u64((uint64_t)w1.x | ((uint64_t)w1.y << 32));
+        e1[a][1] = gauss_from_u64((uint64_t)w1.z | ((uint64_t)w1.w << 32));
+    }
+#pragma unroll 1
     for (uint32_t j = 0; j < c.L; j++) {
         const LimbDev &lb = c.limb[j];
         const uint64_t q = lb.q;
-        ulonglong2 *c0 = reinterpret_cast<ulonglong2 *>(ct + ((tl * 2 + 0) * c.L + j) * c.N + 2 * (size_t)b);
-        ulonglong2 *c1 = reinterpret_cast<ulonglong2 *>(ct + ((tl * 2 + 1) * c.L + j) * c.N + 2 * (size_t)b);
-        ulonglong2 v0 = *c0, v1 = *c1;
-        v0.x = addmod(v0.x, signed_residue(mm.x + e0a, q, lb.mu), q);
-        v0.y = addmod(v0.y, signed_residue(mm.y + e0b, q, lb.mu), q);
-        v1.x = addmod(v1.x, small_residue(e1a, q), q);
-        v1.y = addmod(v1.y, small_residue(e1b, q), q);
-        *c0 = v0;
-        *c1 = v1;
+#pragma unroll 1
+        for (uint32_t comp = 0; comp < 2; comp++) {
+            uint64_t *p = ct + ((tl * 2 + comp) * c.L + j) * c.N + col;
+            u64x2 x[rows];
+#pragma unroll
+            for (uint32_t a = 0; a < rows; a++) x[a] = *reinterpret_cast<const u64x2 *>(p + (size_t)a * B);
+            outer_inverse<A>(x, lb);
+#pragma unroll
+            for (uint32_t a = 0; a < rows; a++) {
+                u64x2 o;
+                if (comp == 0) {
+                    o.x = addmod(x[a].x, signed_residue(me0[a][0], q, lb.mu), q);
+                    o.y = addmod(x[a].y, signed_residue(me0[a][1], q, lb.mu), q);
+                } else {
+                    o.x = addmod(x[a].x, small_residue(e1[a][0], q), q);
+                    o.y = addmod(x[a].y, small_residue(e1[a][1], q), q);
+                }
+                *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = o;
+            }
+        }
     }
 }
 
@@ -921,17 +1007,21 @@ cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const int64_t *m, 
         return launch_encrypt_fused<Lay<13, 3>, 2, true>(c, k, m, t0, T, seed, client, ct, s);
     }
     cudaError_t e;
-    const size_t ctw = 2 * (size_t)c.L * c.N;
-    size_t total = T * (c.N >> 2);
-    enc_sample_u_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, t0, seed, client, ct, total);
+    const size_t cols = T * ((size_t)1 << (c.LOGB - 1));      // pairs of columns
+    FEDHE_FOR_A(c, (enc_outer_sample_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, t0, seed, client, ct, cols)));
     if ((e = FEDHE_LAUNCHED())) return e;
-    if ((e = launch_ntt(c, true, ct + (size_t)c.L * c.N, T, ctw, 0, c.L, s))) return e;   // the c1 halves
-    total = T * (size_t)c.L * c.N;
-    enc_pointwise_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, k, ct, total);
-    if ((e = FEDHE_LAUNCHED())) return e;
-    if ((e = launch_ntt(c, false, ct, 2 * T, (size_t)c.L * c.N, 0, c.L, s))) return e;
-    total = T * (c.N >> 1);
-    enc_add_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, m, t0, seed, client, ct, total);
+    {
+        using L = Lay<13, 3>;                                 // long rings are cut into 2^13 blocks
+        constexpr int V = 2;
+        const size_t smem = sizeof(uint64_t) << L::LOGB;
+        auto kern = enc_block_forward_kernel<L, V>;
+        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+        kern<<<(unsigned)((T * c.L) << c.A), L::NT / V, smem, s>>>(c, k, ct);
+        if ((e = FEDHE_LAUNCHED())) return e;
+    }
+    if ((e = launch_ntt_inner(c, false, ct, 2 * T, (size_t)c.L * c.N, 0, c.L, s))) return e;
+    FEDHE_FOR_A(c, (enc_outer_inverse_add_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, m, t0, seed, client, ct,
+                                                                                          cols)));
     return FEDHE_LAUNCHED();
 }
 
