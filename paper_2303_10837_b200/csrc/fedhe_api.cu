@@ -117,6 +117,18 @@ int he_ctx_create(const he_params *p, he_ctx **out) {
             }
             rc = upload(ctx, reinterpret_cast<const tw_t *>(hl.fwd.data()), hl.fwd.size(), &ld.fwd);
             if (rc == HE_OK) rc = upload(ctx, reinterpret_cast<const tw_t *>(hl.inv.data()), hl.inv.size(), &ld.inv);
+            if (rc == HE_OK && hl.q < F64_PRIME_LIMIT) {
+                // every value is below 2^46, so the conversions are exact
+                std::vector<double> fd(hl.fwd.size()), id(hl.inv.size());
+                for (size_t i = 0; i < fd.size(); i++) fd[i] = (double)hl.fwd[i].w;
+                for (size_t i = 0; i < id.size(); i++) id[i] = (double)hl.inv[i].w;
+                ld.qd = (double)hl.q;
+                ld.qi = 1.0 / ld.qd;
+                ld.ninv_d = (double)hl.ninv.w;
+                ld.wn_d = (double)hl.wn.w;
+                rc = upload(ctx, fd.data(), fd.size(), &ld.fwd_d);
+                if (rc == HE_OK) rc = upload(ctx, id.data(), id.size(), &ld.inv_d);
+            }
         }
         if (rc != HE_OK) break;
         std::vector<double> roots, ftw;

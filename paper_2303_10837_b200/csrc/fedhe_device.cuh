@@ -6,6 +6,11 @@
 #pragma once
 
 #include <stdint.h>
+#include <string.h>
+
+#if !defined(__CUDA_ARCH__)
+#include <cmath>
+#endif
 
 #if defined(__CUDACC__)
 #define HD __host__ __device__ __forceinline__
@@ -106,27 +111,94 @@ HD void ct_butterfly(uint64_t &x, uint64_t &y, uint64_t w, uint64_t wp, uint64_t
     y = add64(sub64(u, v), q2);
 }
 
-// The same butterflies without any conditional subtraction, for primes small
-// enough that the values may simply grow: forward, every stage adds at most
-// 2q to the bound; inverse, the sum doubles it, and the difference is kept
-// non-negative by adding `bound`, a multiple of q not below the inputs.
-HD void ct_butterfly_grow(uint64_t &x, uint64_t &y, uint64_t w, uint64_t wp, uint64_t q, uint64_t q2) {
-    const uint64_t u = x, v = shoup_lazy(y, w, wp, q);
-    x = add64(u, v);
-    y = add64(sub64(u, v), q2);
-}
-HD void gs_butterfly_grow(uint64_t &x, uint64_t &y, uint64_t w, uint64_t wp, uint64_t q, uint64_t bound) {
-    const uint64_t u = x, v = y;
-    x = add64(u, v);
-    y = shoup_lazy(add64(sub64(u, v), bound), w, wp, q);
-}
-
 // Inverse (Gentleman-Sande): inputs and outputs in [0, 2q).
 HD void gs_butterfly(uint64_t &x, uint64_t &y, uint64_t w, uint64_t wp, uint64_t q, uint64_t q2) {
     uint64_t u = x, v = y;
     x = csub(add64(u, v), q2);
     y = shoup_lazy(add64(sub64(u, v), q2), w, wp, q);
 }
+
+// ---------------------------------------------------------------------------
+// Residues of a prime below 2^46 as integers held in doubles
+//
+// The double-precision pipe of the SM is separate from the integer multiply
+// pipe that the 64-bit Shoup products saturate, and a modular product costs it
+// six operations against about nineteen 32-bit multiply slots, so limbs whose
+// prime is small enough run their transforms in this arithmetic.  Values are
+// signed integers of magnitude at most 2^50 (exact in a double); every
+// operation below is a single correctly rounded instruction, written with the
+// rounding intrinsics so that nothing is contracted or reordered.
+// ---------------------------------------------------------------------------
+
+constexpr uint64_t F64_PRIME_LIMIT = 1ull << 46;
+constexpr double F64_ROUND = 6755399441055744.0;    // 1.5 * 2^52: x + F64_ROUND - F64_ROUND = rint(x), |x| < 2^51
+constexpr double F64_TWO52 = 4503599627370496.0;
+
+HD double f64_fma(double a, double b, double c) {
+#if defined(__CUDA_ARCH__)
+    return __fma_rn(a, b, c);
+#else
+    return std::fma(a, b, c);
+#endif
+}
+HD double f64_mul(double a, double b) {
+#if defined(__CUDA_ARCH__)
+    return __dmul_rn(a, b);
+#else
+    return a * b;
+#endif
+}
+HD double f64_add(double a, double b) {
+#if defined(__CUDA_ARCH__)
+    return __dadd_rn(a, b);
+#else
+    return a + b;
+#endif
+}
+HD double f64_sub(double a, double b) { return f64_add(a, -b); }
+
+HD double f64_from_bits(uint64_t b) {
+#if defined(__CUDA_ARCH__)
+    return __longlong_as_double((long long)b);
+#else
+    double d;
+    memcpy(&d, &b, 8);
+    return d;
+#endif
+}
+HD uint64_t f64_bits(double d) {
+#if defined(__CUDA_ARCH__)
+    return (uint64_t)__double_as_longlong(d);
+#else
+    uint64_t b;
+    memcpy(&b, &d, 8);
+    return b;
+#endif
+}
+
+// exact conversions of integers 0 <= x < 2^52 through the exponent of 2^52
+HD double f64_from_u64(uint64_t x) { return f64_sub(f64_from_bits(x | 0x4330000000000000ull), F64_TWO52); }
+HD uint64_t f64_to_u64(double r) { return f64_bits(f64_add(r, F64_TWO52)) & 0x000fffffffffffffull; }
+
+// x - q rint(x / q) for |x| < 2^51 with qi = 1/q rounded: exact, magnitude at most q/2 + 1
+HD double f64_reduce(double x, double q, double qi) {
+    const double k = f64_sub(f64_fma(x, qi, F64_ROUND), F64_ROUND);
+    return f64_fma(-k, q, x);
+}
+
+// y w mod q for integers |y| <= 2^50 and 0 <= w < q < 2^46.  The product is
+// taken exactly as h + l; k = rint(h qi) differs from y w / q by at most
+// 1/2 + 2^50 2^-52 = 3/4, so the result, which both fused operations deliver
+// exactly (h - k q is an integer below 2^53), has magnitude at most 3q/4.
+HD double f64_mulmod(double y, double w, double q, double qi) {
+    const double h = f64_mul(y, w);
+    const double l = f64_fma(y, w, -h);
+    const double k = f64_sub(f64_fma(h, qi, F64_ROUND), F64_ROUND);
+    return f64_add(f64_fma(-k, q, h), l);
+}
+
+// the residue in [0, q) of an integer |r| < q
+HD uint64_t f64_canonical(double r, double q) { return f64_to_u64(r < 0.0 ? f64_add(r, q) : r); }
 
 // ---------------------------------------------------------------------------
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11)

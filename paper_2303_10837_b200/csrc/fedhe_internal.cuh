@@ -20,6 +20,32 @@ struct LimbDev {
     tw_t qlinv;          // 1 / q_{L-1} mod q (unused for the last prime)
     const tw_t *fwd;     // psi^brev(i)
     const tw_t *inv;     // psi^-brev(i)
+    // primes below F64_PRIME_LIMIT also carry what the double-precision
+    // transforms need (fwd_d is null for the others)
+    const double *fwd_d; // the same twiddles as doubles
+    const double *inv_d;
+    double qd, qi;       // q and 1/q rounded
+    double ninv_d, wn_d; // 1/N and (inverse twiddle of stage 0)/N
+};
+
+// the pieces of a limb that a transform in arithmetic M needs
+template <class M>
+struct LimbOf;
+template <>
+struct LimbOf<ModInt> {
+    static HD NttArgs args(const LimbDev &lb, bool fwd, uint32_t A, uint32_t blk) {
+        return NttArgs{fwd ? lb.fwd : lb.inv, ModInt{lb.q, 2 * lb.q}, A, blk};
+    }
+    static HD tw_t ninv(const LimbDev &lb) { return lb.ninv; }
+    static HD tw_t wn(const LimbDev &lb) { return lb.wn; }
+};
+template <>
+struct LimbOf<ModF64> {
+    static HD NttArgsF args(const LimbDev &lb, bool fwd, uint32_t A, uint32_t blk) {
+        return NttArgsF{fwd ? lb.fwd_d : lb.inv_d, ModF64{lb.qd, lb.qi}, A, blk};
+    }
+    static HD double ninv(const LimbDev &lb) { return lb.ninv_d; }
+    static HD double wn(const LimbDev &lb) { return lb.wn_d; }
 };
 
 struct CtxDev {

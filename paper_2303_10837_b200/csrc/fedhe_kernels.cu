@@ -5,6 +5,7 @@
 #include "fedhe_launch.h"
 
 #include <atomic>
+#include <type_traits>
 
 namespace fedhe {
 
@@ -98,47 +99,69 @@ __device__ uint64_t shoup_companion(uint64_t w, uint64_t q) {   // floor(w 2^64 
 // batched negacyclic NTT
 // ===========================================================================
 
-// One block of B = 2^LOGB residues per thread block (a whole limb for
-// N <= 2^14), transformed in place in shared memory; every thread plays V
-// virtual threads per phase with E residues in registers at a time.
+// A limb runs in double-precision arithmetic when its prime allows it.
+#define FEDHE_FOR_ARITH(lb, CALL)                               \
+    if ((lb).fwd_d) { using M_ = ModF64; CALL; }                \
+    else { using M_ = ModInt; CALL; }
+
+// Representations in global memory.  What a caller hands in or gets back is
+// canonical residues.  Between the two passes of a long transform the data is
+// in the arithmetic's own form (lazy 64-bit integers, or the bits of signed
+// doubles): forward, outer pass -> block pass; inverse, block pass -> outer
+// pass.  The inverse block pass reads residues below 2q.
+
+// One block of B = 2^LOGB residues (a whole limb for N <= 2^14), transformed
+// in place in shared memory; every thread plays V virtual threads per phase
+// with E residues in registers at a time.
+template <class M, class L, int V, bool FWD, bool SCALED>
+__device__ __forceinline__ void ntt_block(const CtxDev &c, const LimbDev &lb, uint64_t *sm, uint64_t *p,
+                                          uint32_t blk) {
+    using val = typename M::val;
+    const uint32_t tid = threadIdx.x;
+    const auto a = LimbOf<M>::args(lb, FWD, c.A, blk);
+    const M &ar = a.m;
+    if constexpr (FWD) {
+        const bool piece = c.A > 0;
+        smem_ntt_forward<L, V>(
+            sm, tid, a, [&](uint32_t i) { return piece ? M::from_bits(p[i]) : ar.from_residue(p[i]); },
+            [&](uint32_t i, val u, val v) {
+                u64x2 o;
+                o.x = ar.canon_wide(u);
+                o.y = ar.canon_wide(v);
+                *reinterpret_cast<u64x2 *>(p + i) = o;
+            });
+    } else {
+        smem_ntt_inverse<L, V, SCALED>(
+            sm, tid, a, LimbOf<M>::ninv(lb), LimbOf<M>::wn(lb),
+            [&](uint32_t i) {
+                const u64x2 t = *reinterpret_cast<const u64x2 *>(p + i);
+                return pair_of<val>{ar.from_residue(t.x), ar.from_residue(t.y)};
+            },
+            [&](uint32_t i, val v) { p[i] = SCALED ? ar.canon(v) : M::bits(v); });
+    }
+}
+
 template <class L, int V, bool FWD, bool SCALED>
 __global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
 ntt_block_kernel(const __grid_constant__ CtxDev c, uint64_t *data, size_t poly_stride, uint32_t limb0,
                          uint32_t nlimbs) {
     extern __shared__ __align__(16) uint64_t sm[];
-    const uint32_t tid = threadIdx.x;
     uint32_t b = blockIdx.x;
     const uint32_t blk = b & ((1u << c.A) - 1u);
     b >>= c.A;
     const uint32_t limb = b % nlimbs;
     const size_t poly = b / nlimbs;
     const LimbDev &lb = c.limb[limb0 + limb];
-    const uint64_t q = lb.q, q2 = 2 * q;
     uint64_t *p = data + poly * poly_stride + (size_t)limb * c.N + ((size_t)blk << L::LOGB);
-    if constexpr (FWD) {
-        const NttArgs a = {lb.fwd, q, q2, c.A, blk};
-        smem_ntt_forward<L, V>(
-            sm, tid, a, [&](uint32_t i) { return p[i]; },
-            [&](uint32_t i, uint64_t u, uint64_t v) {
-                u64x2 o;
-                o.x = csub(csub(u, q2), q);
-                o.y = csub(csub(v, q2), q);
-                *reinterpret_cast<u64x2 *>(p + i) = o;
-            });
-    } else {
-        const NttArgs a = {lb.inv, q, q2, c.A, blk};
-        smem_ntt_inverse<L, V, SCALED>(
-            sm, tid, a, lb.ninv, lb.wn, [&](uint32_t i) { return *reinterpret_cast<const u64x2 *>(p + i); },
-            [&](uint32_t i, uint64_t v) { p[i] = SCALED ? csub(v, q) : v; });
-    }
+    FEDHE_FOR_ARITH(lb, (ntt_block<M_, L, V, FWD, SCALED>(c, lb, sm, p, blk)));
 }
 
 // The A = logN - LOGB outer stages of a long transform on two neighbouring
-// columns of the 2^A x B matrix view (x[a] = row a): forward in [0, 4q) out,
-// inverse [0, 2q) in and canonical out with 1/N folded into stage 0.
-template <uint32_t A>
-__device__ __forceinline__ void outer_forward(u64x2 (&x)[1u << A], const LimbDev &lb) {
-    const uint64_t q = lb.q, q2 = 2 * q;
+// columns of the 2^A x B matrix view (x[a], y[a] = row a): forward from
+// canonical input, inverse with 1/N folded into stage 0.
+template <uint32_t A, class M>
+__device__ __forceinline__ void outer_forward(typename M::val (&x)[1u << A], typename M::val (&y)[1u << A],
+                                              const NttArgsT<M> &t) {
     constexpr uint32_t rows = 1u << A;
 #pragma unroll
     for (uint32_t s = 0; s < A; s++) {
@@ -146,16 +169,16 @@ __device__ __forceinline__ void outer_forward(u64x2 (&x)[1u << A], const LimbDev
 #pragma unroll
         for (uint32_t a = 0; a < rows; a++) {
             if (a & bit) continue;
-            tw_t w = load_tw(lb.fwd + (1u << s) + (a >> (A - s)));
-            ct_butterfly(x[a].x, x[a | bit].x, w.w, w.wp, q, q2);
-            ct_butterfly(x[a].y, x[a | bit].y, w.w, w.wp, q, q2);
+            const auto w = M::load(t.tw + (1u << s) + (a >> (A - s)));
+            t.m.fwd(x[a], x[a | bit], w);
+            t.m.fwd(y[a], y[a | bit], w);
         }
     }
 }
 
-template <uint32_t A>
-__device__ __forceinline__ void outer_inverse(u64x2 (&x)[1u << A], const LimbDev &lb) {
-    const uint64_t q = lb.q, q2 = 2 * q;
+template <uint32_t A, class M, class T>
+__device__ __forceinline__ void outer_inverse(typename M::val (&x)[1u << A], typename M::val (&y)[1u << A],
+                                              const NttArgsT<M> &t, const T &ninv, const T &wn) {
     constexpr uint32_t rows = 1u << A;
 #pragma unroll
     for (int s = (int)A - 1; s >= 1; s--) {
@@ -163,25 +186,45 @@ __device__ __forceinline__ void outer_inverse(u64x2 (&x)[1u << A], const LimbDev
 #pragma unroll
         for (uint32_t a = 0; a < rows; a++) {
             if (a & bit) continue;
-            tw_t w = load_tw(lb.inv + (1u << s) + (a >> (A - s)));
-            gs_butterfly(x[a].x, x[a | bit].x, w.w, w.wp, q, q2);
-            gs_butterfly(x[a].y, x[a | bit].y, w.w, w.wp, q, q2);
+            const auto w = M::load(t.tw + (1u << s) + (a >> (A - s)));
+            t.m.inv(x[a], x[a | bit], w);
+            t.m.inv(y[a], y[a | bit], w);
         }
     }
-    const uint32_t bit = 1u << (A - 1);      // stage 0 with 1/N folded in
+    constexpr uint32_t bit = 1u << (A - 1);      // stage 0 with 1/N folded in
 #pragma unroll
     for (uint32_t a = 0; a < rows; a++) {
         if (a & bit) continue;
-        const uint64_t u0 = x[a].x, v0 = x[a | bit].x, u1 = x[a].y, v1 = x[a | bit].y;
-        x[a].x = shoup(u0 + v0, lb.ninv.w, lb.ninv.wp, q);
-        x[a | bit].x = shoup(u0 - v0 + q2, lb.wn.w, lb.wn.wp, q);
-        x[a].y = shoup(u1 + v1, lb.ninv.w, lb.ninv.wp, q);
-        x[a | bit].y = shoup(u1 - v1 + q2, lb.wn.w, lb.wn.wp, q);
+        t.m.inv_scaled(x[a], x[a | bit], ninv, wn);
+        t.m.inv_scaled(y[a], y[a | bit], ninv, wn);
     }
 }
 
 // The outer stages as an elementwise pass over HBM: every thread owns two
 // neighbouring columns and reads and writes whole 16-byte words.
+template <class M, bool FWD, uint32_t A>
+__device__ __forceinline__ void ntt_outer(const LimbDev &lb, uint64_t *p, uint32_t B) {
+    using val = typename M::val;
+    constexpr uint32_t rows = 1u << A;
+    const auto t = LimbOf<M>::args(lb, FWD, 0, 0);
+    val x[rows], y[rows];
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++) {
+        const u64x2 v = *reinterpret_cast<const u64x2 *>(p + (size_t)a * B);
+        x[a] = FWD ? t.m.from_residue(v.x) : M::from_bits(v.x);
+        y[a] = FWD ? t.m.from_residue(v.y) : M::from_bits(v.y);
+    }
+    if constexpr (FWD) outer_forward<A>(x, y, t);
+    else outer_inverse<A>(x, y, t, LimbOf<M>::ninv(lb), LimbOf<M>::wn(lb));
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++) {
+        u64x2 v;
+        v.x = FWD ? M::bits(x[a]) : t.m.canon(x[a]);
+        v.y = FWD ? M::bits(y[a]) : t.m.canon(y[a]);
+        *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = v;
+    }
+}
+
 template <bool FWD, uint32_t A>
 __global__ void __launch_bounds__(256)
 ntt_outer_kernel(const __grid_constant__ CtxDev c, uint64_t *data, size_t poly_stride, uint32_t limb0,
@@ -194,16 +237,8 @@ ntt_outer_kernel(const __grid_constant__ CtxDev c, uint64_t *data, size_t poly_s
     const uint32_t limb = (uint32_t)(g % nlimbs);
     const size_t poly = g / nlimbs;
     const LimbDev &lb = c.limb[limb0 + limb];
-    const uint64_t q = lb.q, q2 = 2 * q;
     uint64_t *p = data + poly * poly_stride + (size_t)limb * c.N + col;
-    constexpr uint32_t rows = 1u << A;
-    u64x2 x[rows];
-#pragma unroll
-    for (uint32_t a = 0; a < rows; a++) x[a] = *reinterpret_cast<const u64x2 *>(p + (size_t)a * B);
-    if (FWD) outer_forward<A>(x, lb);
-    else outer_inverse<A>(x, lb);
-#pragma unroll
-    for (uint32_t a = 0; a < rows; a++) *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = x[a];
+    FEDHE_FOR_ARITH(lb, (ntt_outer<M_, FWD, A>(lb, p, B)));
 }
 
 // launches kern<A> for the context's A (1, 2 or 3)
@@ -638,6 +673,59 @@ cudaError_t launch_decode(const CtxDev &c, const int64_t *d, size_t T, double2 *
 // encryption:  c0 = pk0 u + e0 + m,  c1 = pk1 u + e1   (mod every q_j)
 // ===========================================================================
 
+// One (ciphertext, limb) unit of the fused path in the limb's arithmetic.
+// u^ pk1^ is parked, in the arithmetic's own form, in the c1 slot it will
+// finally occupy while u^ pk0^ stays in shared memory; then two passes over
+// one copy of the inverse-transform code: h = 0 gives c0 = pk0 u + e0 + m from
+// shared memory, h = 1 reloads the parked product and gives c1 = pk1 u + e1.
+template <class M, class L, int V>
+__device__ __forceinline__ void encrypt_unit(const LimbDev &lb, const tw_t *p0, const tw_t *p1, uint64_t *sm,
+                                             const int8_t *su, const int8_t *se0, const int64_t *mt,
+                                             uint64_t *cbase, size_t cstride) {
+    using val = typename M::val;
+    constexpr uint32_t B = 1u << L::LOGB;
+    const uint32_t tid = threadIdx.x;
+    const uint64_t q = lb.q;
+    {
+        uint64_t *c1 = cbase + cstride;
+        const auto fa = LimbOf<M>::args(lb, true, 0, 0);
+        const M &ar = fa.m;
+        smem_ntt_forward<L, V>(
+            sm, tid, fa, [&](uint32_t i) { return ar.small(su[i]); },
+            [&](uint32_t p, val a, val b) {
+                const auto a0 = M::load_key(p1 + p), a1 = M::load_key(p1 + p + 1);
+                u64x2 v;
+                v.x = M::bits(ar.mul_key(a, a0));
+                v.y = M::bits(ar.mul_key(b, a1));
+                *reinterpret_cast<u64x2 *>(c1 + p) = v;
+                const auto b0 = M::load_key(p0 + p), b1 = M::load_key(p0 + p + 1);
+                sm[swz(p)] = M::bits(ar.mul_key(a, b0));
+                sm[swz(p + 1)] = M::bits(ar.mul_key(b, b1));
+            });
+    }
+#pragma unroll 1
+    for (int h = 0; h < 2; h++) {
+        uint64_t *cc = cbase + h * cstride;
+        const int8_t *se = se0 + h * B;
+        const auto ia = LimbOf<M>::args(lb, false, 0, 0);
+        const M &ar = ia.m;
+        smem_ntt_inverse<L, V, true>(
+            sm, tid, ia, LimbOf<M>::ninv(lb), LimbOf<M>::wn(lb),
+            [&](uint32_t p) {
+                if (h == 0) return pair_of<val>{M::from_bits(sm[swz(p)]), M::from_bits(sm[swz(p + 1)])};
+                const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + p);
+                return pair_of<val>{M::from_bits(t.x), M::from_bits(t.y)};
+            },
+            [&](uint32_t i, val v) {
+                // e1 is a small value; e0 + m needs a full reduction
+                const uint64_t add = h == 0 ? signed_residue(mt[i] + (int64_t)se[i], q, lb.mu)
+                                            : small_residue(se[i], q);
+                cc[i] = ar.canon_add(v, add);
+            });
+        __syncthreads();   // phase-0 readers are done before the next transform writes
+    }
+}
+
 // Fused path for N <= 2^14 (one block holds a whole limb): a thread block
 // draws u, e0, e1 of a ciphertext once into shared memory, then for every
 // limb of it transforms u, multiplies by both halves of the public key,
@@ -689,51 +777,86 @@ encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const in
             }
             __syncthreads();
         }
-        const int64_t *mt = m + (size_t)tl * B;
         const LimbDev &lb = c.limb[j];
-        const uint64_t q = lb.q, q2 = 2 * q;
         uint64_t *cbase = ct + (((size_t)tl * 2 + 0) * c.L + j) * B;
-        {
-            const tw_t *p0 = k.pk0_hat + (size_t)j * B, *p1 = k.pk1_hat + (size_t)j * B;
-            uint64_t *c1 = cbase + cstride;
-            const NttArgs fa = {lb.fwd, q, q2, 0, 0};
-            smem_ntt_forward<L, V>(
-                sm, tid, fa, [&](uint32_t i) { return small_residue(su[i], q); },
-                [&](uint32_t p, uint64_t a, uint64_t b) {
-                    // u^ pk1^ is parked in its final c1 slot until the second pass
-                    // below; u^ pk0^ stays in shared memory for the first pass
-                    const tw_t a0 = load_tw(p1 + p), a1 = load_tw(p1 + p + 1);
-                    u64x2 v;
-                    v.x = shoup_lazy(a, a0.w, a0.wp, q);
-                    v.y = shoup_lazy(b, a1.w, a1.wp, q);
-                    *reinterpret_cast<u64x2 *>(c1 + p) = v;
-                    const tw_t b0 = load_tw(p0 + p), b1 = load_tw(p0 + p + 1);
-                    sm[swz(p)] = shoup_lazy(a, b0.w, b0.wp, q);
-                    sm[swz(p + 1)] = shoup_lazy(b, b1.w, b1.wp, q);
-                });
-        }
-        // two passes over one copy of the inverse-transform code: h = 0 gives
-        // c0 = pk0 u + e0 + m from shared memory, h = 1 reloads the parked
-        // product and gives c1 = pk1 u + e1
+        FEDHE_FOR_ARITH(lb, (encrypt_unit<M_, L, V>(lb, k.pk0_hat + (size_t)j * B, k.pk1_hat + (size_t)j * B, sm, su,
+                                                    se0, m + (size_t)tl * B, cbase, cstride)));
+    }
+}
+
+// One (ciphertext, limb) unit of the two-group kernel below (N = 2 * 2^LOGB).
+template <class M, class L, int V>
+__device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0, const tw_t *pk1, uint64_t *sm,
+                                              const int8_t *su, const int8_t *se0, const int64_t *mt,
+                                              uint64_t *cbase, size_t cstride) {
+    using val = typename M::val;
+    constexpr uint32_t H = 1u << L::LOGB, B = 2 * H;
+    constexpr uint32_t GT = L::NT / V, RT = 2 * GT;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t grp = tid / GT, gt = tid % GT;
+    uint64_t *smg = sm + grp * H;                          // this group's half
+    const GroupSync gsync = {1 + grp, GT};
+    const uint64_t q = lb.q;
+    {
+        const tw_t *p0 = pk0 + grp * H, *p1 = pk1 + grp * H;
+        uint64_t *c1 = cbase + cstride + grp * H;
+        const auto fa = LimbOf<M>::args(lb, true, 1, grp);
+        const M &ar = fa.m;
+        const auto w0 = M::load(fa.tw + 1);                // twiddle of the stage that pairs the halves
+        auto src = [&](uint32_t i) {
+            // u is ternary: the twiddle product is 0, w or -w
+            const int b = su[i + H];
+            if constexpr (std::is_same<M, ModF64>::value) {
+                return f64_fma(grp == 0 ? (double)b : (double)-b, w0, (double)su[i]);
+            } else {
+                const uint64_t u = small_residue(su[i], q);
+                const uint64_t v = b == 0 ? 0 : (b > 0 ? w0.w : q - w0.w);
+                return grp == 0 ? u + v : u - v + ar.q2;
+            }
+        };
+        auto dst = [&](uint32_t p, val a, val b) {
+            const auto a0 = M::load_key(p1 + p), a1 = M::load_key(p1 + p + 1);
+            u64x2 v;
+            v.x = M::bits(ar.mul_key(a, a0));
+            v.y = M::bits(ar.mul_key(b, a1));
+            *reinterpret_cast<u64x2 *>(c1 + p) = v;      // parked until the second pass
+            const auto b0 = M::load_key(p0 + p), b1 = M::load_key(p0 + p + 1);
+            smg[swz(p)] = M::bits(ar.mul_key(a, b0));
+            smg[swz(p + 1)] = M::bits(ar.mul_key(b, b1));
+        };
+        smem_ntt_forward<L, V>(smg, gt, fa, src, dst, gsync);
+    }
 #pragma unroll 1
-        for (int h = 0; h < 2; h++) {
-            uint64_t *cc = cbase + h * cstride;
-            const int8_t *se = se0 + h * B;
-            const NttArgs ia = {lb.inv, q, q2, 0, 0};
-            smem_ntt_inverse<L, V, true>(
-                sm, tid, ia, lb.ninv, lb.wn,
-                [&](uint32_t p) {
-                    if (h == 0) return u64x2{sm[swz(p)], sm[swz(p + 1)]};
-                    return *reinterpret_cast<const u64x2 *>(cc + p);
-                },
-                [&](uint32_t i, uint64_t v) {
-                    // e1 is a small value; e0 + m needs a full reduction
-                    const uint64_t add = h == 0 ? signed_residue(mt[i] + (int64_t)se[i], q, lb.mu)
-                                                : small_residue(se[i], q);
-                    cc[i] = addmod(csub(v, q), add, q);
-                });
-            __syncthreads();   // phase-0 readers are done before the next transform writes
+    for (int h = 0; h < 2; h++) {
+        uint64_t *cc = cbase + h * cstride;
+        const int8_t *se = se0 + h * B;
+        const auto ia = LimbOf<M>::args(lb, false, 1, grp);
+        const M &ar = ia.m;
+        const auto ninv = LimbOf<M>::ninv(lb), wn = LimbOf<M>::wn(lb);
+        auto isrc = [&](uint32_t p) {
+            if (h == 0) return pair_of<val>{M::from_bits(smg[swz(p)]), M::from_bits(smg[swz(p + 1)])};
+            const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + grp * H + p);
+            return pair_of<val>{M::from_bits(t.x), M::from_bits(t.y)};
+        };
+        auto idst = [&](uint32_t i, val v) { smg[swz(i)] = M::bits(v); };
+        smem_ntt_inverse<L, V, false>(smg, gt, ia, ninv, wn, isrc, idst, gsync);
+        __syncthreads();
+        // last stage across the halves with 1/N folded in, then the error / message terms
+        for (uint32_t e = tid; e < H; e += RT) {
+            val lo = M::from_bits(sm[swz(e)]), hi = M::from_bits(sm[H + swz(e)]);
+            ar.inv_scaled(lo, hi, ninv, wn);
+            uint64_t add_lo, add_hi;
+            if (h == 0) {
+                add_lo = signed_residue(mt[e] + (int64_t)se[e], q, lb.mu);
+                add_hi = signed_residue(mt[e + H] + (int64_t)se[e + H], q, lb.mu);
+            } else {
+                add_lo = small_residue(se[e], q);
+                add_hi = small_residue(se[e + H], q);
+            }
+            cc[e] = ar.canon_add(lo, add_lo);
+            cc[e + H] = ar.canon_add(hi, add_hi);
         }
+        __syncthreads();
     }
 }
 
@@ -755,9 +878,6 @@ encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const i
     int8_t *su = reinterpret_cast<int8_t *>(sm + B);
     int8_t *se0 = su + B, *se1 = se0 + B;
     const uint32_t tid = threadIdx.x;
-    const uint32_t grp = tid / GT, gt = tid % GT;
-    uint64_t *smg = sm + grp * H;                          // this group's half
-    const GroupSync gsync = {1 + grp, GT};
     __shared__ GaussTables gt_tab;
     gauss_tables_init(gt_tab, tid);
 
@@ -790,69 +910,10 @@ encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const i
             }
             __syncthreads();
         }
-        const int64_t *mt = m + (size_t)tl * B;
         const LimbDev &lb = c.limb[j];
-        const uint64_t q = lb.q, q2 = 2 * q;
-        // primes below 2^45 run the transforms without conditional subtractions:
-        // 13 growing stages keep every value below 2^14 q < 2^59
-        const bool small_q = q < (1ull << 45);
-        const uint64_t diff_bound = small_q ? q << L::LOGB + 1 : q2;
         uint64_t *cbase = ct + (((size_t)tl * 2 + 0) * c.L + j) * B;
-        {
-            const tw_t *p0 = k.pk0_hat + (size_t)j * B + grp * H, *p1 = k.pk1_hat + (size_t)j * B + grp * H;
-            uint64_t *c1 = cbase + cstride + grp * H;
-            const uint64_t w0 = load_tw(lb.fwd + 1).w;     // twiddle of the stage that pairs the halves
-            const NttArgs fa = {lb.fwd, q, q2, 1, grp};
-            auto src = [&](uint32_t i) {
-                const int b = su[i + H];
-                const uint64_t u = small_residue(su[i], q);
-                const uint64_t v = b == 0 ? 0 : (b > 0 ? w0 : q - w0);
-                return grp == 0 ? u + v : u - v + q2;
-            };
-            auto dst = [&](uint32_t p, uint64_t a, uint64_t b) {
-                const tw_t a0 = load_tw(p1 + p), a1 = load_tw(p1 + p + 1);
-                u64x2 v;
-                v.x = shoup_lazy(a, a0.w, a0.wp, q);
-                v.y = shoup_lazy(b, a1.w, a1.wp, q);
-                *reinterpret_cast<u64x2 *>(c1 + p) = v;      // parked until the second pass
-                const tw_t b0 = load_tw(p0 + p), b1 = load_tw(p0 + p + 1);
-                smg[swz(p)] = shoup_lazy(a, b0.w, b0.wp, q);
-                smg[swz(p + 1)] = shoup_lazy(b, b1.w, b1.wp, q);
-            };
-            if (small_q) smem_ntt_forward<L, V, true>(smg, gt, fa, src, dst, gsync);
-            else smem_ntt_forward<L, V, false>(smg, gt, fa, src, dst, gsync);
-        }
-#pragma unroll 1
-        for (int h = 0; h < 2; h++) {
-            uint64_t *cc = cbase + h * cstride;
-            const int8_t *se = se0 + h * B;
-            const NttArgs ia = {lb.inv, q, q2, 1, grp};
-            auto isrc = [&](uint32_t p) {
-                if (h == 0) return u64x2{smg[swz(p)], smg[swz(p + 1)]};
-                return *reinterpret_cast<const u64x2 *>(cc + grp * H + p);
-            };
-            auto idst = [&](uint32_t i, uint64_t v) { smg[swz(i)] = v; };
-            if (small_q) smem_ntt_inverse<L, V, false, true>(smg, gt, ia, lb.ninv, lb.wn, isrc, idst, gsync);
-            else smem_ntt_inverse<L, V, false, false>(smg, gt, ia, lb.ninv, lb.wn, isrc, idst, gsync);
-            __syncthreads();
-            // last stage across the halves with 1/N folded in, then the error / message terms
-            for (uint32_t e = tid; e < H; e += RT) {
-                const uint64_t a = sm[swz(e)], b = sm[H + swz(e)];
-                const uint64_t lo = shoup(a + b, lb.ninv.w, lb.ninv.wp, q);
-                const uint64_t hi = shoup(a - b + diff_bound, lb.wn.w, lb.wn.wp, q);
-                uint64_t add_lo, add_hi;
-                if (h == 0) {
-                    add_lo = signed_residue(mt[e] + (int64_t)se[e], q, lb.mu);
-                    add_hi = signed_residue(mt[e + H] + (int64_t)se[e + H], q, lb.mu);
-                } else {
-                    add_lo = small_residue(se[e], q);
-                    add_hi = small_residue(se[e + H], q);
-                }
-                cc[e] = addmod(lo, add_lo, q);
-                cc[e + H] = addmod(hi, add_hi, q);
-            }
-            __syncthreads();
-        }
+        FEDHE_FOR_ARITH(lb, (encrypt_unit2<M_, L, V>(lb, k.pk0_hat + (size_t)j * B, k.pk1_hat + (size_t)j * B, sm, su,
+                                                     se0, m + (size_t)tl * B, cbase, cstride)));
     }
 }
 
@@ -862,6 +923,23 @@ encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const i
 // (2) block transforms of the c1 slots whose last phase writes both products
 // u^ pk0^ -> c0 and u^ pk1^ -> c1; (3) inverse block transforms of all slots;
 // (4) outer inverse stages fused with the error and message terms.
+
+template <class M, uint32_t A>
+__device__ __forceinline__ void enc_outer_sample_limb(const LimbDev &lb, const int (&u)[1u << A][2], uint64_t *p,
+                                                      uint32_t B) {
+    constexpr uint32_t rows = 1u << A;
+    const auto t = LimbOf<M>::args(lb, true, 0, 0);
+    typename M::val x[rows], y[rows];
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++) {
+        x[a] = t.m.small(u[a][0]);
+        y[a] = t.m.small(u[a][1]);
+    }
+    outer_forward<A>(x, y, t);
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++)
+        *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = u64x2{M::bits(x[a]), M::bits(y[a])};
+}
 
 // (1) one thread per pair of neighbouring columns of one ciphertext, all limbs
 template <uint32_t A>
@@ -885,47 +963,78 @@ enc_outer_sample_kernel(const __grid_constant__ CtxDev c, uint32_t t0, uint64_t 
 #pragma unroll 1
     for (uint32_t j = 0; j < c.L; j++) {
         const LimbDev &lb = c.limb[j];
-        u64x2 x[rows];
-#pragma unroll
-        for (uint32_t a = 0; a < rows; a++) x[a] = u64x2{small_residue(u[a][0], lb.q), small_residue(u[a][1], lb.q)};
-        outer_forward<A>(x, lb);
         uint64_t *p = ct + ((tl * 2 + 1) * c.L + j) * c.N + col;
-#pragma unroll
-        for (uint32_t a = 0; a < rows; a++) *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = x[a];
+        FEDHE_FOR_ARITH(lb, (enc_outer_sample_limb<M_, A>(lb, u, p, B)));
     }
 }
 
 // (2) one thread block per (ciphertext, limb, block): forward block transform of
 // the c1 slot, products with both halves of the public key on the way out
+template <class M, class L, int V>
+__device__ __forceinline__ void enc_block_forward(const CtxDev &c, const LimbDev &lb, uint64_t *sm, uint32_t blk,
+                                                  const tw_t *p0, const tw_t *p1, uint64_t *c0, uint64_t *c1) {
+    using val = typename M::val;
+    const auto a = LimbOf<M>::args(lb, true, c.A, blk);
+    const M &ar = a.m;
+    smem_ntt_forward<L, V>(
+        sm, threadIdx.x, a, [&](uint32_t i) { return M::from_bits(c1[i]); },
+        [&](uint32_t p, val x, val y) {
+            const auto a0 = M::load_key(p0 + p), a1 = M::load_key(p0 + p + 1);
+            const auto b0 = M::load_key(p1 + p), b1 = M::load_key(p1 + p + 1);
+            u64x2 v0, v1;
+            v0.x = ar.to_residue(ar.mul_key(x, a0));
+            v0.y = ar.to_residue(ar.mul_key(y, a1));
+            v1.x = ar.to_residue(ar.mul_key(x, b0));
+            v1.y = ar.to_residue(ar.mul_key(y, b1));
+            *reinterpret_cast<u64x2 *>(c0 + p) = v0;
+            *reinterpret_cast<u64x2 *>(c1 + p) = v1;
+        });
+}
+
 template <class L, int V>
 __global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
 enc_block_forward_kernel(const __grid_constant__ CtxDev c, const KeysDev k, uint64_t *ct) {
     extern __shared__ __align__(16) uint64_t sm[];
-    const uint32_t tid = threadIdx.x;
     uint32_t b = blockIdx.x;
     const uint32_t blk = b & ((1u << c.A) - 1u);
     b >>= c.A;
     const uint32_t j = b % c.L;
     const size_t tl = b / c.L;
     const LimbDev &lb = c.limb[j];
-    const uint64_t q = lb.q, q2 = 2 * q;
     const size_t off = ((size_t)blk << L::LOGB);
     uint64_t *c0 = ct + ((tl * 2 + 0) * c.L + j) * c.N + off;
     uint64_t *c1 = ct + ((tl * 2 + 1) * c.L + j) * c.N + off;
     const tw_t *p0 = k.pk0_hat + (size_t)j * c.N + off, *p1 = k.pk1_hat + (size_t)j * c.N + off;
-    const NttArgs a = {lb.fwd, q, q2, c.A, blk};
-    smem_ntt_forward<L, V>(
-        sm, tid, a, [&](uint32_t i) { return c1[i]; },
-        [&](uint32_t p, uint64_t x, uint64_t y) {
-            const tw_t a0 = load_tw(p0 + p), a1 = load_tw(p0 + p + 1), b0 = load_tw(p1 + p), b1 = load_tw(p1 + p + 1);
-            u64x2 v0, v1;
-            v0.x = shoup_lazy(x, a0.w, a0.wp, q);
-            v0.y = shoup_lazy(y, a1.w, a1.wp, q);
-            v1.x = shoup_lazy(x, b0.w, b0.wp, q);
-            v1.y = shoup_lazy(y, b1.w, b1.wp, q);
-            *reinterpret_cast<u64x2 *>(c0 + p) = v0;
-            *reinterpret_cast<u64x2 *>(c1 + p) = v1;
-        });
+    FEDHE_FOR_ARITH(lb, (enc_block_forward<M_, L, V>(c, lb, sm, blk, p0, p1, c0, c1)));
+}
+
+template <class M, uint32_t A>
+__device__ __forceinline__ void enc_outer_inverse_add_limb(const LimbDev &lb, uint64_t *p, uint32_t B, bool first,
+                                                           const int64_t (&me0)[1u << A][2],
+                                                           const int (&e1)[1u << A][2]) {
+    constexpr uint32_t rows = 1u << A;
+    const uint64_t q = lb.q;
+    const auto t = LimbOf<M>::args(lb, false, 0, 0);
+    typename M::val x[rows], y[rows];
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++) {
+        const u64x2 v = *reinterpret_cast<const u64x2 *>(p + (size_t)a * B);
+        x[a] = M::from_bits(v.x);
+        y[a] = M::from_bits(v.y);
+    }
+    outer_inverse<A>(x, y, t, LimbOf<M>::ninv(lb), LimbOf<M>::wn(lb));
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++) {
+        u64x2 o;
+        if (first) {
+            o.x = t.m.canon_add(x[a], signed_residue(me0[a][0], q, lb.mu));
+            o.y = t.m.canon_add(y[a], signed_residue(me0[a][1], q, lb.mu));
+        } else {
+            o.x = t.m.canon_add(x[a], small_residue(e1[a][0], q));
+            o.y = t.m.canon_add(y[a], small_residue(e1[a][1], q));
+        }
+        *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = o;
+    }
 }
 
 // (4) one thread per pair of neighbouring columns of one ciphertext: draws the
@@ -957,26 +1066,10 @@ enc_outer_inverse_add_kernel(const __grid_constant__ CtxDev c, const int64_t *m,
 #pragma unroll 1
     for (uint32_t j = 0; j < c.L; j++) {
         const LimbDev &lb = c.limb[j];
-        const uint64_t q = lb.q;
 #pragma unroll 1
         for (uint32_t comp = 0; comp < 2; comp++) {
             uint64_t *p = ct + ((tl * 2 + comp) * c.L + j) * c.N + col;
-            u64x2 x[rows];
-#pragma unroll
-            for (uint32_t a = 0; a < rows; a++) x[a] = *reinterpret_cast<const u64x2 *>(p + (size_t)a * B);
-            outer_inverse<A>(x, lb);
-#pragma unroll
-            for (uint32_t a = 0; a < rows; a++) {
-                u64x2 o;
-                if (comp == 0) {
-                    o.x = addmod(x[a].x, signed_residue(me0[a][0], q, lb.mu), q);
-                    o.y = addmod(x[a].y, signed_residue(me0[a][1], q, lb.mu), q);
-                } else {
-                    o.x = addmod(x[a].x, small_residue(e1[a][0], q), q);
-                    o.y = addmod(x[a].y, small_residue(e1[a][1], q), q);
-                }
-                *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = o;
-            }
+            FEDHE_FOR_ARITH(lb, (enc_outer_inverse_add_limb<M_, A>(lb, p, B, comp == 0, me0, e1)));
         }
     }
 }
@@ -1200,7 +1293,7 @@ decrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const ui
     const uint64_t q = lb.q, q2 = 2 * q;
     const uint64_t *c0 = ct + ((t * 2 + 0) * level) * B, *c1 = ct + ((t * 2 + 1) * level) * B;
     {
-        const NttArgs fa = {lb.fwd, q, q2, 0, 0};
+        const NttArgs fa = LimbOf<ModInt>::args(lb, true, 0, 0);   // limb 0 carries the message
         smem_ntt_forward<L, V>(
             sm, tid, fa, [&](uint32_t i) { return c1[i]; },
             [&](uint32_t p, uint64_t a, uint64_t b) {
@@ -1211,7 +1304,7 @@ decrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const ui
     }
     int64_t *d = reinterpret_cast<int64_t *>(sm);
     {
-        const NttArgs ia = {lb.inv, q, q2, 0, 0};
+        const NttArgs ia = LimbOf<ModInt>::args(lb, false, 0, 0);
         smem_ntt_inverse<L, V, true>(
             sm, tid, ia, lb.ninv, lb.wn, [&](uint32_t p) { return u64x2{sm[swz(p)], sm[swz(p + 1)]}; },
             [&](uint32_t i, uint64_t v) {

@@ -39,6 +39,8 @@ __device__ __forceinline__ tw_t load_tw(const tw_t *p) {
 #endif
 
 struct alignas(16) u64x2 { uint64_t x, y; };   // two neighbouring residues
+template <class V>
+struct pair_of { V x, y; };                      // two neighbouring values of an arithmetic
 
 // shared-memory index swizzle: makes all phase layouts free of bank conflicts
 // for 8-byte accesses (xor the low nibble with the next one)
@@ -75,20 +77,112 @@ struct Lay {
     }
 };
 
-// ---- phases ----------------------------------------------------------------
+// ---- arithmetic of one limb ---------------------------------------------------
+//
+// ModInt: any prime below 2^62; 64-bit integers in the lazy Harvey ranges
+// (forward [0, 4q), inverse [0, 2q)), table entries {w, floor(w 2^64 / q)}.
+// ModF64: primes below 2^46; signed integers in doubles, table entries the
+// twiddles as doubles.  Forward, every stage adds at most 3q/4 to the bound
+// (q at the input, at most 13q after 16 stages); inverse, sums double and
+// differences go through the product, so after the at most three stages of a
+// phase the sums are brought back below q (settle) before they are stored.
 
-struct NttArgs {
-    const tw_t *tw;      // table of this limb and direction, indexed by the global twiddle index
-    uint64_t q, q2;      // modulus and twice the modulus
-    uint32_t A;          // log2 of the number of blocks the whole transform is cut into
-    uint32_t blk;        // which block this is
+struct ModInt {
+    using val = uint64_t;
+    using tab = tw_t;
+    uint64_t q, q2;
+    static HD val from_bits(uint64_t b) { return b; }
+    static HD uint64_t bits(val v) { return v; }
+    static HD tw_t load(const tw_t *p) { return FEDHE_LD_TW(p); }
+    HD void fwd(val &x, val &y, const tw_t &w) const { ct_butterfly(x, y, w.w, w.wp, q, q2); }
+    HD void inv(val &x, val &y, const tw_t &w) const { gs_butterfly(x, y, w.w, w.wp, q, q2); }
+    // x <- (x + y) a, y <- (x - y) b for inputs below 2q; outputs below 2q
+    HD void inv_scaled(val &x, val &y, const tw_t &a, const tw_t &b) const {
+        const uint64_t u = x, v = y;
+        x = shoup_lazy(u + v, a.w, a.wp, q);
+        y = shoup_lazy(u - v + q2, b.w, b.wp, q);
+    }
+    HD val settle(val v) const { return v; }
+    // conversions: a residue below 2q <-> the value; a small signed integer -> the value
+    HD val from_residue(uint64_t r) const { return r; }
+    HD uint64_t to_residue(val v) const { return v; }
+    HD val small(int v) const { return small_residue(v, q); }
+    // canonical residue of a forward output (below 4q) / of an inverse output (below 2q),
+    // and of an inverse output plus a residue in [0, q)
+    HD uint64_t canon_wide(val v) const { return csub(csub(v, q2), q); }
+    HD uint64_t canon(val v) const { return csub(v, q); }
+    HD uint64_t canon_add(val v, uint64_t add) const { return csub(csub(v, q) + add, q); }
+    // product with an entry of a key table, below 2q for any v
+    using key = tw_t;
+    static HD key load_key(const tw_t *p) { return FEDHE_LD_TW(p); }
+    HD val mul_key(val v, const key &k) const { return shoup_lazy(v, k.w, k.wp, q); }
 };
 
-// GROW: no conditional subtractions (small primes only, see the *_grow
-// butterflies): a sub-block's inverse input must lie below 2q, and after k
-// inverse stages the values lie below 2^(k+1) q.
-template <class L, int P, int I, bool GROW = false>
-HD void fwd_stage(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
+struct ModF64 {
+    using val = double;
+    using tab = double;
+    double q, qi;        // the prime and its rounded reciprocal
+    static HD val from_bits(uint64_t b) { return f64_from_bits(b); }
+    static HD uint64_t bits(val v) { return f64_bits(v); }
+    static HD double load(const double *p) {
+#if defined(__CUDA_ARCH__)
+        return __ldg(p);
+#else
+        return *p;
+#endif
+    }
+    HD double mul(double y, double w) const { return f64_mulmod(y, w, q, qi); }
+    HD void fwd(val &x, val &y, double w) const {
+        const double u = x, t = mul(y, w);
+        x = f64_add(u, t);
+        y = f64_sub(u, t);
+    }
+    HD void inv(val &x, val &y, double w) const {
+        const double u = x, v = y;
+        x = f64_add(u, v);
+        y = mul(f64_sub(u, v), w);
+    }
+    HD void inv_scaled(val &x, val &y, double a, double b) const {
+        const double u = x, v = y;
+        x = mul(f64_add(u, v), a);
+        y = mul(f64_sub(u, v), b);
+    }
+    HD val settle(val v) const { return f64_reduce(v, q, qi); }
+    HD val from_residue(uint64_t r) const { return f64_from_u64(r); }
+    HD uint64_t to_residue(val v) const { return f64_canonical(v, q); }          // |v| < q
+    HD val small(int v) const { return (double)v; }
+    HD uint64_t canon_wide(val v) const { return f64_canonical(f64_reduce(v, q, qi), q); }
+    HD uint64_t canon(val v) const { return f64_canonical(v, q); }               // |v| < q
+    HD uint64_t canon_add(val v, uint64_t add) const {                           // |v| < q
+        const double r = f64_add(v, f64_from_u64(add));
+        return f64_canonical(r >= q ? f64_sub(r, q) : r, q);
+    }
+    // only the value of a key-table entry is read; |result| <= 3q/4
+    using key = double;
+    static HD key load_key(const tw_t *p) {
+#if defined(__CUDA_ARCH__)
+        return f64_from_u64(__ldg(&p->w));
+#else
+        return f64_from_u64(p->w);
+#endif
+    }
+    HD val mul_key(val v, key k) const { return mul(v, k); }
+};
+
+// ---- phases ----------------------------------------------------------------
+
+template <class M>
+struct NttArgsT {
+    const typename M::tab *tw;   // table of this limb and direction, indexed by the global twiddle index
+    M m;                         // the limb's arithmetic
+    uint32_t A;                  // log2 of the number of blocks the whole transform is cut into
+    uint32_t blk;                // which block this is
+};
+using NttArgs = NttArgsT<ModInt>;
+using NttArgsF = NttArgsT<ModF64>;
+
+template <class L, int P, int I, class M>
+HD void fwd_stage(typename M::val (&x)[L::E], uint32_t tid, const NttArgsT<M> &a) {
     constexpr int s = P * L::LE + I;
     constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
     constexpr int bit = nst - 1 - I;              // register bit of the pair
@@ -98,15 +192,13 @@ HD void fwd_stage(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
         if (r & (1 << bit)) continue;
         // all registers that agree above the pair bit share one twiddle; the
         // compiler merges the equal loads of an unrolled group
-        const tw_t *pw = a.tw + base + L::template top<P, I>(tid, r);
-        tw_t w = FEDHE_LD_TW(pw);
-        if constexpr (GROW) ct_butterfly_grow(x[r], x[r | (1 << bit)], w.w, w.wp, a.q, a.q2);
-        else ct_butterfly(x[r], x[r | (1 << bit)], w.w, w.wp, a.q, a.q2);
+        const auto w = M::load(a.tw + base + L::template top<P, I>(tid, r));
+        a.m.fwd(x[r], x[r | (1 << bit)], w);
     }
 }
 
-template <class L, int P, int I, bool GROW = false>
-HD void inv_stage(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
+template <class L, int P, int I, class M>
+HD void inv_stage(typename M::val (&x)[L::E], uint32_t tid, const NttArgsT<M> &a) {
     constexpr int s = P * L::LE + I;
     constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
     constexpr int bit = nst - 1 - I;
@@ -114,51 +206,52 @@ HD void inv_stage(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
 #pragma unroll
     for (int r = 0; r < L::E; r++) {
         if (r & (1 << bit)) continue;
-        const tw_t *pw = a.tw + base + L::template top<P, I>(tid, r);
-        tw_t w = FEDHE_LD_TW(pw);
-        // local stage s is the (LOGB - 1 - s)-th to run: inputs lie below 2^(LOGB - s) q
-        if constexpr (GROW) gs_butterfly_grow(x[r], x[r | (1 << bit)], w.w, w.wp, a.q, a.q << (L::LOGB - s));
-        else gs_butterfly(x[r], x[r | (1 << bit)], w.w, w.wp, a.q, a.q2);
+        const auto w = M::load(a.tw + base + L::template top<P, I>(tid, r));
+        a.m.inv(x[r], x[r | (1 << bit)], w);
     }
 }
 
 // last inverse stage of a whole transform (global stage 0) with the factor
 // 1/N folded in: x <- (x + y)/N, y <- (x - y) w /N.  ninv = 1/N, wn = w/N.
-template <class L>
-HD void inv_stage0_scaled(uint64_t (&x)[L::E], tw_t ninv, tw_t wn, uint64_t q, uint64_t q2) {
+template <class L, class M, class T>
+HD void inv_stage0_scaled(typename M::val (&x)[L::E], const M &m, const T &ninv, const T &wn) {
     constexpr int bit = L::LE - 1;
 #pragma unroll
     for (int r = 0; r < L::E; r++) {
         if (r & (1 << bit)) continue;
-        uint64_t u = x[r], v = x[r | (1 << bit)];
-        x[r] = shoup_lazy(u + v, ninv.w, ninv.wp, q);
-        x[r | (1 << bit)] = shoup_lazy(u - v + q2, wn.w, wn.wp, q);
+        m.inv_scaled(x[r], x[r | (1 << bit)], ninv, wn);
     }
 }
 
-template <class L, int P, int I = 0, bool GROW = false>
-HD void fwd_phase(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
+template <class L, int P, int I = 0, class M>
+HD void fwd_phase(typename M::val (&x)[L::E], uint32_t tid, const NttArgsT<M> &a) {
     constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
     if constexpr (I < nst) {
-        fwd_stage<L, P, I, GROW>(x, tid, a);
-        fwd_phase<L, P, I + 1, GROW>(x, tid, a);
+        fwd_stage<L, P, I>(x, tid, a);
+        fwd_phase<L, P, I + 1>(x, tid, a);
     }
 }
 
 // inverse phase: stages nst-1 down to STOP (STOP = 1 leaves stage 0 of the
-// phase to the caller)
-template <class L, int P, int STOP, int I, bool GROW = false>
-HD void inv_phase_from(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
+// phase to the caller); a phase that ends with an ordinary stage settles the
+// sums of that stage (the registers whose pair bit is clear)
+template <class L, int P, int STOP, int I, class M>
+HD void inv_phase_from(typename M::val (&x)[L::E], uint32_t tid, const NttArgsT<M> &a) {
     if constexpr (I >= STOP) {
-        inv_stage<L, P, I, GROW>(x, tid, a);
-        inv_phase_from<L, P, STOP, I - 1, GROW>(x, tid, a);
+        inv_stage<L, P, I>(x, tid, a);
+        inv_phase_from<L, P, STOP, I - 1>(x, tid, a);
+    } else if constexpr (STOP == 0) {
+        constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
+#pragma unroll
+        for (int r = 0; r < L::E; r++)
+            if (!(r & (1 << (nst - 1)))) x[r] = a.m.settle(x[r]);
     }
 }
 
-template <class L, int P, int STOP = 0, bool GROW = false>
-HD void inv_phase(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
+template <class L, int P, int STOP = 0, class M>
+HD void inv_phase(typename M::val (&x)[L::E], uint32_t tid, const NttArgsT<M> &a) {
     constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
-    inv_phase_from<L, P, STOP, nst - 1, GROW>(x, tid, a);
+    inv_phase_from<L, P, STOP, nst - 1>(x, tid, a);
 }
 
 #if defined(__CUDACC__)
@@ -171,7 +264,8 @@ HD void inv_phase(uint64_t (&x)[L::E], uint32_t tid, const NttArgs &a) {
 // no spills) and no separate exchange buffer is needed.  The first phase takes its input
 // from `src`, the last hands its output to `dst`:
 //   forward:  src(i) -> residue i;            dst(i, a, b): residues i, i+1
-//   inverse:  src(i) -> residues i, i+1;      dst(i, a): residue i
+//   inverse:  src(i) -> residues i, i+1 (members x, y);   dst(i, a): residue i
+// all in the value type of the limb's arithmetic
 // (pairs always start at an even index and are neighbours in memory).
 // ---------------------------------------------------------------------------
 
@@ -188,74 +282,73 @@ struct GroupSync {
     }
 };
 
-template <class L, int V, bool GROW = false, class Src, class Dst, class Sync = BlockSync, int P = 0>
-__device__ __forceinline__ void smem_ntt_forward(uint64_t *sm, uint32_t tid, const NttArgs &a, const Src &src,
+template <class L, int V, class M, class Src, class Dst, class Sync = BlockSync, int P = 0>
+__device__ __forceinline__ void smem_ntt_forward(uint64_t *sm, uint32_t tid, const NttArgsT<M> &a, const Src &src,
                                                  const Dst &dst, const Sync &sync = Sync()) {
     constexpr int RT = L::NT / V, LAST = L::NPH - 1;
 #pragma unroll 1
     for (int v = 0; v < V; v++) {
         const uint32_t vt = tid + v * RT;
-        uint64_t x[L::E];
+        typename M::val x[L::E];
 #pragma unroll
         for (int r = 0; r < L::E; r++) {
             const uint32_t i = L::template idx<P>(vt, r);
             if constexpr (P == 0) x[r] = src(i);
-            else x[r] = sm[swz(i)];
+            else x[r] = M::from_bits(sm[swz(i)]);
         }
-        fwd_phase<L, P, 0, GROW>(x, vt, a);
+        fwd_phase<L, P>(x, vt, a);
         if constexpr (P == LAST) {
 #pragma unroll
             for (int r = 0; r < L::E; r += 2) dst(L::template idx<P>(vt, r), x[r], x[r + 1]);
         } else {
 #pragma unroll
-            for (int r = 0; r < L::E; r++) sm[swz(L::template idx<P>(vt, r))] = x[r];
+            for (int r = 0; r < L::E; r++) sm[swz(L::template idx<P>(vt, r))] = M::bits(x[r]);
         }
     }
     if constexpr (P < LAST) {
         sync();
-        smem_ntt_forward<L, V, GROW, Src, Dst, Sync, P + 1>(sm, tid, a, src, dst, sync);
+        smem_ntt_forward<L, V, M, Src, Dst, Sync, P + 1>(sm, tid, a, src, dst, sync);
     }
 }
 
-template <class L, int V, bool SCALED, bool GROW = false, class Src, class Dst, class Sync = BlockSync,
+template <class L, int V, bool SCALED, class M, class T, class Src, class Dst, class Sync = BlockSync,
           int P = L::NPH - 1>
-__device__ __forceinline__ void smem_ntt_inverse(uint64_t *sm, uint32_t tid, const NttArgs &a, tw_t ninv,
-                                                 tw_t wn, const Src &src, const Dst &dst,
+__device__ __forceinline__ void smem_ntt_inverse(uint64_t *sm, uint32_t tid, const NttArgsT<M> &a, const T &ninv,
+                                                 const T &wn, const Src &src, const Dst &dst,
                                                  const Sync &sync = Sync()) {
     constexpr int RT = L::NT / V, LAST = L::NPH - 1;
 #pragma unroll 1
     for (int v = 0; v < V; v++) {
         const uint32_t vt = tid + v * RT;
-        uint64_t x[L::E];
+        typename M::val x[L::E];
         if constexpr (P == LAST) {
 #pragma unroll
             for (int r = 0; r < L::E; r += 2) {
-                const u64x2 t = src(L::template idx<P>(vt, r));
+                const auto t = src(L::template idx<P>(vt, r));
                 x[r] = t.x;
                 x[r + 1] = t.y;
             }
         } else {
 #pragma unroll
-            for (int r = 0; r < L::E; r++) x[r] = sm[swz(L::template idx<P>(vt, r))];
+            for (int r = 0; r < L::E; r++) x[r] = M::from_bits(sm[swz(L::template idx<P>(vt, r))]);
         }
-        static_assert(!(SCALED && GROW), "the scaled last stage expects inputs below 2q");
         if constexpr (P == 0 && SCALED) {
             inv_phase<L, 0, 1>(x, vt, a);
-            inv_stage0_scaled<L>(x, ninv, wn, a.q, a.q2);
+            inv_stage0_scaled<L>(x, a.m, ninv, wn);
         } else {
-            inv_phase<L, P, 0, GROW>(x, vt, a);
+            inv_phase<L, P, 0>(x, vt, a);
         }
         if constexpr (P == 0) {
 #pragma unroll
             for (int r = 0; r < L::E; r++) dst(L::template idx<0>(vt, r), x[r]);
         } else {
 #pragma unroll
-            for (int r = 0; r < L::E; r++) sm[swz(L::template idx<P>(vt, r))] = x[r];
+            for (int r = 0; r < L::E; r++) sm[swz(L::template idx<P>(vt, r))] = M::bits(x[r]);
         }
     }
     if constexpr (P > 0) {
         sync();
-        smem_ntt_inverse<L, V, SCALED, GROW, Src, Dst, Sync, P - 1>(sm, tid, a, ninv, wn, src, dst, sync);
+        smem_ntt_inverse<L, V, SCALED, M, T, Src, Dst, Sync, P - 1>(sm, tid, a, ninv, wn, src, dst, sync);
     }
 }
 #endif
