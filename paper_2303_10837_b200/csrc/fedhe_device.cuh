@@ -96,7 +96,9 @@ HD uint64_t barrett64(uint64_t x, uint64_t q, uint64_t mu) {
 // residue in [0, q) of a signed 64-bit integer
 HD uint64_t signed_residue(int64_t v, uint64_t q, uint64_t mu) {
     uint64_t a = v < 0 ? (uint64_t)0 - (uint64_t)v : (uint64_t)v;
-    uint64_t r = barrett64(a, q, mu);
+    // encoded updates are far below the primes, so a warp rarely needs the reduction
+    uint64_t r = a;
+    if (a >= q) r = barrett64(a, q, mu);
     return (v < 0 && r != 0) ? q - r : r;
 }
 

@@ -77,6 +77,48 @@ struct Lay {
     }
 };
 
+// ---- runs of consecutive table entries ---------------------------------------
+//
+// Inside a phase the twiddles of stage I of one thread are 2^I consecutive
+// table entries starting at a multiple of 2^I, so they come in with 16- and
+// 32-byte loads (one address computation each) instead of one load per entry.
+template <int K>
+HD void load_run(const double *p, double (&w)[K]) {
+#if defined(__CUDA_ARCH__)
+    if constexpr (K == 1) {
+        w[0] = __ldg(p);
+    } else if constexpr (K == 2) {
+        const double2 v = __ldg(reinterpret_cast<const double2 *>(p));
+        w[0] = v.x;
+        w[1] = v.y;
+    } else {
+#pragma unroll
+        for (int i = 0; i < K; i += 4)
+            asm("ld.global.nc.v4.f64 {%0,%1,%2,%3}, [%4];"
+                : "=d"(w[i]), "=d"(w[i + 1]), "=d"(w[i + 2]), "=d"(w[i + 3])
+                : "l"(p + i));
+    }
+#else
+    for (int i = 0; i < K; i++) w[i] = p[i];
+#endif
+}
+template <int K>
+HD void load_run(const tw_t *p, tw_t (&w)[K]) {
+#if defined(__CUDA_ARCH__)
+    if constexpr (K == 1) {
+        w[0] = load_tw(p);
+    } else {
+#pragma unroll
+        for (int i = 0; i < K; i += 2)
+            asm("ld.global.nc.v4.u64 {%0,%1,%2,%3}, [%4];"
+                : "=l"(w[i].w), "=l"(w[i].wp), "=l"(w[i + 1].w), "=l"(w[i + 1].wp)
+                : "l"(p + i));
+    }
+#else
+    for (int i = 0; i < K; i++) w[i] = p[i];
+#endif
+}
+
 // ---- arithmetic of one limb ---------------------------------------------------
 //
 // ModInt: any prime below 2^62; 64-bit integers in the lazy Harvey ranges
@@ -181,33 +223,64 @@ struct NttArgsT {
 using NttArgs = NttArgsT<ModInt>;
 using NttArgsF = NttArgsT<ModF64>;
 
+// twiddles of local stage s = P LE + I for the registers of one thread:
+// w[g] serves the butterflies whose lower register has r >> (nst - I) == g
+template <class L, int P, int I, class M>
+HD void stage_twiddles(typename M::tab (&w)[1 << I], uint32_t tid, const NttArgsT<M> &a) {
+    constexpr int s = P * L::LE + I;
+    const uint32_t base = (1u << (a.A + s)) + (a.blk << s);
+    static_assert(P < L::NPH - 1, "in the last phase the registers of a group are far apart in the index");
+    constexpr int lo = L::LOGB - (P + 1) * L::LE;
+    load_run<1 << I>(a.tw + base + ((tid >> lo) << I), w);
+}
+
 template <class L, int P, int I, class M>
 HD void fwd_stage(typename M::val (&x)[L::E], uint32_t tid, const NttArgsT<M> &a) {
-    constexpr int s = P * L::LE + I;
     constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
     constexpr int bit = nst - 1 - I;              // register bit of the pair
-    const uint32_t base = (1u << (a.A + s)) + (a.blk << s);
+    if constexpr (P < L::NPH - 1) {
+        typename M::tab w[1 << I];
+        stage_twiddles<L, P, I>(w, tid, a);
 #pragma unroll
-    for (int r = 0; r < L::E; r++) {
-        if (r & (1 << bit)) continue;
-        // all registers that agree above the pair bit share one twiddle; the
-        // compiler merges the equal loads of an unrolled group
-        const auto w = M::load(a.tw + base + L::template top<P, I>(tid, r));
-        a.m.fwd(x[r], x[r | (1 << bit)], w);
+        for (int r = 0; r < L::E; r++) {
+            if (r & (1 << bit)) continue;
+            a.m.fwd(x[r], x[r | (1 << bit)], w[r >> (nst - I)]);
+        }
+    } else {
+        constexpr int s = P * L::LE + I;
+        const uint32_t base = (1u << (a.A + s)) + (a.blk << s);
+#pragma unroll
+        for (int r = 0; r < L::E; r++) {
+            if (r & (1 << bit)) continue;
+            // registers that agree above the pair bit share one twiddle; the
+            // compiler merges the equal loads of an unrolled group
+            const auto w = M::load(a.tw + base + L::template top<P, I>(tid, r));
+            a.m.fwd(x[r], x[r | (1 << bit)], w);
+        }
     }
 }
 
 template <class L, int P, int I, class M>
 HD void inv_stage(typename M::val (&x)[L::E], uint32_t tid, const NttArgsT<M> &a) {
-    constexpr int s = P * L::LE + I;
     constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
     constexpr int bit = nst - 1 - I;
-    const uint32_t base = (1u << (a.A + s)) + (a.blk << s);
+    if constexpr (P < L::NPH - 1) {
+        typename M::tab w[1 << I];
+        stage_twiddles<L, P, I>(w, tid, a);
 #pragma unroll
-    for (int r = 0; r < L::E; r++) {
-        if (r & (1 << bit)) continue;
-        const auto w = M::load(a.tw + base + L::template top<P, I>(tid, r));
-        a.m.inv(x[r], x[r | (1 << bit)], w);
+        for (int r = 0; r < L::E; r++) {
+            if (r & (1 << bit)) continue;
+            a.m.inv(x[r], x[r | (1 << bit)], w[r >> (nst - I)]);
+        }
+    } else {
+        constexpr int s = P * L::LE + I;
+        const uint32_t base = (1u << (a.A + s)) + (a.blk << s);
+#pragma unroll
+        for (int r = 0; r < L::E; r++) {
+            if (r & (1 << bit)) continue;
+            const auto w = M::load(a.tw + base + L::template top<P, I>(tid, r));
+            a.m.inv(x[r], x[r | (1 << bit)], w);
+        }
     }
 }
 

@@ -147,6 +147,30 @@ def test_encrypt_aggregate_decrypt_bit_exact(he, w):
     assert he.he_ctx_status(g) == he.HE_OK
 
 
+@pytest.mark.parametrize("base", [si.TINY, si.RESNET18, si.bert(1.0)], ids=lambda w: w.name)
+def test_encrypt_large_messages_bit_exact(he, base):
+    """Encoded coefficients above the small primes and close to the large ones: the full
+    reduction of m + e0 and every wrap of the final additions, next to a ciphertext of
+    ordinary small updates in the same call."""
+    w = si.scaled(base, 3 * base.n, clients=1)
+    g, o = contexts(he, w.N, w.primes, w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    _, pk_o = o.keygen(w.key_seed)
+    rng = np.random.default_rng(77)
+    big = 2.0 ** (58.7 - w.log2_delta) * np.sqrt(w.n)  # slot deviation that gives coefficients up to about 2^60.3
+    x = np.concatenate([rng.normal(0, 0.01, w.n), rng.normal(0, big, w.n),
+                        np.where(rng.random(w.n) < 0.05, rng.normal(0, big, w.n), 0.0)])
+    x = x.astype(np.float32)
+    m = he.he_encode(g, dev_f32(x)).cpu().numpy()
+    assert he.he_ctx_status(g) == he.HE_OK
+    assert np.abs(m[0]).max() < min(w.primes) and np.abs(m[2]).max() > min(w.primes)
+    assert max(w.primes) < np.abs(m[1]).max() < 2**62
+    ct = he.he_encrypt(g, keys, dev_f32(x), w.enc_seed, 0)
+    ct_o, bad = o.encrypt(pk_o, x, w.enc_seed, 0)
+    assert bad == 0
+    assert np.array_equal(to_host_u64(ct), ct_o)
+
+
 def test_dropout_subset_of_clients(he):
     """Aggregating any subset with renormalised weights needs no new keys."""
     w = si.scaled(si.RESNET18, 8192 + 11, clients=4, name="r18-dropout")
