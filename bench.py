@@ -37,20 +37,38 @@ import synthetic_inputs as si
 METRIC = "HE-agg params/s (encrypt+weighted sum+decrypt); NTT % of HBM roofline"
 UNIT = "params/s"
 
-# Integer roofline of the transforms.  On B200 every integer multiply goes
-# through one pipe that retires 64 32-bit multiply-adds per SM and clock
-# (measured: 63.8), and a 32x32->64 multiply-add costs 2.5 of those slots
-# (measured: 25.5 per SM and clock) with the int_pipe_bench tool of the package.
-# A 64-bit Shoup butterfly needs at least the high half of x*w' (4 wide
-# products) and the low halves of x*w and hi*q (1 wide + 2 narrow each):
-# 6 wide + 4 narrow = 19 multiply slots.  Additions go to another pipe.
-# DRAM bytes (read + write) per ciphertext of encrypt_fused_kernel at N = 16384,
+# Roofline of the transforms.  On B200 integer multiplies and double-precision
+# operations draw on one budget of 64 slots per SM and clock (measured with the
+# int_pipe_bench tool of the package: 63.7 32-bit multiply-adds, 63.6
+# double-precision FMAs, and no gain from running half of each side by side);
+# a 32x32->64 multiply-add costs 2.5 of those slots.  A 64-bit Shoup butterfly
+# needs the high half of x*w' (4 wide products) and the low halves of x*w and
+# hi*q (1 wide + 2 narrow each): 6 wide + 4 narrow = 19 slots.  Limbs whose
+# prime is below 2^46 run in exact double-precision arithmetic instead: 6
+# operations for the modular product, 2 for the sum and difference, and in the
+# inverse transform 1 more per butterfly for keeping the sums small.
+# Additions, shifts and logic go to another pipe.
+# DRAM bytes (read + write) per ciphertext of encrypt_fused2_kernel at N = 16384,
 # L = 4, from an ncu capture of the profile_case.py encrypt case (summary under profiles/)
-# (363.6 MB for 296 ciphertexts; traffic grows in proportion to the count).
-ENCRYPT_DRAM_BYTES_PER_CT_N16384_L4 = 363.57248e6 / 296
-IMAD_PER_SM_CLK = 64.0
+# (374.5 MB for 296 ciphertexts; traffic grows in proportion to the count).
+ENCRYPT_DRAM_BYTES_PER_CT_N16384_L4 = 374.5472e6 / 296
+SLOTS_PER_SM_CLK = 64.0
 WIDE_COST = 2.5
-MUL_SLOTS_PER_BUTTERFLY = 6 * WIDE_COST + 4
+INT_SLOTS_PER_BUTTERFLY = 6 * WIDE_COST + 4
+F64_SLOTS_FORWARD, F64_SLOTS_INVERSE = 8.0, 9.0
+F64_PRIME_LIMIT = 1 << 46
+
+
+def transform_slots(primes, N, forward, inverse):
+    """Pipe slots of `forward` forward and `inverse` inverse transforms of every limb."""
+    bf = (N // 2) * (N.bit_length() - 1)
+    total = 0.0
+    for q in primes:
+        if q < F64_PRIME_LIMIT:
+            total += bf * (forward * F64_SLOTS_FORWARD + inverse * F64_SLOTS_INVERSE)
+        else:
+            total += bf * (forward + inverse) * INT_SLOTS_PER_BUTTERFLY
+    return total
 
 
 def fallback_peaks():
@@ -357,17 +375,18 @@ def run_ours(args, w):
             dist.destroy_process_group()
         return
 
-    # roofline of the dominant kernel (bound by the integer-multiply pipe)
+    # roofline of the dominant kernel (bound by the multiply / double-precision pipe)
     logN = w.N.bit_length() - 1
     butterflies = 3 * w.L * (w.N // 2) * logN * T           # per launch: 3 limb transforms per limb
-    achieved = butterflies * MUL_SLOTS_PER_BUTTERFLY / (kern_ms * 1e-3) / 1e12
+    achieved = transform_slots(w.primes, w.N, 1, 2) * T / (kern_ms * 1e-3) / 1e12
     n_sm = torch.cuda.get_device_properties(local).multi_processor_count
-    peak = n_sm * IMAD_PER_SM_CLK * peaks["sm_max_mhz"] * 1e6 / 1e12
+    peak = n_sm * SLOTS_PER_SM_CLK * peaks["sm_max_mhz"] * 1e6 / 1e12
     alg_bytes = (16.0 + 32.0 * w.L) * n * T          # read m, write the ciphertext
     roofline = {
-        "kernel": "encrypt_fused_kernel" if w.N <= 16384 else "ntt_block_kernel (inside he_encrypt)",
+        "kernel": ("encrypt_fused2_kernel" if w.N == 16384 else "encrypt_fused_kernel") if w.N <= 16384
+                  else "enc_block_forward_kernel + ntt_block_kernel (inside he_encrypt)",
         "bound": "alu", "achieved": achieved, "peak": peak,
-        "unit": "T multiply-slots/s (32-bit integer multiply pipe)",
+        "unit": "T slots/s (integer-multiply / double-precision pipe)",
         "frac": achieved / peak,
         "traffic": ENCRYPT_DRAM_BYTES_PER_CT_N16384_L4 * T if (w.N == 16384 and w.L == 4) else None,
         "algorithmic_bytes": alg_bytes,
@@ -376,9 +395,10 @@ def run_ours(args, w):
         "hbm_frac_of_kernel": alg_bytes / (kern_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
         "ntt_standalone": {"gbs": ntt_gbs, "hbm_frac": ntt_gbs / peaks["hbm_gbs"], "ms": ntt_ms,
                            "batch_polys": B, "bytes_per_launch": pass_bytes,
-                           "mul_pipe_frac": (B * w.L * (w.N // 2) * logN * MUL_SLOTS_PER_BUTTERFLY
+                           "mul_pipe_frac": (B * transform_slots(w.primes, w.N, 0.5, 0.5)
                                              / (ntt_ms * 1e-3) / 1e12) / peak},
-        "peak_source": "integer-multiply pipe: SM count x 64 per clock (microbenchmark) x max SM clock; "
+        "f64_limbs": sum(1 for q in w.primes if q < F64_PRIME_LIMIT),
+        "peak_source": "multiply / double-precision pipe: SM count x 64 per clock (microbenchmark) x max SM clock; "
                        + peaks["source"] + " hbm_gbs for the HBM fractions",
     }
 
@@ -390,7 +410,7 @@ def run_ours(args, w):
     line = {
         "metric": METRIC, "value": units / job_secs, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * job_secs / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": "u64 (limbs below 2^46: exact f64)", "data": "synthetic",
         "config": config_dict(w, "every rank runs its own full batch; no collective on the path"),
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"] or peaks["sm_max_mhz"],
                    "reasons": clocks["reasons"], "samples": clocks["samples"]},

@@ -130,6 +130,7 @@ HD void load_run(const tw_t *p, tw_t (&w)[K]) {
 // phase the sums are brought back below q (settle) before they are stored.
 
 struct ModInt {
+    static constexpr int UNROLL_V = 1;   // virtual threads of a phase one after the other
     using val = uint64_t;
     using tab = tw_t;
     uint64_t q, q2;
@@ -161,6 +162,7 @@ struct ModInt {
 };
 
 struct ModF64 {
+    static constexpr int UNROLL_V = 2;
     using val = double;
     using tab = double;
     double q, qi;        // the prime and its rounded reciprocal
@@ -359,7 +361,7 @@ template <class L, int V, class M, class Src, class Dst, class Sync = BlockSync,
 __device__ __forceinline__ void smem_ntt_forward(uint64_t *sm, uint32_t tid, const NttArgsT<M> &a, const Src &src,
                                                  const Dst &dst, const Sync &sync = Sync()) {
     constexpr int RT = L::NT / V, LAST = L::NPH - 1;
-#pragma unroll 1
+#pragma unroll M::UNROLL_V
     for (int v = 0; v < V; v++) {
         const uint32_t vt = tid + v * RT;
         typename M::val x[L::E];
@@ -390,7 +392,7 @@ __device__ __forceinline__ void smem_ntt_inverse(uint64_t *sm, uint32_t tid, con
                                                  const T &wn, const Src &src, const Dst &dst,
                                                  const Sync &sync = Sync()) {
     constexpr int RT = L::NT / V, LAST = L::NPH - 1;
-#pragma unroll 1
+#pragma unroll M::UNROLL_V
     for (int v = 0; v < V; v++) {
         const uint32_t vt = tid + v * RT;
         typename M::val x[L::E];
