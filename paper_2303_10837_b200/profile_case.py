@@ -3,7 +3,7 @@
     python paper_2303_10837_b200/profile_case.py encrypt [--cts 296] [--reps 2]
     python paper_2303_10837_b200/profile_case.py ntt [--polys 256]
     python paper_2303_10837_b200/profile_case.py aggregate [--cts 64]
-    python paper_2303_10837_b200/profile_case.py sweep            # kernel sweep table (no profiler)
+    python paper_2303_10837_b200/profile_case.py sweep [--prime-bits 45]   # kernel sweep table (no profiler)
 
 Each case touches more memory than the L2 holds so that DRAM counters mean something,
 launches the kernel of interest a handful of times and exits.
@@ -45,24 +45,24 @@ def timed(fn, reps):
     return ev0.elapsed_time(ev1) / reps
 
 
-def sweep():
+def sweep(bits=60):
     """Batched forward+inverse NTT and encode+encrypt over ring degrees, limb counts and batch
     sizes; GB/s counts 16 N bytes per limb transform (32 N for N > 2^14: two passes) and the
     ciphertext bytes written per encryption."""
     peak, src = read_hbm_peak()
-    print("HBM peak %.1f GB/s (%s)" % (peak, src))
+    print("HBM peak %.1f GB/s (%s); %d-bit primes" % (peak, src, bits))
     print("%6s %3s %6s | %10s %9s %7s | %10s %9s %7s" % ("N", "L", "batch", "ntt us", "GB/s", "%HBM", "encrypt us", "GB/s", "%HBM"))
     for logn in (13, 14, 15, 16):
         N = 1 << logn
         for L in (2, 4, 8, 12):
-            primes = si.PRIMES_SWEEP[:L]
+            primes = (si.PRIMES_SWEEP if bits == 60 else si.PRIMES_SWEEP_45)[:L]
             g = he.he_ctx_create(N, list(primes), 40)
             keys = he.he_keygen(g, 5)
             for B in (1, 4, 16, 64, 256, 1024, 4096):
                 words = B * L * N
                 if words * 8 > 8 << 30 or 2 * words * 8 > 12 << 30:
                     continue
-                polys = torch.randint(0, 1 << 59, (B, L, N), dtype=torch.int64, device="cuda")
+                polys = torch.randint(0, 1 << (bits - 1), (B, L, N), dtype=torch.int64, device="cuda")   # below every prime
                 reps = 3 if words > (1 << 26) else 10
 
                 def both():
@@ -90,9 +90,11 @@ def main():
     ap.add_argument("--polys", type=int, default=256)
     ap.add_argument("--reps", type=int, default=2)
     ap.add_argument("--workload", choices=["resnet18", "tiny", "bert"], default="resnet18")
+    ap.add_argument("--prime-bits", type=int, choices=[60, 45], default=60,
+                    help="sweep: 60-bit primes (integer transforms) or 45-bit primes (double-precision transforms)")
     a = ap.parse_args()
     if a.case == "sweep":
-        sweep()
+        sweep(a.prime_bits)
         return
     base = {"resnet18": si.RESNET18, "tiny": si.TINY, "bert": si.bert(1.0)}[a.workload]
     w = si.scaled(base, a.cts * base.n, clients=base.clients)

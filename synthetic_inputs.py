@@ -63,6 +63,10 @@ PRIMES_N32768 = (0xffffffffffc0001, 0x1fffffcf0001, 0x1fffffc20001, 0x1fffffbf00
 PRIMES_SWEEP = (0xffffffffffc0001, 0xfffffffff840001, 0xfffffffff6a0001, 0xfffffffff5a0001,
                 0xfffffffff2a0001, 0xfffffffff240001, 0xffffffffefe0001, 0xffffffffeca0001,
                 0xffffffffe9e0001, 0xffffffffe7c0001, 0xffffffffe740001, 0xffffffffe520001)
+# the same with twelve 45-bit primes
+PRIMES_SWEEP_45 = (0x1fffffc20001, 0x1fffff980001, 0x1fffff7e0001, 0x1fffff360001,
+                   0x1fffff060001, 0x1ffffede0001, 0x1ffffeca0001, 0x1ffffeb40001,
+                   0x1ffffe760001, 0x1ffffe640001, 0x1ffffe520001, 0x1ffffe0c0001)
 
 TINY = Workload("tiny-3c-100k", 8192, PRIMES_N8192, 40, 3, 100_000, 0.02,
                 weights="dataset", seed=1, key_seed=11, enc_seed=12)
