@@ -1,7 +1,9 @@
 // CUDA kernels (sm_100a) of the FedML-HE secure-aggregation hot path and their
 // launch wrappers.  Nothing here is a dense floating-point contraction, so no
-// tensor-core path exists: the transforms are bound by 64-bit integer
-// multiply throughput, the pointwise passes by HBM bandwidth.
+// tensor-core path exists: the transforms are bound by the issue rate of
+// integer multiplies (limbs with large primes) and double-precision
+// operations (limbs with primes below 2^46), the pointwise passes by HBM
+// bandwidth.
 #include "fedhe_launch.h"
 
 #include <atomic>
