@@ -170,6 +170,27 @@ int he_decrypt(he_ctx *ctx, const he_keys *keys, const uint64_t *agg_dev, size_t
 int he_decrypt_level(he_ctx *ctx, const he_keys *keys, const uint64_t *ct_dev, uint32_t level, size_t T,
                      double *z_dev, void *stream);
 
+/* Transform-domain wire format (an alternative to the coefficient-domain
+ * ciphertexts above; the paper leaves the ciphertext representation to its HE
+ * library, Section 3.2 / API table).  Same layout and sizes, but every limb
+ * polynomial is stored as its negacyclic transform
+ *   A^[k] = sum_j a_j psi^((2 brev(k) + 1) j) mod q,
+ * psi the smallest primitive 2N-th root of unity, brev over log2 N bits, i.e.
+ * exactly he_ntt_forward of the coefficient-domain ciphertext.  The three
+ * calls mirror he_encrypt, he_weighted_aggregate and he_decrypt_level:
+ * encryption costs the same 3L limb transforms (all forward), the server's
+ * weighted sum stays pointwise but its rescale needs 2L limb transforms per
+ * ciphertext index (last limb back, rounding term forward for every other
+ * limb), decryption saves one transform.  Arguments, ownership and errors as
+ * for the coefficient-domain calls; mixing the two formats in one call is not
+ * detected (the bytes are valid residues either way). */
+int he_encrypt_ntt(he_ctx *ctx, const he_keys *keys, const float *sel_dev, size_t k, uint64_t seed,
+                   uint32_t client_id, uint64_t *ct_dev, void *stream);
+int he_weighted_aggregate_ntt(he_ctx *ctx, const uint64_t *const *cts_host, const double *alpha_host,
+                              int C, size_t T, uint64_t *agg_dev, void *stream);
+int he_decrypt_level_ntt(he_ctx *ctx, const he_keys *keys, const uint64_t *ct_dev, uint32_t level, size_t T,
+                         double *z_dev, void *stream);
+
 /* (No counterpart in the paper.)  he_decrypt for callers that must not
  * allocate: a process that has given all free device memory to its own pool,
  * or a latency-critical loop that cannot take the device-wide synchronisation

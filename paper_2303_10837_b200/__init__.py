@@ -70,6 +70,9 @@ _SIGS = {
     "he_encrypt": (C.c_int, [_vp, _vp, _vp, _sz, _u64, _u32, _vp, _vp]),
     "he_encrypt_range": (C.c_int, [_vp, _vp, _vp, _sz, _sz, _u64, _u32, _vp, _vp]),
     "he_weighted_aggregate": (C.c_int, [_vp, _vp, _vp, C.c_int, _sz, _vp, _vp]),
+    "he_encrypt_ntt": (C.c_int, [_vp, _vp, _vp, _sz, _u64, _u32, _vp, _vp]),
+    "he_weighted_aggregate_ntt": (C.c_int, [_vp, _vp, _vp, C.c_int, _sz, _vp, _vp]),
+    "he_decrypt_level_ntt": (C.c_int, [_vp, _vp, _vp, _u32, _sz, _vp, _vp]),
     "he_plain_aggregate": (C.c_int, [_vp, _vp, _vp, C.c_int, _sz, _vp, _vp]),
     "he_decrypt": (C.c_int, [_vp, _vp, _vp, _sz, _vp, _vp]),
     "he_decrypt_level": (C.c_int, [_vp, _vp, _vp, _u32, _sz, _vp, _vp]),
@@ -256,6 +259,17 @@ def he_encrypt(ctx: Ctx, keys: Keys, sel: torch.Tensor, seed: int, client_id: in
     return out
 
 
+def he_encrypt_ntt(ctx: Ctx, keys: Keys, sel: torch.Tensor, seed: int, client_id: int,
+                   out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """The same ciphertexts in the transform-domain wire format."""
+    T = sel.numel() // ctx.n
+    if out is None:
+        out = torch.empty((T, 2, ctx.L, ctx.N), dtype=torch.int64, device="cuda")
+    _check(_lib.he_encrypt_ntt(ctx.handle, keys.handle, _dev(sel, torch.float32), sel.numel(), seed, client_id,
+                               _dev(out, torch.int64), _stream()), "he_encrypt_ntt")
+    return out
+
+
 def he_encrypt_range(ctx: Ctx, keys: Keys, sel: torch.Tensor, t_begin: int, t_count: int, seed: int,
                      client_id: int, out: torch.Tensor) -> torch.Tensor:
     """`sel` holds the slots of ciphertexts t_begin .. t_begin+t_count-1."""
@@ -274,6 +288,19 @@ def he_weighted_aggregate(ctx: Ctx, cts: List[torch.Tensor], alpha: Sequence[flo
         out = torch.empty((T, 2, ctx.L - 1, ctx.N), dtype=torch.int64, device="cuda")
     _check(_lib.he_weighted_aggregate(ctx.handle, C.cast(ptrs, _vp), C.cast(al, _vp), Cn, T,
                                       _dev(out, torch.int64), _stream()), "he_weighted_aggregate")
+    return out
+
+
+def he_weighted_aggregate_ntt(ctx: Ctx, cts: List[torch.Tensor], alpha: Sequence[float],
+                              out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    Cn = len(cts)
+    T = cts[0].shape[0]
+    ptrs = (_vp * Cn)(*[_dev(c, torch.int64) for c in cts])
+    al = (C.c_double * Cn)(*[float(a) for a in alpha])
+    if out is None:
+        out = torch.empty((T, 2, ctx.L - 1, ctx.N), dtype=torch.int64, device="cuda")
+    _check(_lib.he_weighted_aggregate_ntt(ctx.handle, C.cast(ptrs, _vp), C.cast(al, _vp), Cn, T,
+                                          _dev(out, torch.int64), _stream()), "he_weighted_aggregate_ntt")
     return out
 
 
@@ -303,6 +330,16 @@ def he_decrypt_level(ctx: Ctx, keys: Keys, ct: torch.Tensor, level: int) -> torc
     _check(_lib.he_decrypt_level(ctx.handle, keys.handle, _dev(ct, torch.int64), level, T, z.data_ptr(),
                                  _stream()), "he_decrypt_level")
     return z
+
+
+def he_decrypt_level_ntt(ctx: Ctx, keys: Keys, ct: torch.Tensor, level: int,
+                         out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    T = ct.shape[0]
+    if out is None:
+        out = torch.empty(T * ctx.n, dtype=torch.float64, device="cuda")
+    _check(_lib.he_decrypt_level_ntt(ctx.handle, keys.handle, _dev(ct, torch.int64), level, T,
+                                     _dev(out, torch.float64), _stream()), "he_decrypt_level_ntt")
+    return out
 
 
 def he_threshold_split(ctx: Ctx, keys: Keys, seed: int):

@@ -423,21 +423,38 @@ int he_encode(he_ctx *ctx, const float *sel_dev, size_t k, int64_t *m_dev, void 
     return HE_OK;
 }
 
-int he_encrypt_range(he_ctx *ctx, const he_keys *keys, const float *sel_dev, size_t t_begin, size_t t_count,
-                     uint64_t seed, uint32_t client_id, uint64_t *ct_dev, void *stream) {
+static int encrypt_range(he_ctx *ctx, const he_keys *keys, const float *sel_dev, size_t t_begin, size_t t_count,
+                         uint64_t seed, uint32_t client_id, bool ntt_out, uint64_t *ct_dev, void *stream) {
     if (!good(ctx) || !good(keys) || keys->ctx != ctx || keys->is_share) return HE_ERR_INVALID_ARG;
     if (t_begin + t_count >= (1ull << 32)) return HE_ERR_SIZE;
     if (t_count == 0) return HE_OK;
     if (!sel_dev || !ct_dev) return HE_ERR_INVALID_ARG;
     const CtxDev &d = ctx->dev;
-    int rc = ensure(&ctx->ws, &ctx->ws_bytes, work_bytes(ctx, t_count));
+    // transform-domain output on the long rings transforms u in a work buffer of its own
+    const size_t u_words = (ntt_out && d.A > 0) ? t_count * (size_t)d.L * d.N : 0;
+    int rc = ensure(&ctx->ws, &ctx->ws_bytes, work_bytes(ctx, t_count) + u_words * sizeof(uint64_t));
     if (rc != HE_OK) return rc;
     int64_t *m = static_cast<int64_t *>(ctx->ws);
     double2 *cplx = reinterpret_cast<double2 *>(m + t_count * d.N);
+    uint64_t *ubuf = reinterpret_cast<uint64_t *>(m + 2 * t_count * d.N);
     cudaStream_t st = as_stream(stream);
     CU(launch_encode(d, sel_dev, t_count, cplx, m, st));
-    CU(launch_encrypt(d, keys->dev, m, (uint32_t)t_begin, t_count, seed, client_id, ct_dev, st));
+    if (ntt_out)
+        CU(launch_encrypt_ntt(d, keys->dev, m, (uint32_t)t_begin, t_count, seed, client_id, ubuf, ct_dev, st));
+    else
+        CU(launch_encrypt(d, keys->dev, m, (uint32_t)t_begin, t_count, seed, client_id, ct_dev, st));
     return HE_OK;
+}
+
+int he_encrypt_range(he_ctx *ctx, const he_keys *keys, const float *sel_dev, size_t t_begin, size_t t_count,
+                     uint64_t seed, uint32_t client_id, uint64_t *ct_dev, void *stream) {
+    return encrypt_range(ctx, keys, sel_dev, t_begin, t_count, seed, client_id, false, ct_dev, stream);
+}
+
+int he_encrypt_ntt(he_ctx *ctx, const he_keys *keys, const float *sel_dev, size_t k, uint64_t seed,
+                   uint32_t client_id, uint64_t *ct_dev, void *stream) {
+    if (!good(ctx)) return HE_ERR_INVALID_ARG;
+    return encrypt_range(ctx, keys, sel_dev, 0, he_num_ct(ctx, k), seed, client_id, true, ct_dev, stream);
 }
 
 int he_encrypt(he_ctx *ctx, const he_keys *keys, const float *sel_dev, size_t k, uint64_t seed,
@@ -446,8 +463,8 @@ int he_encrypt(he_ctx *ctx, const he_keys *keys, const float *sel_dev, size_t k,
     return he_encrypt_range(ctx, keys, sel_dev, 0, he_num_ct(ctx, k), seed, client_id, ct_dev, stream);
 }
 
-int he_weighted_aggregate(he_ctx *ctx, const uint64_t *const *cts_host, const double *alpha_host, int C,
-                          size_t T, uint64_t *agg_dev, void *stream) {
+static int weighted_aggregate(he_ctx *ctx, const uint64_t *const *cts_host, const double *alpha_host, int C,
+                              size_t T, bool ntt, uint64_t *agg_dev, void *stream) {
     if (!good(ctx) || !cts_host || !alpha_host || C < 1) return HE_ERR_INVALID_ARG;
     if (C > HE_MAX_CLIENTS) return HE_ERR_SIZE;
     if (T && !agg_dev) return HE_ERR_INVALID_ARG;
@@ -475,8 +492,24 @@ int he_weighted_aggregate(he_ctx *ctx, const uint64_t *const *cts_host, const do
     CU(cudaMemcpyAsync(ctx->tab, host.data(), host.size(), cudaMemcpyHostToDevice, st));
     const uint64_t *const *dptrs = static_cast<const uint64_t *const *>(ctx->tab);
     const tw_t *dw = reinterpret_cast<const tw_t *>(static_cast<unsigned char *>(ctx->tab) + C * sizeof(void *));
-    CU(launch_aggregate(d, dptrs, dw, C, T, agg_dev, st));
+    if (ntt) {
+        int rc = ensure(&ctx->ws, &ctx->ws_bytes, 2 * T * (size_t)L * d.N * sizeof(uint64_t));
+        if (rc != HE_OK) return rc;
+        CU(launch_aggregate_ntt(d, dptrs, dw, C, T, static_cast<uint64_t *>(ctx->ws), agg_dev, st));
+    } else {
+        CU(launch_aggregate(d, dptrs, dw, C, T, agg_dev, st));
+    }
     return HE_OK;
+}
+
+int he_weighted_aggregate(he_ctx *ctx, const uint64_t *const *cts_host, const double *alpha_host, int C,
+                          size_t T, uint64_t *agg_dev, void *stream) {
+    return weighted_aggregate(ctx, cts_host, alpha_host, C, T, false, agg_dev, stream);
+}
+
+int he_weighted_aggregate_ntt(he_ctx *ctx, const uint64_t *const *cts_host, const double *alpha_host, int C,
+                              size_t T, uint64_t *agg_dev, void *stream) {
+    return weighted_aggregate(ctx, cts_host, alpha_host, C, T, true, agg_dev, stream);
 }
 
 int he_plain_aggregate(he_ctx *ctx, const float *const *rests_host, const double *alpha_host, int C,
@@ -503,15 +536,15 @@ int he_plain_aggregate(he_ctx *ctx, const float *const *rests_host, const double
     return HE_OK;
 }
 
-int he_decrypt_level(he_ctx *ctx, const he_keys *keys, const uint64_t *ct_dev, uint32_t level, size_t T,
-                     double *z_dev, void *stream) {
+static int decrypt_level(he_ctx *ctx, const he_keys *keys, const uint64_t *ct_dev, uint32_t level, size_t T,
+                         bool ntt_in, double *z_dev, void *stream) {
     if (!good(ctx) || !good(keys) || keys->ctx != ctx || keys->is_share) return HE_ERR_INVALID_ARG;
     if (level < 1 || level > ctx->dev.L) return HE_ERR_LEVEL;
     if (T == 0) return HE_OK;
     if (!ct_dev || !z_dev) return HE_ERR_INVALID_ARG;
     const CtxDev &d = ctx->dev;
     if (d.logN <= 14) {                 // one fused kernel, no work buffer
-        CU(launch_decrypt_fused(d, keys->dev, ct_dev, level, T, z_dev, as_stream(stream)));
+        CU(launch_decrypt_fused(d, keys->dev, ct_dev, level, T, ntt_in, z_dev, as_stream(stream)));
         return HE_OK;
     }
     int rc = ensure(&ctx->ws, &ctx->ws_bytes, work_bytes(ctx, T));
@@ -519,9 +552,20 @@ int he_decrypt_level(he_ctx *ctx, const he_keys *keys, const uint64_t *ct_dev, u
     uint64_t *scratch = static_cast<uint64_t *>(ctx->ws);
     double2 *cplx = reinterpret_cast<double2 *>(scratch + T * d.N);
     cudaStream_t st = as_stream(stream);
-    CU(launch_decrypt(d, keys->dev, ct_dev, level, T, scratch, st));
+    if (ntt_in) CU(launch_decrypt_ntt(d, keys->dev, ct_dev, level, T, scratch, st));
+    else CU(launch_decrypt(d, keys->dev, ct_dev, level, T, scratch, st));
     CU(launch_decode(d, reinterpret_cast<const int64_t *>(scratch), T, cplx, z_dev, st));
     return HE_OK;
+}
+
+int he_decrypt_level(he_ctx *ctx, const he_keys *keys, const uint64_t *ct_dev, uint32_t level, size_t T,
+                     double *z_dev, void *stream) {
+    return decrypt_level(ctx, keys, ct_dev, level, T, false, z_dev, stream);
+}
+
+int he_decrypt_level_ntt(he_ctx *ctx, const he_keys *keys, const uint64_t *ct_dev, uint32_t level, size_t T,
+                         double *z_dev, void *stream) {
+    return decrypt_level(ctx, keys, ct_dev, level, T, true, z_dev, stream);
 }
 
 int he_decrypt(he_ctx *ctx, const he_keys *keys, const uint64_t *agg_dev, size_t T, double *z_dev, void *stream) {

@@ -680,7 +680,7 @@ cudaError_t launch_decode(const CtxDev &c, const int64_t *d, size_t T, double2 *
 // finally occupy while u^ pk0^ stays in shared memory; then two passes over
 // one copy of the inverse-transform code: h = 0 gives c0 = pk0 u + e0 + m from
 // shared memory, h = 1 reloads the parked product and gives c1 = pk1 u + e1.
-template <class M, class L, int V>
+template <class M, class L, int V, bool NTT_OUT>
 __device__ __forceinline__ void encrypt_unit(const LimbDev &lb, const tw_t *p0, const tw_t *p1, uint64_t *sm,
                                              const int8_t *su, const int8_t *se0, const int64_t *mt,
                                              uint64_t *cbase, size_t cstride) {
@@ -688,6 +688,40 @@ __device__ __forceinline__ void encrypt_unit(const LimbDev &lb, const tw_t *p0, 
     constexpr uint32_t B = 1u << L::LOGB;
     const uint32_t tid = threadIdx.x;
     const uint64_t q = lb.q;
+    if constexpr (NTT_OUT) {
+        // transform-domain output: c0^ = pk0^ u^ + (e0 + m)^, c1^ = pk1^ u^ + e1^.  Both
+        // products wait in their final slots for the transforms of the error terms.
+        const auto fa = LimbOf<M>::args(lb, true, 0, 0);
+        const M &ar = fa.m;
+        smem_ntt_forward<L, V>(
+            sm, tid, fa, [&](uint32_t i) { return ar.small(su[i]); },
+            [&](uint32_t p, val a, val b) {
+                const auto a0 = M::load_key(p0 + p), a1 = M::load_key(p0 + p + 1);
+                const auto b0 = M::load_key(p1 + p), b1 = M::load_key(p1 + p + 1);
+                *reinterpret_cast<u64x2 *>(cbase + p) = u64x2{M::bits(ar.mul_key(a, a0)), M::bits(ar.mul_key(b, a1))};
+                *reinterpret_cast<u64x2 *>(cbase + cstride + p) =
+                    u64x2{M::bits(ar.mul_key(a, b0)), M::bits(ar.mul_key(b, b1))};
+            });
+#pragma unroll 1
+        for (int h = 0; h < 2; h++) {
+            uint64_t *cc = cbase + h * cstride;
+            const int8_t *se = se0 + h * B;
+            __syncthreads();   // last-phase readers are done before the next transform writes
+            smem_ntt_forward<L, V>(
+                sm, tid, fa,
+                [&](uint32_t i) {
+                    return h == 0 ? ar.from_residue(signed_residue(mt[i] + (int64_t)se[i], q, lb.mu))
+                                  : ar.small(se[i]);
+                },
+                [&](uint32_t p, val a, val b) {
+                    const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + p);
+                    *reinterpret_cast<u64x2 *>(cc + p) =
+                        u64x2{ar.canon_sum(a, M::from_bits(t.x)), ar.canon_sum(b, M::from_bits(t.y))};
+                });
+        }
+        __syncthreads();
+        return;
+    }
     {
         uint64_t *c1 = cbase + cstride;
         const auto fa = LimbOf<M>::args(lb, true, 0, 0);
@@ -734,7 +768,7 @@ __device__ __forceinline__ void encrypt_unit(const LimbDev &lb, const tw_t *p0, 
 // transforms back and adds the error (and message) terms.  Only the
 // ciphertext itself is written to global memory; the second product waits,
 // in transform order, in the c1 slot it will finally occupy.
-template <class L, int V>
+template <class L, int V, bool NTT_OUT>
 __global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
 encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const int64_t *m, uint32_t t0,
                      uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
@@ -781,13 +815,13 @@ encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const in
         }
         const LimbDev &lb = c.limb[j];
         uint64_t *cbase = ct + (((size_t)tl * 2 + 0) * c.L + j) * B;
-        FEDHE_FOR_ARITH(lb, (encrypt_unit<M_, L, V>(lb, k.pk0_hat + (size_t)j * B, k.pk1_hat + (size_t)j * B, sm, su,
+        FEDHE_FOR_ARITH(lb, (encrypt_unit<M_, L, V, NTT_OUT>(lb, k.pk0_hat + (size_t)j * B, k.pk1_hat + (size_t)j * B, sm, su,
                                                     se0, m + (size_t)tl * B, cbase, cstride)));
     }
 }
 
 // One (ciphertext, limb) unit of the two-group kernel below (N = 2 * 2^LOGB).
-template <class M, class L, int V>
+template <class M, class L, int V, bool NTT_OUT>
 __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0, const tw_t *pk1, uint64_t *sm,
                                               const int8_t *su, const int8_t *se0, const int64_t *mt,
                                               uint64_t *cbase, size_t cstride) {
@@ -816,6 +850,47 @@ __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0
                 return grp == 0 ? u + v : u - v + ar.q2;
             }
         };
+        if constexpr (NTT_OUT) {
+            // transform-domain output: both products wait in their final slots for the
+            // transforms of e0 + m and e1, whose pairing stage costs one product per element
+            uint64_t *c0 = cbase + grp * H;
+            smem_ntt_forward<L, V>(smg, gt, fa, src, [&](uint32_t p, val a, val b) {
+                const auto a0 = M::load_key(p0 + p), a1 = M::load_key(p0 + p + 1);
+                const auto b0 = M::load_key(p1 + p), b1 = M::load_key(p1 + p + 1);
+                *reinterpret_cast<u64x2 *>(c0 + p) = u64x2{M::bits(ar.mul_key(a, a0)), M::bits(ar.mul_key(b, a1))};
+                *reinterpret_cast<u64x2 *>(c1 + p) = u64x2{M::bits(ar.mul_key(a, b0)), M::bits(ar.mul_key(b, b1))};
+            }, gsync);
+#pragma unroll 1
+            for (int h = 0; h < 2; h++) {
+                uint64_t *cc = cbase + h * cstride + grp * H;
+                const int8_t *se = se0 + h * B;
+                auto value = [&](uint32_t i) {
+                    return h == 0 ? ar.from_residue(signed_residue(mt[i] + (int64_t)se[i], q, lb.mu))
+                                  : ar.small(se[i]);
+                };
+                gsync();   // last-phase readers of this half are done before phase 0 writes
+                smem_ntt_forward<L, V>(
+                    smg, gt, fa,
+                    [&](uint32_t i) {
+                        const val lo = value(i), hi = value(i + H);
+                        if constexpr (std::is_same<M, ModF64>::value) {
+                            const double t = ar.mul(hi, w0);
+                            return grp == 0 ? f64_add(lo, t) : f64_sub(lo, t);
+                        } else {
+                            const uint64_t t = shoup_lazy(hi, w0.w, w0.wp, q);
+                            return grp == 0 ? lo + t : lo - t + ar.q2;
+                        }
+                    },
+                    [&](uint32_t p, val a, val b) {
+                        const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + p);
+                        *reinterpret_cast<u64x2 *>(cc + p) =
+                            u64x2{ar.canon_sum(a, M::from_bits(t.x)), ar.canon_sum(b, M::from_bits(t.y))};
+                    },
+                    gsync);
+            }
+            __syncthreads();
+            return;
+        }
         auto dst = [&](uint32_t p, val a, val b) {
             const auto a0 = M::load_key(p1 + p), a1 = M::load_key(p1 + p + 1);
             u64x2 v;
@@ -870,7 +945,7 @@ __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0
 // way in for the forward transform (u is ternary, so the twiddle product is
 // 0, w or q-w, computed by both groups from the shared samples) and by the
 // whole block after the two inverse sub-transforms, fused with the epilogue.
-template <class L, int V>
+template <class L, int V, bool NTT_OUT>
 __global__ void __launch_bounds__(2 * L::NT / V, 1)
 encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const int64_t *m, uint32_t t0,
                       uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
@@ -914,7 +989,7 @@ encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const i
         }
         const LimbDev &lb = c.limb[j];
         uint64_t *cbase = ct + (((size_t)tl * 2 + 0) * c.L + j) * B;
-        FEDHE_FOR_ARITH(lb, (encrypt_unit2<M_, L, V>(lb, k.pk0_hat + (size_t)j * B, k.pk1_hat + (size_t)j * B, sm, su,
+        FEDHE_FOR_ARITH(lb, (encrypt_unit2<M_, L, V, NTT_OUT>(lb, k.pk0_hat + (size_t)j * B, k.pk1_hat + (size_t)j * B, sm, su,
                                                      se0, m + (size_t)tl * B, cbase, cstride)));
     }
 }
@@ -943,11 +1018,12 @@ __device__ __forceinline__ void enc_outer_sample_limb(const LimbDev &lb, const i
         *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = u64x2{M::bits(x[a]), M::bits(y[a])};
 }
 
-// (1) one thread per pair of neighbouring columns of one ciphertext, all limbs
+// (1) one thread per pair of neighbouring columns of one ciphertext, all limbs;
+// the limbs of ciphertext tl go to dst + tl * ct_stride
 template <uint32_t A>
 __global__ void __launch_bounds__(256)
 enc_outer_sample_kernel(const __grid_constant__ CtxDev c, uint32_t t0, uint64_t seed, uint32_t client,
-                        uint64_t *ct, size_t total) {
+                        uint64_t *dst, size_t ct_stride, size_t total) {
     size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= total) return;
     const uint32_t B = 1u << c.LOGB, half = B >> 1;
@@ -965,37 +1041,49 @@ enc_outer_sample_kernel(const __grid_constant__ CtxDev c, uint32_t t0, uint64_t 
 #pragma unroll 1
     for (uint32_t j = 0; j < c.L; j++) {
         const LimbDev &lb = c.limb[j];
-        uint64_t *p = ct + ((tl * 2 + 1) * c.L + j) * c.N + col;
+        uint64_t *p = dst + tl * ct_stride + (size_t)j * c.N + col;   // limb j of ciphertext tl
         FEDHE_FOR_ARITH(lb, (enc_outer_sample_limb<M_, A>(lb, u, p, B)));
     }
 }
 
 // (2) one thread block per (ciphertext, limb, block): forward block transform of
 // the c1 slot, products with both halves of the public key on the way out
-template <class M, class L, int V>
+template <class M, class L, int V, bool ACC>
 __device__ __forceinline__ void enc_block_forward(const CtxDev &c, const LimbDev &lb, uint64_t *sm, uint32_t blk,
-                                                  const tw_t *p0, const tw_t *p1, uint64_t *c0, uint64_t *c1) {
+                                                  const tw_t *p0, const tw_t *p1, const uint64_t *u,
+                                                  uint64_t *c0, uint64_t *c1) {
     using val = typename M::val;
     const auto a = LimbOf<M>::args(lb, true, c.A, blk);
     const M &ar = a.m;
     smem_ntt_forward<L, V>(
-        sm, threadIdx.x, a, [&](uint32_t i) { return M::from_bits(c1[i]); },
+        sm, threadIdx.x, a, [&](uint32_t i) { return M::from_bits(u[i]); },
         [&](uint32_t p, val x, val y) {
             const auto a0 = M::load_key(p0 + p), a1 = M::load_key(p0 + p + 1);
             const auto b0 = M::load_key(p1 + p), b1 = M::load_key(p1 + p + 1);
             u64x2 v0, v1;
-            v0.x = ar.to_residue(ar.mul_key(x, a0));
-            v0.y = ar.to_residue(ar.mul_key(y, a1));
-            v1.x = ar.to_residue(ar.mul_key(x, b0));
-            v1.y = ar.to_residue(ar.mul_key(y, b1));
+            if constexpr (ACC) {       // the slots hold canonical residues to add to
+                v0 = *reinterpret_cast<const u64x2 *>(c0 + p);
+                v1 = *reinterpret_cast<const u64x2 *>(c1 + p);
+                v0.x = ar.canon_add(ar.mul_key(x, a0), v0.x);
+                v0.y = ar.canon_add(ar.mul_key(y, a1), v0.y);
+                v1.x = ar.canon_add(ar.mul_key(x, b0), v1.x);
+                v1.y = ar.canon_add(ar.mul_key(y, b1), v1.y);
+            } else {
+                v0.x = ar.to_residue(ar.mul_key(x, a0));
+                v0.y = ar.to_residue(ar.mul_key(y, a1));
+                v1.x = ar.to_residue(ar.mul_key(x, b0));
+                v1.y = ar.to_residue(ar.mul_key(y, b1));
+            }
             *reinterpret_cast<u64x2 *>(c0 + p) = v0;
             *reinterpret_cast<u64x2 *>(c1 + p) = v1;
         });
 }
 
-template <class L, int V>
+// ACC = false: u comes from the c1 slot and the products replace both slots;
+// ACC = true: u comes from `ubuf` ([T][L][N]) and the products are added to the slots
+template <class L, int V, bool ACC>
 __global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
-enc_block_forward_kernel(const __grid_constant__ CtxDev c, const KeysDev k, uint64_t *ct) {
+enc_block_forward_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const uint64_t *ubuf, uint64_t *ct) {
     extern __shared__ __align__(16) uint64_t sm[];
     uint32_t b = blockIdx.x;
     const uint32_t blk = b & ((1u << c.A) - 1u);
@@ -1006,8 +1094,37 @@ enc_block_forward_kernel(const __grid_constant__ CtxDev c, const KeysDev k, uint
     const size_t off = ((size_t)blk << L::LOGB);
     uint64_t *c0 = ct + ((tl * 2 + 0) * c.L + j) * c.N + off;
     uint64_t *c1 = ct + ((tl * 2 + 1) * c.L + j) * c.N + off;
+    const uint64_t *u = ACC ? ubuf + (tl * c.L + j) * c.N + off : c1;
     const tw_t *p0 = k.pk0_hat + (size_t)j * c.N + off, *p1 = k.pk1_hat + (size_t)j * c.N + off;
-    FEDHE_FOR_ARITH(lb, (enc_block_forward<M_, L, V>(c, lb, sm, blk, p0, p1, c0, c1)));
+    FEDHE_FOR_ARITH(lb, (enc_block_forward<M_, L, V, ACC>(c, lb, sm, blk, p0, p1, u, c0, c1)));
+}
+
+// long rings, transform-domain format: residues of e0 + m into the c0 slots and
+// of e1 into the c1 slots; one thread per pair of neighbouring coefficients
+__global__ void __launch_bounds__(256)
+enc_fill_errors_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint32_t t0, uint64_t seed,
+                       uint32_t client, uint64_t *ct, size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t pairs = c.N >> 1;
+    const uint32_t b = (uint32_t)(g % pairs), i = 2 * b;   // one Philox block per pair
+    const size_t tl = g / pairs;
+    const uint32_t t = t0 + (uint32_t)tl;
+    const u32x4 w0 = stream_block(seed, b, t, client, TAG_ENC_E0);
+    const u32x4 w1 = stream_block(seed, b, t, client, TAG_ENC_E1);
+    const longlong2 mm = *reinterpret_cast<const longlong2 *>(m + tl * c.N + i);
+    const int64_t ax = mm.x + gauss_from_u64((uint64_t)w0.x | ((uint64_t)w0.y << 32));
+    const int64_t ay = mm.y + gauss_from_u64((uint64_t)w0.z | ((uint64_t)w0.w << 32));
+    const int ex = gauss_from_u64((uint64_t)w1.x | ((uint64_t)w1.y << 32));
+    const int ey = gauss_from_u64((uint64_t)w1.z | ((uint64_t)w1.w << 32));
+    for (uint32_t j = 0; j < c.L; j++) {
+        const LimbDev &lb = c.limb[j];
+        const uint64_t q = lb.q;
+        *reinterpret_cast<u64x2 *>(ct + ((tl * 2 + 0) * c.L + j) * c.N + i) =
+            u64x2{signed_residue(ax, q, lb.mu), signed_residue(ay, q, lb.mu)};
+        *reinterpret_cast<u64x2 *>(ct + ((tl * 2 + 1) * c.L + j) * c.N + i) =
+            u64x2{small_residue(ex, q), small_residue(ey, q)};
+    }
 }
 
 template <class M, uint32_t A>
@@ -1076,12 +1193,12 @@ enc_outer_inverse_add_kernel(const __grid_constant__ CtxDev c, const int64_t *m,
     }
 }
 
-template <class L, int V, bool TWO_GROUPS>
+template <class L, int V, bool TWO_GROUPS, bool NTT_OUT>
 static cudaError_t launch_encrypt_fused(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0,
                                         size_t T, uint64_t seed, uint32_t client, uint64_t *ct,
                                         cudaStream_t s) {
     const size_t smem = ((sizeof(uint64_t) << L::LOGB) + (3u << L::LOGB)) * (TWO_GROUPS ? 2 : 1);
-    auto kern = TWO_GROUPS ? encrypt_fused2_kernel<L, V> : encrypt_fused_kernel<L, V>;
+    auto kern = TWO_GROUPS ? encrypt_fused2_kernel<L, V, NTT_OUT> : encrypt_fused_kernel<L, V, NTT_OUT>;
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
     // one block per SM (the kernel's shared memory allows no more), fewer if there is less work
@@ -1094,30 +1211,65 @@ static cudaError_t launch_encrypt_fused(const CtxDev &c, const KeysDev &k, const
     return FEDHE_LAUNCHED();
 }
 
+// launches the block forward kernel of the long-ring paths
+template <bool ACC>
+static cudaError_t launch_enc_block_forward(const CtxDev &c, const KeysDev &k, const uint64_t *ubuf, size_t T,
+                                            uint64_t *ct, cudaStream_t s) {
+    using L = Lay<13, 3>;                                 // long rings are cut into 2^13 blocks
+    constexpr int V = 2;
+    const size_t smem = sizeof(uint64_t) << L::LOGB;
+    auto kern = enc_block_forward_kernel<L, V, ACC>;
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+    kern<<<(unsigned)((T * c.L) << c.A), L::NT / V, smem, s>>>(c, k, ubuf, ct);
+    return FEDHE_LAUNCHED();
+}
+
 cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0, size_t T,
                            uint64_t seed, uint32_t client, uint64_t *ct, cudaStream_t s) {
     if (T == 0) return cudaSuccess;
     if (c.A == 0) {
-        if (c.LOGB == 13) return launch_encrypt_fused<Lay<13, 3>, 2, false>(c, k, m, t0, T, seed, client, ct, s);
-        return launch_encrypt_fused<Lay<13, 3>, 2, true>(c, k, m, t0, T, seed, client, ct, s);
+        if (c.LOGB == 13)
+            return launch_encrypt_fused<Lay<13, 3>, 2, false, false>(c, k, m, t0, T, seed, client, ct, s);
+        return launch_encrypt_fused<Lay<13, 3>, 2, true, false>(c, k, m, t0, T, seed, client, ct, s);
     }
     cudaError_t e;
     const size_t cols = T * ((size_t)1 << (c.LOGB - 1));      // pairs of columns
-    FEDHE_FOR_A(c, (enc_outer_sample_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, t0, seed, client, ct, cols)));
+    const size_t LN = (size_t)c.L * c.N;
+    FEDHE_FOR_A(c, (enc_outer_sample_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, t0, seed, client, ct + LN,
+                                                                                     2 * LN, cols)));
     if ((e = FEDHE_LAUNCHED())) return e;
-    {
-        using L = Lay<13, 3>;                                 // long rings are cut into 2^13 blocks
-        constexpr int V = 2;
-        const size_t smem = sizeof(uint64_t) << L::LOGB;
-        auto kern = enc_block_forward_kernel<L, V>;
-        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-        kern<<<(unsigned)((T * c.L) << c.A), L::NT / V, smem, s>>>(c, k, ct);
-        if ((e = FEDHE_LAUNCHED())) return e;
-    }
-    if ((e = launch_ntt_inner(c, false, ct, 2 * T, (size_t)c.L * c.N, 0, c.L, s))) return e;
+    if ((e = launch_enc_block_forward<false>(c, k, nullptr, T, ct, s))) return e;
+    if ((e = launch_ntt_inner(c, false, ct, 2 * T, LN, 0, c.L, s))) return e;
     FEDHE_FOR_A(c, (enc_outer_inverse_add_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, m, t0, seed, client, ct,
                                                                                           cols)));
     return FEDHE_LAUNCHED();
+}
+
+// Transform-domain wire format: the same ciphertext with every limb polynomial
+// stored as its negacyclic transform.  N <= 2^14: the fused kernels with three
+// forward transforms per limb.  Longer rings: the error terms go into the
+// ciphertext slots and are transformed there; u is transformed in the work
+// buffer `ubuf` ([T][L][N]) and its key products are added on the way out.
+cudaError_t launch_encrypt_ntt(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0, size_t T,
+                               uint64_t seed, uint32_t client, uint64_t *ubuf, uint64_t *ct, cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    if (c.A == 0) {
+        if (c.LOGB == 13)
+            return launch_encrypt_fused<Lay<13, 3>, 2, false, true>(c, k, m, t0, T, seed, client, ct, s);
+        return launch_encrypt_fused<Lay<13, 3>, 2, true, true>(c, k, m, t0, T, seed, client, ct, s);
+    }
+    cudaError_t e;
+    const size_t LN = (size_t)c.L * c.N;
+    const size_t pairs = T * (size_t)(c.N >> 1);
+    enc_fill_errors_kernel<<<blocks_for(pairs, 256), 256, 0, s>>>(c, m, t0, seed, client, ct, pairs);
+    if ((e = FEDHE_LAUNCHED())) return e;
+    if ((e = launch_ntt(c, true, ct, 2 * T, LN, 0, c.L, s))) return e;
+    const size_t cols = T * ((size_t)1 << (c.LOGB - 1));
+    FEDHE_FOR_A(c, (enc_outer_sample_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, t0, seed, client, ubuf, LN,
+                                                                                     cols)));
+    if ((e = FEDHE_LAUNCHED())) return e;
+    return launch_enc_block_forward<true>(c, k, ubuf, T, ct, s);
 }
 
 // ===========================================================================
@@ -1207,6 +1359,92 @@ cudaError_t launch_aggregate(const CtxDev &c, const uint64_t *const *ptrs, const
     return FEDHE_LAUNCHED();
 }
 
+// ---------------------------------------------------------------------------
+// The same on transform-domain ciphertexts.  The weighted sum is pointwise in
+// either domain; the rounding term of the rescale is not: the last limb is
+// brought back to coefficients, centred, and its residues are transformed
+// for every other limb (2L limb transforms per ciphertext index that the
+// coefficient format does not need).
+// ---------------------------------------------------------------------------
+
+// acc_j = sum_i W_i ct_i for all limbs: limbs below the last go to `out`
+// ([T][2][L-1][N]), the last limb to `last` ([T][2][N])
+__global__ void __launch_bounds__(256)
+aggregate_sum_kernel(const __grid_constant__ CtxDev c, const uint64_t *const *ptrs, const tw_t *wtab, int C,
+                     uint64_t *out, uint64_t *last, size_t total) {
+    extern __shared__ __align__(16) unsigned char agg_sm[];
+    const uint32_t L = c.L;
+    tw_t *sw = reinterpret_cast<tw_t *>(agg_sm);
+    const uint64_t **sp = reinterpret_cast<const uint64_t **>(sw + (size_t)C * L);
+    for (int e = threadIdx.x; e < C * (int)L; e += blockDim.x) sw[e] = wtab[e];
+    for (int e = threadIdx.x; e < C; e += blockDim.x) sp[e] = ptrs[e];
+    __syncthreads();
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t pairs = c.N >> 1;
+    const uint32_t i = (uint32_t)(g % pairs) * 2;
+    const size_t tc = g / pairs;
+    for (uint32_t j = 0; j < L; j++) {
+        u64x2 o;
+        weighted_sum_pair(sp, sw, C, L, j, (tc * L + j) * c.N + i, c.limb[j].q, o.x, o.y);
+        uint64_t *dst = j + 1 < L ? out + (tc * (L - 1) + j) * c.N + i : last + tc * c.N + i;
+        *reinterpret_cast<u64x2 *>(dst) = o;
+    }
+}
+
+// residues modulo every remaining prime of the centred last-limb coefficients
+__global__ void __launch_bounds__(256)
+aggregate_spread_kernel(const __grid_constant__ CtxDev c, const uint64_t *last, uint64_t *rem, size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t i = (uint32_t)(g % c.N);
+    const size_t tc = g / c.N;
+    const uint32_t L = c.L;
+    const uint64_t ql = c.limb[L - 1].q, r = last[g];
+    const bool neg = r > ql / 2;
+    const uint64_t mag = neg ? ql - r : r;
+    for (uint32_t j = 0; j + 1 < L; j++) {
+        const LimbDev &lb = c.limb[j];
+        const uint64_t v = barrett64(mag, lb.q, lb.mu);
+        rem[(tc * (L - 1) + j) * c.N + i] = (neg && v) ? lb.q - v : v;
+    }
+}
+
+// out_j = (acc_j - rem_j) / q_{L-1}
+__global__ void __launch_bounds__(256)
+aggregate_finish_kernel(const __grid_constant__ CtxDev c, const uint64_t *rem, uint64_t *out, size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t j = (uint32_t)((g / c.N) % (c.L - 1));
+    const LimbDev &lb = c.limb[j];
+    out[g] = shoup(submod(out[g], rem[g], lb.q), lb.qlinv.w, lb.qlinv.wp, lb.q);
+}
+
+// scratch: [T][2][N] + [T][2][L-1][N] words
+cudaError_t launch_aggregate_ntt(const CtxDev &c, const uint64_t *const *ptrs, const tw_t *wtab, int C,
+                                 size_t T, uint64_t *scratch, uint64_t *out, cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    uint64_t *last = scratch, *rem = scratch + 2 * T * c.N;
+    const size_t smem = (size_t)C * c.L * sizeof(tw_t) + (size_t)C * sizeof(void *);
+    cudaError_t e;
+    if (smem > 48 * 1024 &&
+        (e = cudaFuncSetAttribute(aggregate_sum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)))
+        return e;
+    const size_t pairs = T * 2 * (c.N >> 1);
+    aggregate_sum_kernel<<<blocks_for(pairs, 256), 256, smem, s>>>(c, ptrs, wtab, C, out, last, pairs);
+    if ((e = FEDHE_LAUNCHED())) return e;
+    if ((e = launch_ntt(c, false, last, 2 * T, c.N, c.L - 1, 1, s))) return e;
+    if (c.L > 1) {
+        const size_t n_last = 2 * T * c.N, n_out = n_last * (c.L - 1);
+        aggregate_spread_kernel<<<blocks_for(n_last, 256), 256, 0, s>>>(c, last, rem, n_last);
+        if ((e = FEDHE_LAUNCHED())) return e;
+        if ((e = launch_ntt(c, true, rem, 2 * T, (size_t)(c.L - 1) * c.N, 0, c.L - 1, s))) return e;
+        aggregate_finish_kernel<<<blocks_for(n_out, 256), 256, 0, s>>>(c, rem, out, n_out);
+        if ((e = FEDHE_LAUNCHED())) return e;
+    }
+    return cudaSuccess;
+}
+
 // plaintext remainder: out = sum_i alpha_i * (double) rest_i, client order,
 // separate multiply and add
 __global__ void __launch_bounds__(256)
@@ -1248,6 +1486,21 @@ dec_pointwise_kernel(const __grid_constant__ CtxDev c, const KeysDev k, uint64_t
     scratch[g] = shoup_lazy(scratch[g], s.w, s.wp, c.limb[0].q);
 }
 
+// transform-domain ciphertext: scratch = c0^ + c1^ s^ on limb 0
+__global__ void __launch_bounds__(256)
+dec_pointwise_ntt_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const uint64_t *ct, uint32_t level,
+                         uint64_t *scratch, size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t i = (uint32_t)(g % c.N);
+    const size_t t = g / c.N;
+    const uint64_t q = c.limb[0].q;
+    const tw_t s = load_tw(k.s_hat + i);
+    const uint64_t p = shoup(ct[((t * 2 + 1) * level + 0) * c.N + i], s.w, s.wp, q);
+    scratch[g] = addmod(p, ct[((t * 2 + 0) * level + 0) * c.N + i], q);
+}
+
+// centred d = scratch (+ c0 when the ciphertext is in the coefficient domain: ct != null)
 __global__ void __launch_bounds__(256)
 dec_finish_kernel(const __grid_constant__ CtxDev c, const uint64_t *ct, uint32_t level, uint64_t *scratch,
                   size_t total) {
@@ -1256,7 +1509,7 @@ dec_finish_kernel(const __grid_constant__ CtxDev c, const uint64_t *ct, uint32_t
     const uint32_t i = (uint32_t)(g % c.N);
     const size_t t = g / c.N;
     const uint64_t q = c.limb[0].q;
-    const uint64_t r = addmod(scratch[g], ct[((t * 2 + 0) * level + 0) * c.N + i], q);
+    const uint64_t r = ct ? addmod(scratch[g], ct[((t * 2 + 0) * level + 0) * c.N + i], q) : scratch[g];
     const int64_t d = r > q / 2 ? -(int64_t)(q - r) : (int64_t)r;
     reinterpret_cast<int64_t *>(scratch)[g] = d;
 }
@@ -1276,13 +1529,27 @@ cudaError_t launch_decrypt(const CtxDev &c, const KeysDev &k, const uint64_t *ct
     return FEDHE_LAUNCHED();
 }
 
+cudaError_t launch_decrypt_ntt(const CtxDev &c, const KeysDev &k, const uint64_t *ct, uint32_t level,
+                               size_t T, uint64_t *scratch, cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    cudaError_t e;
+    const size_t total = T * c.N;
+    dec_pointwise_ntt_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, k, ct, level, scratch, total);
+    if ((e = FEDHE_LAUNCHED())) return e;
+    if ((e = launch_ntt(c, false, scratch, T, c.N, 0, 1, s))) return e;
+    dec_finish_kernel<<<blocks_for(total, 256), 256, 0, s>>>(c, nullptr, level, scratch, total);
+    return FEDHE_LAUNCHED();
+}
+
 // Fused path for N <= 2^14: one thread block per ciphertext transforms c1
 // (limb 0), multiplies by the secret key, transforms back, adds c0, centres,
 // and runs the slot transform on the result without leaving the SM; only the
 // two limb-0 polynomials are read and the n decoded values written.
 // L: layout of the length-N integer transform (played by L::NT / V threads),
 // LF: layout of the length-n complex transform with LF::NT == L::NT / V.
-template <class L, int V, class LF>
+// NTT_IN: the ciphertext is in the transform domain, so the forward transform
+// falls away and c0^ + c1^ s^ feeds the inverse transform directly.
+template <class L, int V, class LF, bool NTT_IN>
 __global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
 decrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const uint64_t *ct, uint32_t level,
                      double *z) {
@@ -1294,7 +1561,7 @@ decrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const ui
     const LimbDev &lb = c.limb[0];
     const uint64_t q = lb.q, q2 = 2 * q;
     const uint64_t *c0 = ct + ((t * 2 + 0) * level) * B, *c1 = ct + ((t * 2 + 1) * level) * B;
-    {
+    if constexpr (!NTT_IN) {
         const NttArgs fa = LimbOf<ModInt>::args(lb, true, 0, 0);   // limb 0 carries the message
         smem_ntt_forward<L, V>(
             sm, tid, fa, [&](uint32_t i) { return c1[i]; },
@@ -1308,9 +1575,19 @@ decrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const ui
     {
         const NttArgs ia = LimbOf<ModInt>::args(lb, false, 0, 0);
         smem_ntt_inverse<L, V, true>(
-            sm, tid, ia, lb.ninv, lb.wn, [&](uint32_t p) { return u64x2{sm[swz(p)], sm[swz(p + 1)]}; },
+            sm, tid, ia, lb.ninv, lb.wn,
+            [&](uint32_t p) {
+                if constexpr (NTT_IN) {
+                    const u64x2 a = *reinterpret_cast<const u64x2 *>(c0 + p), b = *reinterpret_cast<const u64x2 *>(c1 + p);
+                    const tw_t s0 = load_tw(k.s_hat + p), s1 = load_tw(k.s_hat + p + 1);
+                    return u64x2{csub(a.x + shoup_lazy(b.x, s0.w, s0.wp, q), q2),
+                                 csub(a.y + shoup_lazy(b.y, s1.w, s1.wp, q), q2)};
+                } else {
+                    return u64x2{sm[swz(p)], sm[swz(p + 1)]};
+                }
+            },
             [&](uint32_t i, uint64_t v) {
-                const uint64_t r = addmod(csub(v, q), c0[i], q);
+                const uint64_t r = NTT_IN ? csub(v, q) : addmod(csub(v, q), c0[i], q);
                 d[swz(i)] = r > q / 2 ? -(int64_t)(q - r) : (int64_t)r;
             });
     }
@@ -1329,11 +1606,11 @@ decrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const ui
     for (int r = 0; r < LF::E; r++) z[t * n + LF::template idx<0>(tid, r)] = x[r].re;
 }
 
-template <class L, int V, class LF>
+template <class L, int V, class LF, bool NTT_IN>
 static cudaError_t launch_decrypt_fused_t(const CtxDev &c, const KeysDev &k, const uint64_t *ct, uint32_t level,
                                           size_t T, double *z, cudaStream_t s) {
     const size_t smem = sizeof(uint64_t) << L::LOGB;
-    auto kern = decrypt_fused_kernel<L, V, LF>;
+    auto kern = decrypt_fused_kernel<L, V, LF, NTT_IN>;
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
     kern<<<(unsigned)T, L::NT / V, smem, s>>>(c, k, ct, level, z);
@@ -1341,10 +1618,14 @@ static cudaError_t launch_decrypt_fused_t(const CtxDev &c, const KeysDev &k, con
 }
 
 cudaError_t launch_decrypt_fused(const CtxDev &c, const KeysDev &k, const uint64_t *ct, uint32_t level,
-                                 size_t T, double *z, cudaStream_t s) {
+                                 size_t T, bool ntt_in, double *z, cudaStream_t s) {
     if (T == 0) return cudaSuccess;
-    if (c.logN == 13) return launch_decrypt_fused_t<Lay<13, 3>, 2, Lay<12, 3>>(c, k, ct, level, T, z, s);
-    return launch_decrypt_fused_t<Lay<14, 3>, 2, Lay<13, 3>>(c, k, ct, level, T, z, s);
+    if (c.logN == 13) {
+        if (ntt_in) return launch_decrypt_fused_t<Lay<13, 3>, 2, Lay<12, 3>, true>(c, k, ct, level, T, z, s);
+        return launch_decrypt_fused_t<Lay<13, 3>, 2, Lay<12, 3>, false>(c, k, ct, level, T, z, s);
+    }
+    if (ntt_in) return launch_decrypt_fused_t<Lay<14, 3>, 2, Lay<13, 3>, true>(c, k, ct, level, T, z, s);
+    return launch_decrypt_fused_t<Lay<14, 3>, 2, Lay<13, 3>, false>(c, k, ct, level, T, z, s);
 }
 
 // ===========================================================================

@@ -32,9 +32,17 @@ cudaError_t launch_decode(const CtxDev &c, const int64_t *d, size_t T, double2 *
 cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0, size_t T,
                            uint64_t seed, uint32_t client, uint64_t *ct, cudaStream_t s);
 
+// the same with every limb polynomial of the result in the transform domain;
+// ubuf: uint64 [T][L][N] work space, used for N > 2^14 only
+cudaError_t launch_encrypt_ntt(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0, size_t T,
+                               uint64_t seed, uint32_t client, uint64_t *ubuf, uint64_t *ct, cudaStream_t s);
+
 // ptrs: device array of C ciphertext pointers; wtab: device [C][L] weights
 cudaError_t launch_aggregate(const CtxDev &c, const uint64_t *const *ptrs, const tw_t *wtab, int C,
                              size_t T, uint64_t *out, cudaStream_t s);
+// transform-domain ciphertexts in and out; scratch: uint64 [T][2][L][N]
+cudaError_t launch_aggregate_ntt(const CtxDev &c, const uint64_t *const *ptrs, const tw_t *wtab, int C,
+                                 size_t T, uint64_t *scratch, uint64_t *out, cudaStream_t s);
 cudaError_t launch_plain_aggregate(const float *const *ptrs, const double *alpha, int C, size_t len,
                                    double *out, cudaStream_t s);
 
@@ -42,9 +50,14 @@ cudaError_t launch_plain_aggregate(const float *const *ptrs, const double *alpha
 cudaError_t launch_decrypt(const CtxDev &c, const KeysDev &k, const uint64_t *ct, uint32_t level,
                            size_t T, uint64_t *scratch, cudaStream_t s);
 
-// fused decrypt + decode for N <= 2^14 (no scratch): z double [T][n]
+// the same for a transform-domain ciphertext
+cudaError_t launch_decrypt_ntt(const CtxDev &c, const KeysDev &k, const uint64_t *ct, uint32_t level,
+                               size_t T, uint64_t *scratch, cudaStream_t s);
+
+// fused decrypt + decode for N <= 2^14 (no scratch): z double [T][n];
+// ntt_in: the ciphertext is in the transform domain
 cudaError_t launch_decrypt_fused(const CtxDev &c, const KeysDev &k, const uint64_t *ct, uint32_t level,
-                                 size_t T, double *z, cudaStream_t s);
+                                 size_t T, bool ntt_in, double *z, cudaStream_t s);
 
 // two-party threshold decryption.  tmp: uint64 [2][L][N] (shares as residues)
 cudaError_t launch_threshold_split(const CtxDev &c, const int8_t *s8, uint64_t seed, uint64_t *tmp,

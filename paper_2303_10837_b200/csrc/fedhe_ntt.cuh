@@ -155,6 +155,8 @@ struct ModInt {
     HD uint64_t canon_wide(val v) const { return csub(csub(v, q2), q); }
     HD uint64_t canon(val v) const { return csub(v, q); }
     HD uint64_t canon_add(val v, uint64_t add) const { return csub(csub(v, q) + add, q); }
+    // canonical residue of a forward output plus a key product
+    HD uint64_t canon_sum(val a, val b) const { return csub(canon_wide(a) + csub(b, q), q); }
     // product with an entry of a key table, below 2q for any v
     using key = tw_t;
     static HD key load_key(const tw_t *p) { return FEDHE_LD_TW(p); }
@@ -201,6 +203,7 @@ struct ModF64 {
         const double r = f64_add(v, f64_from_u64(add));
         return f64_canonical(r >= q ? f64_sub(r, q) : r, q);
     }
+    HD uint64_t canon_sum(val a, val b) const { return canon_wide(f64_add(a, b)); }
     // only the value of a key-table entry is read; |result| <= 3q/4
     using key = double;
     static HD key load_key(const tw_t *p) {

@@ -171,6 +171,49 @@ def test_encrypt_large_messages_bit_exact(he, base):
     assert np.array_equal(to_host_u64(ct), ct_o)
 
 
+def oracle_ntt_of(o, ct):
+    """Every limb polynomial of an oracle ciphertext [T][2][level][N] through the oracle's forward transform."""
+    out = np.empty_like(ct)
+    for t in range(ct.shape[0]):
+        for c in range(2):
+            for j in range(ct.shape[2]):
+                out[t, c, j] = o.ntt_forward(j, ct[t, c, j])
+    return out
+
+
+@pytest.mark.parametrize("w", workload_cases(), ids=lambda w: w.name)
+def test_transform_domain_format_bit_exact(he, w):
+    """The alternative wire format: each step equals the transform of the oracle's coefficient-domain
+    result, and the decrypted slots are those of the coefficient path."""
+    g, o = contexts(he, w.N, w.primes, w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    s_o, pk_o = o.keygen(w.key_seed)
+    xs = si.client_updates(w)
+    alpha = si.client_weights(w)
+    cts, cts_o = [], []
+    for i, x in enumerate(xs):
+        sel, _ = he.he_pack(g, None, dev_f32(x))
+        ct = he.he_encrypt_ntt(g, keys, sel, w.enc_seed, i)
+        ct_o, bad = o.encrypt(pk_o, o.pack(None, w.P, x)[0], w.enc_seed, i)
+        assert bad == 0
+        assert np.array_equal(to_host_u64(ct), oracle_ntt_of(o, ct_o)), "ciphertext of client %d" % i
+        # the same bytes as transforming the coefficient-domain ciphertext
+        ref = he.he_encrypt(g, keys, sel, w.enc_seed, i)
+        he.he_ntt_forward(g, ref.view(-1, w.L, w.N))
+        assert torch.equal(ct, ref)
+        cts.append(ct)
+        cts_o.append(ct_o)
+    agg = he.he_weighted_aggregate_ntt(g, cts, alpha)
+    agg_o = o.rescale(o.weighted_sum(cts_o, o.weights(alpha)))
+    assert np.array_equal(to_host_u64(agg), oracle_ntt_of(o, agg_o))
+    z = he.he_decrypt_level_ntt(g, keys, agg, w.L - 1).cpu().numpy()
+    z_o = o.decode(o.decrypt(s_o, agg_o, w.L - 1)).reshape(-1)
+    assert np.abs(z - z_o).max() <= DECODE_TOL
+    z0 = he.he_decrypt_level_ntt(g, keys, cts[0], w.L).cpu().numpy()
+    assert np.abs(z0[: w.P] - xs[0].astype(np.float64)).max() <= FEDAVG_TOL
+    assert he.he_ctx_status(g) == he.HE_OK
+
+
 def test_dropout_subset_of_clients(he):
     """Aggregating any subset with renormalised weights needs no new keys."""
     w = si.scaled(si.RESNET18, 8192 + 11, clients=4, name="r18-dropout")
