@@ -275,6 +275,11 @@ def run_ours(args, w):
             he.he_decrypt(g, keys, agg[:tc], out=z[t0 * n:(t0 + tc) * n])
         he.he_unpack(g, mask, z, None, w.P, out=out)
 
+    transform = args.format == "transform"
+    if transform and Tc < T:
+        raise SystemExit("bench: --format transform is not wired to the streamed (chunked) round")
+    enc = he.he_encrypt_ntt if transform else he.he_encrypt
+
     def step(record):
         if Tc < T:
             return step_streamed(record)
@@ -284,13 +289,17 @@ def run_ours(args, w):
             if record:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
-            he.he_encrypt(g, keys, sel, enc_seed, i, out=cts[i])
+            enc(g, keys, sel, enc_seed, i, out=cts[i])
             if record:
                 e1.record()
                 enc_events.append((e0, e1, T))
             rests.append(rest)
-        he.he_weighted_aggregate(g, cts, alpha, out=agg)
-        he.he_decrypt(g, keys, agg, out=z)
+        if transform:
+            he.he_weighted_aggregate_ntt(g, cts, alpha, out=agg)
+            he.he_decrypt_level_ntt(g, keys, agg, w.L - 1, out=z)
+        else:
+            he.he_weighted_aggregate(g, cts, alpha, out=agg)
+            he.he_decrypt(g, keys, agg, out=z)
         avg = he.he_plain_aggregate(g, rests, alpha) if mask is not None else None
         he.he_unpack(g, mask, z, avg, w.P, out=out)
 
@@ -378,7 +387,8 @@ def run_ours(args, w):
     # roofline of the dominant kernel (bound by the multiply / double-precision pipe)
     logN = w.N.bit_length() - 1
     butterflies = 3 * w.L * (w.N // 2) * logN * T           # per launch: 3 limb transforms per limb
-    achieved = transform_slots(w.primes, w.N, 1, 2) * T / (kern_ms * 1e-3) / 1e12
+    # coefficient format: one forward and two inverse transforms per limb; transform format: three forward
+    achieved = transform_slots(w.primes, w.N, 3 if transform else 1, 0 if transform else 2) * T / (kern_ms * 1e-3) / 1e12
     n_sm = torch.cuda.get_device_properties(local).multi_processor_count
     peak = n_sm * SLOTS_PER_SM_CLK * peaks["sm_max_mhz"] * 1e6 / 1e12
     alg_bytes = (16.0 + 32.0 * w.L) * n * T          # read m, write the ciphertext
@@ -411,7 +421,8 @@ def run_ours(args, w):
         "metric": METRIC, "value": units / job_secs, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * job_secs / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u64 (limbs below 2^46: exact f64)", "data": "synthetic",
-        "config": config_dict(w, "every rank runs its own full batch; no collective on the path"),
+        "config": dict(config_dict(w, "every rank runs its own full batch; no collective on the path"),
+                       format=args.format),
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"] or peaks["sm_max_mhz"],
                    "reasons": clocks["reasons"], "samples": clocks["samples"]},
         "e2e": {"value": e2e_units / e2e_job, "unit": UNIT, "h2d_bytes_per_step": 4 * w.P * w.clients,
@@ -433,6 +444,9 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=["resnet18", "tiny", "resnet50-top10", "bert-1", "bert-10", "bert-100"],
                     default="resnet18")
+    ap.add_argument("--format", choices=["coefficient", "transform"], default="coefficient",
+                    help="ciphertext wire format of the timed round (the host-buffer leg always runs "
+                         "he_round_host, which implements the coefficient format)")
     args = ap.parse_args()
     w = {"resnet18": si.RESNET18, "tiny": si.TINY, "resnet50-top10": si.RESNET50_TOP10,
          "bert-1": si.bert(0.01), "bert-10": si.bert(0.10), "bert-100": si.bert(1.0)}[args.workload]

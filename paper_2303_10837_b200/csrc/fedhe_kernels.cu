@@ -689,37 +689,38 @@ __device__ __forceinline__ void encrypt_unit(const LimbDev &lb, const tw_t *p0, 
     const uint32_t tid = threadIdx.x;
     const uint64_t q = lb.q;
     if constexpr (NTT_OUT) {
-        // transform-domain output: c0^ = pk0^ u^ + (e0 + m)^, c1^ = pk1^ u^ + e1^.  Both
-        // products wait in their final slots for the transforms of the error terms.
+        // transform-domain output: c0^ = pk0^ u^ + (e0 + m)^, c1^ = pk1^ u^ + e1^.  Three
+        // passes over one copy of the forward-transform code: u (both products wait in
+        // their final slots), then e0 + m and e1, each added to its product.
         const auto fa = LimbOf<M>::args(lb, true, 0, 0);
         const M &ar = fa.m;
-        smem_ntt_forward<L, V>(
-            sm, tid, fa, [&](uint32_t i) { return ar.small(su[i]); },
-            [&](uint32_t p, val a, val b) {
-                const auto a0 = M::load_key(p0 + p), a1 = M::load_key(p0 + p + 1);
-                const auto b0 = M::load_key(p1 + p), b1 = M::load_key(p1 + p + 1);
-                *reinterpret_cast<u64x2 *>(cbase + p) = u64x2{M::bits(ar.mul_key(a, a0)), M::bits(ar.mul_key(b, a1))};
-                *reinterpret_cast<u64x2 *>(cbase + cstride + p) =
-                    u64x2{M::bits(ar.mul_key(a, b0)), M::bits(ar.mul_key(b, b1))};
-            });
 #pragma unroll 1
-        for (int h = 0; h < 2; h++) {
-            uint64_t *cc = cbase + h * cstride;
-            const int8_t *se = se0 + h * B;
-            __syncthreads();   // last-phase readers are done before the next transform writes
+        for (int h = 0; h < 3; h++) {
+            uint64_t *cc = cbase + (h == 2 ? cstride : 0);
+            const int8_t *se = se0 + (h == 2 ? B : 0);
             smem_ntt_forward<L, V>(
                 sm, tid, fa,
                 [&](uint32_t i) {
-                    return h == 0 ? ar.from_residue(signed_residue(mt[i] + (int64_t)se[i], q, lb.mu))
-                                  : ar.small(se[i]);
+                    if (h == 0) return ar.small(su[i]);
+                    if (h == 2) return ar.small(se[i]);
+                    return ar.from_residue(signed_residue(mt[i] + (int64_t)se[i], q, lb.mu));
                 },
                 [&](uint32_t p, val a, val b) {
-                    const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + p);
-                    *reinterpret_cast<u64x2 *>(cc + p) =
-                        u64x2{ar.canon_sum(a, M::from_bits(t.x)), ar.canon_sum(b, M::from_bits(t.y))};
+                    if (h == 0) {
+                        const auto a0 = M::load_key(p0 + p), a1 = M::load_key(p0 + p + 1);
+                        const auto b0 = M::load_key(p1 + p), b1 = M::load_key(p1 + p + 1);
+                        *reinterpret_cast<u64x2 *>(cbase + p) =
+                            u64x2{M::bits(ar.mul_key(a, a0)), M::bits(ar.mul_key(b, a1))};
+                        *reinterpret_cast<u64x2 *>(cbase + cstride + p) =
+                            u64x2{M::bits(ar.mul_key(a, b0)), M::bits(ar.mul_key(b, b1))};
+                    } else {
+                        const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + p);
+                        *reinterpret_cast<u64x2 *>(cc + p) =
+                            u64x2{ar.canon_sum(a, M::from_bits(t.x)), ar.canon_sum(b, M::from_bits(t.y))};
+                    }
                 });
+            __syncthreads();   // last-phase readers are done before the next transform writes
         }
-        __syncthreads();
         return;
     }
     {
@@ -851,27 +852,22 @@ __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0
             }
         };
         if constexpr (NTT_OUT) {
-            // transform-domain output: both products wait in their final slots for the
-            // transforms of e0 + m and e1, whose pairing stage costs one product per element
+            // transform-domain output: three passes over one copy of the forward code: u
+            // (both products wait in their final slots), then e0 + m and e1, whose pairing
+            // stage costs one product per element, each added to its product
             uint64_t *c0 = cbase + grp * H;
-            smem_ntt_forward<L, V>(smg, gt, fa, src, [&](uint32_t p, val a, val b) {
-                const auto a0 = M::load_key(p0 + p), a1 = M::load_key(p0 + p + 1);
-                const auto b0 = M::load_key(p1 + p), b1 = M::load_key(p1 + p + 1);
-                *reinterpret_cast<u64x2 *>(c0 + p) = u64x2{M::bits(ar.mul_key(a, a0)), M::bits(ar.mul_key(b, a1))};
-                *reinterpret_cast<u64x2 *>(c1 + p) = u64x2{M::bits(ar.mul_key(a, b0)), M::bits(ar.mul_key(b, b1))};
-            }, gsync);
 #pragma unroll 1
-            for (int h = 0; h < 2; h++) {
-                uint64_t *cc = cbase + h * cstride + grp * H;
-                const int8_t *se = se0 + h * B;
+            for (int h = 0; h < 3; h++) {
+                uint64_t *cc = h == 2 ? c1 : c0;
+                const int8_t *se = se0 + (h == 2 ? B : 0);
                 auto value = [&](uint32_t i) {
-                    return h == 0 ? ar.from_residue(signed_residue(mt[i] + (int64_t)se[i], q, lb.mu))
-                                  : ar.small(se[i]);
+                    if (h == 2) return ar.small(se[i]);
+                    return ar.from_residue(signed_residue(mt[i] + (int64_t)se[i], q, lb.mu));
                 };
-                gsync();   // last-phase readers of this half are done before phase 0 writes
                 smem_ntt_forward<L, V>(
                     smg, gt, fa,
                     [&](uint32_t i) {
+                        if (h == 0) return src(i);
                         const val lo = value(i), hi = value(i + H);
                         if constexpr (std::is_same<M, ModF64>::value) {
                             const double t = ar.mul(hi, w0);
@@ -882,11 +878,21 @@ __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0
                         }
                     },
                     [&](uint32_t p, val a, val b) {
-                        const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + p);
-                        *reinterpret_cast<u64x2 *>(cc + p) =
-                            u64x2{ar.canon_sum(a, M::from_bits(t.x)), ar.canon_sum(b, M::from_bits(t.y))};
+                        if (h == 0) {
+                            const auto a0 = M::load_key(p0 + p), a1 = M::load_key(p0 + p + 1);
+                            const auto b0 = M::load_key(p1 + p), b1 = M::load_key(p1 + p + 1);
+                            *reinterpret_cast<u64x2 *>(c0 + p) =
+                                u64x2{M::bits(ar.mul_key(a, a0)), M::bits(ar.mul_key(b, a1))};
+                            *reinterpret_cast<u64x2 *>(c1 + p) =
+                                u64x2{M::bits(ar.mul_key(a, b0)), M::bits(ar.mul_key(b, b1))};
+                        } else {
+                            const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + p);
+                            *reinterpret_cast<u64x2 *>(cc + p) =
+                                u64x2{ar.canon_sum(a, M::from_bits(t.x)), ar.canon_sum(b, M::from_bits(t.y))};
+                        }
                     },
                     gsync);
+                gsync();   // last-phase readers of this half are done before phase 0 writes
             }
             __syncthreads();
             return;
