@@ -42,9 +42,18 @@ struct alignas(16) u64x2 { uint64_t x, y; };   // two neighbouring residues
 template <class V>
 struct pair_of { V x, y; };                      // two neighbouring values of an arithmetic
 
-// shared-memory index swizzle: makes all phase layouts free of bank conflicts
-// for 8-byte accesses (xor the low nibble with the next one)
-HD uint32_t swz(uint32_t i) { return i ^ ((i >> 4) & 15u); }
+// Shared-memory index swizzle.  A 64-bit access of a warp is served half-warp
+// by half-warp from 16 banks of 8 bytes (the low four index bits), and the 16
+// lanes of a half-warp differ in four index bits that depend on the phase:
+// bits {0,1,2,3}, {0,4,5,6}, {1,2,3,4}, {0,1,5,6} or {2,3,4,5} for the layouts
+// in use.  XOR-ing t ^ (t << 1), t = index bits 4..6, into the low nibble makes
+// the bank a bijection of each of these sets (as linear maps over GF(2): the
+// columns 0011, 0110, 1100 for bits 4, 5, 6 next to the identity), so no
+// phase has bank conflicts; the map permutes every aligned group of 16 words.
+HD uint32_t swz(uint32_t i) {
+    const uint32_t t = (i >> 4) & 7u;
+    return i ^ t ^ ((t << 1) & 15u);
+}
 
 template <int LOGB_, int LE_>
 struct Lay {
