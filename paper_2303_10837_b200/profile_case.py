@@ -4,6 +4,7 @@
     python paper_2303_10837_b200/profile_case.py ntt [--polys 256]
     python paper_2303_10837_b200/profile_case.py aggregate [--cts 64]
     python paper_2303_10837_b200/profile_case.py sweep [--prime-bits 45]   # kernel sweep table (no profiler)
+    python paper_2303_10837_b200/profile_case.py kernels [--workload W]    # every step alone, % of the HBM peak
 
 Each case touches more memory than the L2 holds so that DRAM counters mean something,
 launches the kernel of interest a handful of times and exits.
@@ -83,9 +84,55 @@ def sweep(bits=60):
             del keys, g
 
 
+def kernels(workload):
+    """Every step of the round timed alone on one workload: algorithmic bytes (the minimum the
+    step must move) / time as a share of the HBM peak, median of 11 runs."""
+    peak, src = read_hbm_peak()
+    base = {"resnet18": si.RESNET18, "tiny": si.TINY, "bert": si.bert(1.0)}[workload]
+    w = si.scaled(base, min(base.P, 11_700_000), clients=base.clients)        # full encryption of at most 11.7 M parameters
+    g = he.he_ctx_create(w.N, list(w.primes), w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    C, L, N, n, T, P = w.clients, w.L, w.N, w.n, w.T, w.P
+    xs = [torch.from_numpy(si.client_update(w, i)).cuda() for i in range(C)]
+    alpha = si.client_weights(w)
+    score = torch.rand(P, device="cuda")
+    mask = he.he_select_mask(g, score, P // 10)
+    sel, _ = he.he_pack(g, None, xs[0])
+    cts = [he.he_encrypt(g, keys, he.he_pack(g, None, xs[i])[0], w.enc_seed, i) for i in range(C)]
+    agg = he.he_weighted_aggregate(g, cts, alpha)
+    z = he.he_decrypt(g, keys, agg)
+    rests = [he.he_pack(g, mask, xs[i])[1] for i in range(C)]
+    out = torch.empty(P, dtype=torch.float64, device="cuda")
+
+    def med(fn):
+        ts = sorted(timed(fn, 1) for _ in range(11))
+        return ts[5]
+
+    rows = [
+        ("he_select_mask (k = P/10)", lambda: he.he_select_mask(g, score, P // 10), 6 * 4.0 * P),
+        ("he_pack (full)", lambda: he.he_pack(g, None, xs[0]), 8.0 * P),
+        ("he_pack (masked, 10 %)", lambda: he.he_pack(g, mask, xs[0]), 8.0 * P + 4.0 * P / 10),
+        ("he_encode", lambda: he.he_encode(g, sel), 4.0 * T * n + 8.0 * T * N),
+        ("he_encrypt (encode + encrypt)", lambda: he.he_encrypt(g, keys, sel, w.enc_seed, 0, out=cts[0]),
+         4.0 * T * n + 16.0 * L * N * T),
+        ("he_weighted_aggregate", lambda: he.he_weighted_aggregate(g, cts, alpha, out=agg),
+         16.0 * N * T * (L * C + (L - 1))),
+        ("he_plain_aggregate (90 %)", lambda: he.he_plain_aggregate(g, rests, alpha), rests[0].numel() * (4.0 * C + 8)),
+        ("he_decrypt (decrypt + decode)", lambda: he.he_decrypt(g, keys, agg, out=z), 16.0 * N * T + 8.0 * n * T),
+        ("he_unpack (full)", lambda: he.he_unpack(g, None, z, None, P, out=out), 16.0 * P),
+    ]
+    print("workload %s: N %d, L %d, %d clients, %d ciphertexts per client; HBM peak %.1f GB/s (%s)"
+          % (w.name, N, L, C, T, peak, src))
+    print("%-34s %10s %12s %9s %7s" % ("call", "ms", "alg. MB", "GB/s", "%HBM"))
+    for name, fn, nbytes in rows:
+        ms = med(fn)
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        print("%-34s %10.3f %12.1f %9.1f %6.1f%%" % (name, ms, nbytes / 1e6, gbs, 100 * gbs / peak))
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["encrypt", "ntt", "aggregate", "decrypt", "sweep"])
+    ap.add_argument("case", choices=["encrypt", "ntt", "aggregate", "decrypt", "sweep", "kernels"])
     ap.add_argument("--cts", type=int, default=296)
     ap.add_argument("--polys", type=int, default=256)
     ap.add_argument("--reps", type=int, default=2)
@@ -95,6 +142,9 @@ def main():
     a = ap.parse_args()
     if a.case == "sweep":
         sweep(a.prime_bits)
+        return
+    if a.case == "kernels":
+        kernels(a.workload)
         return
     base = {"resnet18": si.RESNET18, "tiny": si.TINY, "bert": si.bert(1.0)}[a.workload]
     w = si.scaled(base, a.cts * base.n, clients=base.clients)
