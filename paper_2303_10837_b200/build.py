@@ -10,15 +10,18 @@ import os
 import shutil
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libfedhe.so")
 BUILD = os.path.join(HERE, "_build")
 
-CUDA_SOURCES = ["fedhe_kernels.cu", "fedhe_api.cu", "fedhe_noalloc.cu"]
+CUDA_SOURCES = ["fedhe_transform.cu", "fedhe_slots.cu", "fedhe_encrypt.cu", "fedhe_server.cu", "fedhe_decrypt.cu",
+                "fedhe_mask.cu", "fedhe_api.cu", "fedhe_noalloc.cu"]
 HOST_SOURCES = ["fedhe_host.cpp"]
 HEADERS = ["fedhe_device.cuh", "fedhe_ntt.cuh", "fedhe_internal.cuh", "fedhe_launch.h", "fedhe_host.h",
+           "fedhe_kernels.cuh", "fedhe_slots.cuh",
            os.path.join("..", "..", "include", "fedhe.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -43,7 +46,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(BUILD, exist_ok=True)
     headers = [os.path.join(CSRC, h) for h in HEADERS] + [os.path.abspath(__file__)]
     objs = []
-    for src in CUDA_SOURCES:
+
+    def compile_cuda(src):
         s = os.path.join(CSRC, src)
         o = os.path.join(BUILD, src + ".o")
         if force or _stale(o, [s] + headers):
@@ -55,7 +59,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
                 sys.stderr.write(r.stdout + r.stderr)
             if r.returncode:
                 raise RuntimeError("nvcc failed on " + src)
-        objs.append(o)
+        return o
+
+    # the translation units are independent: compile them side by side
+    with ThreadPoolExecutor(max_workers=min(len(CUDA_SOURCES), os.cpu_count() or 1)) as pool:
+        objs.extend(pool.map(compile_cuda, CUDA_SOURCES))
     for src in HOST_SOURCES:
         s = os.path.join(CSRC, src)
         o = os.path.join(BUILD, src + ".o")

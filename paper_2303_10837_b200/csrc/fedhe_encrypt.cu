@@ -1,0 +1,613 @@
+// Encryption kernels (part 3 of the kernels).
+#include "fedhe_kernels.cuh"
+
+namespace fedhe {
+
+// ===========================================================================
+// encryption:  c0 = pk0 u + e0 + m,  c1 = pk1 u + e1   (mod every q_j)
+// ===========================================================================
+
+// One (ciphertext, limb) unit of the fused path in the limb's arithmetic.
+// u^ pk1^ is parked, in the arithmetic's own form, in the c1 slot it will
+// finally occupy while u^ pk0^ stays in shared memory; then two passes over
+// one copy of the inverse-transform code: h = 0 gives c0 = pk0 u + e0 + m from
+// shared memory, h = 1 reloads the parked product and gives c1 = pk1 u + e1.
+template <class M, class L, int V, bool NTT_OUT>
+__device__ __forceinline__ void encrypt_unit(const LimbDev &lb, const tw_t *p0, const tw_t *p1, uint64_t *sm,
+                                             const int8_t *su, const int8_t *se0, const int64_t *mt,
+                                             uint64_t *cbase, size_t cstride) {
+    using val = typename M::val;
+    constexpr uint32_t B = 1u << L::LOGB;
+    const uint32_t tid = threadIdx.x;
+    const uint64_t q = lb.q;
+    if constexpr (NTT_OUT) {
+        // transform-domain output: c0^ = pk0^ u^ + (e0 + m)^, c1^ = pk1^ u^ + e1^.  Three
+        // passes over one copy of the forward-transform code: u (both products wait in
+        // their final slots), then e0 + m and e1, each added to its product.
+        const auto fa = LimbOf<M>::args(lb, true, 0, 0);
+        const M &ar = fa.m;
+#pragma unroll 1
+        for (int h = 0; h < 3; h++) {
+            uint64_t *cc = cbase + (h == 2 ? cstride : 0);
+            const int8_t *se = se0 + (h == 2 ? B : 0);
+            smem_ntt_forward<L, V>(
+                sm, tid, fa,
+                [&](uint32_t i) {
+                    if (h == 0) return ar.small(su[i]);
+                    if (h == 2) return ar.small(se[i]);
+                    return ar.from_residue(signed_residue(mt[i] + (int64_t)se[i], q, lb.mu));
+                },
+                [&](uint32_t p, val a, val b) {
+                    if (h == 0) {
+                        const auto a0 = M::load_key(p0 + p), a1 = M::load_key(p0 + p + 1);
+                        const auto b0 = M::load_key(p1 + p), b1 = M::load_key(p1 + p + 1);
+                        *reinterpret_cast<u64x2 *>(cbase + p) =
+                            u64x2{M::bits(ar.mul_key(a, a0)), M::bits(ar.mul_key(b, a1))};
+                        *reinterpret_cast<u64x2 *>(cbase + cstride + p) =
+                            u64x2{M::bits(ar.mul_key(a, b0)), M::bits(ar.mul_key(b, b1))};
+                    } else {
+                        const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + p);
+                        *reinterpret_cast<u64x2 *>(cc + p) =
+                            u64x2{ar.canon_sum(a, M::from_bits(t.x)), ar.canon_sum(b, M::from_bits(t.y))};
+                    }
+                });
+            __syncthreads();   // last-phase readers are done before the next transform writes
+        }
+        return;
+    }
+    {
+        uint64_t *c1 = cbase + cstride;
+        const auto fa = LimbOf<M>::args(lb, true, 0, 0);
+        const M &ar = fa.m;
+        smem_ntt_forward<L, V>(
+            sm, tid, fa, [&](uint32_t i) { return ar.small(su[i]); },
+            [&](uint32_t p, val a, val b) {
+                const auto a0 = M::load_key(p1 + p), a1 = M::load_key(p1 + p + 1);
+                u64x2 v;
+                v.x = M::bits(ar.mul_key(a, a0));
+                v.y = M::bits(ar.mul_key(b, a1));
+                *reinterpret_cast<u64x2 *>(c1 + p) = v;
+                const auto b0 = M::load_key(p0 + p), b1 = M::load_key(p0 + p + 1);
+                sm[swz(p)] = M::bits(ar.mul_key(a, b0));
+                sm[swz(p + 1)] = M::bits(ar.mul_key(b, b1));
+            });
+    }
+#pragma unroll 1
+    for (int h = 0; h < 2; h++) {
+        uint64_t *cc = cbase + h * cstride;
+        const int8_t *se = se0 + h * B;
+        const auto ia = LimbOf<M>::args(lb, false, 0, 0);
+        const M &ar = ia.m;
+        smem_ntt_inverse<L, V, true>(
+            sm, tid, ia, LimbOf<M>::ninv(lb), LimbOf<M>::wn(lb),
+            [&](uint32_t p) {
+                if (h == 0) return pair_of<val>{M::from_bits(sm[swz(p)]), M::from_bits(sm[swz(p + 1)])};
+                const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + p);
+                return pair_of<val>{M::from_bits(t.x), M::from_bits(t.y)};
+            },
+            [&](uint32_t i, val v) {
+                // e1 is a small value; e0 + m needs a full reduction
+                const uint64_t add = h == 0 ? signed_residue(mt[i] + (int64_t)se[i], q, lb.mu)
+                                            : small_residue(se[i], q);
+                cc[i] = ar.canon_add(v, add);
+            });
+        __syncthreads();   // phase-0 readers are done before the next transform writes
+    }
+}
+
+// Fused path for N <= 2^14 (one block holds a whole limb): a thread block
+// draws u, e0, e1 of a ciphertext once into shared memory, then for every
+// limb of it transforms u, multiplies by both halves of the public key,
+// transforms back and adds the error (and message) terms.  Only the
+// ciphertext itself is written to global memory; the second product waits,
+// in transform order, in the c1 slot it will finally occupy.
+template <class L, int V, bool NTT_OUT>
+__global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
+encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const int64_t *m, uint32_t t0,
+                     uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
+    extern __shared__ __align__(16) uint64_t sm[];
+    constexpr uint32_t B = 1u << L::LOGB, RT = L::NT / V;
+    int8_t *su = reinterpret_cast<int8_t *>(sm + B);
+    int8_t *se0 = su + B, *se1 = se0 + B;
+    const uint32_t tid = threadIdx.x;
+    __shared__ GaussTables gt;
+    gauss_tables_init(gt, tid);
+
+    // Work units are (ciphertext, limb) pairs in ciphertext-major order, dealt
+    // evenly to the blocks of the grid (one block per SM), so that the last
+    // wave is as full as the others; a block re-draws u, e0, e1 whenever its
+    // range moves on to the next ciphertext.
+    const uint64_t units = (uint64_t)T * c.L;
+    const uint32_t u_begin = (uint32_t)(units * blockIdx.x / gridDim.x);
+    const uint32_t u_end = (uint32_t)(units * (blockIdx.x + 1) / gridDim.x);
+    const size_t cstride = (size_t)c.L * B;          // from c0 to c1 of the same limb
+    uint32_t sampled = 0xffffffffu;
+    for (uint32_t unit = u_begin; unit < u_end; unit++) {
+        const uint32_t tl = unit / c.L, j = unit % c.L;   // ciphertext within this call, limb
+        if (tl != sampled) {
+            sampled = tl;
+            const uint32_t t = t0 + tl;                   // stream coordinate
+            __syncthreads();                              // tables ready / previous samples no longer read
+            for (uint32_t b = tid; b < B / 4; b += RT) {
+                u32x4 w = stream_block(seed, b, t, client, TAG_ENC_U);
+                char4 v = make_char4((signed char)ternary_from_word(w.x), (signed char)ternary_from_word(w.y),
+                                     (signed char)ternary_from_word(w.z), (signed char)ternary_from_word(w.w));
+                reinterpret_cast<char4 *>(su)[b] = v;
+            }
+            for (uint32_t b = tid; b < B / 2; b += RT) {
+                u32x4 w0 = stream_block(seed, b, t, client, TAG_ENC_E0);
+                u32x4 w1 = stream_block(seed, b, t, client, TAG_ENC_E1);
+                char2 a = make_char2((signed char)gauss_from_u64(gt, (uint64_t)w0.x | ((uint64_t)w0.y << 32)),
+                                     (signed char)gauss_from_u64(gt, (uint64_t)w0.z | ((uint64_t)w0.w << 32)));
+                char2 e = make_char2((signed char)gauss_from_u64(gt, (uint64_t)w1.x | ((uint64_t)w1.y << 32)),
+                                     (signed char)gauss_from_u64(gt, (uint64_t)w1.z | ((uint64_t)w1.w << 32)));
+                reinterpret_cast<char2 *>(se0)[b] = a;
+                reinterpret_cast<char2 *>(se1)[b] = e;
+            }
+            __syncthreads();
+        }
+        const LimbDev &lb = c.limb[j];
+        uint64_t *cbase = ct + (((size_t)tl * 2 + 0) * c.L + j) * B;
+        FEDHE_FOR_ARITH(lb, (encrypt_unit<M_, L, V, NTT_OUT>(lb, k.pk0_hat + (size_t)j * B, k.pk1_hat + (size_t)j * B, sm, su,
+                                                    se0, m + (size_t)tl * B, cbase, cstride)));
+    }
+}
+
+// One (ciphertext, limb) unit of the two-group kernel below (N = 2 * 2^LOGB).
+template <class M, class L, int V, bool NTT_OUT>
+__device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0, const tw_t *pk1, uint64_t *sm,
+                                              const int8_t *su, const int8_t *se0, const int64_t *mt,
+                                              uint64_t *cbase, size_t cstride) {
+    using val = typename M::val;
+    constexpr uint32_t H = 1u << L::LOGB, B = 2 * H;
+    constexpr uint32_t GT = L::NT / V, RT = 2 * GT;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t grp = tid / GT, gt = tid % GT;
+    uint64_t *smg = sm + grp * H;                          // this group's half
+    const GroupSync gsync = {1 + grp, GT};
+    const uint64_t q = lb.q;
+    {
+        const tw_t *p0 = pk0 + grp * H, *p1 = pk1 + grp * H;
+        uint64_t *c1 = cbase + cstride + grp * H;
+        const auto fa = LimbOf<M>::args(lb, true, 1, grp);
+        const M &ar = fa.m;
+        const auto w0 = M::load(fa.tw + 1);                // twiddle of the stage that pairs the halves
+        auto src = [&](uint32_t i) {
+            // u is ternary: the twiddle product is 0, w or -w
+            const int b = su[i + H];
+            if constexpr (std::is_same<M, ModF64>::value) {
+                return f64_fma(grp == 0 ? (double)b : (double)-b, w0, (double)su[i]);
+            } else {
+                const uint64_t u = small_residue(su[i], q);
+                const uint64_t v = b == 0 ? 0 : (b > 0 ? w0.w : q - w0.w);
+                return grp == 0 ? u + v : u - v + ar.q2;
+            }
+        };
+        if constexpr (NTT_OUT) {
+            // transform-domain output: three passes over one copy of the forward code: u
+            // (both products wait in their final slots), then e0 + m and e1, whose pairing
+            // stage costs one product per element, each added to its product
+            uint64_t *c0 = cbase + grp * H;
+#pragma unroll 1
+            for (int h = 0; h < 3; h++) {
+                uint64_t *cc = h == 2 ? c1 : c0;
+                const int8_t *se = se0 + (h == 2 ? B : 0);
+                auto value = [&](uint32_t i) {
+                    if (h == 2) return ar.small(se[i]);
+                    return ar.from_residue(signed_residue(mt[i] + (int64_t)se[i], q, lb.mu));
+                };
+                smem_ntt_forward<L, V>(
+                    smg, gt, fa,
+                    [&](uint32_t i) {
+                        if (h == 0) return src(i);
+                        const val lo = value(i), hi = value(i + H);
+                        if constexpr (std::is_same<M, ModF64>::value) {
+                            const double t = ar.mul(hi, w0);
+                            return grp == 0 ? f64_add(lo, t) : f64_sub(lo, t);
+                        } else {
+                            const uint64_t t = shoup_lazy(hi, w0.w, w0.wp, q);
+                            return grp == 0 ? lo + t : lo - t + ar.q2;
+                        }
+                    },
+                    [&](uint32_t p, val a, val b) {
+                        if (h == 0) {
+                            const auto a0 = M::load_key(p0 + p), a1 = M::load_key(p0 + p + 1);
+                            const auto b0 = M::load_key(p1 + p), b1 = M::load_key(p1 + p + 1);
+                            *reinterpret_cast<u64x2 *>(c0 + p) =
+                                u64x2{M::bits(ar.mul_key(a, a0)), M::bits(ar.mul_key(b, a1))};
+                            *reinterpret_cast<u64x2 *>(c1 + p) =
+                                u64x2{M::bits(ar.mul_key(a, b0)), M::bits(ar.mul_key(b, b1))};
+                        } else {
+                            const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + p);
+                            *reinterpret_cast<u64x2 *>(cc + p) =
+                                u64x2{ar.canon_sum(a, M::from_bits(t.x)), ar.canon_sum(b, M::from_bits(t.y))};
+                        }
+                    },
+                    gsync);
+                gsync();   // last-phase readers of this half are done before phase 0 writes
+            }
+            __syncthreads();
+            return;
+        }
+        auto dst = [&](uint32_t p, val a, val b) {
+            const auto a0 = M::load_key(p1 + p), a1 = M::load_key(p1 + p + 1);
+            u64x2 v;
+            v.x = M::bits(ar.mul_key(a, a0));
+            v.y = M::bits(ar.mul_key(b, a1));
+            *reinterpret_cast<u64x2 *>(c1 + p) = v;      // parked until the second pass
+            const auto b0 = M::load_key(p0 + p), b1 = M::load_key(p0 + p + 1);
+            smg[swz(p)] = M::bits(ar.mul_key(a, b0));
+            smg[swz(p + 1)] = M::bits(ar.mul_key(b, b1));
+        };
+        smem_ntt_forward<L, V>(smg, gt, fa, src, dst, gsync);
+    }
+#pragma unroll 1
+    for (int h = 0; h < 2; h++) {
+        uint64_t *cc = cbase + h * cstride;
+        const int8_t *se = se0 + h * B;
+        const auto ia = LimbOf<M>::args(lb, false, 1, grp);
+        const M &ar = ia.m;
+        const auto ninv = LimbOf<M>::ninv(lb), wn = LimbOf<M>::wn(lb);
+        auto isrc = [&](uint32_t p) {
+            if (h == 0) return pair_of<val>{M::from_bits(smg[swz(p)]), M::from_bits(smg[swz(p + 1)])};
+            const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + grp * H + p);
+            return pair_of<val>{M::from_bits(t.x), M::from_bits(t.y)};
+        };
+        auto idst = [&](uint32_t i, val v) { smg[swz(i)] = M::bits(v); };
+        smem_ntt_inverse<L, V, false>(smg, gt, ia, ninv, wn, isrc, idst, gsync);
+        __syncthreads();
+        // last stage across the halves with 1/N folded in, then the error / message terms
+        for (uint32_t e = tid; e < H; e += RT) {
+            val lo = M::from_bits(sm[swz(e)]), hi = M::from_bits(sm[H + swz(e)]);
+            ar.inv_scaled(lo, hi, ninv, wn);
+            uint64_t add_lo, add_hi;
+            if (h == 0) {
+                add_lo = signed_residue(mt[e] + (int64_t)se[e], q, lb.mu);
+                add_hi = signed_residue(mt[e + H] + (int64_t)se[e + H], q, lb.mu);
+            } else {
+                add_lo = small_residue(se[e], q);
+                add_hi = small_residue(se[e + H], q);
+            }
+            cc[e] = ar.canon_add(lo, add_lo);
+            cc[e + H] = ar.canon_add(hi, add_hi);
+        }
+        __syncthreads();
+    }
+}
+
+// The same for N = 2 * 2^LOGB (N = 2^14 with LOGB = 13): the thread block is
+// two groups of threads, each of which transforms one half of the limb as a
+// sub-block of the long transform on its own schedule (named barriers), so
+// that one group's barrier and memory waits overlap the other's arithmetic.
+// The stage that pairs the two halves is done where both are at hand: on the
+// way in for the forward transform (u is ternary, so the twiddle product is
+// 0, w or q-w, computed by both groups from the shared samples) and by the
+// whole block after the two inverse sub-transforms, fused with the epilogue.
+template <class L, int V, bool NTT_OUT>
+__global__ void __launch_bounds__(2 * L::NT / V, 1)
+encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const int64_t *m, uint32_t t0,
+                      uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
+    extern __shared__ __align__(16) uint64_t sm[];
+    constexpr uint32_t H = 1u << L::LOGB, B = 2 * H;       // half and whole limb
+    constexpr uint32_t GT = L::NT / V, RT = 2 * GT;        // threads per group, per block
+    int8_t *su = reinterpret_cast<int8_t *>(sm + B);
+    int8_t *se0 = su + B, *se1 = se0 + B;
+    const uint32_t tid = threadIdx.x;
+    __shared__ GaussTables gt_tab;
+    gauss_tables_init(gt_tab, tid);
+
+    const uint64_t units = (uint64_t)T * c.L;
+    const uint32_t u_begin = (uint32_t)(units * blockIdx.x / gridDim.x);
+    const uint32_t u_end = (uint32_t)(units * (blockIdx.x + 1) / gridDim.x);
+    const size_t cstride = (size_t)c.L * B;
+    uint32_t sampled = 0xffffffffu;
+    for (uint32_t unit = u_begin; unit < u_end; unit++) {
+        const uint32_t tl = unit / c.L, j = unit % c.L;
+        if (tl != sampled) {
+            sampled = tl;
+            const uint32_t t = t0 + tl;
+            __syncthreads();
+            for (uint32_t b = tid; b < B / 4; b += RT) {
+                u32x4 w = stream_block(seed, b, t, client, TAG_ENC_U);
+                char4 v = make_char4((signed char)ternary_from_word(w.x), (signed char)ternary_from_word(w.y),
+                                     (signed char)ternary_from_word(w.z), (signed char)ternary_from_word(w.w));
+                reinterpret_cast<char4 *>(su)[b] = v;
+            }
+            for (uint32_t b = tid; b < B / 2; b += RT) {
+                u32x4 w0 = stream_block(seed, b, t, client, TAG_ENC_E0);
+                u32x4 w1 = stream_block(seed, b, t, client, TAG_ENC_E1);
+                char2 a = make_char2((signed char)gauss_from_u64(gt_tab, (uint64_t)w0.x | ((uint64_t)w0.y << 32)),
+                                     (signed char)gauss_from_u64(gt_tab, (uint64_t)w0.z | ((uint64_t)w0.w << 32)));
+                char2 e = make_char2((signed char)gauss_from_u64(gt_tab, (uint64_t)w1.x | ((uint64_t)w1.y << 32)),
+                                     (signed char)gauss_from_u64(gt_tab, (uint64_t)w1.z | ((uint64_t)w1.w << 32)));
+                reinterpret_cast<char2 *>(se0)[b] = a;
+                reinterpret_cast<char2 *>(se1)[b] = e;
+            }
+            __syncthreads();
+        }
+        const LimbDev &lb = c.limb[j];
+        uint64_t *cbase = ct + (((size_t)tl * 2 + 0) * c.L + j) * B;
+        FEDHE_FOR_ARITH(lb, (encrypt_unit2<M_, L, V, NTT_OUT>(lb, k.pk0_hat + (size_t)j * B, k.pk1_hat + (size_t)j * B, sm, su,
+                                                     se0, m + (size_t)tl * B, cbase, cstride)));
+    }
+}
+
+// Long rings (N = 2^15, 2^16), where a limb does not fit one SM: the ciphertext
+// buffer itself is the only work space and every pass over it does as much as
+// it can.  (1) draw u and run the outer forward stages into the c1 slots;
+// (2) block transforms of the c1 slots whose last phase writes both products
+// u^ pk0^ -> c0 and u^ pk1^ -> c1; (3) inverse block transforms of all slots;
+// (4) outer inverse stages fused with the error and message terms.
+
+template <class M, uint32_t A>
+__device__ __forceinline__ void enc_outer_sample_limb(const LimbDev &lb, const int (&u)[1u << A][2], uint64_t *p,
+                                                      uint32_t B) {
+    constexpr uint32_t rows = 1u << A;
+    const auto t = LimbOf<M>::args(lb, true, 0, 0);
+    typename M::val x[rows], y[rows];
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++) {
+        x[a] = t.m.small(u[a][0]);
+        y[a] = t.m.small(u[a][1]);
+    }
+    outer_forward<A>(x, y, t);
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++)
+        *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = u64x2{M::bits(x[a]), M::bits(y[a])};
+}
+
+// (1) one thread per pair of neighbouring columns of one ciphertext, all limbs;
+// the limbs of ciphertext tl go to dst + tl * ct_stride
+template <uint32_t A>
+__global__ void __launch_bounds__(256)
+enc_outer_sample_kernel(const __grid_constant__ CtxDev c, uint32_t t0, uint64_t seed, uint32_t client,
+                        uint64_t *dst, size_t ct_stride, size_t total) {
+    size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t B = 1u << c.LOGB, half = B >> 1;
+    constexpr uint32_t rows = 1u << A;
+    const uint32_t col = (uint32_t)(g % half) * 2;
+    const size_t tl = g / half;
+    int u[rows][2];
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++) {
+        const uint32_t i = a * B + col;               // even: both columns share a Philox block
+        const u32x4 w = stream_block(seed, i >> 2, t0 + (uint32_t)tl, client, TAG_ENC_U);
+        u[a][0] = ternary_from_word((i & 2) ? w.z : w.x);
+        u[a][1] = ternary_from_word((i & 2) ? w.w : w.y);
+    }
+#pragma unroll 1
+    for (uint32_t j = 0; j < c.L; j++) {
+        const LimbDev &lb = c.limb[j];
+        uint64_t *p = dst + tl * ct_stride + (size_t)j * c.N + col;   // limb j of ciphertext tl
+        FEDHE_FOR_ARITH(lb, (enc_outer_sample_limb<M_, A>(lb, u, p, B)));
+    }
+}
+
+// (2) one thread block per (ciphertext, limb, block): forward block transform of
+// the c1 slot, products with both halves of the public key on the way out
+template <class M, class L, int V, bool ACC>
+__device__ __forceinline__ void enc_block_forward(const CtxDev &c, const LimbDev &lb, uint64_t *sm, uint32_t blk,
+                                                  const tw_t *p0, const tw_t *p1, const uint64_t *u,
+                                                  uint64_t *c0, uint64_t *c1) {
+    using val = typename M::val;
+    const auto a = LimbOf<M>::args(lb, true, c.A, blk);
+    const M &ar = a.m;
+    smem_ntt_forward<L, V>(
+        sm, threadIdx.x, a, [&](uint32_t i) { return M::from_bits(u[i]); },
+        [&](uint32_t p, val x, val y) {
+            const auto a0 = M::load_key(p0 + p), a1 = M::load_key(p0 + p + 1);
+            const auto b0 = M::load_key(p1 + p), b1 = M::load_key(p1 + p + 1);
+            u64x2 v0, v1;
+            if constexpr (ACC) {       // the slots hold canonical residues to add to
+                v0 = *reinterpret_cast<const u64x2 *>(c0 + p);
+                v1 = *reinterpret_cast<const u64x2 *>(c1 + p);
+                v0.x = ar.canon_add(ar.mul_key(x, a0), v0.x);
+                v0.y = ar.canon_add(ar.mul_key(y, a1), v0.y);
+                v1.x = ar.canon_add(ar.mul_key(x, b0), v1.x);
+                v1.y = ar.canon_add(ar.mul_key(y, b1), v1.y);
+            } else {
+                v0.x = ar.to_residue(ar.mul_key(x, a0));
+                v0.y = ar.to_residue(ar.mul_key(y, a1));
+                v1.x = ar.to_residue(ar.mul_key(x, b0));
+                v1.y = ar.to_residue(ar.mul_key(y, b1));
+            }
+            *reinterpret_cast<u64x2 *>(c0 + p) = v0;
+            *reinterpret_cast<u64x2 *>(c1 + p) = v1;
+        });
+}
+
+// ACC = false: u comes from the c1 slot and the products replace both slots;
+// ACC = true: u comes from `ubuf` ([T][L][N]) and the products are added to the slots
+template <class L, int V, bool ACC>
+__global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
+enc_block_forward_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const uint64_t *ubuf, uint64_t *ct) {
+    extern __shared__ __align__(16) uint64_t sm[];
+    uint32_t b = blockIdx.x;
+    const uint32_t blk = b & ((1u << c.A) - 1u);
+    b >>= c.A;
+    const uint32_t j = b % c.L;
+    const size_t tl = b / c.L;
+    const LimbDev &lb = c.limb[j];
+    const size_t off = ((size_t)blk << L::LOGB);
+    uint64_t *c0 = ct + ((tl * 2 + 0) * c.L + j) * c.N + off;
+    uint64_t *c1 = ct + ((tl * 2 + 1) * c.L + j) * c.N + off;
+    const uint64_t *u = ACC ? ubuf + (tl * c.L + j) * c.N + off : c1;
+    const tw_t *p0 = k.pk0_hat + (size_t)j * c.N + off, *p1 = k.pk1_hat + (size_t)j * c.N + off;
+    FEDHE_FOR_ARITH(lb, (enc_block_forward<M_, L, V, ACC>(c, lb, sm, blk, p0, p1, u, c0, c1)));
+}
+
+// long rings, transform-domain format: residues of e0 + m into the c0 slots and
+// of e1 into the c1 slots; one thread per pair of neighbouring coefficients
+__global__ void __launch_bounds__(256)
+enc_fill_errors_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint32_t t0, uint64_t seed,
+                       uint32_t client, uint64_t *ct, size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t pairs = c.N >> 1;
+    const uint32_t b = (uint32_t)(g % pairs), i = 2 * b;   // one Philox block per pair
+    const size_t tl = g / pairs;
+    const uint32_t t = t0 + (uint32_t)tl;
+    const u32x4 w0 = stream_block(seed, b, t, client, TAG_ENC_E0);
+    const u32x4 w1 = stream_block(seed, b, t, client, TAG_ENC_E1);
+    const longlong2 mm = *reinterpret_cast<const longlong2 *>(m + tl * c.N + i);
+    const int64_t ax = mm.x + gauss_from_u64((uint64_t)w0.x | ((uint64_t)w0.y << 32));
+    const int64_t ay = mm.y + gauss_from_u64((uint64_t)w0.z | ((uint64_t)w0.w << 32));
+    const int ex = gauss_from_u64((uint64_t)w1.x | ((uint64_t)w1.y << 32));
+    const int ey = gauss_from_u64((uint64_t)w1.z | ((uint64_t)w1.w << 32));
+    for (uint32_t j = 0; j < c.L; j++) {
+        const LimbDev &lb = c.limb[j];
+        const uint64_t q = lb.q;
+        *reinterpret_cast<u64x2 *>(ct + ((tl * 2 + 0) * c.L + j) * c.N + i) =
+            u64x2{signed_residue(ax, q, lb.mu), signed_residue(ay, q, lb.mu)};
+        *reinterpret_cast<u64x2 *>(ct + ((tl * 2 + 1) * c.L + j) * c.N + i) =
+            u64x2{small_residue(ex, q), small_residue(ey, q)};
+    }
+}
+
+template <class M, uint32_t A>
+__device__ __forceinline__ void enc_outer_inverse_add_limb(const LimbDev &lb, uint64_t *p, uint32_t B, bool first,
+                                                           const int64_t (&me0)[1u << A][2],
+                                                           const int (&e1)[1u << A][2]) {
+    constexpr uint32_t rows = 1u << A;
+    const uint64_t q = lb.q;
+    const auto t = LimbOf<M>::args(lb, false, 0, 0);
+    typename M::val x[rows], y[rows];
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++) {
+        const u64x2 v = *reinterpret_cast<const u64x2 *>(p + (size_t)a * B);
+        x[a] = M::from_bits(v.x);
+        y[a] = M::from_bits(v.y);
+    }
+    outer_inverse<A>(x, y, t, LimbOf<M>::ninv(lb), LimbOf<M>::wn(lb));
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++) {
+        u64x2 o;
+        if (first) {
+            o.x = t.m.canon_add(x[a], signed_residue(me0[a][0], q, lb.mu));
+            o.y = t.m.canon_add(y[a], signed_residue(me0[a][1], q, lb.mu));
+        } else {
+            o.x = t.m.canon_add(x[a], small_residue(e1[a][0], q));
+            o.y = t.m.canon_add(y[a], small_residue(e1[a][1], q));
+        }
+        *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = o;
+    }
+}
+
+// (4) one thread per pair of neighbouring columns of one ciphertext: draws the
+// errors once, then for every limb finishes both components
+template <uint32_t A>
+__global__ void __launch_bounds__(256, 2)
+enc_outer_inverse_add_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint32_t t0, uint64_t seed,
+                             uint32_t client, uint64_t *ct, size_t total) {
+    size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t B = 1u << c.LOGB, half = B >> 1;
+    constexpr uint32_t rows = 1u << A;
+    const uint32_t col = (uint32_t)(g % half) * 2;
+    const size_t tl = g / half;
+    const uint32_t t = t0 + (uint32_t)tl;
+    int e1[rows][2];
+    int64_t me0[rows][2];                              // m + e0
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++) {
+        const uint32_t i = a * B + col;               // one Philox block per pair of coefficients
+        const u32x4 w0 = stream_block(seed, i >> 1, t, client, TAG_ENC_E0);
+        const u32x4 w1 = stream_block(seed, i >> 1, t, client, TAG_ENC_E1);
+        const longlong2 mm = *reinterpret_cast<const longlong2 *>(m + tl * c.N + i);
+        me0[a][0] = mm.x + gauss_from_u64((uint64_t)w0.x | ((uint64_t)w0.y << 32));
+        me0[a][1] = mm.y + gauss_from_u64((uint64_t)w0.z | ((uint64_t)w0.w << 32));
+        e1[a][0] = gauss_from_u64((uint64_t)w1.x | ((uint64_t)w1.y << 32));
+        e1[a][1] = gauss_from_u64((uint64_t)w1.z | ((uint64_t)w1.w << 32));
+    }
+#pragma unroll 1
+    for (uint32_t j = 0; j < c.L; j++) {
+        const LimbDev &lb = c.limb[j];
+#pragma unroll 1
+        for (uint32_t comp = 0; comp < 2; comp++) {
+            uint64_t *p = ct + ((tl * 2 + comp) * c.L + j) * c.N + col;
+            FEDHE_FOR_ARITH(lb, (enc_outer_inverse_add_limb<M_, A>(lb, p, B, comp == 0, me0, e1)));
+        }
+    }
+}
+
+template <class L, int V, bool TWO_GROUPS, bool NTT_OUT>
+static cudaError_t launch_encrypt_fused(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0,
+                                        size_t T, uint64_t seed, uint32_t client, uint64_t *ct,
+                                        cudaStream_t s) {
+    const size_t smem = ((sizeof(uint64_t) << L::LOGB) + (3u << L::LOGB)) * (TWO_GROUPS ? 2 : 1);
+    auto kern = TWO_GROUPS ? encrypt_fused2_kernel<L, V, NTT_OUT> : encrypt_fused_kernel<L, V, NTT_OUT>;
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+    // one block per SM (the kernel's shared memory allows no more), fewer if there is less work
+    int dev = 0, n_sm = 0;
+    if ((e = cudaGetDevice(&dev)) || (e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev))) return e;
+    const size_t per_sm = (size_t)(227 * 1024) / smem;               // blocks that fit one SM
+    size_t grid = (size_t)n_sm * (per_sm ? per_sm : 1);
+    if (grid > T * c.L) grid = T * c.L;
+    kern<<<(unsigned)grid, (TWO_GROUPS ? 2 : 1) * L::NT / V, smem, s>>>(c, k, m, t0, seed, client, ct, (uint32_t)T);
+    return FEDHE_LAUNCHED();
+}
+
+// launches the block forward kernel of the long-ring paths
+template <bool ACC>
+static cudaError_t launch_enc_block_forward(const CtxDev &c, const KeysDev &k, const uint64_t *ubuf, size_t T,
+                                            uint64_t *ct, cudaStream_t s) {
+    using L = Lay<13, 3>;                                 // long rings are cut into 2^13 blocks
+    constexpr int V = 2;
+    const size_t smem = sizeof(uint64_t) << L::LOGB;
+    auto kern = enc_block_forward_kernel<L, V, ACC>;
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+    kern<<<(unsigned)((T * c.L) << c.A), L::NT / V, smem, s>>>(c, k, ubuf, ct);
+    return FEDHE_LAUNCHED();
+}
+
+cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0, size_t T,
+                           uint64_t seed, uint32_t client, uint64_t *ct, cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    if (c.A == 0) {
+        if (c.LOGB == 13)
+            return launch_encrypt_fused<Lay<13, 3>, 2, false, false>(c, k, m, t0, T, seed, client, ct, s);
+        return launch_encrypt_fused<Lay<13, 3>, 2, true, false>(c, k, m, t0, T, seed, client, ct, s);
+    }
+    cudaError_t e;
+    const size_t cols = T * ((size_t)1 << (c.LOGB - 1));      // pairs of columns
+    const size_t LN = (size_t)c.L * c.N;
+    FEDHE_FOR_A(c, (enc_outer_sample_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, t0, seed, client, ct + LN,
+                                                                                     2 * LN, cols)));
+    if ((e = FEDHE_LAUNCHED())) return e;
+    if ((e = launch_enc_block_forward<false>(c, k, nullptr, T, ct, s))) return e;
+    if ((e = launch_ntt_inner(c, false, ct, 2 * T, LN, 0, c.L, s))) return e;
+    FEDHE_FOR_A(c, (enc_outer_inverse_add_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, m, t0, seed, client, ct,
+                                                                                          cols)));
+    return FEDHE_LAUNCHED();
+}
+
+// Transform-domain wire format: the same ciphertext with every limb polynomial
+// stored as its negacyclic transform.  N <= 2^14: the fused kernels with three
+// forward transforms per limb.  Longer rings: the error terms go into the
+// ciphertext slots and are transformed there; u is transformed in the work
+// buffer `ubuf` ([T][L][N]) and its key products are added on the way out.
+cudaError_t launch_encrypt_ntt(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0, size_t T,
+                               uint64_t seed, uint32_t client, uint64_t *ubuf, uint64_t *ct, cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    if (c.A == 0) {
+        if (c.LOGB == 13)
+            return launch_encrypt_fused<Lay<13, 3>, 2, false, true>(c, k, m, t0, T, seed, client, ct, s);
+        return launch_encrypt_fused<Lay<13, 3>, 2, true, true>(c, k, m, t0, T, seed, client, ct, s);
+    }
+    cudaError_t e;
+    const size_t LN = (size_t)c.L * c.N;
+    const size_t pairs = T * (size_t)(c.N >> 1);
+    enc_fill_errors_kernel<<<blocks_for(pairs, 256), 256, 0, s>>>(c, m, t0, seed, client, ct, pairs);
+    if ((e = FEDHE_LAUNCHED())) return e;
+    if ((e = launch_ntt(c, true, ct, 2 * T, LN, 0, c.L, s))) return e;
+    const size_t cols = T * ((size_t)1 << (c.LOGB - 1));
+    FEDHE_FOR_A(c, (enc_outer_sample_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, t0, seed, client, ubuf, LN,
+                                                                                     cols)));
+    if ((e = FEDHE_LAUNCHED())) return e;
+    return launch_enc_block_forward<true>(c, k, ubuf, T, ct, s);
+}
+
+}  // namespace fedhe

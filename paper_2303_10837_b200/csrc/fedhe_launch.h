@@ -1,4 +1,4 @@
-// Launch wrappers of the CUDA kernels (implemented in fedhe_kernels.cu),
+// Launch wrappers of the CUDA kernels (implemented in fedhe_transform.cu, fedhe_slots.cu, fedhe_encrypt.cu, fedhe_server.cu, fedhe_decrypt.cu and fedhe_mask.cu),
 // called by the C ABI in fedhe_api.cu.  All of them enqueue work on `s` and
 // return the launch status; none synchronises.
 #pragma once

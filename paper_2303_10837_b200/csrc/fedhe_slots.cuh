@@ -1,0 +1,119 @@
+// Device code of the CKKS slot transform: complex arithmetic with one rounding
+// per operation, the register-tiled butterfly network and its shared-memory
+// exchange.  Used by the encode / decode kernels and by the fused decrypt.
+#pragma once
+
+#include "fedhe_kernels.cuh"
+
+namespace fedhe {
+
+// ===========================================================================
+// CKKS slot transform (fp64).  Encoding must reproduce one fixed radix-2
+// network operation by operation (separate IEEE multiply and add, no fused
+// multiply-add), because the rounded integers are compared bit for bit.
+// ===========================================================================
+
+struct cpx { double re, im; };
+
+__device__ __forceinline__ cpx cadd_rn(cpx a, cpx b) { return cpx{__dadd_rn(a.re, b.re), __dadd_rn(a.im, b.im)}; }
+__device__ __forceinline__ cpx csub_rn(cpx a, cpx b) { return cpx{__dsub_rn(a.re, b.re), __dsub_rn(a.im, b.im)}; }
+// (a + bi)(c + di) = (ac - bd) + (ad + bc) i, data operand first
+__device__ __forceinline__ cpx cmul_rn(cpx x, cpx w) {
+    cpx r;
+    r.re = __dsub_rn(__dmul_rn(x.re, w.re), __dmul_rn(x.im, w.im));
+    r.im = __dadd_rn(__dmul_rn(x.re, w.im), __dmul_rn(x.im, w.re));
+    return r;
+}
+__device__ __forceinline__ cpx load_ftw(const double2 *ftw, uint32_t i) {
+    double2 v = __ldg(ftw + i);
+    return cpx{v.x, v.y};
+}
+
+// decimation-in-frequency stage of the inverse (encoding) network
+template <class L, int P, int I>
+__device__ __forceinline__ void dif_stage(cpx (&x)[L::E], uint32_t tid, const double2 *ftw) {
+    constexpr int s = P * L::LE + I;
+    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
+    constexpr int bit = nst - 1 - I;
+    constexpr uint32_t half = 1u << (L::LOGB - 1 - s);
+#pragma unroll
+    for (int r = 0; r < L::E; r++) {
+        if (r & (1 << bit)) continue;
+        const uint32_t j = L::template idx<P>(tid, r) & (half - 1u);
+        cpx w = load_ftw(ftw, half + j);
+        w.im = -w.im;
+        const cpx U = x[r], V = x[r | (1 << bit)];
+        x[r] = cadd_rn(U, V);
+        x[r | (1 << bit)] = cmul_rn(csub_rn(U, V), w);
+    }
+}
+
+// decimation-in-time stage of the forward (decoding) network
+template <class L, int P, int I>
+__device__ __forceinline__ void dit_stage(cpx (&x)[L::E], uint32_t tid, const double2 *ftw) {
+    constexpr int s = P * L::LE + I;
+    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
+    constexpr int bit = nst - 1 - I;
+    constexpr uint32_t half = 1u << (L::LOGB - 1 - s);
+#pragma unroll
+    for (int r = 0; r < L::E; r++) {
+        if (r & (1 << bit)) continue;
+        const uint32_t j = L::template idx<P>(tid, r) & (half - 1u);
+        const cpx w = load_ftw(ftw, half + j);
+        const cpx U = x[r], V = cmul_rn(x[r | (1 << bit)], w);
+        x[r] = cadd_rn(U, V);
+        x[r | (1 << bit)] = csub_rn(U, V);
+    }
+}
+
+template <class L, int P, int I = 0>
+__device__ __forceinline__ void dif_phase(cpx (&x)[L::E], uint32_t tid, const double2 *ftw) {
+    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
+    if constexpr (I < nst) {
+        dif_stage<L, P, I>(x, tid, ftw);
+        dif_phase<L, P, I + 1>(x, tid, ftw);
+    }
+}
+template <class L, int P, int I>
+__device__ __forceinline__ void dit_phase_from(cpx (&x)[L::E], uint32_t tid, const double2 *ftw) {
+    if constexpr (I >= 0) {
+        dit_stage<L, P, I>(x, tid, ftw);
+        dit_phase_from<L, P, I - 1>(x, tid, ftw);
+    }
+}
+
+template <class L, int PF, int PT>
+__device__ __forceinline__ void cpx_exchange(cpx (&x)[L::E], cpx *sm, uint32_t tid) {
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < L::E; r++) sm[swz(L::template idx<PF>(tid, r))] = x[r];
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < L::E; r++) x[r] = sm[swz(L::template idx<PT>(tid, r))];
+}
+
+template <class L, int P = 0>
+__device__ __forceinline__ void block_dif(cpx (&x)[L::E], cpx *sm, uint32_t tid, const double2 *ftw) {
+    dif_phase<L, P>(x, tid, ftw);
+    if constexpr (P + 1 < L::NPH) {
+        cpx_exchange<L, P, P + 1>(x, sm, tid);
+        block_dif<L, P + 1>(x, sm, tid, ftw);
+    }
+}
+template <class L, int P = L::NPH - 1>
+__device__ __forceinline__ void block_dit(cpx (&x)[L::E], cpx *sm, uint32_t tid, const double2 *ftw) {
+    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
+    dit_phase_from<L, P, nst - 1>(x, tid, ftw);
+    if constexpr (P > 0) {
+        cpx_exchange<L, P, P - 1>(x, sm, tid);
+        block_dit<L, P - 1>(x, sm, tid, ftw);
+    }
+}
+
+__device__ __forceinline__ uint32_t bitrev(uint32_t v, int bits) { return __brev(v) >> (32 - bits); }
+// index swizzle of the encoder's output staging buffer: bit-reversed writes of
+// a warp differ only in high index bits; folding them into the low nibble
+// spreads them over the banks (checked exhaustively for both block sizes)
+__device__ __forceinline__ uint32_t stage_swz(uint32_t k) { return k ^ (((k >> 8) ^ (k >> 4)) & 15u); }
+
+}  // namespace fedhe
