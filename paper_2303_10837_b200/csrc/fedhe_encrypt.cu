@@ -442,6 +442,9 @@ enc_block_forward_kernel(const __grid_constant__ CtxDev c, const KeysDev k, cons
 __global__ void __launch_bounds__(256)
 enc_fill_errors_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint32_t t0, uint64_t seed,
                        uint32_t client, uint64_t *ct, size_t total) {
+    __shared__ GaussTables gt;
+    gauss_tables_init(gt, threadIdx.x);
+    __syncthreads();
     const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= total) return;
     const uint32_t pairs = c.N >> 1;
@@ -451,10 +454,10 @@ enc_fill_errors_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint3
     const u32x4 w0 = stream_block(seed, b, t, client, TAG_ENC_E0);
     const u32x4 w1 = stream_block(seed, b, t, client, TAG_ENC_E1);
     const longlong2 mm = *reinterpret_cast<const longlong2 *>(m + tl * c.N + i);
-    const int64_t ax = mm.x + gauss_from_u64((uint64_t)w0.x | ((uint64_t)w0.y << 32));
-    const int64_t ay = mm.y + gauss_from_u64((uint64_t)w0.z | ((uint64_t)w0.w << 32));
-    const int ex = gauss_from_u64((uint64_t)w1.x | ((uint64_t)w1.y << 32));
-    const int ey = gauss_from_u64((uint64_t)w1.z | ((uint64_t)w1.w << 32));
+    const int64_t ax = mm.x + gauss_from_u64(gt, (uint64_t)w0.x | ((uint64_t)w0.y << 32));
+    const int64_t ay = mm.y + gauss_from_u64(gt, (uint64_t)w0.z | ((uint64_t)w0.w << 32));
+    const int ex = gauss_from_u64(gt, (uint64_t)w1.x | ((uint64_t)w1.y << 32));
+    const int ey = gauss_from_u64(gt, (uint64_t)w1.z | ((uint64_t)w1.w << 32));
     for (uint32_t j = 0; j < c.L; j++) {
         const LimbDev &lb = c.limb[j];
         const uint64_t q = lb.q;
@@ -466,9 +469,8 @@ enc_fill_errors_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint3
 }
 
 template <class M, uint32_t A>
-__device__ __forceinline__ void enc_outer_inverse_add_limb(const LimbDev &lb, uint64_t *p, uint32_t B, bool first,
-                                                           const int64_t (&me0)[1u << A][2],
-                                                           const int (&e1)[1u << A][2]) {
+__device__ __forceinline__ void enc_outer_inverse_add_limb(const LimbDev &lb, uint64_t *p, uint32_t B,
+                                                           const int64_t (&add)[1u << A][2]) {
     constexpr uint32_t rows = 1u << A;
     const uint64_t q = lb.q;
     const auto t = LimbOf<M>::args(lb, false, 0, 0);
@@ -483,23 +485,21 @@ __device__ __forceinline__ void enc_outer_inverse_add_limb(const LimbDev &lb, ui
 #pragma unroll
     for (uint32_t a = 0; a < rows; a++) {
         u64x2 o;
-        if (first) {
-            o.x = t.m.canon_add(x[a], signed_residue(me0[a][0], q, lb.mu));
-            o.y = t.m.canon_add(y[a], signed_residue(me0[a][1], q, lb.mu));
-        } else {
-            o.x = t.m.canon_add(x[a], small_residue(e1[a][0], q));
-            o.y = t.m.canon_add(y[a], small_residue(e1[a][1], q));
-        }
+        o.x = t.m.canon_add(x[a], signed_residue(add[a][0], q, lb.mu));
+        o.y = t.m.canon_add(y[a], signed_residue(add[a][1], q, lb.mu));
         *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = o;
     }
 }
 
-// (4) one thread per pair of neighbouring columns of one ciphertext: draws the
-// errors once, then for every limb finishes both components
+// (4) one thread per pair of neighbouring columns of one ciphertext: for each
+// component draws its error terms once (e0 + m, then e1), then finishes every limb
 template <uint32_t A>
-__global__ void __launch_bounds__(256, 2)
+__global__ void __launch_bounds__(256, A == 3 ? 2 : 4)
 enc_outer_inverse_add_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint32_t t0, uint64_t seed,
                              uint32_t client, uint64_t *ct, size_t total) {
+    __shared__ GaussTables gt;
+    gauss_tables_init(gt, threadIdx.x);
+    __syncthreads();
     size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= total) return;
     const uint32_t B = 1u << c.LOGB, half = B >> 1;
@@ -507,26 +507,26 @@ enc_outer_inverse_add_kernel(const __grid_constant__ CtxDev c, const int64_t *m,
     const uint32_t col = (uint32_t)(g % half) * 2;
     const size_t tl = g / half;
     const uint32_t t = t0 + (uint32_t)tl;
-    int e1[rows][2];
-    int64_t me0[rows][2];                              // m + e0
+#pragma unroll 1
+    for (uint32_t comp = 0; comp < 2; comp++) {
+        int64_t add[rows][2];                          // e0 + m, or e1
 #pragma unroll
-    for (uint32_t a = 0; a < rows; a++) {
-        const uint32_t i = a * B + col;               // one Philox block per pair of coefficients
-        const u32x4 w0 = stream_block(seed, i >> 1, t, client, TAG_ENC_E0);
-        const u32x4 w1 = stream_block(seed, i >> 1, t, client, TAG_ENC_E1);
-        const longlong2 mm = *reinterpret_cast<const longlong2 *>(m + tl * c.N + i);
-        me0[a][0] = mm.x + gauss_from_u64((uint64_t)w0.x | ((uint64_t)w0.y << 32));
-        me0[a][1] = mm.y + gauss_from_u64((uint64_t)w0.z | ((uint64_t)w0.w << 32));
-        e1[a][0] = gauss_from_u64((uint64_t)w1.x | ((uint64_t)w1.y << 32));
-        e1[a][1] = gauss_from_u64((uint64_t)w1.z | ((uint64_t)w1.w << 32));
-    }
+        for (uint32_t a = 0; a < rows; a++) {
+            const uint32_t i = a * B + col;           // one Philox block per pair of coefficients
+            const u32x4 w = stream_block(seed, i >> 1, t, client, comp == 0 ? TAG_ENC_E0 : TAG_ENC_E1);
+            add[a][0] = gauss_from_u64(gt, (uint64_t)w.x | ((uint64_t)w.y << 32));
+            add[a][1] = gauss_from_u64(gt, (uint64_t)w.z | ((uint64_t)w.w << 32));
+            if (comp == 0) {
+                const longlong2 mm = *reinterpret_cast<const longlong2 *>(m + tl * c.N + i);
+                add[a][0] += mm.x;
+                add[a][1] += mm.y;
+            }
+        }
 #pragma unroll 1
-    for (uint32_t j = 0; j < c.L; j++) {
-        const LimbDev &lb = c.limb[j];
-#pragma unroll 1
-        for (uint32_t comp = 0; comp < 2; comp++) {
+        for (uint32_t j = 0; j < c.L; j++) {
+            const LimbDev &lb = c.limb[j];
             uint64_t *p = ct + ((tl * 2 + comp) * c.L + j) * c.N + col;
-            FEDHE_FOR_ARITH(lb, (enc_outer_inverse_add_limb<M_, A>(lb, p, B, comp == 0, me0, e1)));
+            FEDHE_FOR_ARITH(lb, (enc_outer_inverse_add_limb<M_, A>(lb, p, B, add)));
         }
     }
 }
