@@ -167,6 +167,7 @@ int he_ctx_destroy(he_ctx *ctx) {
         if (ctx->ev_ready[i]) cudaEventDestroy(ctx->ev_ready[i]);
         if (ctx->ev_free[i]) cudaEventDestroy(ctx->ev_free[i]);
     }
+    if (ctx->ev_chunk) cudaEventDestroy(ctx->ev_chunk);
     ctx->magic = 0;
     delete ctx;
     return HE_OK;
@@ -711,6 +712,10 @@ int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const f
     // ciphertexts of a chunk within about 8 GiB; a chunk is a whole number of
     // waves of one thread block per SM
     size_t Tc = ((size_t)8 << 30) / (C * ctw * sizeof(uint64_t));
+    // at least four chunks when there is enough work, so that the download of
+    // one chunk's result hides behind the next chunk's arithmetic
+    const size_t quarter = (T + 3) / 4;
+    if (Tc > quarter && quarter >= (size_t)ctx->sm_count) Tc = quarter + ctx->sm_count - 1;
     if (Tc > (size_t)ctx->sm_count) Tc -= Tc % ctx->sm_count;
     if (Tc < 1) Tc = 1;
     if (Tc > T) Tc = T;
@@ -744,6 +749,7 @@ int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const f
             CU(cudaEventCreateWithFlags(&ctx->ev_ready[i], cudaEventDisableTiming));
             CU(cudaEventCreateWithFlags(&ctx->ev_free[i], cudaEventDisableTiming));
         }
+        CU(cudaEventCreateWithFlags(&ctx->ev_chunk, cudaEventDisableTiming));
     }
     for (int i = 0; i < C; i++)
         if (!xs_host[i]) return HE_ERR_INVALID_ARG;
@@ -776,6 +782,20 @@ int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const f
         if (rc != HE_OK) return rc;
         rc = he_decrypt(ctx, keys, agg, tc, z + t0 * n, stream);
         if (rc != HE_OK) return rc;
+        if (!mask) {
+            // full encryption: the decoded slots are the result, in order; send this
+            // chunk's part home on the copy stream while the next chunk is computed
+            const size_t first = t0 * n, count = P - first < tc * n ? P - first : tc * n;
+            CU(cudaEventRecord(ctx->ev_chunk, st));
+            CU(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_chunk, 0));
+            CU(cudaMemcpyAsync(w_glob_host + first, z + first, count * sizeof(double), cudaMemcpyDeviceToHost,
+                               ctx->copy_stream));
+        }
+    }
+    if (!mask) {
+        CU(cudaStreamSynchronize(ctx->copy_stream));
+        CU(cudaStreamSynchronize(st));
+        return HE_OK;
     }
     if (restlen) {
         std::vector<const float *> rptr(rest.begin(), rest.end());

@@ -83,6 +83,7 @@ struct he_ctx {
     int sm_count = 0;
     cudaStream_t copy_stream = nullptr;   // uploads of he_round_host, overlapped with compute
     cudaEvent_t ev_ready[2] = {nullptr, nullptr}, ev_free[2] = {nullptr, nullptr};
+    cudaEvent_t ev_chunk = nullptr;       // a chunk's result is ready for download
 };
 
 struct he_keys {

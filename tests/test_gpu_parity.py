@@ -327,6 +327,22 @@ def test_tiny_config_whole_round(he):
     assert np.array_equal(host.numpy(), out)
 
 
+def test_host_round_in_several_chunks(he):
+    """The host-buffer entry point splits a large round into chunks of ciphertext indices (here
+    296 + 296 + 8, ragged tail in the last ciphertext) and downloads each chunk's slots while the
+    next is computed: same result as the device calls on the whole range, bit for bit, and FedAvg."""
+    w = si.scaled(si.TINY, 600 * 4096 - 37, clients=2, name="tiny-600cts")
+    g = he.he_ctx_create(w.N, list(w.primes), w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    xs, alpha = si.client_updates(w), si.client_weights(w)
+    out = run_round_gpu(he, g, keys, None, xs, alpha, w)
+    host = torch.full((w.P,), np.nan, dtype=torch.float64).pin_memory()
+    he.he_round_host(g, keys, None, [torch.from_numpy(x).pin_memory() for x in xs], alpha, w.enc_seed, host)
+    assert np.array_equal(host.numpy(), out)
+    want = sum(a * x.astype(np.float64) for a, x in zip(alpha, xs))
+    assert np.abs(out - want).max() <= FEDAVG_TOL
+
+
 def test_selective_round_with_mask(he):
     """Config 3 shape at reduced size: top-10 % encrypted, the rest averaged in plaintext."""
     w = si.scaled(si.RESNET50_TOP10, 300_000, clients=4)
