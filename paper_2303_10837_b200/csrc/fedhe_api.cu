@@ -708,17 +708,22 @@ int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const f
     const CtxDev &d = ctx->dev;
     const size_t n = d.N / 2, T = he_num_ct(ctx, k), padded = T * n, restlen = P - k;
     const size_t ctw = 2 * (size_t)d.L * d.N, aggw = 2 * (size_t)(d.L - 1) * d.N;
-    // ciphertext indices are processed in chunks that keep all clients'
+    // Ciphertext indices are processed in chunks that keep all clients'
     // ciphertexts of a chunk within about 8 GiB; a chunk is a whole number of
-    // waves of one thread block per SM
-    size_t Tc = ((size_t)8 << 30) / (C * ctw * sizeof(uint64_t));
-    // at least four chunks when there is enough work, so that the download of
-    // one chunk's result hides behind the next chunk's arithmetic
-    const size_t quarter = (T + 3) / 4;
-    if (Tc > quarter && quarter >= (size_t)ctx->sm_count) Tc = quarter + ctx->sm_count - 1;
-    if (Tc > (size_t)ctx->sm_count) Tc -= Tc % ctx->sm_count;
-    if (Tc < 1) Tc = 1;
+    // waves of one thread block per SM.  When there is enough work the first
+    // chunk takes half of it, so that encrypting a client's share of it
+    // outlasts the upload of the next client's update, and the rest goes in two
+    // chunks, so that the download of a chunk's result hides behind the next.
+    const size_t sm = (size_t)ctx->sm_count;
+    auto whole_waves = [&](size_t want, size_t cap) {
+        size_t v = want < cap ? want : cap;
+        if (v > sm) v -= v % sm;
+        return v < 1 ? (size_t)1 : v;
+    };
+    const size_t cap = ((size_t)8 << 30) / (C * ctw * sizeof(uint64_t));
+    size_t Tc = (T < 4 * sm && T <= cap) ? T : whole_waves((T + 1) / 2 + sm - 1, cap);   // first chunk, the largest
     if (Tc > T) Tc = T;
+    const size_t Tc_rest = T > Tc ? whole_waves((T - Tc + 1) / 2 + sm - 1, Tc) : Tc;
     auto align = [](size_t b) { return (b + 255) & ~(size_t)255; };
     const size_t b_x = align(P * sizeof(float)), b_sel = align(padded * sizeof(float)),
                  b_rest = align(restlen * sizeof(float)), b_cts = align(C * Tc * ctw * sizeof(uint64_t)),
@@ -758,24 +763,40 @@ int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const f
     CU(cudaEventRecord(ctx->ev_free[0], st));       // earlier work on `st` may still use the buffers
     CU(cudaEventRecord(ctx->ev_free[1], st));
     std::vector<const uint64_t *> cptr(C);
-    for (size_t t0 = 0; t0 < T || t0 == 0; t0 += Tc) {
-        const size_t tc = T - t0 < Tc ? T - t0 : Tc;
+    for (size_t t0 = 0, step = Tc; t0 < T || t0 == 0; t0 += step, step = Tc_rest) {
+        const size_t tc = T - t0 < step ? T - t0 : step;
         for (int i = 0; i < C; i++) {
+            // With full encryption the first client's update is uploaded in two pieces so
+            // that its first chunk can be encrypted while the rest is still on its way
+            // (every later upload hides behind the arithmetic of the client before).
+            size_t head = P;
+            const int b = i & 1;
             if (t0 == 0) {
-                const int b = i & 1;
+                if (!mask && i == 0 && Tc < T) head = Tc * n;
                 CU(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_free[b], 0));
-                CU(cudaMemcpyAsync(x[b], xs_host[i], P * sizeof(float), cudaMemcpyHostToDevice, ctx->copy_stream));
+                CU(cudaMemcpyAsync(x[b], xs_host[i], head * sizeof(float), cudaMemcpyHostToDevice, ctx->copy_stream));
                 CU(cudaEventRecord(ctx->ev_ready[b], ctx->copy_stream));
+                if (head < P) {
+                    CU(cudaMemcpyAsync(x[b] + head, xs_host[i] + head, (P - head) * sizeof(float),
+                                       cudaMemcpyHostToDevice, ctx->copy_stream));
+                    CU(cudaEventRecord(ctx->ev_chunk, ctx->copy_stream));
+                }
                 CU(cudaStreamWaitEvent(st, ctx->ev_ready[b], 0));
-                rc = he_pack(ctx, mask, x[b], P, sel[i], restlen ? rest[i] : nullptr, stream);
+                rc = he_pack(ctx, mask, x[b], head, sel[i], restlen ? rest[i] : nullptr, stream);
                 if (rc != HE_OK) return rc;
-                CU(cudaEventRecord(ctx->ev_free[b], st));
+                if (head == P) CU(cudaEventRecord(ctx->ev_free[b], st));
             }
             if (tc == 0) continue;
             uint64_t *ci = cts + (size_t)i * Tc * ctw;
             rc = he_encrypt_range(ctx, keys, sel[i] + t0 * n, t0, tc, enc_seed, (uint32_t)i, ci, stream);
             if (rc != HE_OK) return rc;
             cptr[i] = ci;
+            if (t0 == 0 && head < P) {          // the rest of the first client's slots
+                CU(cudaStreamWaitEvent(st, ctx->ev_chunk, 0));
+                rc = he_pack(ctx, nullptr, x[b] + head, P - head, sel[i] + head, nullptr, stream);
+                if (rc != HE_OK) return rc;
+                CU(cudaEventRecord(ctx->ev_free[b], st));
+            }
         }
         if (tc == 0) break;
         rc = he_weighted_aggregate(ctx, cptr.data(), alpha_host, C, tc, agg, stream);
