@@ -108,8 +108,8 @@ decrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const ui
             sm, tid, fa, [&](uint32_t i) { return c1[i]; },
             [&](uint32_t p, uint64_t a, uint64_t b) {
                 const tw_t s0 = load_tw(k.s_hat + p), s1 = load_tw(k.s_hat + p + 1);
-                sm[swz(p)] = shoup_lazy(a, s0.w, s0.wp, q);
-                sm[swz(p + 1)] = shoup_lazy(b, s1.w, s1.wp, q);
+                sm[wswz(p)] = shoup_lazy(a, s0.w, s0.wp, q);
+                sm[wswz(p + 1)] = shoup_lazy(b, s1.w, s1.wp, q);
             });
     }
     int64_t *d = reinterpret_cast<int64_t *>(sm);
@@ -124,12 +124,12 @@ decrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const ui
                     return u64x2{csub(a.x + shoup_lazy(b.x, s0.w, s0.wp, q), q2),
                                  csub(a.y + shoup_lazy(b.y, s1.w, s1.wp, q), q2)};
                 } else {
-                    return u64x2{sm[swz(p)], sm[swz(p + 1)]};
+                    return u64x2{sm[wswz(p)], sm[wswz(p + 1)]};
                 }
             },
             [&](uint32_t i, uint64_t v) {
                 const uint64_t r = NTT_IN ? csub(v, q) : addmod(csub(v, q), c0[i], q);
-                d[swz(i)] = r > q / 2 ? -(int64_t)(q - r) : (int64_t)r;
+                d[wswz(i)] = r > q / 2 ? -(int64_t)(q - r) : (int64_t)r;
             });
     }
     __syncthreads();
@@ -139,7 +139,7 @@ decrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const ui
 #pragma unroll
     for (int r = 0; r < LF::E; r++) {
         const uint32_t kk = bitrev(LF::template idx<LF::NPH - 1>(tid, r), LF::LOGB);
-        x[r] = cpx{(double)d[swz(kk)] * inv_delta, (double)d[swz(kk + n)] * inv_delta};
+        x[r] = cpx{(double)d[wswz(kk)] * inv_delta, (double)d[wswz(kk + n)] * inv_delta};
     }
     __syncthreads();                      // all inputs are in registers: the buffer becomes the exchange buffer
     block_dit<LF>(x, reinterpret_cast<cpx *>(sm), tid, c.ftw);
@@ -162,11 +162,11 @@ cudaError_t launch_decrypt_fused(const CtxDev &c, const KeysDev &k, const uint64
                                  size_t T, bool ntt_in, double *z, cudaStream_t s) {
     if (T == 0) return cudaSuccess;
     if (c.logN == 13) {
-        if (ntt_in) return launch_decrypt_fused_t<Lay<13, 3>, 2, Lay<12, 3>, true>(c, k, ct, level, T, z, s);
-        return launch_decrypt_fused_t<Lay<13, 3>, 2, Lay<12, 3>, false>(c, k, ct, level, T, z, s);
+        if (ntt_in) return launch_decrypt_fused_t<WLay<13>, 2, Lay<12, 3>, true>(c, k, ct, level, T, z, s);
+        return launch_decrypt_fused_t<WLay<13>, 2, Lay<12, 3>, false>(c, k, ct, level, T, z, s);
     }
-    if (ntt_in) return launch_decrypt_fused_t<Lay<14, 3>, 2, Lay<13, 3>, true>(c, k, ct, level, T, z, s);
-    return launch_decrypt_fused_t<Lay<14, 3>, 2, Lay<13, 3>, false>(c, k, ct, level, T, z, s);
+    if (ntt_in) return launch_decrypt_fused_t<WLay<14>, 2, Lay<13, 3>, true>(c, k, ct, level, T, z, s);
+    return launch_decrypt_fused_t<WLay<14>, 2, Lay<13, 3>, false>(c, k, ct, level, T, z, s);
 }
 
 // ===========================================================================

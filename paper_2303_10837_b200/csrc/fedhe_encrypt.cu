@@ -7,6 +7,13 @@ namespace fedhe {
 // encryption:  c0 = pk0 u + e0 + m,  c1 = pk1 u + e1   (mod every q_j)
 // ===========================================================================
 
+// Index swizzle of the one-byte sample arrays in shared memory (banks of four
+// bytes, i.e. index bits 2..6): the first phase of a transform reads them with
+// lanes that differ in index bits 0, 1 and three bits from 7 upwards, the
+// epilogues with consecutive lanes; folding bits 7..11 into bits 2..6 keeps
+// both patterns free of bank conflicts and leaves aligned groups of four intact.
+__device__ __forceinline__ uint32_t bswz(uint32_t i) { return i ^ (((i >> 7) & 31u) << 2); }
+
 // One (ciphertext, limb) unit of the fused path in the limb's arithmetic.
 // u^ pk1^ is parked, in the arithmetic's own form, in the c1 slot it will
 // finally occupy while u^ pk0^ stays in shared memory; then two passes over
@@ -33,9 +40,9 @@ __device__ __forceinline__ void encrypt_unit(const LimbDev &lb, const tw_t *p0, 
             smem_ntt_forward<L, V>(
                 sm, tid, fa,
                 [&](uint32_t i) {
-                    if (h == 0) return ar.small(su[i]);
-                    if (h == 2) return ar.small(se[i]);
-                    return ar.from_residue(signed_residue(mt[i] + (int64_t)se[i], q, lb.mu));
+                    if (h == 0) return ar.small(su[bswz(i)]);
+                    if (h == 2) return ar.small(se[bswz(i)]);
+                    return ar.from_residue(signed_residue(mt[i] + (int64_t)se[bswz(i)], q, lb.mu));
                 },
                 [&](uint32_t p, val a, val b) {
                     if (h == 0) {
@@ -60,7 +67,7 @@ __device__ __forceinline__ void encrypt_unit(const LimbDev &lb, const tw_t *p0, 
         const auto fa = LimbOf<M>::args(lb, true, 0, 0);
         const M &ar = fa.m;
         smem_ntt_forward<L, V>(
-            sm, tid, fa, [&](uint32_t i) { return ar.small(su[i]); },
+            sm, tid, fa, [&](uint32_t i) { return ar.small(su[bswz(i)]); },
             [&](uint32_t p, val a, val b) {
                 const auto a0 = M::load_key(p1 + p), a1 = M::load_key(p1 + p + 1);
                 u64x2 v;
@@ -68,8 +75,8 @@ __device__ __forceinline__ void encrypt_unit(const LimbDev &lb, const tw_t *p0, 
                 v.y = M::bits(ar.mul_key(b, a1));
                 *reinterpret_cast<u64x2 *>(c1 + p) = v;
                 const auto b0 = M::load_key(p0 + p), b1 = M::load_key(p0 + p + 1);
-                sm[swz(p)] = M::bits(ar.mul_key(a, b0));
-                sm[swz(p + 1)] = M::bits(ar.mul_key(b, b1));
+                sm[wswz(p)] = M::bits(ar.mul_key(a, b0));
+                sm[wswz(p + 1)] = M::bits(ar.mul_key(b, b1));
             });
     }
 #pragma unroll 1
@@ -81,14 +88,14 @@ __device__ __forceinline__ void encrypt_unit(const LimbDev &lb, const tw_t *p0, 
         smem_ntt_inverse<L, V, true>(
             sm, tid, ia, LimbOf<M>::ninv(lb), LimbOf<M>::wn(lb),
             [&](uint32_t p) {
-                if (h == 0) return pair_of<val>{M::from_bits(sm[swz(p)]), M::from_bits(sm[swz(p + 1)])};
+                if (h == 0) return pair_of<val>{M::from_bits(sm[wswz(p)]), M::from_bits(sm[wswz(p + 1)])};
                 const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + p);
                 return pair_of<val>{M::from_bits(t.x), M::from_bits(t.y)};
             },
             [&](uint32_t i, val v) {
                 // e1 is a small value; e0 + m needs a full reduction
-                const uint64_t add = h == 0 ? signed_residue(mt[i] + (int64_t)se[i], q, lb.mu)
-                                            : small_residue(se[i], q);
+                const uint64_t add = h == 0 ? signed_residue(mt[i] + (int64_t)se[bswz(i)], q, lb.mu)
+                                            : small_residue(se[bswz(i)], q);
                 cc[i] = ar.canon_add(v, add);
             });
         __syncthreads();   // phase-0 readers are done before the next transform writes
@@ -132,7 +139,7 @@ encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const in
                 u32x4 w = stream_block(seed, b, t, client, TAG_ENC_U);
                 char4 v = make_char4((signed char)ternary_from_word(w.x), (signed char)ternary_from_word(w.y),
                                      (signed char)ternary_from_word(w.z), (signed char)ternary_from_word(w.w));
-                reinterpret_cast<char4 *>(su)[b] = v;
+                *reinterpret_cast<char4 *>(su + bswz(4 * b)) = v;
             }
             for (uint32_t b = tid; b < B / 2; b += RT) {
                 u32x4 w0 = stream_block(seed, b, t, client, TAG_ENC_E0);
@@ -141,8 +148,8 @@ encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const in
                                      (signed char)gauss_from_u64(gt, (uint64_t)w0.z | ((uint64_t)w0.w << 32)));
                 char2 e = make_char2((signed char)gauss_from_u64(gt, (uint64_t)w1.x | ((uint64_t)w1.y << 32)),
                                      (signed char)gauss_from_u64(gt, (uint64_t)w1.z | ((uint64_t)w1.w << 32)));
-                reinterpret_cast<char2 *>(se0)[b] = a;
-                reinterpret_cast<char2 *>(se1)[b] = e;
+                *reinterpret_cast<char2 *>(se0 + bswz(2 * b)) = a;
+                *reinterpret_cast<char2 *>(se1 + bswz(2 * b)) = e;
             }
             __syncthreads();
         }
@@ -174,11 +181,11 @@ __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0
         const auto w0 = M::load(fa.tw + 1);                // twiddle of the stage that pairs the halves
         auto src = [&](uint32_t i) {
             // u is ternary: the twiddle product is 0, w or -w
-            const int b = su[i + H];
+            const int b = su[bswz(i + H)];
             if constexpr (std::is_same<M, ModF64>::value) {
-                return f64_fma(grp == 0 ? (double)b : (double)-b, w0, (double)su[i]);
+                return f64_fma(grp == 0 ? (double)b : (double)-b, w0, (double)su[bswz(i)]);
             } else {
-                const uint64_t u = small_residue(su[i], q);
+                const uint64_t u = small_residue(su[bswz(i)], q);
                 const uint64_t v = b == 0 ? 0 : (b > 0 ? w0.w : q - w0.w);
                 return grp == 0 ? u + v : u - v + ar.q2;
             }
@@ -193,8 +200,8 @@ __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0
                 uint64_t *cc = h == 2 ? c1 : c0;
                 const int8_t *se = se0 + (h == 2 ? B : 0);
                 auto value = [&](uint32_t i) {
-                    if (h == 2) return ar.small(se[i]);
-                    return ar.from_residue(signed_residue(mt[i] + (int64_t)se[i], q, lb.mu));
+                    if (h == 2) return ar.small(se[bswz(i)]);
+                    return ar.from_residue(signed_residue(mt[i] + (int64_t)se[bswz(i)], q, lb.mu));
                 };
                 smem_ntt_forward<L, V>(
                     smg, gt, fa,
@@ -236,8 +243,8 @@ __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0
             v.y = M::bits(ar.mul_key(b, a1));
             *reinterpret_cast<u64x2 *>(c1 + p) = v;      // parked until the second pass
             const auto b0 = M::load_key(p0 + p), b1 = M::load_key(p0 + p + 1);
-            smg[swz(p)] = M::bits(ar.mul_key(a, b0));
-            smg[swz(p + 1)] = M::bits(ar.mul_key(b, b1));
+            smg[wswz(p)] = M::bits(ar.mul_key(a, b0));
+            smg[wswz(p + 1)] = M::bits(ar.mul_key(b, b1));
         };
         smem_ntt_forward<L, V>(smg, gt, fa, src, dst, gsync);
     }
@@ -249,24 +256,24 @@ __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0
         const M &ar = ia.m;
         const auto ninv = LimbOf<M>::ninv(lb), wn = LimbOf<M>::wn(lb);
         auto isrc = [&](uint32_t p) {
-            if (h == 0) return pair_of<val>{M::from_bits(smg[swz(p)]), M::from_bits(smg[swz(p + 1)])};
+            if (h == 0) return pair_of<val>{M::from_bits(smg[wswz(p)]), M::from_bits(smg[wswz(p + 1)])};
             const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + grp * H + p);
             return pair_of<val>{M::from_bits(t.x), M::from_bits(t.y)};
         };
-        auto idst = [&](uint32_t i, val v) { smg[swz(i)] = M::bits(v); };
+        auto idst = [&](uint32_t i, val v) { smg[wswz(i)] = M::bits(v); };
         smem_ntt_inverse<L, V, false>(smg, gt, ia, ninv, wn, isrc, idst, gsync);
         __syncthreads();
         // last stage across the halves with 1/N folded in, then the error / message terms
         for (uint32_t e = tid; e < H; e += RT) {
-            val lo = M::from_bits(sm[swz(e)]), hi = M::from_bits(sm[H + swz(e)]);
+            val lo = M::from_bits(sm[wswz(e)]), hi = M::from_bits(sm[H + wswz(e)]);
             ar.inv_scaled(lo, hi, ninv, wn);
             uint64_t add_lo, add_hi;
             if (h == 0) {
-                add_lo = signed_residue(mt[e] + (int64_t)se[e], q, lb.mu);
-                add_hi = signed_residue(mt[e + H] + (int64_t)se[e + H], q, lb.mu);
+                add_lo = signed_residue(mt[e] + (int64_t)se[bswz(e)], q, lb.mu);
+                add_hi = signed_residue(mt[e + H] + (int64_t)se[bswz(e + H)], q, lb.mu);
             } else {
-                add_lo = small_residue(se[e], q);
-                add_hi = small_residue(se[e + H], q);
+                add_lo = small_residue(se[bswz(e)], q);
+                add_hi = small_residue(se[bswz(e + H)], q);
             }
             cc[e] = ar.canon_add(lo, add_lo);
             cc[e + H] = ar.canon_add(hi, add_hi);
@@ -311,7 +318,7 @@ encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const i
                 u32x4 w = stream_block(seed, b, t, client, TAG_ENC_U);
                 char4 v = make_char4((signed char)ternary_from_word(w.x), (signed char)ternary_from_word(w.y),
                                      (signed char)ternary_from_word(w.z), (signed char)ternary_from_word(w.w));
-                reinterpret_cast<char4 *>(su)[b] = v;
+                *reinterpret_cast<char4 *>(su + bswz(4 * b)) = v;
             }
             for (uint32_t b = tid; b < B / 2; b += RT) {
                 u32x4 w0 = stream_block(seed, b, t, client, TAG_ENC_E0);
@@ -320,8 +327,8 @@ encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const i
                                      (signed char)gauss_from_u64(gt_tab, (uint64_t)w0.z | ((uint64_t)w0.w << 32)));
                 char2 e = make_char2((signed char)gauss_from_u64(gt_tab, (uint64_t)w1.x | ((uint64_t)w1.y << 32)),
                                      (signed char)gauss_from_u64(gt_tab, (uint64_t)w1.z | ((uint64_t)w1.w << 32)));
-                reinterpret_cast<char2 *>(se0)[b] = a;
-                reinterpret_cast<char2 *>(se1)[b] = e;
+                *reinterpret_cast<char2 *>(se0 + bswz(2 * b)) = a;
+                *reinterpret_cast<char2 *>(se1 + bswz(2 * b)) = e;
             }
             __syncthreads();
         }
@@ -553,7 +560,7 @@ static cudaError_t launch_encrypt_fused(const CtxDev &c, const KeysDev &k, const
 template <bool ACC>
 static cudaError_t launch_enc_block_forward(const CtxDev &c, const KeysDev &k, const uint64_t *ubuf, size_t T,
                                             uint64_t *ct, cudaStream_t s) {
-    using L = Lay<13, 3>;                                 // long rings are cut into 2^13 blocks
+    using L = WLay<13>;                                 // long rings are cut into 2^13 blocks
     constexpr int V = 2;
     const size_t smem = sizeof(uint64_t) << L::LOGB;
     auto kern = enc_block_forward_kernel<L, V, ACC>;
@@ -568,8 +575,8 @@ cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const int64_t *m, 
     if (T == 0) return cudaSuccess;
     if (c.A == 0) {
         if (c.LOGB == 13)
-            return launch_encrypt_fused<Lay<13, 3>, 2, false, false>(c, k, m, t0, T, seed, client, ct, s);
-        return launch_encrypt_fused<Lay<13, 3>, 2, true, false>(c, k, m, t0, T, seed, client, ct, s);
+            return launch_encrypt_fused<WLay<13>, 2, false, false>(c, k, m, t0, T, seed, client, ct, s);
+        return launch_encrypt_fused<WLay<13>, 2, true, false>(c, k, m, t0, T, seed, client, ct, s);
     }
     cudaError_t e;
     const size_t cols = T * ((size_t)1 << (c.LOGB - 1));      // pairs of columns
@@ -594,8 +601,8 @@ cudaError_t launch_encrypt_ntt(const CtxDev &c, const KeysDev &k, const int64_t 
     if (T == 0) return cudaSuccess;
     if (c.A == 0) {
         if (c.LOGB == 13)
-            return launch_encrypt_fused<Lay<13, 3>, 2, false, true>(c, k, m, t0, T, seed, client, ct, s);
-        return launch_encrypt_fused<Lay<13, 3>, 2, true, true>(c, k, m, t0, T, seed, client, ct, s);
+            return launch_encrypt_fused<WLay<13>, 2, false, true>(c, k, m, t0, T, seed, client, ct, s);
+        return launch_encrypt_fused<WLay<13>, 2, true, true>(c, k, m, t0, T, seed, client, ct, s);
     }
     cudaError_t e;
     const size_t LN = (size_t)c.L * c.N;

@@ -1,7 +1,8 @@
 // Register-tiled negacyclic NTT of one block of B = 2^LOGB residues held by
-// one thread block in shared memory: a thread takes E = 2^LE residues into
-// registers, does LE butterfly stages on them and puts them back; between
-// such phases the index bits are re-dealt among the threads.
+// one thread block in shared memory: a thread takes E = 8 residues into
+// registers, does up to three butterfly stages on them and puts them back;
+// between such phases the elements change hands, inside a warp where the
+// layout allows it and across the block once per transform.
 //
 // Index conventions (forward transform, natural order in, bit-reversed out):
 // stage s (0-based) of a length-N transform pairs the elements whose indices
@@ -11,11 +12,6 @@
 // longer transform (N = 2^A B) whose first A stages were done elsewhere; then
 // the local stage s' is the global stage A + s' and the block index enters
 // the twiddle index.
-//
-// Phase p < NPH-1 keeps in registers the elements that differ in index bits
-// [lo, lo+LE), lo = LOGB - (p+1) LE; the last phase holds the remaining R low
-// bits plus the LE-R top bits (so that a thread owns runs of 2^R consecutive
-// elements and a warp covers whole 128-byte lines).
 #pragma once
 
 #include "fedhe_device.cuh"
@@ -42,19 +38,19 @@ struct alignas(16) u64x2 { uint64_t x, y; };   // two neighbouring residues
 template <class V>
 struct pair_of { V x, y; };                      // two neighbouring values of an arithmetic
 
-// Shared-memory index swizzle.  A 64-bit access of a warp is served half-warp
-// by half-warp from 16 banks of 8 bytes (the low four index bits), and the 16
-// lanes of a half-warp differ in four index bits that depend on the phase:
-// bits {0,1,2,3}, {0,4,5,6}, {1,2,3,4}, {0,1,5,6} or {2,3,4,5} for the layouts
-// in use.  XOR-ing t ^ (t << 1), t = index bits 4..6, into the low nibble makes
-// the bank a bijection of each of these sets (as linear maps over GF(2): the
-// columns 0011, 0110, 1100 for bits 4, 5, 6 next to the identity), so no
-// phase has bank conflicts; the map permutes every aligned group of 16 words.
+// Index swizzle and thread layout of the complex slot transform (its kernels
+// keep their values in registers across phases and exchange them through
+// shared memory between phases).  XOR-ing t ^ (t << 1), t = index bits 4..6,
+// into the low nibble spreads the accesses of every phase layout over the
+// banks; the map permutes every aligned group of 16 words.
 HD uint32_t swz(uint32_t i) {
     const uint32_t t = (i >> 4) & 7u;
     return i ^ t ^ ((t << 1) & 15u);
 }
 
+// Phase p < NPH-1 keeps in registers the elements that differ in index bits
+// [lo, lo+LE), lo = LOGB - (p+1) LE; the last phase holds the remaining R low
+// bits plus the LE-R top bits.
 template <int LOGB_, int LE_>
 struct Lay {
     static constexpr int LOGB = LOGB_, LE = LE_;
@@ -225,6 +221,99 @@ struct ModF64 {
     HD val mul_key(val v, key k) const { return mul(v, k); }
 };
 
+// ---- warp-local layout --------------------------------------------------------
+//
+// The 3 * 4 + R stages of a block run in five phases of (3, 3, 3, 3, R) stages,
+// R = LOGB - 12.  In every phase a virtual thread holds E = 8 elements that
+// differ in three index bits (the register bits: the bits the phase's
+// butterflies pair, plus 3 - R idle bits in the last phase), the 32 lanes of
+// its virtual warp differ in five more (the lane bits), and the remaining
+// LOGB - 8 bits number the virtual warp.  Register and lane bits are chosen so
+// that a virtual warp works on one and the same set of 256 elements
+// throughout phases 0-1 and on another throughout phases 2-4: inside such a
+// super-phase the elements change hands between the lanes of one warp only, a
+// warp-level barrier orders the exchange, and the warps of a block drift apart
+// (one warp's shared-memory traffic overlaps another's arithmetic).  Only the
+// step from phase 1 to phase 2 needs a barrier over the whole block.
+//
+// Register bits:  phase P < 4: LOGB - 3 (P + 1) + {0, 1, 2};
+//                 phase 4: {0 .. R-1} (paired) and the top 3 - R bits below bit 8.
+// Lane bits (lane bit 0 first) and virtual-warp bits:
+//   LOGB 14: {0,1,8,9,10} {0,1,11,12,13} | {0,1,2,3,4} {0,1,5,6,7} {2,3,4,5,6};  warp: 2..7 | 8..13
+//   LOGB 13: {0,1,8,9,7}  {0,1,11,12,10} | {0,1,2,3,7} {0,4,5,6,7} {1,2,3,4,5};  warp: 2..6 | 8..12
+// In the last phase a thread owns runs of 2^R neighbouring elements and the
+// lanes of a warp follow one another, so that a warp reads and writes whole
+// lines of global memory.
+
+// Shared-memory index swizzle for 8-byte words.  A 64-bit access of a warp is
+// served half-warp by half-warp from 16 banks of 8 bytes (the low four index
+// bits); the 16 lanes of a half-warp differ in the index bits named first in
+// the lists above.  The map XORs into the low nibble, as linear maps over
+// GF(2), the columns 0011, 0110, 1100 for index bits 4, 5, 6 and 0100, 1000
+// for bits 8, 9 and again for bits 11, 12, which makes the bank a bijection of
+// each of those sets of four bits; it permutes every aligned group of 16 words.
+HD uint32_t wswz(uint32_t i) {
+    const uint32_t t = (i >> 4) & 7u;
+    return i ^ t ^ ((t << 1) & 15u) ^ ((((i >> 8) ^ (i >> 11)) & 3u) << 2);
+}
+
+template <int LOGB_>
+struct WLay {
+    static_assert(LOGB_ == 13 || LOGB_ == 14, "blocks of 2^13 or 2^14 elements");
+    static constexpr int LOGB = LOGB_, LE = 3, E = 8, NPH = 5;
+    static constexpr int SPLIT = 2;                       // phases [0, SPLIT) and [SPLIT, NPH) are the super-phases
+    static constexpr int NT = 1 << (LOGB - LE);           // virtual threads
+    static constexpr int NW = NT / 32;                    // virtual warps
+    static constexpr int WB = LOGB - 8;                   // index bits that number the virtual warp
+    static constexpr int R = LOGB - 12;                   // stages of the last phase
+
+    static HD constexpr int nst(int P) { return P < NPH - 1 ? LE : R; }
+    static HD constexpr int reg_bit(int P, int k) {
+        if (P < NPH - 1) return LOGB - LE * (P + 1) + k;
+        return k < R ? k : 8 - (LE - R) + (k - R);
+    }
+    static HD constexpr int lane_bit(int P, int k) {
+        constexpr int t14[5][5] = {{0, 1, 8, 9, 10}, {0, 1, 11, 12, 13}, {0, 1, 2, 3, 4}, {0, 1, 5, 6, 7}, {2, 3, 4, 5, 6}};
+        constexpr int t13[5][5] = {{0, 1, 8, 9, 7}, {0, 1, 11, 12, 10}, {0, 1, 2, 3, 7}, {0, 4, 5, 6, 7}, {1, 2, 3, 4, 5}};
+        return LOGB == 14 ? t14[P][k] : t13[P][k];
+    }
+    static HD constexpr int warp_bit(int P, int k) { return (P < SPLIT ? 2 : 8) + k; }
+
+    // bits [K, K + len) of x go to consecutive index bits: one shift and mask per run
+    template <int P, bool LANE, int K>
+    static HD constexpr int run() {
+        constexpr int NB = LANE ? 5 : WB;
+        int len = 1;
+        while (K + len < NB &&
+               (LANE ? lane_bit(P, K + len) : warp_bit(P, K + len)) == (LANE ? lane_bit(P, K) : warp_bit(P, K)) + len)
+            len++;
+        return len;
+    }
+    template <int P, bool LANE, int K = 0>
+    static HD uint32_t deposit(uint32_t x) {
+        constexpr int NB = LANE ? 5 : WB;
+        if constexpr (K >= NB) {
+            return 0u;
+        } else {
+            constexpr int len = run<P, LANE, K>();
+            constexpr int pos = LANE ? lane_bit(P, K) : warp_bit(P, K);
+            return (((x >> K) & ((1u << len) - 1u)) << pos) | deposit<P, LANE, K + len>(x);
+        }
+    }
+    // index of the element in register 0 of a lane of a virtual warp in phase P
+    template <int P>
+    static HD uint32_t base(uint32_t vwarp, uint32_t lane) {
+        return deposit<P, true>(lane) | deposit<P, false>(vwarp);
+    }
+    // what register r adds to that index
+    template <int P>
+    static HD constexpr uint32_t reg(int r) {
+        uint32_t i = 0;
+        for (int k = 0; k < LE; k++) i |= (uint32_t)((r >> k) & 1) << reg_bit(P, k);
+        return i;
+    }
+};
+
 // ---- phases ----------------------------------------------------------------
 
 template <class M>
@@ -237,63 +326,67 @@ struct NttArgsT {
 using NttArgs = NttArgsT<ModInt>;
 using NttArgsF = NttArgsT<ModF64>;
 
-// twiddles of local stage s = P LE + I for the registers of one thread:
-// w[g] serves the butterflies whose lower register has r >> (nst - I) == g
+// Local stage s = 3 P + I pairs the elements that differ in index bit
+// LOGB - 1 - s and uses the twiddle with index 2^(A+s) + (blk << s) +
+// (index >> (LOGB - s)).  In the phases before the last, the indices of a
+// thread's registers agree above the register bits, so the 2^I twiddles of
+// stage I are consecutive table entries: w[g] serves the butterflies whose
+// lower register has r >> (3 - I) == g.
 template <class L, int P, int I, class M>
-HD void stage_twiddles(typename M::tab (&w)[1 << I], uint32_t tid, const NttArgsT<M> &a) {
-    constexpr int s = P * L::LE + I;
-    const uint32_t base = (1u << (a.A + s)) + (a.blk << s);
+HD void stage_twiddles(typename M::tab (&w)[1 << I], uint32_t base, const NttArgsT<M> &a) {
     static_assert(P < L::NPH - 1, "in the last phase the registers of a group are far apart in the index");
-    constexpr int lo = L::LOGB - (P + 1) * L::LE;
-    load_run<1 << I>(a.tw + base + ((tid >> lo) << I), w);
+    constexpr int s = P * L::LE + I;
+    constexpr int above = L::reg_bit(P, 0) + L::LE;        // index bits above the register bits
+    load_run<1 << I>(a.tw + (1u << (a.A + s)) + (a.blk << s) + ((base >> above) << I), w);
+}
+
+// twiddle of a butterfly of the last phase whose lower element has index i
+template <class L, int I, class M>
+HD auto last_twiddle(uint32_t i, const NttArgsT<M> &a) {
+    constexpr int s = (L::NPH - 1) * L::LE + I;
+    return M::load(a.tw + (1u << (a.A + s)) + (a.blk << s) + (i >> (L::LOGB - s)));
 }
 
 template <class L, int P, int I, class M>
-HD void fwd_stage(typename M::val (&x)[L::E], uint32_t tid, const NttArgsT<M> &a) {
-    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
+HD void fwd_stage(typename M::val (&x)[L::E], uint32_t base, const NttArgsT<M> &a) {
+    constexpr int nst = L::nst(P);
     constexpr int bit = nst - 1 - I;              // register bit of the pair
     if constexpr (P < L::NPH - 1) {
         typename M::tab w[1 << I];
-        stage_twiddles<L, P, I>(w, tid, a);
+        stage_twiddles<L, P, I>(w, base, a);
 #pragma unroll
         for (int r = 0; r < L::E; r++) {
             if (r & (1 << bit)) continue;
             a.m.fwd(x[r], x[r | (1 << bit)], w[r >> (nst - I)]);
         }
     } else {
-        constexpr int s = P * L::LE + I;
-        const uint32_t base = (1u << (a.A + s)) + (a.blk << s);
 #pragma unroll
         for (int r = 0; r < L::E; r++) {
             if (r & (1 << bit)) continue;
             // registers that agree above the pair bit share one twiddle; the
             // compiler merges the equal loads of an unrolled group
-            const auto w = M::load(a.tw + base + L::template top<P, I>(tid, r));
-            a.m.fwd(x[r], x[r | (1 << bit)], w);
+            a.m.fwd(x[r], x[r | (1 << bit)], last_twiddle<L, I>(base | L::template reg<P>(r), a));
         }
     }
 }
 
 template <class L, int P, int I, class M>
-HD void inv_stage(typename M::val (&x)[L::E], uint32_t tid, const NttArgsT<M> &a) {
-    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
+HD void inv_stage(typename M::val (&x)[L::E], uint32_t base, const NttArgsT<M> &a) {
+    constexpr int nst = L::nst(P);
     constexpr int bit = nst - 1 - I;
     if constexpr (P < L::NPH - 1) {
         typename M::tab w[1 << I];
-        stage_twiddles<L, P, I>(w, tid, a);
+        stage_twiddles<L, P, I>(w, base, a);
 #pragma unroll
         for (int r = 0; r < L::E; r++) {
             if (r & (1 << bit)) continue;
             a.m.inv(x[r], x[r | (1 << bit)], w[r >> (nst - I)]);
         }
     } else {
-        constexpr int s = P * L::LE + I;
-        const uint32_t base = (1u << (a.A + s)) + (a.blk << s);
 #pragma unroll
         for (int r = 0; r < L::E; r++) {
             if (r & (1 << bit)) continue;
-            const auto w = M::load(a.tw + base + L::template top<P, I>(tid, r));
-            a.m.inv(x[r], x[r | (1 << bit)], w);
+            a.m.inv(x[r], x[r | (1 << bit)], last_twiddle<L, I>(base | L::template reg<P>(r), a));
         }
     }
 }
@@ -311,11 +404,10 @@ HD void inv_stage0_scaled(typename M::val (&x)[L::E], const M &m, const T &ninv,
 }
 
 template <class L, int P, int I = 0, class M>
-HD void fwd_phase(typename M::val (&x)[L::E], uint32_t tid, const NttArgsT<M> &a) {
-    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
-    if constexpr (I < nst) {
-        fwd_stage<L, P, I>(x, tid, a);
-        fwd_phase<L, P, I + 1>(x, tid, a);
+HD void fwd_phase(typename M::val (&x)[L::E], uint32_t base, const NttArgsT<M> &a) {
+    if constexpr (I < L::nst(P)) {
+        fwd_stage<L, P, I>(x, base, a);
+        fwd_phase<L, P, I + 1>(x, base, a);
     }
 }
 
@@ -323,37 +415,37 @@ HD void fwd_phase(typename M::val (&x)[L::E], uint32_t tid, const NttArgsT<M> &a
 // phase to the caller); a phase that ends with an ordinary stage settles the
 // sums of that stage (the registers whose pair bit is clear)
 template <class L, int P, int STOP, int I, class M>
-HD void inv_phase_from(typename M::val (&x)[L::E], uint32_t tid, const NttArgsT<M> &a) {
+HD void inv_phase_from(typename M::val (&x)[L::E], uint32_t base, const NttArgsT<M> &a) {
     if constexpr (I >= STOP) {
-        inv_stage<L, P, I>(x, tid, a);
-        inv_phase_from<L, P, STOP, I - 1>(x, tid, a);
+        inv_stage<L, P, I>(x, base, a);
+        inv_phase_from<L, P, STOP, I - 1>(x, base, a);
     } else if constexpr (STOP == 0) {
-        constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
 #pragma unroll
         for (int r = 0; r < L::E; r++)
-            if (!(r & (1 << (nst - 1)))) x[r] = a.m.settle(x[r]);
+            if (!(r & (1 << (L::nst(P) - 1)))) x[r] = a.m.settle(x[r]);
     }
 }
 
 template <class L, int P, int STOP = 0, class M>
-HD void inv_phase(typename M::val (&x)[L::E], uint32_t tid, const NttArgsT<M> &a) {
-    constexpr int nst = (P < L::NPH - 1) ? L::LE : L::R;
-    inv_phase_from<L, P, STOP, nst - 1>(x, tid, a);
+HD void inv_phase(typename M::val (&x)[L::E], uint32_t base, const NttArgsT<M> &a) {
+    inv_phase_from<L, P, STOP, L::nst(P) - 1>(x, base, a);
 }
 
 #if defined(__CUDACC__)
 // ---------------------------------------------------------------------------
 // Whole-block transforms.  The block's residues stay in shared memory
-// (swizzled) and every thread plays V "virtual threads" per phase, each of
-// which loads its E residues, does the phase's butterflies in registers and
-// stores them back to the same places, so that only E residues are live per
-// thread at a time (E = 8 keeps a 1024-thread block within 64 registers with
-// no spills) and no separate exchange buffer is needed.  The first phase takes its input
-// from `src`, the last hands its output to `dst`:
+// (swizzled) and every warp plays V virtual warps per phase; a virtual thread
+// loads its E residues, does the phase's butterflies in registers and stores
+// them back to the same places, so that only E residues are live per thread
+// at a time (E = 8 keeps a 1024-thread block within 64 registers with no
+// spills) and no separate exchange buffer is needed.  The first phase takes
+// its input from `src`, the last hands its output to `dst`:
 //   forward:  src(i) -> residue i;            dst(i, a, b): residues i, i+1
 //   inverse:  src(i) -> residues i, i+1 (members x, y);   dst(i, a): residue i
-// all in the value type of the limb's arithmetic
-// (pairs always start at an even index and are neighbours in memory).
+// all in the value type of the limb's arithmetic (pairs always start at an
+// even index and are neighbours in memory).  The thread that hands element i
+// to `dst` is the one that read it from `src` or from shared memory word
+// wswz(i) in the same phase, so `dst` may overwrite that word.
 // ---------------------------------------------------------------------------
 
 // Barrier over the whole thread block, or over one of its halves / quarters
@@ -369,76 +461,95 @@ struct GroupSync {
     }
 };
 
-template <class L, int V, class M, class Src, class Dst, class Sync = BlockSync, int P = 0>
-__device__ __forceinline__ void smem_ntt_forward(uint64_t *sm, uint32_t tid, const NttArgsT<M> &a, const Src &src,
-                                                 const Dst &dst, const Sync &sync = Sync()) {
-    constexpr int RT = L::NT / V, LAST = L::NPH - 1;
+// phases [P, PEND) of a forward transform, a warp-level barrier between them
+template <class L, int V, int P, int PEND, class M, class Src, class Dst>
+__device__ __forceinline__ void forward_phases(uint64_t *sm, uint32_t warp, uint32_t lane, const NttArgsT<M> &a,
+                                               const Src &src, const Dst &dst) {
+    constexpr int LAST = L::NPH - 1;
 #pragma unroll M::UNROLL_V
     for (int v = 0; v < V; v++) {
-        const uint32_t vt = tid + v * RT;
+        const uint32_t base = L::template base<P>(warp + v * (L::NW / V), lane);
+        const uint32_t sb = wswz(base);
         typename M::val x[L::E];
 #pragma unroll
         for (int r = 0; r < L::E; r++) {
-            const uint32_t i = L::template idx<P>(vt, r);
-            if constexpr (P == 0) x[r] = src(i);
-            else x[r] = M::from_bits(sm[swz(i)]);
+            if constexpr (P == 0) x[r] = src(base | L::template reg<P>(r));
+            else x[r] = M::from_bits(sm[sb ^ wswz(L::template reg<P>(r))]);
         }
-        fwd_phase<L, P>(x, vt, a);
+        fwd_phase<L, P>(x, base, a);
         if constexpr (P == LAST) {
 #pragma unroll
-            for (int r = 0; r < L::E; r += 2) dst(L::template idx<P>(vt, r), x[r], x[r + 1]);
+            for (int r = 0; r < L::E; r += 2) dst(base | L::template reg<P>(r), x[r], x[r + 1]);
         } else {
 #pragma unroll
-            for (int r = 0; r < L::E; r++) sm[swz(L::template idx<P>(vt, r))] = M::bits(x[r]);
+            for (int r = 0; r < L::E; r++) sm[sb ^ wswz(L::template reg<P>(r))] = M::bits(x[r]);
         }
     }
-    if constexpr (P < LAST) {
-        sync();
-        smem_ntt_forward<L, V, M, Src, Dst, Sync, P + 1>(sm, tid, a, src, dst, sync);
+    if constexpr (P + 1 < PEND) {
+        __syncwarp();
+        forward_phases<L, V, P + 1, PEND>(sm, warp, lane, a, src, dst);
     }
 }
 
-template <class L, int V, bool SCALED, class M, class T, class Src, class Dst, class Sync = BlockSync,
-          int P = L::NPH - 1>
-__device__ __forceinline__ void smem_ntt_inverse(uint64_t *sm, uint32_t tid, const NttArgsT<M> &a, const T &ninv,
-                                                 const T &wn, const Src &src, const Dst &dst,
-                                                 const Sync &sync = Sync()) {
-    constexpr int RT = L::NT / V, LAST = L::NPH - 1;
+template <class L, int V, class M, class Src, class Dst, class Sync = BlockSync>
+__device__ __forceinline__ void smem_ntt_forward(uint64_t *sm, uint32_t tid, const NttArgsT<M> &a, const Src &src,
+                                                 const Dst &dst, const Sync &sync = Sync()) {
+    const uint32_t warp = tid >> 5, lane = tid & 31u;
+    forward_phases<L, V, 0, L::SPLIT>(sm, warp, lane, a, src, dst);
+    sync();
+    forward_phases<L, V, L::SPLIT, L::NPH>(sm, warp, lane, a, src, dst);
+}
+
+// phases P down to PEND of an inverse transform
+template <class L, int V, bool SCALED, int P, int PEND, class M, class T, class Src, class Dst>
+__device__ __forceinline__ void inverse_phases(uint64_t *sm, uint32_t warp, uint32_t lane, const NttArgsT<M> &a,
+                                               const T &ninv, const T &wn, const Src &src, const Dst &dst) {
+    constexpr int LAST = L::NPH - 1;
 #pragma unroll M::UNROLL_V
     for (int v = 0; v < V; v++) {
-        const uint32_t vt = tid + v * RT;
+        const uint32_t base = L::template base<P>(warp + v * (L::NW / V), lane);
+        const uint32_t sb = wswz(base);
         typename M::val x[L::E];
         if constexpr (P == LAST) {
 #pragma unroll
             for (int r = 0; r < L::E; r += 2) {
-                const auto t = src(L::template idx<P>(vt, r));
+                const auto t = src(base | L::template reg<P>(r));
                 x[r] = t.x;
                 x[r + 1] = t.y;
             }
         } else {
 #pragma unroll
-            for (int r = 0; r < L::E; r++) x[r] = M::from_bits(sm[swz(L::template idx<P>(vt, r))]);
+            for (int r = 0; r < L::E; r++) x[r] = M::from_bits(sm[sb ^ wswz(L::template reg<P>(r))]);
         }
         if constexpr (P == 0 && SCALED) {
-            inv_phase<L, 0, 1>(x, vt, a);
+            inv_phase<L, 0, 1>(x, base, a);
             inv_stage0_scaled<L>(x, a.m, ninv, wn);
         } else {
-            inv_phase<L, P, 0>(x, vt, a);
+            inv_phase<L, P, 0>(x, base, a);
         }
         if constexpr (P == 0) {
 #pragma unroll
-            for (int r = 0; r < L::E; r++) dst(L::template idx<0>(vt, r), x[r]);
+            for (int r = 0; r < L::E; r++) dst(base | L::template reg<P>(r), x[r]);
         } else {
 #pragma unroll
-            for (int r = 0; r < L::E; r++) sm[swz(L::template idx<P>(vt, r))] = M::bits(x[r]);
+            for (int r = 0; r < L::E; r++) sm[sb ^ wswz(L::template reg<P>(r))] = M::bits(x[r]);
         }
     }
-    if constexpr (P > 0) {
-        sync();
-        smem_ntt_inverse<L, V, SCALED, M, T, Src, Dst, Sync, P - 1>(sm, tid, a, ninv, wn, src, dst, sync);
+    if constexpr (P > PEND) {
+        __syncwarp();
+        inverse_phases<L, V, SCALED, P - 1, PEND>(sm, warp, lane, a, ninv, wn, src, dst);
     }
 }
-#endif
 
+template <class L, int V, bool SCALED, class M, class T, class Src, class Dst, class Sync = BlockSync>
+__device__ __forceinline__ void smem_ntt_inverse(uint64_t *sm, uint32_t tid, const NttArgsT<M> &a, const T &ninv,
+                                                 const T &wn, const Src &src, const Dst &dst,
+                                                 const Sync &sync = Sync()) {
+    const uint32_t warp = tid >> 5, lane = tid & 31u;
+    inverse_phases<L, V, SCALED, L::NPH - 1, L::SPLIT>(sm, warp, lane, a, ninv, wn, src, dst);
+    sync();
+    inverse_phases<L, V, SCALED, L::SPLIT - 1, 0>(sm, warp, lane, a, ninv, wn, src, dst);
+}
+#endif
 
 }  // namespace fedhe

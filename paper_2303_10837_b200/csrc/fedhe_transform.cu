@@ -130,8 +130,8 @@ static cudaError_t launch_ntt_blocks(const CtxDev &c, bool forward, uint64_t *da
 // the block (inner) stages only
 cudaError_t launch_ntt_inner(const CtxDev &c, bool forward, uint64_t *data, size_t npoly, size_t poly_stride,
                              uint32_t limb0, uint32_t nlimbs, cudaStream_t s) {
-    if (c.LOGB == 13) return launch_ntt_blocks<Lay<13, 3>, 2>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
-    return launch_ntt_blocks<Lay<14, 3>, 2>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
+    if (c.LOGB == 13) return launch_ntt_blocks<WLay<13>, 2>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
+    return launch_ntt_blocks<WLay<14>, 2>(c, forward, data, npoly, poly_stride, limb0, nlimbs, s);
 }
 
 cudaError_t launch_ntt(const CtxDev &c, bool forward, uint64_t *data, size_t npoly, size_t poly_stride,

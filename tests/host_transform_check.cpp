@@ -1,18 +1,21 @@
 // Host-side check of the CUDA library's transform core (no GPU): the header
-// that the kernels are built from is compiled for the CPU, every virtual
-// thread of a block is played in turn with a plain array as shared memory,
+// that the kernels are built from is compiled for the CPU, every lane of every
+// virtual warp of a block is played in turn with a plain array as shared memory,
 // and the result is compared with the transform's definition
 //   A^[k] = sum_j a_j psi^((2 brev(k) + 1) j) mod q
 // evaluated directly.  Covers both limb arithmetics (64-bit integers, and
 // signed integers in doubles for primes below 2^46), whole blocks and the
 // pieces of a longer transform, the scaled inverse, the bounds that the
-// double-precision arithmetic relies on, and the shared-memory swizzle.
+// double-precision arithmetic relies on, the shared-memory swizzle, and that a
+// virtual warp keeps to its own words between the phases that only a
+// warp-level barrier separates.
 //
 // Built and run by tests/test_host_transform.py:  prints "ok" and exits 0.
 #include <cmath>
 #include <cstdint>
 #include <cstdio>
 #include <cstdlib>
+#include <algorithm>
 #include <vector>
 
 #include "../paper_2303_10837_b200/csrc/fedhe_host.h"
@@ -122,23 +125,56 @@ struct Tables<ModF64> {
     }
 };
 
+// the shared-memory words one virtual warp touches in phase P (sorted)
+template <class L, int P>
+static std::vector<uint32_t> warp_words(uint32_t vw) {
+    std::vector<uint32_t> w;
+    for (uint32_t lane = 0; lane < 32; lane++)
+        for (int r = 0; r < L::E; r++) w.push_back(wswz(L::template base<P>(vw, lane) | L::template reg<P>(r)));
+    std::sort(w.begin(), w.end());
+    return w;
+}
+
+// Inside a super-phase only a warp-level barrier separates the phases, so a
+// virtual warp must work on the same words in all of them.
+template <class L, int P = 0>
+static void check_closure() {
+    if constexpr (P + 1 < L::NPH && P + 1 != L::SPLIT) {
+        for (uint32_t vw = 0; vw < (uint32_t)L::NW; vw++)
+        {
+            const std::vector<uint32_t> here = warp_words<L, P>(vw), next = warp_words<L, P + 1>(vw);
+            CHECK(here == next, "warp %u leaves its words between phases %d and %d", vw, P, P + 1);
+        }
+    }
+    if constexpr (P + 1 < L::NPH) check_closure<L, P + 1>();
+}
+
 // one block of 2^LOGB values, piece `blk` of a transform cut into 2^A blocks, all phases
 template <class L, class M, int P = 0>
 static void forward_block(std::vector<uint64_t> &sm, const NttArgsT<M> &a, double *max_abs) {
     std::vector<uint64_t> out(sm.size());
     std::vector<int> writers(sm.size(), 0);
-    for (uint32_t vt = 0; vt < (uint32_t)L::NT; vt++) {
-        typename M::val x[L::E];
-        for (int r = 0; r < L::E; r++) x[r] = M::from_bits(sm[swz(L::template idx<P>(vt, r))]);
-        fwd_phase<L, P>(x, vt, a);
-        for (int r = 0; r < L::E; r++) {
-            const uint32_t i = swz(L::template idx<P>(vt, r));
-            CHECK(i < sm.size(), "index out of the block");
-            writers[i]++;
-            out[i] = M::bits(x[r]);
-            if (max_abs) *max_abs = std::fmax(*max_abs, std::fabs((double)x[r]));
+    for (uint32_t vw = 0; vw < (uint32_t)L::NW; vw++)
+        for (uint32_t lane = 0; lane < 32; lane++) {
+            const uint32_t base = L::template base<P>(vw, lane);
+            typename M::val x[L::E];
+            for (int r = 0; r < L::E; r++) {
+                CHECK((base & L::template reg<P>(r)) == 0, "register bits overlap the thread's bits");
+                x[r] = M::from_bits(sm[wswz(base | L::template reg<P>(r))]);
+            }
+            fwd_phase<L, P>(x, base, a);
+            for (int r = 0; r < L::E; r++) {
+                const uint32_t i = wswz(base | L::template reg<P>(r));
+                CHECK(i < sm.size(), "index out of the block");
+                writers[i]++;
+                out[i] = M::bits(x[r]);
+                if (max_abs) *max_abs = std::fmax(*max_abs, std::fabs((double)x[r]));
+            }
+            if (P == L::NPH - 1)
+                for (int r = 0; r < L::E; r += 2)
+                    CHECK((L::template reg<P>(r) & 1u) == 0 && L::template reg<P>(r + 1) == (L::template reg<P>(r) | 1u),
+                          "the last phase hands out pairs of neighbours");
         }
-    }
     for (int wcount : writers) CHECK(wcount == 1, "every word has exactly one owner per phase");
     sm = out;
     if constexpr (P + 1 < L::NPH) forward_block<L, M, P + 1>(sm, a, max_abs);
@@ -148,20 +184,22 @@ template <class L, class M, class T, bool SCALED, int P = L::NPH - 1>
 static void inverse_block(std::vector<uint64_t> &sm, const NttArgsT<M> &a, const T &ninv, const T &wn,
                           double *max_abs) {
     std::vector<uint64_t> out(sm.size());
-    for (uint32_t vt = 0; vt < (uint32_t)L::NT; vt++) {
-        typename M::val x[L::E];
-        for (int r = 0; r < L::E; r++) x[r] = M::from_bits(sm[swz(L::template idx<P>(vt, r))]);
-        if constexpr (P == 0 && SCALED) {
-            inv_phase<L, 0, 1>(x, vt, a);
-            inv_stage0_scaled<L>(x, a.m, ninv, wn);
-        } else {
-            inv_phase<L, P, 0>(x, vt, a);
+    for (uint32_t vw = 0; vw < (uint32_t)L::NW; vw++)
+        for (uint32_t lane = 0; lane < 32; lane++) {
+            const uint32_t base = L::template base<P>(vw, lane);
+            typename M::val x[L::E];
+            for (int r = 0; r < L::E; r++) x[r] = M::from_bits(sm[wswz(base | L::template reg<P>(r))]);
+            if constexpr (P == 0 && SCALED) {
+                inv_phase<L, 0, 1>(x, base, a);
+                inv_stage0_scaled<L>(x, a.m, ninv, wn);
+            } else {
+                inv_phase<L, P, 0>(x, base, a);
+            }
+            for (int r = 0; r < L::E; r++) {
+                out[wswz(base | L::template reg<P>(r))] = M::bits(x[r]);
+                if (max_abs) *max_abs = std::fmax(*max_abs, std::fabs((double)x[r]));
+            }
         }
-        for (int r = 0; r < L::E; r++) {
-            out[swz(L::template idx<P>(vt, r))] = M::bits(x[r]);
-            if (max_abs) *max_abs = std::fmax(*max_abs, std::fabs((double)x[r]));
-        }
-    }
     sm = out;
     if constexpr (P > 0) inverse_block<L, M, T, SCALED, P - 1>(sm, a, ninv, wn, max_abs);
 }
@@ -194,10 +232,10 @@ static void check_transform(uint32_t A, uint64_t q, int samples) {
     double max_fwd = 0;
     for (uint32_t blk = 0; blk < (1u << A); blk++) {
         std::vector<uint64_t> sm(B);
-        for (uint32_t i = 0; i < B; i++) sm[swz(i)] = M::bits(x[blk * B + i]);
+        for (uint32_t i = 0; i < B; i++) sm[wswz(i)] = M::bits(x[blk * B + i]);
         const NttArgsT<M> args{tab.fwd.data(), tab.m, A, blk};
         forward_block<L, M>(sm, args, &max_fwd);
-        for (uint32_t i = 0; i < B; i++) hat[blk * B + i] = tab.m.canon_wide(M::from_bits(sm[swz(i)]));
+        for (uint32_t i = 0; i < B; i++) hat[blk * B + i] = tab.m.canon_wide(M::from_bits(sm[wswz(i)]));
     }
     if (std::is_same<M, ModF64>::value)
         CHECK(max_fwd <= 13.0 * (double)q, "forward values stay below 13 q (%.2f q)", max_fwd / (double)q);
@@ -211,11 +249,11 @@ static void check_transform(uint32_t A, uint64_t q, int samples) {
     double max_inv = 0;
     for (uint32_t blk = 0; blk < (1u << A); blk++) {
         std::vector<uint64_t> sm(B);
-        for (uint32_t i = 0; i < B; i++) sm[swz(i)] = M::bits(tab.m.from_residue(hat[blk * B + i]));
+        for (uint32_t i = 0; i < B; i++) sm[wswz(i)] = M::bits(tab.m.from_residue(hat[blk * B + i]));
         const NttArgsT<M> args{tab.inv.data(), tab.m, A, blk};
         if (A == 0) inverse_block<L, M, decltype(tab.ninv), true>(sm, args, tab.ninv, tab.wn, &max_inv);
         else inverse_block<L, M, decltype(tab.ninv), false>(sm, args, tab.ninv, tab.wn, &max_inv);
-        for (uint32_t i = 0; i < B; i++) y[blk * B + i] = M::from_bits(sm[swz(i)]);
+        for (uint32_t i = 0; i < B; i++) y[blk * B + i] = M::from_bits(sm[wswz(i)]);
     }
     if (std::is_same<M, ModF64>::value)
         CHECK(max_inv <= (double)q, "inverse values are back below q after every phase (%.2f q)", max_inv / (double)q);
@@ -234,13 +272,13 @@ static void check_transform(uint32_t A, uint64_t q, int samples) {
 // 8 bytes in every phase layout, and permutes every aligned group of 16 words
 template <class L, int P = 0>
 static void check_banks() {
-    for (uint32_t warp = 0; warp < (uint32_t)L::NT / 32; warp++)
+    for (uint32_t vw = 0; vw < (uint32_t)L::NW; vw++)
         for (int r = 0; r < L::E; r++)
             for (int halfwarp = 0; halfwarp < 2; halfwarp++) {
                 uint32_t seen = 0;
-                for (uint32_t lane = 0; lane < 16; lane++) {
-                    const uint32_t tid = warp * 32 + halfwarp * 16 + lane;
-                    const uint32_t bank = swz(L::template idx<P>(tid, r)) & 15u;   // 16 banks of 8 bytes
+                for (uint32_t l = 0; l < 16; l++) {
+                    const uint32_t i = L::template base<P>(vw, halfwarp * 16 + l) | L::template reg<P>(r);
+                    const uint32_t bank = wswz(i) & 15u;   // 16 banks of 8 bytes
                     CHECK(!(seen & (1u << bank)), "bank conflict in phase %d", P);
                     seen |= 1u << bank;
                 }
@@ -252,8 +290,8 @@ int main() {
     for (uint32_t g = 0; g < (1u << 14); g += 16) {
         uint32_t seen = 0;
         for (uint32_t i = 0; i < 16; i++) {
-            CHECK((swz(g + i) & ~15u) == g, "swizzle leaves its group");
-            seen |= 1u << (swz(g + i) & 15u);
+            CHECK((wswz(g + i) & ~15u) == g, "swizzle leaves its group");
+            seen |= 1u << (wswz(g + i) & 15u);
         }
         CHECK(seen == 0xffffu, "swizzle is not a permutation");
     }
@@ -261,20 +299,22 @@ int main() {
     check_f64_primitives(q45);
     check_f64_primitives(q40);
     check_f64_primitives((1ull << 46) - 2 * 65536 * 3 + 1);   // any odd modulus below 2^46 serves the arithmetic
-    check_banks<Lay<13, 3>>();
-    check_banks<Lay<14, 3>>();
+    check_banks<WLay<13>>();
+    check_banks<WLay<14>>();
+    check_closure<WLay<13>>();
+    check_closure<WLay<14>>();
     // whole blocks
-    check_transform<Lay<13, 3>, ModInt>(0, q60, 24);
-    check_transform<Lay<13, 3>, ModF64>(0, q45, 24);
-    check_transform<Lay<14, 3>, ModInt>(0, q60, 12);
-    check_transform<Lay<14, 3>, ModF64>(0, q40, 12);
-    check_transform<Lay<13, 3>, ModInt>(0, q40, 12);          // a small prime in integer arithmetic
+    check_transform<WLay<13>, ModInt>(0, q60, 24);
+    check_transform<WLay<13>, ModF64>(0, q45, 24);
+    check_transform<WLay<14>, ModInt>(0, q60, 12);
+    check_transform<WLay<14>, ModF64>(0, q40, 12);
+    check_transform<WLay<13>, ModInt>(0, q40, 12);          // a small prime in integer arithmetic
     // pieces of longer transforms (the two-group encrypt and the long rings)
-    check_transform<Lay<13, 3>, ModInt>(1, q60, 8);
-    check_transform<Lay<13, 3>, ModF64>(1, q40, 8);
-    check_transform<Lay<13, 3>, ModF64>(2, q45, 6);
-    check_transform<Lay<13, 3>, ModInt>(3, q60, 4);
-    check_transform<Lay<13, 3>, ModF64>(3, q45, 4);
+    check_transform<WLay<13>, ModInt>(1, q60, 8);
+    check_transform<WLay<13>, ModF64>(1, q40, 8);
+    check_transform<WLay<13>, ModF64>(2, q45, 6);
+    check_transform<WLay<13>, ModInt>(3, q60, 4);
+    check_transform<WLay<13>, ModF64>(3, q45, 4);
     printf("ok\n");
     return 0;
 }
