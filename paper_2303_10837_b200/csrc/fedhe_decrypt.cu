@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
 decrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const uint64_t *ct, uint32_t level,
                      double *z) {
     static_assert(LF::NT == L::NT / V && LF::LOGB + 1 == L::LOGB, "thread counts and sizes must match");
-    extern __shared__ __align__(16) uint64_t sm[];
+    extern __shared__ __align__(128) uint64_t sm[];
     constexpr uint32_t B = 1u << L::LOGB, n = B >> 1;
     const uint32_t tid = threadIdx.x;
     const size_t t = blockIdx.x;

@@ -9,10 +9,11 @@ namespace fedhe {
 
 // Index swizzle of the one-byte sample arrays in shared memory (banks of four
 // bytes, i.e. index bits 2..6): the first phase of a transform reads them with
-// lanes that differ in index bits 0, 1 and three bits from 7 upwards, the
-// epilogues with consecutive lanes; folding bits 7..11 into bits 2..6 keeps
-// both patterns free of bank conflicts and leaves aligned groups of four intact.
-__device__ __forceinline__ uint32_t bswz(uint32_t i) { return i ^ (((i >> 7) & 31u) << 2); }
+// lanes that differ in index bits 0, 1, 7, 8 and 9, the epilogues with
+// consecutive lanes; folding bits 7..9 into bits 2..4 keeps both patterns free
+// of bank conflicts, leaves aligned groups of four intact, and does not involve
+// the first phase's register bits (10 and up), so a thread computes it once.
+__device__ __forceinline__ uint32_t bswz(uint32_t i) { return i ^ (((i >> 7) & 7u) << 2); }
 
 // One (ciphertext, limb) unit of the fused path in the limb's arithmetic.
 // u^ pk1^ is parked, in the arithmetic's own form, in the c1 slot it will
@@ -112,7 +113,7 @@ template <class L, int V, bool NTT_OUT>
 __global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
 encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const int64_t *m, uint32_t t0,
                      uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
-    extern __shared__ __align__(16) uint64_t sm[];
+    extern __shared__ __align__(128) uint64_t sm[];
     constexpr uint32_t B = 1u << L::LOGB, RT = L::NT / V;
     int8_t *su = reinterpret_cast<int8_t *>(sm + B);
     int8_t *se0 = su + B, *se1 = se0 + B;
@@ -294,7 +295,7 @@ template <class L, int V, bool NTT_OUT>
 __global__ void __launch_bounds__(2 * L::NT / V, 1)
 encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const int64_t *m, uint32_t t0,
                       uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
-    extern __shared__ __align__(16) uint64_t sm[];
+    extern __shared__ __align__(128) uint64_t sm[];
     constexpr uint32_t H = 1u << L::LOGB, B = 2 * H;       // half and whole limb
     constexpr uint32_t GT = L::NT / V, RT = 2 * GT;        // threads per group, per block
     int8_t *su = reinterpret_cast<int8_t *>(sm + B);
@@ -429,7 +430,7 @@ __device__ __forceinline__ void enc_block_forward(const CtxDev &c, const LimbDev
 template <class L, int V, bool ACC>
 __global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
 enc_block_forward_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const uint64_t *ubuf, uint64_t *ct) {
-    extern __shared__ __align__(16) uint64_t sm[];
+    extern __shared__ __align__(128) uint64_t sm[];
     uint32_t b = blockIdx.x;
     const uint32_t blk = b & ((1u << c.A) - 1u);
     b >>= c.A;

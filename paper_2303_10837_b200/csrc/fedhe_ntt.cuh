@@ -461,6 +461,24 @@ struct GroupSync {
     }
 };
 
+// Word of register r of a thread, given the 32-bit shared-memory address `a0`
+// of its register-0 word (sm + wswz(base)).  The swizzle is linear over GF(2)
+// and `base` is zero at the register bits, so the word index is
+// wswz(base) ^ wswz(reg(r)); of that constant the part above the low nibble
+// only sets bits that are clear in wswz(base), i.e. it adds and folds into the
+// instruction's offset, while the nibble is XOR-ed into the address itself
+// (which needs `sm` on a 128-byte boundary): one logic operation per distinct
+// nibble instead of an XOR and a scaled add per access.
+template <class L, int P>
+__device__ __forceinline__ uint64_t *reg_word(uint32_t a0, int r) {
+    const uint32_t k = wswz(L::template reg<P>(r));
+    const uint32_t a = (a0 ^ ((k & 15u) << 3)) + ((k & ~15u) << 3);
+    return reinterpret_cast<uint64_t *>(__cvta_shared_to_generic((size_t)a));
+}
+__device__ __forceinline__ uint32_t word_address(const uint64_t *sm, uint32_t word) {
+    return (uint32_t)__cvta_generic_to_shared(sm) + (word << 3);
+}
+
 // phases [P, PEND) of a forward transform, a warp-level barrier between them
 template <class L, int V, int P, int PEND, class M, class Src, class Dst>
 __device__ __forceinline__ void forward_phases(uint64_t *sm, uint32_t warp, uint32_t lane, const NttArgsT<M> &a,
@@ -469,12 +487,12 @@ __device__ __forceinline__ void forward_phases(uint64_t *sm, uint32_t warp, uint
 #pragma unroll M::UNROLL_V
     for (int v = 0; v < V; v++) {
         const uint32_t base = L::template base<P>(warp + v * (L::NW / V), lane);
-        const uint32_t sb = wswz(base);
+        const uint32_t a0 = word_address(sm, wswz(base));
         typename M::val x[L::E];
 #pragma unroll
         for (int r = 0; r < L::E; r++) {
             if constexpr (P == 0) x[r] = src(base | L::template reg<P>(r));
-            else x[r] = M::from_bits(sm[sb ^ wswz(L::template reg<P>(r))]);
+            else x[r] = M::from_bits(*reg_word<L, P>(a0, r));
         }
         fwd_phase<L, P>(x, base, a);
         if constexpr (P == LAST) {
@@ -482,7 +500,7 @@ __device__ __forceinline__ void forward_phases(uint64_t *sm, uint32_t warp, uint
             for (int r = 0; r < L::E; r += 2) dst(base | L::template reg<P>(r), x[r], x[r + 1]);
         } else {
 #pragma unroll
-            for (int r = 0; r < L::E; r++) sm[sb ^ wswz(L::template reg<P>(r))] = M::bits(x[r]);
+            for (int r = 0; r < L::E; r++) *reg_word<L, P>(a0, r) = M::bits(x[r]);
         }
     }
     if constexpr (P + 1 < PEND) {
@@ -508,7 +526,7 @@ __device__ __forceinline__ void inverse_phases(uint64_t *sm, uint32_t warp, uint
 #pragma unroll M::UNROLL_V
     for (int v = 0; v < V; v++) {
         const uint32_t base = L::template base<P>(warp + v * (L::NW / V), lane);
-        const uint32_t sb = wswz(base);
+        const uint32_t a0 = word_address(sm, wswz(base));
         typename M::val x[L::E];
         if constexpr (P == LAST) {
 #pragma unroll
@@ -519,7 +537,7 @@ __device__ __forceinline__ void inverse_phases(uint64_t *sm, uint32_t warp, uint
             }
         } else {
 #pragma unroll
-            for (int r = 0; r < L::E; r++) x[r] = M::from_bits(sm[sb ^ wswz(L::template reg<P>(r))]);
+            for (int r = 0; r < L::E; r++) x[r] = M::from_bits(*reg_word<L, P>(a0, r));
         }
         if constexpr (P == 0 && SCALED) {
             inv_phase<L, 0, 1>(x, base, a);
@@ -532,7 +550,7 @@ __device__ __forceinline__ void inverse_phases(uint64_t *sm, uint32_t warp, uint
             for (int r = 0; r < L::E; r++) dst(base | L::template reg<P>(r), x[r]);
         } else {
 #pragma unroll
-            for (int r = 0; r < L::E; r++) sm[sb ^ wswz(L::template reg<P>(r))] = M::bits(x[r]);
+            for (int r = 0; r < L::E; r++) *reg_word<L, P>(a0, r) = M::bits(x[r]);
         }
     }
     if constexpr (P > PEND) {

@@ -55,7 +55,7 @@ template <class L, int V, bool FWD, bool SCALED>
 __global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
 ntt_block_kernel(const __grid_constant__ CtxDev c, uint64_t *data, size_t poly_stride, uint32_t limb0,
                          uint32_t nlimbs) {
-    extern __shared__ __align__(16) uint64_t sm[];
+    extern __shared__ __align__(128) uint64_t sm[];
     uint32_t b = blockIdx.x;
     const uint32_t blk = b & ((1u << c.A) - 1u);
     b >>= c.A;
