@@ -264,20 +264,36 @@ __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0
         auto idst = [&](uint32_t i, val v) { smg[wswz(i)] = M::bits(v); };
         smem_ntt_inverse<L, V, false>(smg, gt, ia, ninv, wn, isrc, idst, gsync);
         __syncthreads();
-        // last stage across the halves with 1/N folded in, then the error / message terms
-        for (uint32_t e = tid; e < H; e += RT) {
-            val lo = M::from_bits(sm[wswz(e)]), hi = M::from_bits(sm[H + wswz(e)]);
-            ar.inv_scaled(lo, hi, ninv, wn);
-            uint64_t add_lo, add_hi;
+        // last stage across the halves with 1/N folded in, then the error / message terms; the
+        // message words of four rounds are requested before the first of them is used
+        constexpr uint32_t ROUNDS = H / RT, AHEAD = ROUNDS < 4 ? ROUNDS : 4;
+#pragma unroll
+        for (uint32_t k0 = 0; k0 < ROUNDS; k0 += AHEAD) {
+            int64_t m_lo[AHEAD], m_hi[AHEAD];
             if (h == 0) {
-                add_lo = signed_residue(mt[e] + (int64_t)se[bswz(e)], q, lb.mu);
-                add_hi = signed_residue(mt[e + H] + (int64_t)se[bswz(e + H)], q, lb.mu);
-            } else {
-                add_lo = small_residue(se[bswz(e)], q);
-                add_hi = small_residue(se[bswz(e + H)], q);
+#pragma unroll
+                for (uint32_t k = 0; k < AHEAD; k++) {
+                    const uint32_t e = tid + (k0 + k) * RT;
+                    m_lo[k] = mt[e];
+                    m_hi[k] = mt[e + H];
+                }
             }
-            cc[e] = ar.canon_add(lo, add_lo);
-            cc[e + H] = ar.canon_add(hi, add_hi);
+#pragma unroll
+            for (uint32_t k = 0; k < AHEAD; k++) {
+                const uint32_t e = tid + (k0 + k) * RT;
+                val lo = M::from_bits(sm[wswz(e)]), hi = M::from_bits(sm[H + wswz(e)]);
+                ar.inv_scaled(lo, hi, ninv, wn);
+                uint64_t add_lo, add_hi;
+                if (h == 0) {
+                    add_lo = signed_residue(m_lo[k] + (int64_t)se[bswz(e)], q, lb.mu);
+                    add_hi = signed_residue(m_hi[k] + (int64_t)se[bswz(e + H)], q, lb.mu);
+                } else {
+                    add_lo = small_residue(se[bswz(e)], q);
+                    add_hi = small_residue(se[bswz(e + H)], q);
+                }
+                cc[e] = ar.canon_add(lo, add_lo);
+                cc[e + H] = ar.canon_add(hi, add_hi);
+            }
         }
         __syncthreads();
     }
