@@ -65,7 +65,7 @@ typedef struct he_mask he_mask;
 typedef struct he_params {
     uint32_t N;                  /* ring degree: power of two, 8192..65536 */
     uint32_t L;                  /* number of RNS primes, 2..HE_MAX_LIMBS */
-    uint64_t q[HE_MAX_LIMBS];    /* distinct primes < 2^62 with q = 1 mod 2N */
+    uint64_t q[HE_MAX_LIMBS];    /* distinct primes < 2^61 with q = 1 mod 2N */
     int32_t log2_delta;          /* scale bits, 1 <= log2_delta, 2^log2_delta < q_0 / 4 */
 } he_params;
 

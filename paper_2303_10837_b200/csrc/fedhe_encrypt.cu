@@ -156,7 +156,7 @@ encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const in
         }
         const LimbDev &lb = c.limb[j];
         uint64_t *cbase = ct + (((size_t)tl * 2 + 0) * c.L + j) * B;
-        FEDHE_FOR_ARITH(lb, (encrypt_unit<M_, L, V, NTT_OUT>(lb, k.pk0_hat + (size_t)j * B, k.pk1_hat + (size_t)j * B, sm, su,
+        FEDHE_FOR_ARITH_SEL(lb, (encrypt_unit<M_, L, V, NTT_OUT>(lb, k.pk0_hat + (size_t)j * B, k.pk1_hat + (size_t)j * B, sm, su,
                                                     se0, m + (size_t)tl * B, cbase, cstride)));
     }
 }
@@ -351,7 +351,7 @@ encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const i
         }
         const LimbDev &lb = c.limb[j];
         uint64_t *cbase = ct + (((size_t)tl * 2 + 0) * c.L + j) * B;
-        FEDHE_FOR_ARITH(lb, (encrypt_unit2<M_, L, V, NTT_OUT>(lb, k.pk0_hat + (size_t)j * B, k.pk1_hat + (size_t)j * B, sm, su,
+        FEDHE_FOR_ARITH_SEL(lb, (encrypt_unit2<M_, L, V, NTT_OUT>(lb, k.pk0_hat + (size_t)j * B, k.pk1_hat + (size_t)j * B, sm, su,
                                                      se0, m + (size_t)tl * B, cbase, cstride)));
     }
 }

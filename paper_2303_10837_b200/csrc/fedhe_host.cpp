@@ -57,7 +57,7 @@ const char *host_check_params(uint32_t N, uint32_t L, const uint64_t *q, int log
     if (L < 2 || L > 16) return "L must be in [2, 16]";
     if (log2_delta < 1 || log2_delta > 58) return "log2_delta out of range";
     for (uint32_t j = 0; j < L; j++) {
-        if (q[j] >= (1ull << 62) || q[j] < (1ull << 20)) return "prime out of range";
+        if (q[j] >= (1ull << 61) || q[j] < (1ull << 20)) return "prime out of range";
         if ((q[j] - 1) % (2ull * N)) return "prime is not 1 mod 2N";
         if (!host_is_prime(q[j])) return "modulus is not prime";
         for (uint32_t i = 0; i < j; i++)

@@ -31,10 +31,10 @@ struct LimbDev {
 // the pieces of a limb that a transform in arithmetic M needs
 template <class M>
 struct LimbOf;
-template <>
-struct LimbOf<ModInt> {
-    static HD NttArgs args(const LimbDev &lb, bool fwd, uint32_t A, uint32_t blk) {
-        return NttArgs{fwd ? lb.fwd : lb.inv, ModInt{lb.q, 2 * lb.q}, A, blk};
+template <bool SEL>
+struct LimbOf<ModIntT<SEL>> {
+    static HD NttArgsT<ModIntT<SEL>> args(const LimbDev &lb, bool fwd, uint32_t A, uint32_t blk) {
+        return NttArgsT<ModIntT<SEL>>{fwd ? lb.fwd : lb.inv, ModIntT<SEL>{lb.q, 2 * lb.q}, A, blk};
     }
     static HD tw_t ninv(const LimbDev &lb) { return lb.ninv; }
     static HD tw_t wn(const LimbDev &lb) { return lb.wn; }

@@ -100,6 +100,11 @@ static __device__ uint64_t shoup_companion(uint64_t w, uint64_t q) {   // floor(
     if ((lb).fwd_d) { using M_ = ModF64; CALL; }                \
     else { using M_ = ModInt; CALL; }
 
+// the same with the select flavour of the integer arithmetic (kernels bound by the multiply pipe)
+#define FEDHE_FOR_ARITH_SEL(lb, CALL)                           \
+    if ((lb).fwd_d) { using M_ = ModF64; CALL; }                \
+    else { using M_ = ModIntSel; CALL; }
+
 // The A = logN - LOGB outer stages of a long transform on two neighbouring
 // columns of the 2^A x B matrix view (x[a], y[a] = row a): forward from
 // canonical input, inverse with 1/N folded into stage 0.

@@ -126,7 +126,7 @@ HD void load_run(const tw_t *p, tw_t (&w)[K]) {
 
 // ---- arithmetic of one limb ---------------------------------------------------
 //
-// ModInt: any prime below 2^62; 64-bit integers in the lazy Harvey ranges
+// ModInt: any prime below 2^61; 64-bit integers in the lazy Harvey ranges
 // (forward [0, 4q), inverse [0, 2q)), table entries {w, floor(w 2^64 / q)}.
 // ModF64: primes below 2^46; signed integers in doubles, table entries the
 // twiddles as doubles.  Forward, every stage adds at most 3q/4 to the bound
@@ -134,7 +134,9 @@ HD void load_run(const tw_t *p, tw_t (&w)[K]) {
 // differences go through the product, so after the at most three stages of a
 // phase the sums are brought back below q (settle) before they are stored.
 
-struct ModInt {
+// SEL: conditional subtractions by bitwise selects (csub_sel) instead of predicated moves
+template <bool SEL>
+struct ModIntT {
     static constexpr int UNROLL_V = 1;   // virtual threads of a phase one after the other
     using val = uint64_t;
     using tab = tw_t;
@@ -142,8 +144,8 @@ struct ModInt {
     static HD val from_bits(uint64_t b) { return b; }
     static HD uint64_t bits(val v) { return v; }
     static HD tw_t load(const tw_t *p) { return FEDHE_LD_TW(p); }
-    HD void fwd(val &x, val &y, const tw_t &w) const { ct_butterfly(x, y, w.w, w.wp, q, q2); }
-    HD void inv(val &x, val &y, const tw_t &w) const { gs_butterfly(x, y, w.w, w.wp, q, q2); }
+    HD void fwd(val &x, val &y, const tw_t &w) const { ct_butterfly<SEL>(x, y, w.w, w.wp, q, q2); }
+    HD void inv(val &x, val &y, const tw_t &w) const { gs_butterfly<SEL>(x, y, w.w, w.wp, q, q2); }
     // x <- (x + y) a, y <- (x - y) b for inputs below 2q; outputs below 2q
     HD void inv_scaled(val &x, val &y, const tw_t &a, const tw_t &b) const {
         const uint64_t u = x, v = y;
@@ -157,16 +159,19 @@ struct ModInt {
     HD val small(int v) const { return small_residue(v, q); }
     // canonical residue of a forward output (below 4q) / of an inverse output (below 2q),
     // and of an inverse output plus a residue in [0, q)
-    HD uint64_t canon_wide(val v) const { return csub(csub(v, q2), q); }
-    HD uint64_t canon(val v) const { return csub(v, q); }
-    HD uint64_t canon_add(val v, uint64_t add) const { return csub(csub(v, q) + add, q); }
+    HD uint64_t canon_wide(val v) const { return csub_as<SEL>(csub_as<SEL>(v, q2), q); }
+    HD uint64_t canon(val v) const { return csub_as<SEL>(v, q); }
+    HD uint64_t canon_add(val v, uint64_t add) const { return csub_as<SEL>(csub_as<SEL>(v, q) + add, q); }
     // canonical residue of a forward output plus a key product
-    HD uint64_t canon_sum(val a, val b) const { return csub(canon_wide(a) + csub(b, q), q); }
+    HD uint64_t canon_sum(val a, val b) const { return csub_as<SEL>(canon_wide(a) + csub_as<SEL>(b, q), q); }
     // product with an entry of a key table, below 2q for any v
     using key = tw_t;
     static HD key load_key(const tw_t *p) { return FEDHE_LD_TW(p); }
     HD val mul_key(val v, const key &k) const { return shoup_lazy(v, k.w, k.wp, q); }
 };
+
+using ModInt = ModIntT<false>;
+using ModIntSel = ModIntT<true>;
 
 struct ModF64 {
     static constexpr int UNROLL_V = 2;
