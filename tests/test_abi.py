@@ -41,6 +41,7 @@ def test_error_strings_and_host_side_parameter_checks():
         (8192, list(si.PRIMES_N8192), 59),                    # scale >= q0 / 4
         (8192, [si.PRIMES_N8192[0]], 40),                     # a single prime leaves nothing after the rescale
         (4096, list(si.PRIMES_N8192), 40),                    # N below the supported range
+        (8192, [0x3fffffffffff0001, si.PRIMES_N8192[1]], 40),  # a prime (= 1 mod 2N) of 62 bits: lazy values must stay below 2^63
     ]
     for N, primes, ld in bad:
         with pytest.raises(he.HeError) as ei:
