@@ -164,53 +164,95 @@ cudaError_t launch_mask_write(size_t P, const uint32_t *bits, const uint32_t *bl
 // ===========================================================================
 
 // one pass over the update: masked parameters go to their slot, the others to
-// the compacted remainder; the tail of the last ciphertext is zeroed
+// the compacted remainder; the tail of the last ciphertext is zeroed.  A
+// thread takes four neighbouring parameters (one 16-byte load when the
+// pointers allow it; they always share one word of the bit mask).
 __global__ void __launch_bounds__(256)
 pack_kernel(const uint32_t *bits, const uint32_t *wpre, const float *x, size_t P, size_t k, size_t padded,
-            float *sel, float *rest) {
-    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < P) {
-        const float v = __ldg(x + i);
-        if (bits == nullptr) {
-            sel[i] = v;
+            float *sel, float *rest, bool vec) {
+    const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t i0 = t * 4;
+    if (i0 < P) {
+        float v[4];
+        const uint32_t cnt = P - i0 < 4 ? (uint32_t)(P - i0) : 4u;
+        if (vec && cnt == 4) {
+            const float4 q = __ldg(reinterpret_cast<const float4 *>(x + i0));
+            v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
         } else {
-            const uint32_t w = bits[i >> 5], lane = (uint32_t)(i & 31);
-            const size_t before = (size_t)wpre[i >> 5] + __popc(w & ((1u << lane) - 1u));
-            if ((w >> lane) & 1u) sel[before] = v;
-            else rest[i - before] = v;
+#pragma unroll
+            for (uint32_t j = 0; j < 4; j++) v[j] = j < cnt ? __ldg(x + i0 + j) : 0.0f;
+        }
+        if (bits == nullptr) {
+            if (vec && cnt == 4) {
+                *reinterpret_cast<float4 *>(sel + i0) = make_float4(v[0], v[1], v[2], v[3]);
+            } else {
+#pragma unroll
+                for (uint32_t j = 0; j < 4; j++)
+                    if (j < cnt) sel[i0 + j] = v[j];
+            }
+        } else {
+            const uint32_t w = bits[i0 >> 5], lane = (uint32_t)(i0 & 31);
+            size_t before = (size_t)wpre[i0 >> 5] + __popc(w & ((1u << lane) - 1u));
+#pragma unroll
+            for (uint32_t j = 0; j < 4; j++) {
+                if (j < cnt) {
+                    if ((w >> (lane + j)) & 1u) sel[before++] = v[j];
+                    else rest[i0 + j - before] = v[j];
+                }
+            }
         }
     }
-    if (i < padded - k) sel[k + i] = 0.0f;
+    if (t < padded - k) sel[k + t] = 0.0f;
 }
 
 cudaError_t launch_pack(const he_mask *mask, const float *x, size_t P, size_t k, size_t padded,
                         float *sel, float *rest, cudaStream_t s) {
-    size_t threads = P > padded - k ? P : padded - k;
+    const size_t quads = (P + 3) / 4;
+    size_t threads = quads > padded - k ? quads : padded - k;
     if (threads == 0) return cudaSuccess;
+    const bool vec = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(sel)) & 15u) == 0;
     pack_kernel<<<blocks_for(threads, 256), 256, 0, s>>>(mask ? mask->bits : nullptr, mask ? mask->wpre : nullptr,
-                                                          x, P, k, padded, sel, rest);
+                                                          x, P, k, padded, sel, rest, vec);
     return FEDHE_LAUNCHED();
 }
 
+// the reverse: two neighbouring parameters per thread (one 16-byte store)
 __global__ void __launch_bounds__(256)
 unpack_kernel(const uint32_t *bits, const uint32_t *wpre, const double *z, const double *rest_avg, size_t P,
-              double *w_glob) {
-    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= P) return;
+              double *w_glob, bool vec) {
+    const size_t i0 = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 2;
+    if (i0 >= P) return;
+    const bool two = i0 + 1 < P;
+    double a, b = 0.0;
     if (bits == nullptr) {
-        w_glob[i] = z[i];
-        return;
+        if (vec && two) {
+            *reinterpret_cast<double2 *>(w_glob + i0) = *reinterpret_cast<const double2 *>(z + i0);
+            return;
+        }
+        a = z[i0];
+        if (two) b = z[i0 + 1];
+    } else {
+        const uint32_t w = bits[i0 >> 5], lane = (uint32_t)(i0 & 31);
+        size_t before = (size_t)wpre[i0 >> 5] + __popc(w & ((1u << lane) - 1u));
+        const bool s0 = (w >> lane) & 1u;
+        a = s0 ? z[before] : rest_avg[i0 - before];
+        before += s0 ? 1 : 0;
+        if (two) b = ((w >> (lane + 1)) & 1u) ? z[before] : rest_avg[i0 + 1 - before];
     }
-    const uint32_t w = bits[i >> 5], lane = (uint32_t)(i & 31);
-    const size_t before = (size_t)wpre[i >> 5] + __popc(w & ((1u << lane) - 1u));
-    w_glob[i] = ((w >> lane) & 1u) ? z[before] : rest_avg[i - before];
+    if (vec && two) {
+        *reinterpret_cast<double2 *>(w_glob + i0) = make_double2(a, b);
+    } else {
+        w_glob[i0] = a;
+        if (two) w_glob[i0 + 1] = b;
+    }
 }
 
 cudaError_t launch_unpack(const he_mask *mask, const double *z, const double *rest_avg, size_t P,
                           double *w_glob, cudaStream_t s) {
     if (P == 0) return cudaSuccess;
-    unpack_kernel<<<blocks_for(P, 256), 256, 0, s>>>(mask ? mask->bits : nullptr, mask ? mask->wpre : nullptr, z,
-                                                     rest_avg, P, w_glob);
+    const bool vec = ((reinterpret_cast<uintptr_t>(z) | reinterpret_cast<uintptr_t>(w_glob)) & 15u) == 0;
+    unpack_kernel<<<blocks_for((P + 1) / 2, 256), 256, 0, s>>>(mask ? mask->bits : nullptr,
+                                                               mask ? mask->wpre : nullptr, z, rest_avg, P, w_glob, vec);
     return FEDHE_LAUNCHED();
 }
 
