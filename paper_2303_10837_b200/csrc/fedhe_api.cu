@@ -283,9 +283,13 @@ static int build_mask(he_ctx *ctx, const float *score, size_t P, size_t k, const
     const size_t nblocks = (P + MASK_BLOCK - 1) / MASK_BLOCK, nwords = (P + 31) / 32;
 
     // scratch: histogram (2048) | totals (2) | blk_a (nblocks) | blk_b (nblocks) | ranges
-    uint32_t *scratch = nullptr;
+    // (it lives in the context's work space: no allocation, and no free that would wait for the device)
     const size_t scratch_words = 2048 + 2 + 2 * nblocks + 4 * 64 + 2;
-    CU(cudaMalloc(reinterpret_cast<void **>(&scratch), scratch_words * sizeof(uint32_t)));
+    {
+        const int erc = ensure(&ctx->ws, &ctx->ws_bytes, scratch_words * sizeof(uint32_t));
+        if (erc != HE_OK) return erc;
+    }
+    uint32_t *scratch = static_cast<uint32_t *>(ctx->ws);
     uint32_t *hist = scratch, *totals = scratch + 2048, *blk_eq = totals + 2, *blk_sel = blk_eq + nblocks;
     uint64_t *ranges_dev = reinterpret_cast<uint64_t *>(scratch + ((2048 + 2 + 2 * nblocks + 1) & ~(size_t)1));
     int rc = HE_OK;
@@ -325,8 +329,9 @@ static int build_mask(he_ctx *ctx, const float *score, size_t P, size_t k, const
             if (fail) { rc = HE_ERR_CUDA; break; }
             tau = prefix;
         }
-        MCU(cudaMalloc(reinterpret_cast<void **>(&bits), nwords * sizeof(uint32_t)));
-        MCU(cudaMalloc(reinterpret_cast<void **>(&wpre), nwords * sizeof(uint32_t)));
+        // bit mask and per-word prefix counts share one allocation
+        MCU(cudaMalloc(reinterpret_cast<void **>(&bits), 2 * nwords * sizeof(uint32_t)));
+        wpre = bits + nwords;
         if (num_ranges)
             MCU(cudaMemcpyAsync(ranges_dev, ranges_host, 2 * num_ranges * sizeof(uint64_t), cudaMemcpyHostToDevice, st));
         MCU(launch_mask_count_eq(score, P, tau, blk_eq, st));
@@ -350,10 +355,8 @@ static int build_mask(he_ctx *ctx, const float *score, size_t P, size_t k, const
         m->wpre = wpre;
 #undef MCU
     } while (0);
-    cudaFree(scratch);
     if (rc != HE_OK) {
         if (bits) cudaFree(bits);
-        if (wpre) cudaFree(wpre);
         if (idx) cudaFree(idx);
         return rc;
     }
@@ -388,8 +391,7 @@ int he_mask_destroy(he_mask *mask) {
     if (!good(mask)) return HE_ERR_INVALID_ARG;
     cudaDeviceSynchronize();
     cudaFree(mask->idx);
-    cudaFree(mask->bits);
-    cudaFree(mask->wpre);
+    cudaFree(mask->bits);      // the prefix counts are the second half of this allocation
     mask->magic = 0;
     delete mask;
     return HE_OK;
