@@ -50,8 +50,8 @@ UNIT = "params/s"
 # Additions, shifts and logic go to another pipe.
 # DRAM bytes (read + write) per ciphertext of encrypt_fused2_kernel at N = 16384,
 # L = 4, from an ncu capture of the profile_case.py encrypt case (summary under profiles/)
-# (360.1 MB for 296 ciphertexts; traffic grows in proportion to the count).
-ENCRYPT_DRAM_BYTES_PER_CT_N16384_L4 = 360.068096e6 / 296
+# (363.1 MB for 296 ciphertexts; traffic grows in proportion to the count).
+ENCRYPT_DRAM_BYTES_PER_CT_N16384_L4 = 363.052288e6 / 296
 SLOTS_PER_SM_CLK = 64.0
 WIDE_COST = 2.5
 INT_SLOTS_PER_BUTTERFLY = 6 * WIDE_COST + 4
