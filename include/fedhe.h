@@ -18,10 +18,23 @@
  *     caller, never freed by the library; "host" pointers are ordinary host
  *     memory.  Handles (he_ctx, he_keys, he_mask) are owned by the library
  *     and released by the matching *_destroy.
+ *   - Alignment: every dev pointer to uint64 words (ciphertexts, aggregates,
+ *     partial decryptions, exported keys, the polynomials of he_ntt_*) must be
+ *     16-byte aligned, because the kernels move two words per access; a
+ *     pointer that is not is refused with HE_ERR_INVALID_ARG before anything is
+ *     launched.  float, double, int64 and index buffers need only their
+ *     natural alignment (the kernels fall back to narrower accesses).
+ *   - The library cannot see how large a caller's buffer is: every size below
+ *     is a requirement on the caller (the Python binding checks them).
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
  *     Calls are asynchronous on it unless stated otherwise.  A context keeps
- *     small library-owned work buffers; calls that share a context must be
- *     issued on one stream at a time.
+ *     library-owned work buffers; calls that share a context must be issued
+ *     on one stream at a time.  A call that needs more work space than the
+ *     context holds (he_encode, he_encrypt*, he_decrypt* on rings above
+ *     N = 16384, he_threshold_combine, he_weighted_aggregate_ntt,
+ *     he_select_mask*, he_round_host with a larger problem than before) frees
+ *     and reallocates it, which synchronises the whole device once;
+ *     he_ctx_reserve does that ahead of time.
  *   - Kernels never trap or assert.  A numeric anomaly (an encoded
  *     coefficient of magnitude >= 2^62, or a non-finite input) sets a sticky
  *     status word read by he_ctx_status().
@@ -260,7 +273,10 @@ int he_ntt_inverse(he_ctx *ctx, uint64_t *polys_dev, size_t B, void *stream);
  * run on a second stream beside the arithmetic; they overlap it only when xs
  * and w_glob are page-locked (pinned) host memory, pageable memory is
  * correct but serialises.  With full encryption parts of w_glob are written
- * before the call returns; after an error return its contents are unspecified. */
+ * before the call returns; after an error return its contents are unspecified.
+ * Bad arguments (a NULL xs[i], a weight outside [0, 1]) are refused before
+ * anything is queued.  On every return, error or not, both streams have been
+ * waited for: no copy is still reading xs or writing w_glob. */
 int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const float *const *xs_host,
                   const double *alpha_host, int C, size_t P, uint64_t enc_seed, double *w_glob_host,
                   void *stream);

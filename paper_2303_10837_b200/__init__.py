@@ -116,6 +116,34 @@ def _dev(t: torch.Tensor, dtype: torch.dtype) -> int:
     return t.data_ptr()
 
 
+# The C ABI takes plain pointers and cannot know how large a buffer is, so this
+# layer is where a short buffer is caught: before the call, on the host, as an
+# error instead of an out-of-bounds access on the device.
+def _sized(t: torch.Tensor, count: int, what: str, exact: bool = False) -> None:
+    have = t.numel()
+    if have != count if exact else have < count:
+        raise HeError(HE_ERR_INVALID_ARG, "%s: %d entries, %s%d needed" % (what, have, "" if exact else "at least ", count))
+
+
+def _same_len(a, b, what: str) -> None:
+    if len(a) != len(b) or len(a) < 1:
+        raise HeError(HE_ERR_INVALID_ARG, "%s: %d and %d entries" % (what, len(a), len(b)))
+
+
+def _whole_cts(ctx: "Ctx", sel: torch.Tensor, what: str) -> int:
+    """Number of ciphertexts of a slot buffer, which must hold whole ciphertexts."""
+    if sel.numel() % ctx.n:
+        raise HeError(HE_ERR_INVALID_ARG, "%s: %d slots is not a multiple of n = %d" % (what, sel.numel(), ctx.n))
+    return sel.numel() // ctx.n
+
+
+def _ct_count(ctx: "Ctx", ct: torch.Tensor, level: int, what: str) -> int:
+    """T of a ciphertext tensor [T][2][level][N] (taken from its first extent, checked against its size)."""
+    T = ct.shape[0] if ct.dim() else 0
+    _sized(ct, T * 2 * level * ctx.N, what, exact=True)
+    return T
+
+
 class Ctx:
     """Owner of a ``he_ctx*``."""
 
@@ -231,6 +259,8 @@ def he_mask_indices(mask: Mask) -> torch.Tensor:
 def he_pack(ctx: Ctx, mask: Optional[Mask], x: torch.Tensor):
     """(sel float32 [T*n], rest float32 [P-k] or None)."""
     P = x.numel()
+    if mask is not None and mask.P != P:
+        raise HeError(HE_ERR_INVALID_ARG, "he_pack: the mask was built for %d parameters, x has %d" % (mask.P, P))
     k = mask.k if mask is not None else P
     sel = torch.empty(he_num_ct(ctx, k) * ctx.n, dtype=torch.float32, device="cuda")
     rest = torch.empty(P - k, dtype=torch.float32, device="cuda") if mask is not None else None
@@ -241,7 +271,7 @@ def he_pack(ctx: Ctx, mask: Optional[Mask], x: torch.Tensor):
 
 
 def he_encode(ctx: Ctx, sel: torch.Tensor) -> torch.Tensor:
-    T = sel.numel() // ctx.n
+    T = _whole_cts(ctx, sel, "he_encode sel")
     m = torch.empty((T, ctx.N), dtype=torch.int64, device="cuda")
     _check(_lib.he_encode(ctx.handle, _dev(sel, torch.float32), sel.numel(), m.data_ptr(), _stream()),
            "he_encode")
@@ -251,9 +281,10 @@ def he_encode(ctx: Ctx, sel: torch.Tensor) -> torch.Tensor:
 def he_encrypt(ctx: Ctx, keys: Keys, sel: torch.Tensor, seed: int, client_id: int,
                out: Optional[torch.Tensor] = None) -> torch.Tensor:
     """Fresh ciphertexts uint64-as-int64 [T][2][L][N]."""
-    T = sel.numel() // ctx.n
+    T = _whole_cts(ctx, sel, "he_encrypt sel")
     if out is None:
         out = torch.empty((T, 2, ctx.L, ctx.N), dtype=torch.int64, device="cuda")
+    _sized(out, T * 2 * ctx.L * ctx.N, "he_encrypt out")
     _check(_lib.he_encrypt(ctx.handle, keys.handle, _dev(sel, torch.float32), sel.numel(), seed, client_id,
                            _dev(out, torch.int64), _stream()), "he_encrypt")
     return out
@@ -262,9 +293,10 @@ def he_encrypt(ctx: Ctx, keys: Keys, sel: torch.Tensor, seed: int, client_id: in
 def he_encrypt_ntt(ctx: Ctx, keys: Keys, sel: torch.Tensor, seed: int, client_id: int,
                    out: Optional[torch.Tensor] = None) -> torch.Tensor:
     """The same ciphertexts in the transform-domain wire format."""
-    T = sel.numel() // ctx.n
+    T = _whole_cts(ctx, sel, "he_encrypt_ntt sel")
     if out is None:
         out = torch.empty((T, 2, ctx.L, ctx.N), dtype=torch.int64, device="cuda")
+    _sized(out, T * 2 * ctx.L * ctx.N, "he_encrypt_ntt out")
     _check(_lib.he_encrypt_ntt(ctx.handle, keys.handle, _dev(sel, torch.float32), sel.numel(), seed, client_id,
                                _dev(out, torch.int64), _stream()), "he_encrypt_ntt")
     return out
@@ -273,6 +305,8 @@ def he_encrypt_ntt(ctx: Ctx, keys: Keys, sel: torch.Tensor, seed: int, client_id
 def he_encrypt_range(ctx: Ctx, keys: Keys, sel: torch.Tensor, t_begin: int, t_count: int, seed: int,
                      client_id: int, out: torch.Tensor) -> torch.Tensor:
     """`sel` holds the slots of ciphertexts t_begin .. t_begin+t_count-1."""
+    _sized(sel, t_count * ctx.n, "he_encrypt_range sel")
+    _sized(out, t_count * 2 * ctx.L * ctx.N, "he_encrypt_range out")
     _check(_lib.he_encrypt_range(ctx.handle, keys.handle, _dev(sel, torch.float32), t_begin, t_count, seed,
                                  client_id, _dev(out, torch.int64), _stream()), "he_encrypt_range")
     return out
@@ -280,12 +314,16 @@ def he_encrypt_range(ctx: Ctx, keys: Keys, sel: torch.Tensor, t_begin: int, t_co
 
 def he_weighted_aggregate(ctx: Ctx, cts: List[torch.Tensor], alpha: Sequence[float],
                           out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    _same_len(cts, alpha, "he_weighted_aggregate cts and alpha")
     Cn = len(cts)
-    T = cts[0].shape[0]
-    ptrs = (_vp * Cn)(*[_dev(c, torch.int64) for c in cts])
-    al = (C.c_double * Cn)(*[float(a) for a in alpha])
+    T = _ct_count(ctx, cts[0], ctx.L, "he_weighted_aggregate cts[0]")
+    for i, c in enumerate(cts):
+        _sized(c, T * 2 * ctx.L * ctx.N, "he_weighted_aggregate cts[%d]" % i, exact=True)
     if out is None:
         out = torch.empty((T, 2, ctx.L - 1, ctx.N), dtype=torch.int64, device="cuda")
+    _sized(out, T * 2 * (ctx.L - 1) * ctx.N, "he_weighted_aggregate out")
+    ptrs = (_vp * Cn)(*[_dev(c, torch.int64) for c in cts])
+    al = (C.c_double * Cn)(*[float(a) for a in alpha])
     _check(_lib.he_weighted_aggregate(ctx.handle, C.cast(ptrs, _vp), C.cast(al, _vp), Cn, T,
                                       _dev(out, torch.int64), _stream()), "he_weighted_aggregate")
     return out
@@ -293,20 +331,27 @@ def he_weighted_aggregate(ctx: Ctx, cts: List[torch.Tensor], alpha: Sequence[flo
 
 def he_weighted_aggregate_ntt(ctx: Ctx, cts: List[torch.Tensor], alpha: Sequence[float],
                               out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    _same_len(cts, alpha, "he_weighted_aggregate_ntt cts and alpha")
     Cn = len(cts)
-    T = cts[0].shape[0]
-    ptrs = (_vp * Cn)(*[_dev(c, torch.int64) for c in cts])
-    al = (C.c_double * Cn)(*[float(a) for a in alpha])
+    T = _ct_count(ctx, cts[0], ctx.L, "he_weighted_aggregate_ntt cts[0]")
+    for i, c in enumerate(cts):
+        _sized(c, T * 2 * ctx.L * ctx.N, "he_weighted_aggregate_ntt cts[%d]" % i, exact=True)
     if out is None:
         out = torch.empty((T, 2, ctx.L - 1, ctx.N), dtype=torch.int64, device="cuda")
+    _sized(out, T * 2 * (ctx.L - 1) * ctx.N, "he_weighted_aggregate_ntt out")
+    ptrs = (_vp * Cn)(*[_dev(c, torch.int64) for c in cts])
+    al = (C.c_double * Cn)(*[float(a) for a in alpha])
     _check(_lib.he_weighted_aggregate_ntt(ctx.handle, C.cast(ptrs, _vp), C.cast(al, _vp), Cn, T,
                                           _dev(out, torch.int64), _stream()), "he_weighted_aggregate_ntt")
     return out
 
 
 def he_plain_aggregate(ctx: Ctx, rests: List[torch.Tensor], alpha: Sequence[float]) -> torch.Tensor:
+    _same_len(rests, alpha, "he_plain_aggregate rests and alpha")
     Cn = len(rests)
     n = rests[0].numel()
+    for i, r in enumerate(rests):
+        _sized(r, n, "he_plain_aggregate rests[%d]" % i, exact=True)
     ptrs = (_vp * Cn)(*[_dev(r, torch.float32) if n else 1 for r in rests])
     al = (C.c_double * Cn)(*[float(a) for a in alpha])
     out = torch.empty(n, dtype=torch.float64, device="cuda")
@@ -316,16 +361,17 @@ def he_plain_aggregate(ctx: Ctx, rests: List[torch.Tensor], alpha: Sequence[floa
 
 
 def he_decrypt(ctx: Ctx, keys: Keys, agg: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
-    T = agg.shape[0]
+    T = _ct_count(ctx, agg, ctx.L - 1, "he_decrypt agg")
     if out is None:
         out = torch.empty(T * ctx.n, dtype=torch.float64, device="cuda")
+    _sized(out, T * ctx.n, "he_decrypt out")
     _check(_lib.he_decrypt(ctx.handle, keys.handle, _dev(agg, torch.int64), T, _dev(out, torch.float64),
                            _stream()), "he_decrypt")
     return out
 
 
 def he_decrypt_level(ctx: Ctx, keys: Keys, ct: torch.Tensor, level: int) -> torch.Tensor:
-    T = ct.shape[0]
+    T = _ct_count(ctx, ct, level, "he_decrypt_level ct")
     z = torch.empty(T * ctx.n, dtype=torch.float64, device="cuda")
     _check(_lib.he_decrypt_level(ctx.handle, keys.handle, _dev(ct, torch.int64), level, T, z.data_ptr(),
                                  _stream()), "he_decrypt_level")
@@ -334,9 +380,10 @@ def he_decrypt_level(ctx: Ctx, keys: Keys, ct: torch.Tensor, level: int) -> torc
 
 def he_decrypt_level_ntt(ctx: Ctx, keys: Keys, ct: torch.Tensor, level: int,
                          out: Optional[torch.Tensor] = None) -> torch.Tensor:
-    T = ct.shape[0]
+    T = _ct_count(ctx, ct, level, "he_decrypt_level_ntt ct")
     if out is None:
         out = torch.empty(T * ctx.n, dtype=torch.float64, device="cuda")
+    _sized(out, T * ctx.n, "he_decrypt_level_ntt out")
     _check(_lib.he_decrypt_level_ntt(ctx.handle, keys.handle, _dev(ct, torch.int64), level, T,
                                      _dev(out, torch.float64), _stream()), "he_decrypt_level_ntt")
     return out
@@ -353,7 +400,7 @@ def he_threshold_split(ctx: Ctx, keys: Keys, seed: int):
 def he_partial_decrypt(ctx: Ctx, share: Keys, party: int, ct: torch.Tensor, level: int, seed: int,
                        smudge_bits: int) -> torch.Tensor:
     """Residues mod q_0, uint64-as-int64 [T][N]."""
-    T = ct.shape[0]
+    T = _ct_count(ctx, ct, level, "he_partial_decrypt ct")
     part = torch.empty((T, ctx.N), dtype=torch.int64, device="cuda")
     _check(_lib.he_partial_decrypt(ctx.handle, share.handle, party, _dev(ct, torch.int64) or None, level, T,
                                    seed, smudge_bits, part.data_ptr() or None, _stream()), "he_partial_decrypt")
@@ -361,7 +408,9 @@ def he_partial_decrypt(ctx: Ctx, share: Keys, party: int, ct: torch.Tensor, leve
 
 
 def he_threshold_combine(ctx: Ctx, ct: torch.Tensor, level: int, parts: List[torch.Tensor]) -> torch.Tensor:
-    T = ct.shape[0]
+    T = _ct_count(ctx, ct, level, "he_threshold_combine ct")
+    for i, p in enumerate(parts):
+        _sized(p, T * ctx.N, "he_threshold_combine parts[%d]" % i, exact=True)
     ptrs = (_vp * len(parts))(*[_dev(p, torch.int64) for p in parts])
     z = torch.empty(T * ctx.n, dtype=torch.float64, device="cuda")
     _check(_lib.he_threshold_combine(ctx.handle, _dev(ct, torch.int64) or None, level, C.cast(ptrs, _vp),
@@ -376,7 +425,8 @@ def he_decrypt_noalloc(ctx: Ctx, keys: Keys, agg: torch.Tensor, out: torch.Tenso
     """he_decrypt without any allocation inside the library: the work buffer is a fixed array
     in the library image, so T * N must not exceed HE_NOALLOC_MAX_WORDS and N must be <= 16384.
     `out` (float64 [T*n]) is supplied by the caller for the same reason."""
-    T = agg.shape[0]
+    T = _ct_count(ctx, agg, ctx.L - 1, "he_decrypt_noalloc agg")
+    _sized(out, T * ctx.n, "he_decrypt_noalloc out")
     _check(_lib.he_decrypt_noalloc(ctx.handle, keys.handle, _dev(agg, torch.int64) or None, T,
                                    _dev(out, torch.float64) or None, _stream()), "he_decrypt_noalloc")
     return out
@@ -384,8 +434,19 @@ def he_decrypt_noalloc(ctx: Ctx, keys: Keys, agg: torch.Tensor, out: torch.Tenso
 
 def he_unpack(ctx: Ctx, mask: Optional[Mask], z: torch.Tensor, rest_avg: Optional[torch.Tensor], P: int,
               out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    k = P
+    if mask is not None:
+        if mask.P != P:
+            raise HeError(HE_ERR_INVALID_ARG, "he_unpack: the mask was built for %d parameters, P is %d" % (mask.P, P))
+        k = mask.k
+        if k < P:
+            if rest_avg is None:
+                raise HeError(HE_ERR_INVALID_ARG, "he_unpack: rest_avg is missing")
+            _sized(rest_avg, P - k, "he_unpack rest_avg")
+    _sized(z, k, "he_unpack z")
     if out is None:
         out = torch.empty(P, dtype=torch.float64, device="cuda")
+    _sized(out, P, "he_unpack out")
     _check(_lib.he_unpack(ctx.handle, mask.handle if mask else None, _dev(z, torch.float64) or None,
                           _dev(rest_avg, torch.float64) if (rest_avg is not None and rest_avg.numel()) else None,
                           P, _dev(out, torch.float64), _stream()), "he_unpack")
@@ -394,12 +455,14 @@ def he_unpack(ctx: Ctx, mask: Optional[Mask], z: torch.Tensor, rest_avg: Optiona
 
 def he_ntt_forward(ctx: Ctx, polys: torch.Tensor) -> torch.Tensor:
     """In place on uint64-as-int64 [B][L][N]."""
+    _sized(polys, (polys.shape[0] if polys.dim() else 0) * ctx.L * ctx.N, "he_ntt_forward polys", exact=True)
     _check(_lib.he_ntt_forward(ctx.handle, _dev(polys, torch.int64), polys.shape[0], _stream()),
            "he_ntt_forward")
     return polys
 
 
 def he_ntt_inverse(ctx: Ctx, polys: torch.Tensor) -> torch.Tensor:
+    _sized(polys, (polys.shape[0] if polys.dim() else 0) * ctx.L * ctx.N, "he_ntt_inverse polys", exact=True)
     _check(_lib.he_ntt_inverse(ctx.handle, _dev(polys, torch.int64), polys.shape[0], _stream()),
            "he_ntt_inverse")
     return polys
@@ -408,8 +471,11 @@ def he_ntt_inverse(ctx: Ctx, polys: torch.Tensor) -> torch.Tensor:
 def he_round_host(ctx: Ctx, keys: Keys, mask: Optional[Mask], xs: List[torch.Tensor],
                   alpha: Sequence[float], enc_seed: int, out: torch.Tensor) -> torch.Tensor:
     """Whole round with HOST tensors in (float32 [P] each, ideally pinned) and out (float64 [P])."""
+    _same_len(xs, alpha, "he_round_host xs and alpha")
     Cn = len(xs)
     P = xs[0].numel()
+    if mask is not None and mask.P != P:
+        raise HeError(HE_ERR_INVALID_ARG, "he_round_host: the mask was built for %d parameters, xs have %d" % (mask.P, P))
     for x in xs:
         if x.is_cuda or x.dtype != torch.float32 or not x.is_contiguous() or x.numel() != P:
             raise TypeError("xs must be contiguous host float32 tensors of one size")

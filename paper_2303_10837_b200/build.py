@@ -79,12 +79,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if force or _stale(tool, [tool_src]):
         subprocess.run([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-o", tool, tool_src],
                        check=True, capture_output=True)
-    loop_src = os.path.join(CSRC, "transform_loop_bench.cu")
-    loop_tool = os.path.join(HERE, "transform_loop_bench")
-    if force or _stale(loop_tool, [loop_src] + headers):
-        subprocess.run([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17",
-                        "--expt-relaxed-constexpr", "-o", loop_tool, loop_src, os.path.join(CSRC, "fedhe_host.cpp"),
-                        "-lquadmath"], check=True, capture_output=True)
     return OUT
 
 

@@ -17,6 +17,8 @@ inline cudaStream_t as_stream(void *s) { return reinterpret_cast<cudaStream_t>(s
 inline bool good(const he_ctx *c) { return c && c->magic == CTX_MAGIC; }
 inline bool good(const he_keys *k) { return k && k->magic == KEYS_MAGIC; }
 inline bool good(const he_mask *m) { return m && m->magic == MASK_MAGIC; }
+// ciphertext-like buffers are read and written with 16-byte accesses
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 #define CU(expr)                                   \
     do {                                           \
@@ -258,6 +260,7 @@ int he_keys_export(he_ctx *ctx, const he_keys *keys, uint64_t *pk_dev, int8_t *s
     const size_t LN = (size_t)d.L * d.N;
     cudaStream_t st = as_stream(stream);
     if (pk_dev) {
+        if (!aligned16(pk_dev)) return HE_ERR_INVALID_ARG;
         // pk0^ and pk1^ are adjacent in the key storage
         CU(launch_extract_values(keys->dev.pk0_hat, pk_dev, 2 * LN, st));
         CU(launch_ntt(d, false, pk_dev, 2, LN, 0, d.L, st));
@@ -431,7 +434,7 @@ static int encrypt_range(he_ctx *ctx, const he_keys *keys, const float *sel_dev,
     if (!good(ctx) || !good(keys) || keys->ctx != ctx || keys->is_share) return HE_ERR_INVALID_ARG;
     if (t_begin + t_count >= (1ull << 32)) return HE_ERR_SIZE;
     if (t_count == 0) return HE_OK;
-    if (!sel_dev || !ct_dev) return HE_ERR_INVALID_ARG;
+    if (!sel_dev || !ct_dev || !aligned16(ct_dev)) return HE_ERR_INVALID_ARG;
     const CtxDev &d = ctx->dev;
     // transform-domain output on the long rings transforms u in a work buffer of its own
     const size_t u_words = (ntt_out && d.A > 0) ? t_count * (size_t)d.L * d.N : 0;
@@ -470,7 +473,7 @@ static int weighted_aggregate(he_ctx *ctx, const uint64_t *const *cts_host, cons
                               size_t T, bool ntt, uint64_t *agg_dev, void *stream) {
     if (!good(ctx) || !cts_host || !alpha_host || C < 1) return HE_ERR_INVALID_ARG;
     if (C > HE_MAX_CLIENTS) return HE_ERR_SIZE;
-    if (T && !agg_dev) return HE_ERR_INVALID_ARG;
+    if (T && (!agg_dev || !aligned16(agg_dev))) return HE_ERR_INVALID_ARG;
     const CtxDev &d = ctx->dev;
     const uint32_t L = d.L;
     // weights as constant polynomials at scale q_{L-1}: W_i = rint(alpha_i * q_{L-1})
@@ -479,7 +482,7 @@ static int weighted_aggregate(he_ctx *ctx, const uint64_t *const *cts_host, cons
     const uint64_t **ptrs = reinterpret_cast<const uint64_t **>(host.data());
     tw_t *wt = reinterpret_cast<tw_t *>(host.data() + C * sizeof(void *));
     for (int i = 0; i < C; i++) {
-        if (T && !cts_host[i]) return HE_ERR_INVALID_ARG;
+        if (T && (!cts_host[i] || !aligned16(cts_host[i]))) return HE_ERR_INVALID_ARG;
         const double a = alpha_host[i];
         if (!(a >= 0.0) || !(a <= 1.0)) return HE_ERR_INVALID_ARG;
         const double prod = a * ql;
@@ -544,7 +547,7 @@ static int decrypt_level(he_ctx *ctx, const he_keys *keys, const uint64_t *ct_de
     if (!good(ctx) || !good(keys) || keys->ctx != ctx || keys->is_share) return HE_ERR_INVALID_ARG;
     if (level < 1 || level > ctx->dev.L) return HE_ERR_LEVEL;
     if (T == 0) return HE_OK;
-    if (!ct_dev || !z_dev) return HE_ERR_INVALID_ARG;
+    if (!ct_dev || !z_dev || !aligned16(ct_dev)) return HE_ERR_INVALID_ARG;
     const CtxDev &d = ctx->dev;
     if (d.logN <= 14) {                 // one fused kernel, no work buffer
         CU(launch_decrypt_fused(d, keys->dev, ct_dev, level, T, ntt_in, z_dev, as_stream(stream)));
@@ -591,7 +594,7 @@ int he_unpack(he_ctx *ctx, const he_mask *mask, const double *z_dev, const doubl
 }
 
 int he_ntt_forward(he_ctx *ctx, uint64_t *polys_dev, size_t B, void *stream) {
-    if (!good(ctx) || !polys_dev) return HE_ERR_INVALID_ARG;
+    if (!good(ctx) || !polys_dev || !aligned16(polys_dev)) return HE_ERR_INVALID_ARG;
     const CtxDev &d = ctx->dev;
     if ((B * d.L) >> (31 - d.A)) return HE_ERR_SIZE;
     CU(launch_ntt(d, true, polys_dev, B, (size_t)d.L * d.N, 0, d.L, as_stream(stream)));
@@ -599,7 +602,7 @@ int he_ntt_forward(he_ctx *ctx, uint64_t *polys_dev, size_t B, void *stream) {
 }
 
 int he_ntt_inverse(he_ctx *ctx, uint64_t *polys_dev, size_t B, void *stream) {
-    if (!good(ctx) || !polys_dev) return HE_ERR_INVALID_ARG;
+    if (!good(ctx) || !polys_dev || !aligned16(polys_dev)) return HE_ERR_INVALID_ARG;
     const CtxDev &d = ctx->dev;
     if ((B * d.L) >> (31 - d.A)) return HE_ERR_SIZE;
     CU(launch_ntt(d, false, polys_dev, B, (size_t)d.L * d.N, 0, d.L, as_stream(stream)));
@@ -663,7 +666,7 @@ int he_partial_decrypt(he_ctx *ctx, const he_keys *share, uint32_t party, const 
     if (level < 1 || level > ctx->dev.L) return HE_ERR_LEVEL;
     if (smudge_bits > 40 || T >= (1ull << 32)) return HE_ERR_SIZE;
     if (T == 0) return HE_OK;
-    if (!ct_dev || !part_dev) return HE_ERR_INVALID_ARG;
+    if (!ct_dev || !part_dev || !aligned16(ct_dev) || !aligned16(part_dev)) return HE_ERR_INVALID_ARG;
     CU(launch_partial_decrypt(ctx->dev, share->dev, party, ct_dev, level, T, seed, smudge_bits, part_dev,
                               as_stream(stream)));
     return HE_OK;
@@ -675,10 +678,10 @@ int he_threshold_combine(he_ctx *ctx, const uint64_t *ct_dev, uint32_t level, co
     if (nparts > 8) return HE_ERR_SIZE;
     if (level < 1 || level > ctx->dev.L) return HE_ERR_LEVEL;
     if (T == 0) return HE_OK;
-    if (!ct_dev || !z_dev) return HE_ERR_INVALID_ARG;
+    if (!ct_dev || !z_dev || !aligned16(ct_dev)) return HE_ERR_INVALID_ARG;
     PartPtrs pp = {};
     for (int p = 0; p < nparts; p++) {
-        if (!parts_host[p]) return HE_ERR_INVALID_ARG;
+        if (!parts_host[p] || !aligned16(parts_host[p])) return HE_ERR_INVALID_ARG;
         pp.p[p] = parts_host[p];
     }
     void *ws = nullptr;
@@ -696,17 +699,10 @@ int he_threshold_combine(he_ctx *ctx, const uint64_t *ct_dev, uint32_t level, co
 // whole round from host memory
 // ---------------------------------------------------------------------------
 
-int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const float *const *xs_host,
-                  const double *alpha_host, int C, size_t P, uint64_t enc_seed, double *w_glob_host,
-                  void *stream) {
-    if (!good(ctx) || !good(keys) || keys->ctx != ctx || keys->is_share || !xs_host || !alpha_host || !w_glob_host || C < 1 || P == 0)
-        return HE_ERR_INVALID_ARG;
-    if (C > HE_MAX_CLIENTS) return HE_ERR_SIZE;
-    size_t k = P;
-    if (mask) {
-        if (!good(mask) || mask->P != P) return HE_ERR_INVALID_ARG;
-        k = mask->k;
-    }
+// The queued part of he_round_host; every argument has been validated.
+static int round_host_queued(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const float *const *xs_host,
+                             const double *alpha_host, int C, size_t P, size_t k, uint64_t enc_seed,
+                             double *w_glob_host, void *stream) {
     const CtxDev &d = ctx->dev;
     const size_t n = d.N / 2, T = he_num_ct(ctx, k), padded = T * n, restlen = P - k;
     const size_t ctw = 2 * (size_t)d.L * d.N, aggw = 2 * (size_t)(d.L - 1) * d.N;
@@ -758,8 +754,6 @@ int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const f
         }
         CU(cudaEventCreateWithFlags(&ctx->ev_chunk, cudaEventDisableTiming));
     }
-    for (int i = 0; i < C; i++)
-        if (!xs_host[i]) return HE_ERR_INVALID_ARG;
     // The upload of client i+1 (copy stream, two staging buffers) overlaps
     // the packing of client i and the encryption of its first chunk.
     CU(cudaEventRecord(ctx->ev_free[0], st));       // earlier work on `st` may still use the buffers
@@ -815,11 +809,7 @@ int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const f
                                ctx->copy_stream));
         }
     }
-    if (!mask) {
-        CU(cudaStreamSynchronize(ctx->copy_stream));
-        CU(cudaStreamSynchronize(st));
-        return HE_OK;
-    }
+    if (!mask) return HE_OK;                        // the caller waits for both streams
     if (restlen) {
         std::vector<const float *> rptr(rest.begin(), rest.end());
         rc = he_plain_aggregate(ctx, rptr.data(), alpha_host, C, restlen, ravg, stream);
@@ -828,8 +818,32 @@ int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const f
     rc = he_unpack(ctx, mask, z, restlen ? ravg : nullptr, P, out, stream);
     if (rc != HE_OK) return rc;
     CU(cudaMemcpyAsync(w_glob_host, out, P * sizeof(double), cudaMemcpyDeviceToHost, st));
-    CU(cudaStreamSynchronize(st));
     return HE_OK;
+}
+
+int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const float *const *xs_host,
+                  const double *alpha_host, int C, size_t P, uint64_t enc_seed, double *w_glob_host,
+                  void *stream) {
+    // everything that can be refused is refused here, before anything is queued
+    if (!good(ctx) || !good(keys) || keys->ctx != ctx || keys->is_share || !xs_host || !alpha_host || !w_glob_host || C < 1 || P == 0)
+        return HE_ERR_INVALID_ARG;
+    if (C > HE_MAX_CLIENTS) return HE_ERR_SIZE;
+    size_t k = P;
+    if (mask) {
+        if (!good(mask) || mask->P != P) return HE_ERR_INVALID_ARG;
+        k = mask->k;
+    }
+    for (int i = 0; i < C; i++) {
+        if (!xs_host[i]) return HE_ERR_INVALID_ARG;
+        if (!(alpha_host[i] >= 0.0) || !(alpha_host[i] <= 1.0)) return HE_ERR_INVALID_ARG;
+    }
+    const int rc = round_host_queued(ctx, keys, mask, xs_host, alpha_host, C, P, k, enc_seed, w_glob_host, stream);
+    // Success or not, nothing may still be reading xs or writing w_glob when the
+    // call returns: wait for both streams (on an error path their status is ignored).
+    cudaError_t e0 = ctx->copy_stream ? cudaStreamSynchronize(ctx->copy_stream) : cudaSuccess;
+    cudaError_t e1 = cudaStreamSynchronize(as_stream(stream));
+    if (rc != HE_OK) return rc;
+    return (e0 == cudaSuccess && e1 == cudaSuccess) ? HE_OK : HE_ERR_CUDA;
 }
 
 }  // extern "C"

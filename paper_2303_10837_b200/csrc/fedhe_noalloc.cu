@@ -60,7 +60,7 @@ extern "C" int he_decrypt_noalloc(he_ctx *ctx, const he_keys *keys, const uint64
     if (d.N > 16384) return HE_ERR_SIZE;
     if (T > HE_NOALLOC_MAX_WORDS / d.N) return HE_ERR_SIZE;
     if (T == 0) return HE_OK;
-    if (!agg_dev || !z_dev) return HE_ERR_INVALID_ARG;
+    if (!agg_dev || !z_dev || (reinterpret_cast<uintptr_t>(agg_dev) & 15u)) return HE_ERR_INVALID_ARG;
     uint64_t *scratch = nullptr;
     const int rc = scratch_for_current_device(&scratch);
     if (rc != HE_OK) return rc;

@@ -67,11 +67,20 @@ def test_keygen_bit_exact(he, N, primes):
 
 # --------------------------------------------------------------------------- encode / encrypt
 
+def long_ring(name, primes, P, clients=2):
+    """N = 65536 (the longest ring of the kernel sweep): the transform is cut into 8 blocks."""
+    return si.Workload(name, 65536, tuple(primes), 40, clients, P, 0.01, seed=6, key_seed=61, enc_seed=62)
+
+
 def workload_cases():
     return [
         si.scaled(si.TINY, 2 * 4096 + 101, name="tiny-ragged"),               # N=8192, 3 cts, ragged tail
         si.scaled(si.RESNET18, 3 * 8192 - 7, clients=3, name="r18-ragged"),    # N=16384, L=4
         si.scaled(si.bert(1.0), 16384 + 33, clients=2, name="bert-ragged"),    # N=32768, L=6, Delta=2^45
+        # N=65536: three 60-bit primes (integer limbs), three 45-bit primes (limbs in doubles), mixed
+        long_ring("n65536-int", si.PRIMES_SWEEP[:3], 32768 + 77),
+        long_ring("n65536-f64", si.PRIMES_SWEEP_45[:3], 2 * 32768 - 5),
+        long_ring("n65536-mixed", (si.PRIMES_SWEEP[0], si.PRIMES_SWEEP_45[0], si.PRIMES_SWEEP[1]), 32768 + 1),
     ]
 
 
@@ -147,7 +156,10 @@ def test_encrypt_aggregate_decrypt_bit_exact(he, w):
     assert he.he_ctx_status(g) == he.HE_OK
 
 
-@pytest.mark.parametrize("base", [si.TINY, si.RESNET18, si.bert(1.0)], ids=lambda w: w.name)
+@pytest.mark.parametrize("base", [si.TINY, si.RESNET18, si.bert(1.0),
+                                  long_ring("n65536-mixed-large", (si.PRIMES_SWEEP[0], si.PRIMES_SWEEP_45[0],
+                                                                   si.PRIMES_SWEEP[1]), 32768)],
+                         ids=lambda w: w.name)
 def test_encrypt_large_messages_bit_exact(he, base):
     """Encoded coefficients above the small primes and close to the large ones: the full
     reduction of m + e0 and every wrap of the final additions, next to a ciphertext of
@@ -401,6 +413,73 @@ def test_empty_and_degenerate_inputs(he):
     assert ei.value.code == he.HE_ERR_INVALID_ARG
 
 
+def test_unaligned_word_buffers_are_refused(he):
+    """Ciphertext-like buffers are moved two words at a time: a pointer at an odd word offset comes
+    back as an error from the host-side check, never as a misaligned access on the device."""
+    w = si.scaled(si.TINY, 4096, clients=1)
+    g, _ = contexts(he, w.N, w.primes, w.log2_delta)
+    keys = he.he_keygen(g, 1)
+    sel, _ = he.he_pack(g, None, dev_f32(si.client_update(w, 0)))
+
+    def odd(shape):
+        count = int(np.prod(shape))
+        return torch.zeros(count + 1, dtype=torch.int64, device="cuda")[1:].view(shape)
+
+    ct = he.he_encrypt(g, keys, sel, 1, 0)
+    agg = he.he_weighted_aggregate(g, [ct], [1.0])
+    ct_odd, agg_odd = odd(ct.shape), odd(agg.shape)
+    ct_odd.copy_(ct)
+    agg_odd.copy_(agg)
+    assert ct_odd.data_ptr() % 16 == 8
+    calls = [
+        lambda: he.he_encrypt(g, keys, sel, 1, 0, out=ct_odd),
+        lambda: he.he_encrypt_ntt(g, keys, sel, 1, 0, out=ct_odd),
+        lambda: he.he_weighted_aggregate(g, [ct_odd], [1.0]),
+        lambda: he.he_weighted_aggregate(g, [ct], [1.0], out=agg_odd),
+        lambda: he.he_decrypt(g, keys, agg_odd),
+        lambda: he.he_decrypt_level(g, keys, ct_odd, w.L),
+        lambda: he.he_decrypt_noalloc(g, keys, agg_odd, torch.empty(w.n, dtype=torch.float64, device="cuda")),
+        lambda: he.he_ntt_forward(g, odd((1, w.L, w.N))),
+        lambda: he.he_ntt_inverse(g, odd((1, w.L, w.N))),
+    ]
+    for call in calls:
+        with pytest.raises(he.HeError) as ei:
+            call()
+        assert ei.value.code == he.HE_ERR_INVALID_ARG
+    # the context is as usable as before
+    z = he.he_decrypt(g, keys, agg).cpu().numpy()
+    assert np.abs(z[: w.P] - si.client_update(w, 0).astype(np.float64)).max() <= FEDAVG_TOL
+
+
+def test_host_round_refuses_bad_arguments_before_queueing(he):
+    """A missing client buffer or a weight outside [0, 1] is an error return with nothing queued,
+    and the same context then runs a correct round."""
+    import ctypes as C
+    w = si.scaled(si.TINY, 3 * 4096 + 5, clients=3)
+    g, _ = contexts(he, w.N, w.primes, w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    xs, alpha = si.client_updates(w), si.client_weights(w)
+    xs_t = [torch.from_numpy(x).pin_memory() for x in xs]
+    host = torch.full((w.P,), np.nan, dtype=torch.float64).pin_memory()
+    lib = C.CDLL(he.LIB_PATH)
+    lib.he_round_host.restype = C.c_int
+    lib.he_round_host.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_size_t,
+                                  C.c_uint64, C.c_void_p, C.c_void_p]
+    al = (C.c_double * 3)(*[float(a) for a in alpha])
+    ptrs = (C.c_void_p * 3)(xs_t[0].data_ptr(), None, xs_t[2].data_ptr())          # client 1 is missing
+    before = he.he_launch_count()
+    rc = lib.he_round_host(g.handle, keys.handle, None, C.cast(ptrs, C.c_void_p), C.cast(al, C.c_void_p), 3, w.P,
+                           w.enc_seed, host.data_ptr(), None)
+    assert rc == he.HE_ERR_INVALID_ARG and he.he_launch_count() == before
+    assert bool(torch.isnan(host).all())                                             # nothing was written
+    with pytest.raises(he.HeError) as ei:
+        he.he_round_host(g, keys, None, xs_t, [0.5, 0.7, -0.2], w.enc_seed, host)
+    assert ei.value.code == he.HE_ERR_INVALID_ARG and he.he_launch_count() == before
+    he.he_round_host(g, keys, None, xs_t, alpha, w.enc_seed, host)
+    want = sum(a * x.astype(np.float64) for a, x in zip(alpha, xs))
+    assert np.abs(host.numpy() - want).max() <= FEDAVG_TOL
+
+
 def test_runs_are_deterministic(he):
     """Bit-identical outputs on repeated runs (a race would show up here)."""
     w = si.scaled(si.RESNET18, 5 * 8192, clients=2)
@@ -448,7 +527,9 @@ def test_sensitivity_map_round(he):
 
 
 @pytest.mark.parametrize("w", [si.scaled(si.TINY, 4096 + 50, name="thr-tiny"),
-                               si.scaled(si.bert(1.0), 16384 + 9, clients=2, name="thr-bert")],
+                               si.scaled(si.bert(1.0), 16384 + 9, clients=2, name="thr-bert"),
+                               long_ring("thr-n65536", (si.PRIMES_SWEEP[0], si.PRIMES_SWEEP_45[0],
+                                                        si.PRIMES_SWEEP[1]), 32768 + 3)],
                          ids=lambda w: w.name)
 def test_threshold_decryption_bit_exact(he, w):
     """Two-party threshold decryption: partial results bit-exact against the oracle, merged result

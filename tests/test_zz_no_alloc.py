@@ -71,3 +71,36 @@ def test_noalloc_decrypt_rejects_what_does_not_fit():
     with pytest.raises(he.HeError) as ei:
         he.he_decrypt_noalloc(gb, kb, aggb, torch.empty(b.n, dtype=torch.float64, device="cuda"))
     assert ei.value.code == he.HE_ERR_SIZE
+
+
+def test_noalloc_decrypt_smallest_ring_and_its_limit():
+    """N = 8192: up to 256 ciphertexts fit the fixed array; 257 are refused, 256 give he_decrypt's result."""
+    import paper_2303_10837_b200 as he
+    w = si.scaled(si.TINY, 256 * 4096 - 11, clients=2, name="noalloc-8192")
+    g = he.he_ctx_create(w.N, list(w.primes), w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    alpha = si.client_weights(w)
+    cts = [he.he_encrypt(g, keys, he.he_pack(g, None, torch.from_numpy(si.client_update(w, i)).cuda())[0], 5, i)
+           for i in range(w.clients)]
+    agg = he.he_weighted_aggregate(g, cts, alpha)
+    assert agg.shape[0] == 256 == he.HE_NOALLOC_MAX_WORDS // w.N
+    want = he.he_decrypt(g, keys, agg)
+    out = torch.empty_like(want)
+    he.he_decrypt_noalloc(g, keys, agg, out)
+    he.he_decrypt_noalloc(g, keys, agg, out)          # again, over the array the first call left behind
+    torch.cuda.synchronize()
+    assert float((out - want).abs().max()) <= DECODE_TOL
+    more = torch.zeros((257, 2, w.L - 1, w.N), dtype=torch.int64, device="cuda")
+    with pytest.raises(he.HeError) as ei:
+        he.he_decrypt_noalloc(g, keys, more, torch.empty(257 * w.n, dtype=torch.float64, device="cuda"))
+    assert ei.value.code == he.HE_ERR_SIZE
+    # nothing to do is not an error; a missing buffer is
+    empty = torch.zeros((0, 2, w.L - 1, w.N), dtype=torch.int64, device="cuda")
+    he.he_decrypt_noalloc(g, keys, empty, torch.empty(0, dtype=torch.float64, device="cuda"))
+    import ctypes as C
+    lib = C.CDLL(he.LIB_PATH)
+    lib.he_decrypt_noalloc.restype = C.c_int
+    lib.he_decrypt_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+    assert lib.he_decrypt_noalloc(g.handle, keys.handle, None, 1, out.data_ptr(), None) == he.HE_ERR_INVALID_ARG
+    assert lib.he_decrypt_noalloc(g.handle, keys.handle, agg.data_ptr(), 1, None, None) == he.HE_ERR_INVALID_ARG
+    assert he.he_ctx_status(g) == he.HE_OK
