@@ -204,13 +204,20 @@ int he_weighted_aggregate_ntt(he_ctx *ctx, const uint64_t *const *cts_host, cons
 int he_decrypt_level_ntt(he_ctx *ctx, const he_keys *keys, const uint64_t *ct_dev, uint32_t level, size_t T,
                          double *z_dev, void *stream);
 
-/* (No counterpart in the paper.)  he_decrypt for callers that must not
+/* (No counterpart in the paper.)  Decryption for callers that must not
  * allocate: a process that has given all free device memory to its own pool,
  * or a latency-critical loop that cannot take the device-wide synchronisation
- * of cudaMalloc/cudaFree.  Same arguments and result as he_decrypt, but the
- * work buffer is a fixed 16 MiB array inside the library image (present on
- * every GPU that loads the library until the process exits), so the call
- * issues no cudaMalloc, cudaFree or allocating library routine.
+ * of cudaMalloc/cudaFree.  Same arguments and result as he_decrypt.  It runs
+ * the multi-kernel decryption path (the one he_decrypt takes on rings above
+ * N = 16384, where it may grow the context's work buffer), with the work
+ * buffer a fixed 16 MiB array inside the library image (present on every GPU
+ * that loads the library until the process exits), so the call issues no
+ * cudaMalloc, cudaFree or allocating library routine whatever kernels the
+ * library picks.  On the rings it accepts, he_decrypt itself is one fused
+ * kernel without a work buffer, allocates nothing either and is faster; this
+ * call costs about three more passes over T * N words.
+ *   A cudaDeviceReset by the caller invalidates the cached address of the
+ *   array together with every handle of the library.
  *   Limits: N <= 16384 and T * N <= HE_NOALLOC_MAX_WORDS (T <= 128 at
  *   N = 16384, T <= 256 at N = 8192); anything larger returns HE_ERR_SIZE.
  *   The context's GPU must be the current device (HE_ERR_INVALID_ARG).

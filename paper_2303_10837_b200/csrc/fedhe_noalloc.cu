@@ -1,19 +1,29 @@
-// he_decrypt_noalloc: decryption whose work buffer is a fixed array inside the
+// he_decrypt_noalloc: the multi-kernel decryption path (gather, transform, key
+// product, inverse transform, centring, slot transform), whose intermediate
+// polynomials need a work buffer, with that buffer a fixed array inside the
 // library image instead of memory obtained from the CUDA allocator.
 //
 // Who needs it: a caller that has handed all remaining device memory to its
 // own pool (a serving process with a pre-partitioned HBM budget, a job under
 // a hard memory cap) cannot let a library call cudaMalloc behind its back,
 // and a caller inside a latency-critical loop cannot afford the device-wide
-// synchronisation that cudaMalloc/cudaFree imply.  he_decrypt may grow the
-// context's work buffer on a call with a larger T than before; this entry
-// point never allocates, at the price of a size limit.
+// synchronisation that cudaMalloc/cudaFree imply.  For the rings this entry
+// point accepts (N <= 16384) he_decrypt itself runs one fused kernel that needs
+// no work buffer and allocates nothing either, and is the faster call; the
+// multi-kernel path is what he_decrypt uses on the longer rings, where it may
+// grow the context's work buffer.  This entry point gives a caller that path
+// with a guarantee that does not depend on which kernel the library picks: it
+// never allocates, at the price of a size limit and of about three extra
+// passes over T * N words.
 //
 // The array costs HE_NOALLOC_MAX_WORDS * 8 bytes (16 MiB) on every GPU that
 // loads the library, until the process exits.  All calls on a device share
 // it and it keeps whatever the previous call left there: nothing in it has to
 // start at zero (every word that is read was written earlier in the same
 // call), but two calls that overlap on the GPU (different streams) race.
+// The array's device address is looked up once per device and kept for the
+// life of the process; a caller that resets the device (cudaDeviceReset)
+// invalidates it together with every context and key handle of the library.
 #include <mutex>
 
 #include "fedhe_launch.h"
