@@ -11,9 +11,19 @@ region.  ``--impl reference`` times the CPU oracle instead.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-For N > 1 launch under ``torch.distributed.run``; every rank processes its own
-full batch (ciphertext indices are independent, so the path shards with no
-collective) and the job time is the maximum over ranks.
+The default line carries the ResNet-18-sized workload (``value``) and, under
+``workloads``, the ResNet-50-sized top-10 % round and the BERT-sized round at
+100 % encryption (streamed in chunks of ciphertext indices), each with its own
+time, roofline block, host-buffer leg and clocks.
+
+For N > 1 launch under ``torch.distributed.run``.  ``--shard index`` (default):
+ONE round is cut over the ranks, rank r taking the contiguous ciphertext
+indices [T r / N, T (r+1) / N) and the same share of the plaintext remainder,
+with context, keys and mask replicated and no collective on the path
+(``--gather`` adds the one all-gather of the decoded pieces, for when one
+place needs the whole model); fixed total work, "scaling": "strong".
+``--shard batch``: every rank runs its own full round ("weak").  The job time
+is the maximum over ranks either way.
 """
 from __future__ import annotations
 
@@ -48,10 +58,11 @@ UNIT = "params/s"
 # operations for the modular product, 2 for the sum and difference, and in the
 # inverse transform 1 more per butterfly for keeping the sums small.
 # Additions, shifts and logic go to another pipe.
-# DRAM bytes (read + write) per ciphertext of encrypt_fused2_kernel at N = 16384,
-# L = 4, from an ncu capture of the profile_case.py encrypt case (summary under profiles/)
-# (363.1 MB for 296 ciphertexts; traffic grows in proportion to the count).
-ENCRYPT_DRAM_BYTES_PER_CT_N16384_L4 = 363.052288e6 / 296
+# DRAM bytes (read + write) per ciphertext of the encrypt kernel, by (N, L), from ncu captures of
+# the profile_case.py encrypt case (summaries under profiles/; traffic grows in proportion to the
+# number of ciphertexts).  An entry is dropped (None is reported) when the kernel has changed
+# since its counters were taken.
+ENCRYPT_DRAM_BYTES_PER_CT = {(16384, 4): 363.052288e6 / 296}
 SLOTS_PER_SM_CLK = 64.0
 WIDE_COST = 2.5
 INT_SLOTS_PER_BUTTERFLY = 6 * WIDE_COST + 4
@@ -217,138 +228,173 @@ def config_dict(w, note):
 
 # --------------------------------------------------------------------------- GPU arm
 
-def run_ours(args, w):
-    import torch
-    import torch.distributed as dist
-    import paper_2303_10837_b200 as he
+class Job:
+    """Process-wide state of one bench run."""
 
-    rank, world, local = dist_env()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    peaks = read_peaks()
+    def __init__(self, args):
+        import torch
+        import torch.distributed as dist
+        self.torch, self.dist = torch, dist
+        self.rank, self.world, self.local = dist_env()
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+        torch.cuda.set_device(self.local)
+        if self.world > 1:
+            dist.init_process_group("nccl", device_id=torch.device("cuda", self.local))
+        self.peaks = read_peaks()
+        self.n_sm = torch.cuda.get_device_properties(self.local).multi_processor_count
+        self.args = args
+
+    def barrier(self):
+        self.torch.cuda.synchronize()
+        if self.world > 1:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+
+def measure(job, w, steps, warmup, with_cpu_baseline):
+    """One workload: W warm-up rounds, K timed rounds, the dominant kernel's roofline, the
+    host-buffer leg.  Returns the fields of a bench line for this workload (rank 0) or None."""
+    import paper_2303_10837_b200 as he
+    from paper_2303_10837_b200.sharding import even_edges, gather_pieces, shard_range, slot_edges, slot_range
+    torch, args = job.torch, job.args
+    rank, world = job.rank, job.world
+    by_index = world > 1 and args.shard == "index"
+    transform = args.format == "transform"
 
     g = he.he_ctx_create(w.N, list(w.primes), w.log2_delta)
     keys = he.he_keygen(g, w.key_seed)
     alpha = si.client_weights(w)
-    enc_seed = w.enc_seed + 1000 * rank
-    # inputs: every rank has its own batch (weak scaling)
+    T, n = w.T, w.n
+    # what this rank works on: everything (one GPU, or one batch per rank), or its range of one round
+    if by_index:
+        tb, te, sb, se = slot_range(T, n, w.k, rank, world)
+        rb, re = shard_range(w.P - w.k, rank, world)
+        batch_seed, enc_seed = 0, w.enc_seed
+    else:
+        tb, te, sb, se = 0, T, 0, w.k
+        rb, re = 0, w.P - w.k
+        batch_seed, enc_seed = rank, w.enc_seed + 1000 * rank
+    Tr = te - tb
     xs_host = []
     for i in range(w.clients):
-        rng = np.random.default_rng([w.seed, 1000 + i, rank])
+        rng = np.random.default_rng([w.seed, 1000 + i, batch_seed])
         x = rng.standard_normal(w.P, dtype=np.float32)
         x *= np.float32(w.std)
         xs_host.append(torch.from_numpy(x).pin_memory())
     xs = [x.cuda() for x in xs_host]
-    mask = None
+    mask, idx = None, None
     if w.k < w.P:
         mask = he.he_select_mask(g, torch.from_numpy(si.sensitivity_scores(w)).cuda(), w.k)
-    T, n = w.T, w.n
-    # ciphertext indices are streamed in chunks when all clients' ciphertexts exceed 40 GB
+        idx = he.he_mask_indices(mask).long()
+    # ciphertext indices are streamed in chunks when all clients' ciphertexts of this rank exceed 40 GB
     ct_bytes = 8 * 2 * w.L * w.N
-    Tc = T
-    if w.clients * T * ct_bytes > 40e9:
-        n_sm = torch.cuda.get_device_properties(local).multi_processor_count
-        Tc = max(n_sm, int(16e9 // (w.clients * ct_bytes)) // n_sm * n_sm)
+    Tc = max(Tr, 1)
+    if w.clients * Tr * ct_bytes > 40e9:
+        Tc = max(job.n_sm, int(16e9 // (w.clients * ct_bytes)) // job.n_sm * job.n_sm)
+    if transform and (Tc < Tr or by_index):
+        raise SystemExit("bench: --format transform is wired to the whole, unchunked round only")
     cts = [torch.empty((Tc, 2, w.L, w.N), dtype=torch.int64, device="cuda") for _ in range(w.clients)]
     agg = torch.empty((Tc, 2, w.L - 1, w.N), dtype=torch.int64, device="cuda")
-    z = torch.empty(T * n, dtype=torch.float64, device="cuda")
+    z = torch.empty(Tr * n, dtype=torch.float64, device="cuda")
     out = torch.empty(w.P, dtype=torch.float64, device="cuda")
-    he.he_ctx_reserve(g, w.k)
+    he.he_ctx_reserve(g, min(Tr, Tc) * n)
     enc_events = []
+    result = {}
 
-    def step_streamed(record):
-        sels = [he.he_pack(g, mask, xs[i])[0] for i in range(w.clients)]
-        for t0 in range(0, T, Tc):
-            tc = min(Tc, T - t0)
+    def step(record):
+        sels, rests = [], []
+        for i in range(w.clients):
+            if by_index and mask is None:           # full encryption: the rank's slots are a slice of x
+                sel, rest = he.he_pack(g, None, xs[i][sb:se])
+            else:
+                sel, rest = he.he_pack(g, mask, xs[i])
+                sel = sel[tb * n:te * n]
+            sels.append(sel)
+            rests.append(rest[rb:re] if rest is not None else None)
+        for t0 in range(0, Tr, Tc):
+            tc = min(Tc, Tr - t0)
             for i in range(w.clients):
                 if record:
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     e0.record()
-                he.he_encrypt_range(g, keys, sels[i][t0 * n:(t0 + tc) * n], t0, tc, enc_seed, i, cts[i][:tc])
+                if transform:
+                    he.he_encrypt_ntt(g, keys, sels[i], enc_seed, i, out=cts[i])
+                else:
+                    he.he_encrypt_range(g, keys, sels[i][t0 * n:(t0 + tc) * n], tb + t0, tc, enc_seed, i, cts[i][:tc])
                 if record:
                     e1.record()
                     enc_events.append((e0, e1, tc))
-            he.he_weighted_aggregate(g, [c[:tc] for c in cts], alpha, out=agg[:tc])
-            he.he_decrypt(g, keys, agg[:tc], out=z[t0 * n:(t0 + tc) * n])
-        he.he_unpack(g, mask, z, None, w.P, out=out)
-
-    transform = args.format == "transform"
-    if transform and Tc < T:
-        raise SystemExit("bench: --format transform is not wired to the streamed (chunked) round")
-    enc = he.he_encrypt_ntt if transform else he.he_encrypt
-
-    def step(record):
-        if Tc < T:
-            return step_streamed(record)
-        rests = []
-        for i in range(w.clients):
-            sel, rest = he.he_pack(g, mask, xs[i])
-            if record:
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-            enc(g, keys, sel, enc_seed, i, out=cts[i])
-            if record:
-                e1.record()
-                enc_events.append((e0, e1, T))
-            rests.append(rest)
-        if transform:
-            he.he_weighted_aggregate_ntt(g, cts, alpha, out=agg)
-            he.he_decrypt_level_ntt(g, keys, agg, w.L - 1, out=z)
+            if transform:
+                he.he_weighted_aggregate_ntt(g, cts, alpha, out=agg)
+                he.he_decrypt_level_ntt(g, keys, agg, w.L - 1, out=z)
+            else:
+                he.he_weighted_aggregate(g, [c[:tc] for c in cts], alpha, out=agg[:tc])
+                he.he_decrypt(g, keys, agg[:tc], out=z[t0 * n:(t0 + tc) * n])
+        avg = he.he_plain_aggregate(g, rests, alpha) if (mask is not None and re > rb) else None
+        if by_index:
+            # the rank's part of the model: z[: se - sb] and avg; gathered only on request
+            if args.gather:
+                zf = gather_pieces(z[: se - sb], slot_edges(T, n, w.k, world), rank)
+                af = gather_pieces(avg, even_edges(w.P - w.k, world), rank) if mask is not None and w.k < w.P else None
+                he.he_unpack(g, mask, zf, af, w.P, out=out)
+            result["z"], result["avg"] = z, avg
         else:
-            he.he_weighted_aggregate(g, cts, alpha, out=agg)
-            he.he_decrypt(g, keys, agg, out=z)
-        avg = he.he_plain_aggregate(g, rests, alpha) if mask is not None else None
-        he.he_unpack(g, mask, z, avg, w.P, out=out)
+            he.he_unpack(g, mask, z, avg, w.P, out=out)
 
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         step(False)
-    barrier()
-    sampler = ClockSampler(local)
+    job.barrier()
+    sampler = ClockSampler(job.local)
     sampler.start()
     launches0 = he.he_launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
-    for _ in range(args.steps):
+    for _ in range(steps):
         step(True)
     ev1.record()
-    barrier()
+    job.barrier()
     launches = he.he_launch_count() - launches0
     secs = ev0.elapsed_time(ev1) * 1e-3
-    # correctness of what was timed: plaintext FedAvg on every parameter
+    # correctness of what was timed: plaintext FedAvg on every parameter this rank produced
     want = sum(float(a) * x.double() for a, x in zip(alpha, xs))
-    err = float((out - want).abs().max())
+    if by_index and not args.gather:
+        pos = torch.arange(sb, se, device="cuda") if idx is None else idx[sb:se]
+        err = float((result["z"][: se - sb] - want[pos]).abs().max()) if se > sb else 0.0
+        if result["avg"] is not None:
+            comp = torch.ones(w.P, dtype=torch.bool, device="cuda")
+            comp[idx] = False
+            err = max(err, float((result["avg"] - want[comp][rb:re]).abs().max()))
+    else:
+        err = float((out - want).abs().max())
     if not err <= 1e-6 or he.he_ctx_status(g) != he.HE_OK:
         raise SystemExit("bench: aggregate differs from plaintext FedAvg by %g" % err)
 
-    # dominant kernel: the fused encrypt.  Its duration = the event-bracketed
-    # he_encrypt calls of the timed region minus the encode kernel that runs in
-    # the same call, timed alone on the same inputs.
-    # time of all he_encrypt calls of one client (T ciphertexts, one call unless streamed)
-    enc_ms = sum(a.elapsed_time(b) for a, b, _ in enc_events) / (args.steps * w.clients)
-    sel0, _ = he.he_pack(g, mask, xs[0])
+    # Dominant kernel: the encryption.  Duration of one client's he_encrypt calls in the timed
+    # region (CUDA events on the launching stream); where the library still runs the encoder as a
+    # launch of its own inside he_encrypt, that launch, timed alone on the same inputs, is taken off.
+    enc_ms = sum(a.elapsed_time(b) for a, b, _ in enc_events) / (steps * w.clients)
+    sel0 = he.he_pack(g, mask, xs[0])[0][tb * n:te * n]
+    probe = min(Tr, Tc)
+    c0 = he.he_launch_count()
+    he.he_encrypt_range(g, keys, sel0[: probe * n], tb, probe, enc_seed, 0, cts[0][:probe])
+    launches_per_encrypt = he.he_launch_count() - c0
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     reps = 5
-    he.he_encode(g, sel0)
-    e0.record()
-    for _ in range(reps):
+    encode_ms = 0.0
+    if launches_per_encrypt > 1 and Tr:
         he.he_encode(g, sel0)
-    e1.record()
-    torch.cuda.synchronize()
-    encode_ms = e0.elapsed_time(e1) / reps
+        e0.record()
+        for _ in range(reps):
+            he.he_encode(g, sel0)
+        e1.record()
+        torch.cuda.synchronize()
+        encode_ms = e0.elapsed_time(e1) / reps
     kern_ms = max(enc_ms - encode_ms, 1e-6)
 
     # standalone transform: forward + inverse over a batch larger than L2
-    B = 256
+    B = 256 if w.N <= 16384 else 64
     polys = torch.from_numpy(si.random_residues(7, (B, w.L, w.N), w.primes).view(np.int64)).cuda()
     he.he_ntt_forward(g, polys)
     he.he_ntt_inverse(g, polys)
@@ -362,78 +408,130 @@ def run_ours(args, w):
     ntt_ms = e0.elapsed_time(e1) / (2 * reps)
     pass_bytes = 16.0 * w.N * w.L * B * (1 if w.N <= 16384 else 2)
     ntt_gbs = pass_bytes / (ntt_ms * 1e-3) / 1e9
+    del polys
     clocks = sampler.stop()
 
-    # e2e through the host entry point
-    host_out = torch.empty(w.P, dtype=torch.float64).pin_memory()
-    he.he_round_host(g, keys, mask, xs_host, alpha, enc_seed, host_out)          # allocates its buffers
-    barrier()
-    e2e_steps = max(1, min(args.steps, 3))
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        he.he_round_host(g, keys, mask, xs_host, alpha, enc_seed, host_out)
-    torch.cuda.synchronize()
-    e2e_secs = time.perf_counter() - t0
-    if not float((host_out.cuda() - want).abs().max()) <= 1e-6:
-        raise SystemExit("bench: host round differs from plaintext FedAvg")
+    # end to end through the host entry point (pinned host buffers, copies inside the timed region)
+    e2e = None
+    del cts, agg
+    torch.cuda.empty_cache()
+    if not by_index or mask is None:
+        if by_index:
+            xh = [x[sb:se] for x in xs_host]             # the rank's slots are a slice of every update
+            Pe = se - sb
+        else:
+            xh, Pe = xs_host, w.P
+        if Pe:
+            host_out = torch.empty(Pe, dtype=torch.float64).pin_memory()
+            he.he_round_host(g, keys, mask, xh, alpha, enc_seed, host_out)          # allocates its buffers
+            job.barrier()
+            e2e_steps = max(1, min(steps, 3))
+            t0 = time.perf_counter()
+            for _ in range(e2e_steps):
+                he.he_round_host(g, keys, mask, xh, alpha, enc_seed, host_out)
+            torch.cuda.synchronize()
+            e2e_secs = time.perf_counter() - t0
+            ref = want[sb:se] if by_index else want
+            if not float((host_out.cuda() - ref).abs().max()) <= 1e-6:
+                raise SystemExit("bench: host round differs from plaintext FedAvg")
+            e2e = (float(Pe) * e2e_steps, e2e_secs, e2e_steps, 4 * Pe * w.clients, 8 * Pe)
 
-    units, job_secs = reduce_job(float(w.P) * args.steps, secs, world, "cuda")
-    e2e_units, e2e_job = reduce_job(float(w.P) * e2e_steps, e2e_secs, world, "cuda")
+    # whole job: units = parameters every rank produced, time = the slowest rank
+    mine = float(w.P) if not by_index else float((se - sb) + (re - rb))
+    units, job_secs = reduce_job(mine * steps, secs, world, "cuda")
+    e2e_line = None
+    if e2e is not None:
+        eu, es = reduce_job(e2e[0], e2e[1], world, "cuda")
+        e2e_line = {"value": eu / es, "unit": UNIT, "h2d_bytes_per_step": e2e[3], "d2h_bytes_per_step": e2e[4],
+                    "steps": e2e[2]}
+        if by_index:
+            e2e_line["note"] = "per rank: he_round_host on the rank's slice of every update (bytes are per rank)"
+    del xs, xs_host, out, z, mask, keys, g
+    torch.cuda.empty_cache()
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
+        return None
 
     # roofline of the dominant kernel (bound by the multiply / double-precision pipe)
     logN = w.N.bit_length() - 1
-    butterflies = 3 * w.L * (w.N // 2) * logN * T           # per launch: 3 limb transforms per limb
+    per_launch = Tr                                          # ciphertexts of one client's he_encrypt calls
+    butterflies = 3 * w.L * (w.N // 2) * logN * per_launch
     # coefficient format: one forward and two inverse transforms per limb; transform format: three forward
-    achieved = transform_slots(w.primes, w.N, 3 if transform else 1, 0 if transform else 2) * T / (kern_ms * 1e-3) / 1e12
-    n_sm = torch.cuda.get_device_properties(local).multi_processor_count
-    peak = n_sm * SLOTS_PER_SM_CLK * peaks["sm_max_mhz"] * 1e6 / 1e12
-    alg_bytes = (16.0 + 32.0 * w.L) * n * T          # read m, write the ciphertext
+    achieved = transform_slots(w.primes, w.N, 3 if transform else 1, 0 if transform else 2) * per_launch / (kern_ms * 1e-3) / 1e12
+    peak = job.n_sm * SLOTS_PER_SM_CLK * job.peaks["sm_max_mhz"] * 1e6 / 1e12
+    alg_bytes = (4.0 + 32.0 * w.L) * n * per_launch          # read the slots, write the ciphertext
+    if w.N <= 16384:
+        kname = "encrypt_fused2_kernel" if w.N == 16384 else "encrypt_fused_kernel"
+    else:
+        kname = "the kernels of he_encrypt on a long ring (N > 16384), timed as one call"
     roofline = {
-        "kernel": ("encrypt_fused2_kernel" if w.N == 16384 else "encrypt_fused_kernel") if w.N <= 16384
-                  else "enc_block_forward_kernel + ntt_block_kernel (inside he_encrypt)",
+        "kernel": kname,
         "bound": "alu", "achieved": achieved, "peak": peak,
         "unit": "T slots/s (integer-multiply / double-precision pipe)",
         "frac": achieved / peak,
-        "traffic": ENCRYPT_DRAM_BYTES_PER_CT_N16384_L4 * T if (w.N == 16384 and w.L == 4) else None,
+        "traffic": ENCRYPT_DRAM_BYTES_PER_CT.get((w.N, w.L), None) and ENCRYPT_DRAM_BYTES_PER_CT[(w.N, w.L)] * per_launch,
         "algorithmic_bytes": alg_bytes,
-        "ms_per_launch": kern_ms, "launches_per_step": w.clients, "butterflies_per_launch": butterflies,
+        "ms_per_launch": kern_ms, "launches_per_step": w.clients, "kernels_per_he_encrypt": int(launches_per_encrypt),
+        "butterflies_per_launch": butterflies,
         "hbm_gbs_of_kernel": alg_bytes / (kern_ms * 1e-3) / 1e9,
-        "hbm_frac_of_kernel": alg_bytes / (kern_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-        "ntt_standalone": {"gbs": ntt_gbs, "hbm_frac": ntt_gbs / peaks["hbm_gbs"], "ms": ntt_ms,
+        "hbm_frac_of_kernel": alg_bytes / (kern_ms * 1e-3) / 1e9 / job.peaks["hbm_gbs"],
+        "ntt_standalone": {"gbs": ntt_gbs, "hbm_frac": ntt_gbs / job.peaks["hbm_gbs"], "ms": ntt_ms,
                            "batch_polys": B, "bytes_per_launch": pass_bytes,
                            "mul_pipe_frac": (B * transform_slots(w.primes, w.N, 0.5, 0.5)
                                              / (ntt_ms * 1e-3) / 1e12) / peak},
         "f64_limbs": sum(1 for q in w.primes if q < F64_PRIME_LIMIT),
         "peak_source": "multiply / double-precision pipe: SM count x 64 per clock (microbenchmark) x max SM clock; "
-                       + peaks["source"] + " hbm_gbs for the HBM fractions",
+                       + job.peaks["source"] + " hbm_gbs for the HBM fractions",
     }
-
-    cpu_ct = min(w.T, 768)
-    cpu_p, cpu_dt, cores = oracle_sample(w, cpu_ct)
-    cpu = {"value": cpu_p / cpu_dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-           "sample": "first %d of %d ciphertext indices (%d params), all %d clients, %.1f s" % (cpu_ct, w.T, cpu_p, w.clients, cpu_dt)}
-
-    line = {
-        "metric": METRIC, "value": units / job_secs, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": 1e3 * job_secs / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "u64 (limbs below 2^46: exact f64)", "data": "synthetic",
-        "config": dict(config_dict(w, "every rank runs its own full batch; no collective on the path"),
-                       format=args.format),
-        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"] or peaks["sm_max_mhz"],
+    if by_index:
+        note = ("one round cut over %d ranks by ciphertext index (rank r: [T r / N, T (r+1) / N) and the same share of "
+                "the plaintext remainder); no collective on the path%s" % (world, "; decoded pieces all-gathered" if args.gather else ""))
+    elif world > 1:
+        note = "every rank runs its own full batch; no collective on the path"
+    else:
+        note = "one GPU"
+    fields = {
+        "value": units / job_secs, "unit": UNIT, "ms_per_step": 1e3 * job_secs / steps, "steps": steps, "warmup": warmup,
+        "config": dict(config_dict(w, note), format=args.format),
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"] or job.peaks["sm_max_mhz"],
                    "reasons": clocks["reasons"], "samples": clocks["samples"]},
-        "e2e": {"value": e2e_units / e2e_job, "unit": UNIT, "h2d_bytes_per_step": 4 * w.P * w.clients,
-                "d2h_bytes_per_step": 8 * w.P, "steps": e2e_steps},
+        "e2e": e2e_line,
         "gpu_launches": int(launches),
-        "roofline": roofline, "cpu_baseline": cpu,
+        "roofline": roofline,
         "max_abs_err_vs_fedavg": err,
     }
-    print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    if with_cpu_baseline:
+        cpu_ct = min(w.T, 768)
+        cpu_p, cpu_dt, cores = oracle_sample(w, cpu_ct)
+        fields["cpu_baseline"] = {"value": cpu_p / cpu_dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                  "sample": "first %d of %d ciphertext indices (%d params), all %d clients, %.1f s"
+                                            % (cpu_ct, w.T, cpu_p, w.clients, cpu_dt)}
+    return fields
+
+
+def run_ours(args, w, extras):
+    job = Job(args)
+    main = measure(job, w, args.steps, args.warmup, with_cpu_baseline=(job.world == 1))
+    others = {}
+    for name, ew in extras:
+        # the further workloads take at most three timed rounds each (a BERT-sized round is 0.4 s)
+        f = measure(job, ew, max(1, min(args.steps, 3)), max(3, min(args.warmup, 3)), with_cpu_baseline=False)
+        if f is not None:
+            others[name] = f
+    if job.rank == 0:
+        by_index = job.world > 1 and args.shard == "index"
+        line = {"metric": METRIC, "n_gpus": job.world, "higher_is_better": True,
+                "scaling": "strong" if by_index else "weak", "vs_baseline": None,
+                "dtype": "u64 (limbs below 2^46: exact f64)", "data": "synthetic"}
+        line.update(main)
+        if others:
+            line["workloads"] = others
+        print(json.dumps(line), flush=True)
+    if job.world > 1:
+        job.dist.destroy_process_group()
+
+
+WORKLOADS = {"resnet18": lambda: si.RESNET18, "tiny": lambda: si.TINY, "resnet50-top10": lambda: si.RESNET50_TOP10,
+             "bert-1": lambda: si.bert(0.01), "bert-10": lambda: si.bert(0.10), "bert-100": lambda: si.bert(1.0)}
 
 
 def main():
@@ -442,18 +540,29 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=["resnet18", "tiny", "resnet50-top10", "bert-1", "bert-10", "bert-100"],
-                    default="resnet18")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="resnet18")
+    ap.add_argument("--also", default=None,
+                    help="comma-separated further workloads reported under `workloads` (default: resnet50-top10,bert-100 "
+                         "on one GPU when --workload is left at its default; 'none' for none)")
+    ap.add_argument("--shard", choices=["index", "batch"], default="index",
+                    help="N > 1: cut one round over the ranks by ciphertext index (strong scaling) or run one full "
+                         "batch per rank (weak scaling)")
+    ap.add_argument("--gather", action="store_true",
+                    help="with --shard index: all-gather the decoded pieces so that every rank holds the whole model")
     ap.add_argument("--format", choices=["coefficient", "transform"], default="coefficient",
                     help="ciphertext wire format of the timed round (the host-buffer leg always runs "
                          "he_round_host, which implements the coefficient format)")
     args = ap.parse_args()
-    w = {"resnet18": si.RESNET18, "tiny": si.TINY, "resnet50-top10": si.RESNET50_TOP10,
-         "bert-1": si.bert(0.01), "bert-10": si.bert(0.10), "bert-100": si.bert(1.0)}[args.workload]
+    w = WORKLOADS[args.workload]()
     if args.impl == "reference":
         run_reference(args, w)
+        return
+    _, world, _ = dist_env()
+    if args.also is None:
+        also = ["resnet50-top10", "bert-100"] if (world == 1 and args.workload == "resnet18" and args.format == "coefficient") else []
     else:
-        run_ours(args, w)
+        also = [a for a in args.also.split(",") if a and a != "none"]
+    run_ours(args, w, [(a, WORKLOADS[a]()) for a in also])
 
 
 if __name__ == "__main__":
