@@ -24,6 +24,17 @@ def he():
     return he
 
 
+def fresh_noise_bound(N, log2_delta):
+    """Bound on the slot error of ONE fresh ciphertext.  The noise polynomial v = e u + e0 + e1 s
+    has per-coefficient variance sigma^2 (4N/3 + 1) and a slot's real part sums N coefficients at
+    half weight, which gives the standard deviation; but a slot sees e(zeta) u(zeta), a product of
+    two near-Gaussian values, so the error is Laplace-tailed, P(|err| > t std) = exp(-sqrt(2) t),
+    and the largest of 3e4 slots sits near 7 std.  18 std leaves 1e-11 per slot.  (The 1e-6 bound is
+    stated for the weighted aggregate; a single ciphertext on the longest ring at scale 2^40 has a
+    standard deviation of 1.6e-7 and exceeds it.)"""
+    return 18.0 * 3.2 * np.sqrt((4.0 * N / 3.0 + 1.0) * N / 2.0) / 2.0 ** log2_delta
+
+
 def contexts(he, N, primes, ld):
     return he.he_ctx_create(N, list(primes), ld), oracle.Context(N, primes, ld)
 
@@ -152,7 +163,7 @@ def test_encrypt_aggregate_decrypt_bit_exact(he, w):
     assert np.array_equal(out, z[: w.P])
     # a fresh ciphertext opens to its own message
     z0 = he.he_decrypt_level(g, keys, cts[0], w.L).cpu().numpy()
-    assert np.abs(z0[: w.P] - xs[0].astype(np.float64)).max() <= FEDAVG_TOL
+    assert np.abs(z0[: w.P] - xs[0].astype(np.float64)).max() <= fresh_noise_bound(w.N, w.log2_delta)
     assert he.he_ctx_status(g) == he.HE_OK
 
 
@@ -222,7 +233,7 @@ def test_transform_domain_format_bit_exact(he, w):
     z_o = o.decode(o.decrypt(s_o, agg_o, w.L - 1)).reshape(-1)
     assert np.abs(z - z_o).max() <= DECODE_TOL
     z0 = he.he_decrypt_level_ntt(g, keys, cts[0], w.L).cpu().numpy()
-    assert np.abs(z0[: w.P] - xs[0].astype(np.float64)).max() <= FEDAVG_TOL
+    assert np.abs(z0[: w.P] - xs[0].astype(np.float64)).max() <= fresh_noise_bound(w.N, w.log2_delta)
     assert he.he_ctx_status(g) == he.HE_OK
 
 
