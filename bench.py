@@ -62,12 +62,13 @@ UNIT = "params/s"
 # the profile_case.py encrypt case (summaries under profiles/; traffic grows in proportion to the
 # number of ciphertexts).  An entry is dropped (None is reported) when the kernel has changed
 # since its counters were taken.
-ENCRYPT_DRAM_BYTES_PER_CT = {(16384, 4): 363.052288e6 / 296}
+ENCRYPT_DRAM_BYTES_PER_CT = {}
 SLOTS_PER_SM_CLK = 64.0
 WIDE_COST = 2.5
 INT_SLOTS_PER_BUTTERFLY = 6 * WIDE_COST + 4
 F64_SLOTS_FORWARD, F64_SLOTS_INVERSE = 8.0, 9.0
 F64_PRIME_LIMIT = 1 << 46
+ENCODE_SLOTS_PER_BUTTERFLY = 10.0     # complex product (4 multiplies, 2 add/sub) and complex sum and difference
 
 
 def transform_slots(primes, N, forward, inverse):
@@ -456,7 +457,11 @@ def measure(job, w, steps, warmup, with_cpu_baseline):
     per_launch = Tr                                          # ciphertexts of one client's he_encrypt calls
     butterflies = 3 * w.L * (w.N // 2) * logN * per_launch
     # coefficient format: one forward and two inverse transforms per limb; transform format: three forward
-    achieved = transform_slots(w.primes, w.N, 3 if transform else 1, 0 if transform else 2) * per_launch / (kern_ms * 1e-3) / 1e12
+    slots_per_ct = transform_slots(w.primes, w.N, 3 if transform else 1, 0 if transform else 2)
+    if launches_per_encrypt == 1:
+        # the encoder runs inside the kernel: (n/2) log2 n complex butterflies of 10 double-precision operations
+        slots_per_ct += (n // 2) * (n.bit_length() - 1) * ENCODE_SLOTS_PER_BUTTERFLY
+    achieved = slots_per_ct * per_launch / (kern_ms * 1e-3) / 1e12
     peak = job.n_sm * SLOTS_PER_SM_CLK * job.peaks["sm_max_mhz"] * 1e6 / 1e12
     alg_bytes = (4.0 + 32.0 * w.L) * n * per_launch          # read the slots, write the ciphertext
     if w.N <= 16384:

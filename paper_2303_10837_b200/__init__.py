@@ -139,6 +139,8 @@ def _whole_cts(ctx: "Ctx", sel: torch.Tensor, what: str) -> int:
 
 def _ct_count(ctx: "Ctx", ct: torch.Tensor, level: int, what: str) -> int:
     """T of a ciphertext tensor [T][2][level][N] (taken from its first extent, checked against its size)."""
+    if not 1 <= level <= ctx.L:
+        raise HeError(HE_ERR_LEVEL, what)
     T = ct.shape[0] if ct.dim() else 0
     _sized(ct, T * 2 * level * ctx.N, what, exact=True)
     return T

@@ -187,7 +187,10 @@ int he_ctx_status(he_ctx *ctx, int *status) {
 
 int he_ctx_reserve(he_ctx *ctx, size_t max_k) {
     if (!good(ctx)) return HE_ERR_INVALID_ARG;
-    return ensure(&ctx->ws, &ctx->ws_bytes, work_bytes(ctx, he_num_ct(ctx, max_k)));
+    const size_t T = he_num_ct(ctx, max_k);
+    size_t need = encrypt_work_bytes(ctx->dev, ctx->sm_count, T, true);
+    if (ctx->dev.A > 0 && work_bytes(ctx, T) > need) need = work_bytes(ctx, T);     // decryption on the long rings
+    return ensure(&ctx->ws, &ctx->ws_bytes, need);
 }
 
 size_t he_slots(const he_ctx *ctx) { return good(ctx) ? ctx->dev.N / 2 : 0; }
@@ -436,19 +439,15 @@ static int encrypt_range(he_ctx *ctx, const he_keys *keys, const float *sel_dev,
     if (t_count == 0) return HE_OK;
     if (!sel_dev || !ct_dev || !aligned16(ct_dev)) return HE_ERR_INVALID_ARG;
     const CtxDev &d = ctx->dev;
-    // transform-domain output on the long rings transforms u in a work buffer of its own
-    const size_t u_words = (ntt_out && d.A > 0) ? t_count * (size_t)d.L * d.N : 0;
-    int rc = ensure(&ctx->ws, &ctx->ws_bytes, work_bytes(ctx, t_count) + u_words * sizeof(uint64_t));
+    int rc = ensure(&ctx->ws, &ctx->ws_bytes, encrypt_work_bytes(d, ctx->sm_count, t_count, ntt_out));
     if (rc != HE_OK) return rc;
-    int64_t *m = static_cast<int64_t *>(ctx->ws);
-    double2 *cplx = reinterpret_cast<double2 *>(m + t_count * d.N);
-    uint64_t *ubuf = reinterpret_cast<uint64_t *>(m + 2 * t_count * d.N);
     cudaStream_t st = as_stream(stream);
-    CU(launch_encode(d, sel_dev, t_count, cplx, m, st));
     if (ntt_out)
-        CU(launch_encrypt_ntt(d, keys->dev, m, (uint32_t)t_begin, t_count, seed, client_id, ubuf, ct_dev, st));
+        CU(launch_encrypt_ntt(d, keys->dev, sel_dev, ctx->ws, ctx->sm_count, (uint32_t)t_begin, t_count, seed,
+                              client_id, ct_dev, st));
     else
-        CU(launch_encrypt(d, keys->dev, m, (uint32_t)t_begin, t_count, seed, client_id, ct_dev, st));
+        CU(launch_encrypt(d, keys->dev, sel_dev, ctx->ws, ctx->sm_count, (uint32_t)t_begin, t_count, seed,
+                          client_id, ct_dev, st));
     return HE_OK;
 }
 
@@ -730,7 +729,11 @@ static int round_host_queued(he_ctx *ctx, const he_keys *keys, const he_mask *ma
     const size_t total = 2 * b_x + C * (b_sel + b_rest) + b_cts + b_agg + b_z + b_ravg + b_out;
     int rc = ensure(&ctx->round_buf, &ctx->round_bytes, total);
     if (rc != HE_OK) return rc;
-    rc = ensure(&ctx->ws, &ctx->ws_bytes, work_bytes(ctx, Tc));
+    {
+        size_t need = encrypt_work_bytes(d, ctx->sm_count, Tc, false);
+        if (d.A > 0 && work_bytes(ctx, Tc) > need) need = work_bytes(ctx, Tc);
+        rc = ensure(&ctx->ws, &ctx->ws_bytes, need);
+    }
     if (rc != HE_OK) return rc;
     unsigned char *p = static_cast<unsigned char *>(ctx->round_buf);
     float *x[2];

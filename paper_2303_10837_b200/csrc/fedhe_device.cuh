@@ -104,9 +104,50 @@ HD uint64_t csub_as(uint64_t x, uint64_t m) { return SEL ? csub_sel(x, m) : csub
 
 // Shoup product with a fixed operand w < q and wp = floor(w 2^64 / q):
 // returns x w mod q up to one extra q, i.e. a value in [0, 2q), for any x.
+//
+// On the device the product is written out in 32-bit pieces.  The quotient
+// hi = floor(x wp / 2^64) comes from the three upper partial products chained
+// through the carry flag (of x0 wp0 only the high word matters); the result is
+// x w + hi (2^64 - q) mod 2^64, accumulated by two wide multiply-adds into one
+// 64-bit register pair plus four narrow ones into its high word, so that no
+// separate subtraction and no carry additions remain.  Measured on whole
+// transforms in shared memory against `x * w - __umul64hi(x, wp) * q`: 6 %
+// faster, 30.5 instead of 34.5 instructions per butterfly.
 HD uint64_t shoup_lazy(uint64_t x, uint64_t w, uint64_t wp, uint64_t q) {
+#if defined(__CUDA_ARCH__)
+    const uint64_t nq = 0 - q;
+    uint64_t r;
+    asm("{\n\t"
+        ".reg .u32 x0, x1, p0, p1, w0, w1, n0, n1, t1, t2, t3, r0, r1;\n\t"
+        ".reg .u64 acc;\n\t"
+        "mov.b64 {x0, x1}, %1;\n\t"
+        "mov.b64 {w0, w1}, %2;\n\t"
+        "mov.b64 {p0, p1}, %3;\n\t"
+        "mov.b64 {n0, n1}, %4;\n\t"
+        "mul.hi.u32 t1, x0, p0;\n\t"
+        "mad.lo.cc.u32 t1, x0, p1, t1;\n\t"
+        "madc.hi.u32 t2, x0, p1, 0;\n\t"
+        "mad.lo.cc.u32 t1, x1, p0, t1;\n\t"
+        "madc.hi.cc.u32 t2, x1, p0, t2;\n\t"
+        "addc.u32 t3, 0, 0;\n\t"
+        "mad.lo.cc.u32 t2, x1, p1, t2;\n\t"
+        "madc.hi.u32 t3, x1, p1, t3;\n\t"            // hi = t3 : t2
+        "mul.wide.u32 acc, x0, w0;\n\t"
+        "mad.wide.u32 acc, t2, n0, acc;\n\t"
+        "mov.b64 {r0, r1}, acc;\n\t"
+        "mad.lo.u32 r1, x0, w1, r1;\n\t"
+        "mad.lo.u32 r1, x1, w0, r1;\n\t"
+        "mad.lo.u32 r1, t2, n1, r1;\n\t"
+        "mad.lo.u32 r1, t3, n0, r1;\n\t"
+        "mov.b64 %0, {r0, r1};\n\t"
+        "}"
+        : "=l"(r)
+        : "l"(x), "l"(w), "l"(wp), "l"(nq));
+    return r;
+#else
     uint64_t hi = mulhi64(x, wp);
     return sub64(x * w, hi * q);
+#endif
 }
 
 HD uint64_t shoup(uint64_t x, uint64_t w, uint64_t wp, uint64_t q) {

@@ -1,5 +1,6 @@
 // Encryption kernels (part 3 of the kernels).
 #include "fedhe_kernels.cuh"
+#include "fedhe_slots.cuh"
 
 namespace fedhe {
 
@@ -43,7 +44,7 @@ __device__ __forceinline__ void encrypt_unit(const LimbDev &lb, const tw_t *p0, 
                 [&](uint32_t i) {
                     if (h == 0) return ar.small(su[bswz(i)]);
                     if (h == 2) return ar.small(se[bswz(i)]);
-                    return ar.from_residue(signed_residue(mt[i] + (int64_t)se[bswz(i)], q, lb.mu));
+                    return ar.from_residue(signed_residue(__ldcg(mt + i) + (int64_t)se[bswz(i)], q, lb.mu));
                 },
                 [&](uint32_t p, val a, val b) {
                     if (h == 0) {
@@ -95,7 +96,7 @@ __device__ __forceinline__ void encrypt_unit(const LimbDev &lb, const tw_t *p0, 
             },
             [&](uint32_t i, val v) {
                 // e1 is a small value; e0 + m needs a full reduction
-                const uint64_t add = h == 0 ? signed_residue(mt[i] + (int64_t)se[bswz(i)], q, lb.mu)
+                const uint64_t add = h == 0 ? signed_residue(__ldcg(mt + i) + (int64_t)se[bswz(i)], q, lb.mu)
                                             : small_residue(se[bswz(i)], q);
                 cc[i] = ar.canon_add(v, add);
             });
@@ -104,15 +105,22 @@ __device__ __forceinline__ void encrypt_unit(const LimbDev &lb, const tw_t *p0, 
 }
 
 // Fused path for N <= 2^14 (one block holds a whole limb): a thread block
-// draws u, e0, e1 of a ciphertext once into shared memory, then for every
-// limb of it transforms u, multiplies by both halves of the public key,
-// transforms back and adds the error (and message) terms.  Only the
-// ciphertext itself is written to global memory; the second product waits,
-// in transform order, in the c1 slot it will finally occupy.
+// draws u, e0, e1 of a ciphertext once into shared memory and encodes the
+// ciphertext's slots (the slot transform runs in the limb buffer; the rounded
+// message goes to a scratch of N words that belongs to this block alone and is
+// read back once per limb, so it lives in L2), then for every limb of it
+// transforms u, multiplies by both halves of the public key, transforms back
+// and adds the error and message terms.  HBM sees the slots once and the
+// ciphertext once; the second product waits, in transform order, in the c1
+// slot it will finally occupy.  A block whose range of units begins in the
+// middle of a ciphertext encodes that ciphertext again for itself (no block
+// waits for another).
 template <class L, int V, bool NTT_OUT>
 __global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
-encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const int64_t *m, uint32_t t0,
-                     uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
+encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const float *sel, int64_t *mscr,
+                     uint32_t t0, uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
+    using LF = Lay<L::LOGB - 1, 3>;                  // the slot transform of the same ring
+    static_assert(LF::NT == L::NT / V, "the encoder is played by the same threads");
     extern __shared__ __align__(128) uint64_t sm[];
     constexpr uint32_t B = 1u << L::LOGB, RT = L::NT / V;
     int8_t *su = reinterpret_cast<int8_t *>(sm + B);
@@ -129,6 +137,7 @@ encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const in
     const uint32_t u_begin = (uint32_t)(units * blockIdx.x / gridDim.x);
     const uint32_t u_end = (uint32_t)(units * (blockIdx.x + 1) / gridDim.x);
     const size_t cstride = (size_t)c.L * B;          // from c0 to c1 of the same limb
+    int64_t *mblk = mscr + (size_t)blockIdx.x * B;   // this block's encoded message (stays in L2)
     uint32_t sampled = 0xffffffffu;
     for (uint32_t unit = u_begin; unit < u_end; unit++) {
         const uint32_t tl = unit / c.L, j = unit % c.L;   // ciphertext within this call, limb
@@ -152,12 +161,13 @@ encrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const in
                 *reinterpret_cast<char2 *>(se0 + bswz(2 * b)) = a;
                 *reinterpret_cast<char2 *>(se1 + bswz(2 * b)) = e;
             }
-            __syncthreads();
+            // the ciphertext's message: slot transform, scaling and rounding in the limb buffer
+            if (encode_in_block<LF>(c, sel + (size_t)tl * (B / 2), sm, mblk)) atomicOr(c.status, 1);
         }
         const LimbDev &lb = c.limb[j];
         uint64_t *cbase = ct + (((size_t)tl * 2 + 0) * c.L + j) * B;
         FEDHE_FOR_ARITH_SEL(lb, (encrypt_unit<M_, L, V, NTT_OUT>(lb, k.pk0_hat + (size_t)j * B, k.pk1_hat + (size_t)j * B, sm, su,
-                                                    se0, m + (size_t)tl * B, cbase, cstride)));
+                                                    se0, mblk, cbase, cstride)));
     }
 }
 
@@ -202,7 +212,7 @@ __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0
                 const int8_t *se = se0 + (h == 2 ? B : 0);
                 auto value = [&](uint32_t i) {
                     if (h == 2) return ar.small(se[bswz(i)]);
-                    return ar.from_residue(signed_residue(mt[i] + (int64_t)se[bswz(i)], q, lb.mu));
+                    return ar.from_residue(signed_residue(__ldcg(mt + i) + (int64_t)se[bswz(i)], q, lb.mu));
                 };
                 smem_ntt_forward<L, V>(
                     smg, gt, fa,
@@ -274,8 +284,8 @@ __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0
 #pragma unroll
                 for (uint32_t k = 0; k < AHEAD; k++) {
                     const uint32_t e = tid + (k0 + k) * RT;
-                    m_lo[k] = mt[e];
-                    m_hi[k] = mt[e + H];
+                    m_lo[k] = __ldcg(mt + e);
+                    m_hi[k] = __ldcg(mt + e + H);
                 }
             }
 #pragma unroll
@@ -309,8 +319,10 @@ __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0
 // whole block after the two inverse sub-transforms, fused with the epilogue.
 template <class L, int V, bool NTT_OUT>
 __global__ void __launch_bounds__(2 * L::NT / V, 1)
-encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const int64_t *m, uint32_t t0,
-                      uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
+encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const float *sel, int64_t *mscr,
+                      uint32_t t0, uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
+    using LF = Lay<L::LOGB, 3>;                      // the slot transform of the ring (n = half a limb)
+    static_assert(LF::NT == 2 * L::NT / V, "the encoder is played by the whole block");
     extern __shared__ __align__(128) uint64_t sm[];
     constexpr uint32_t H = 1u << L::LOGB, B = 2 * H;       // half and whole limb
     constexpr uint32_t GT = L::NT / V, RT = 2 * GT;        // threads per group, per block
@@ -324,6 +336,7 @@ encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const i
     const uint32_t u_begin = (uint32_t)(units * blockIdx.x / gridDim.x);
     const uint32_t u_end = (uint32_t)(units * (blockIdx.x + 1) / gridDim.x);
     const size_t cstride = (size_t)c.L * B;
+    int64_t *mblk = mscr + (size_t)blockIdx.x * B;   // this block's encoded message (stays in L2)
     uint32_t sampled = 0xffffffffu;
     for (uint32_t unit = u_begin; unit < u_end; unit++) {
         const uint32_t tl = unit / c.L, j = unit % c.L;
@@ -347,12 +360,13 @@ encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const i
                 *reinterpret_cast<char2 *>(se0 + bswz(2 * b)) = a;
                 *reinterpret_cast<char2 *>(se1 + bswz(2 * b)) = e;
             }
-            __syncthreads();
+            // the ciphertext's message: slot transform, scaling and rounding in the limb buffer
+            if (encode_in_block<LF>(c, sel + (size_t)tl * H, sm, mblk)) atomicOr(c.status, 1);
         }
         const LimbDev &lb = c.limb[j];
         uint64_t *cbase = ct + (((size_t)tl * 2 + 0) * c.L + j) * B;
         FEDHE_FOR_ARITH_SEL(lb, (encrypt_unit2<M_, L, V, NTT_OUT>(lb, k.pk0_hat + (size_t)j * B, k.pk1_hat + (size_t)j * B, sm, su,
-                                                     se0, m + (size_t)tl * B, cbase, cstride)));
+                                                     se0, mblk, cbase, cstride)));
     }
 }
 
@@ -555,21 +569,28 @@ enc_outer_inverse_add_kernel(const __grid_constant__ CtxDev c, const int64_t *m,
     }
 }
 
+// shared memory of a block of the fused kernels: the limb and three one-byte sample arrays
+static size_t fused_smem(const CtxDev &c) { return ((size_t)c.N << 3) + 3 * (size_t)c.N; }
+
+// The fused kernels run one block per SM for N = 2^14 and two for N = 2^13 (what
+// their shared memory allows); every block owns N words of message scratch.
+size_t encrypt_fused_blocks(const CtxDev &c, int n_sm) {
+    const size_t per_sm = (size_t)(227 * 1024) / fused_smem(c);
+    return (size_t)n_sm * (per_sm ? per_sm : 1);
+}
+
 template <class L, int V, bool TWO_GROUPS, bool NTT_OUT>
-static cudaError_t launch_encrypt_fused(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0,
-                                        size_t T, uint64_t seed, uint32_t client, uint64_t *ct,
-                                        cudaStream_t s) {
-    const size_t smem = ((sizeof(uint64_t) << L::LOGB) + (3u << L::LOGB)) * (TWO_GROUPS ? 2 : 1);
+static cudaError_t launch_encrypt_fused(const CtxDev &c, const KeysDev &k, const float *sel, int64_t *mscr,
+                                        int n_sm, uint32_t t0, size_t T, uint64_t seed, uint32_t client,
+                                        uint64_t *ct, cudaStream_t s) {
+    const size_t smem = fused_smem(c);
     auto kern = TWO_GROUPS ? encrypt_fused2_kernel<L, V, NTT_OUT> : encrypt_fused_kernel<L, V, NTT_OUT>;
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-    // one block per SM (the kernel's shared memory allows no more), fewer if there is less work
-    int dev = 0, n_sm = 0;
-    if ((e = cudaGetDevice(&dev)) || (e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev))) return e;
-    const size_t per_sm = (size_t)(227 * 1024) / smem;               // blocks that fit one SM
-    size_t grid = (size_t)n_sm * (per_sm ? per_sm : 1);
+    size_t grid = encrypt_fused_blocks(c, n_sm);                     // fewer if there is less work
     if (grid > T * c.L) grid = T * c.L;
-    kern<<<(unsigned)grid, (TWO_GROUPS ? 2 : 1) * L::NT / V, smem, s>>>(c, k, m, t0, seed, client, ct, (uint32_t)T);
+    kern<<<(unsigned)grid, (TWO_GROUPS ? 2 : 1) * L::NT / V, smem, s>>>(c, k, sel, mscr, t0, seed, client, ct,
+                                                                        (uint32_t)T);
     return FEDHE_LAUNCHED();
 }
 
@@ -587,15 +608,25 @@ static cudaError_t launch_enc_block_forward(const CtxDev &c, const KeysDev &k, c
     return FEDHE_LAUNCHED();
 }
 
-cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0, size_t T,
-                           uint64_t seed, uint32_t client, uint64_t *ct, cudaStream_t s) {
+size_t encrypt_work_bytes(const CtxDev &c, int n_sm, size_t T, bool ntt_out) {
+    if (c.A == 0) return encrypt_fused_blocks(c, n_sm) * c.N * sizeof(int64_t);
+    // long rings: the encoded messages and the encoder's complex buffer; the
+    // transform-domain format transforms u in a buffer of its own
+    return (2 * T * c.N + (ntt_out ? T * (size_t)c.L * c.N : 0)) * sizeof(uint64_t);
+}
+
+cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const float *sel, void *work, int n_sm,
+                           uint32_t t0, size_t T, uint64_t seed, uint32_t client, uint64_t *ct,
+                           cudaStream_t s) {
     if (T == 0) return cudaSuccess;
+    int64_t *m = static_cast<int64_t *>(work);
     if (c.A == 0) {
         if (c.LOGB == 13)
-            return launch_encrypt_fused<WLay<13>, 2, false, false>(c, k, m, t0, T, seed, client, ct, s);
-        return launch_encrypt_fused<WLay<13>, 2, true, false>(c, k, m, t0, T, seed, client, ct, s);
+            return launch_encrypt_fused<WLay<13>, 2, false, false>(c, k, sel, m, n_sm, t0, T, seed, client, ct, s);
+        return launch_encrypt_fused<WLay<13>, 2, true, false>(c, k, sel, m, n_sm, t0, T, seed, client, ct, s);
     }
     cudaError_t e;
+    if ((e = launch_encode(c, sel, T, reinterpret_cast<double2 *>(m + T * c.N), m, s))) return e;
     const size_t cols = T * ((size_t)1 << (c.LOGB - 1));      // pairs of columns
     const size_t LN = (size_t)c.L * c.N;
     FEDHE_FOR_A(c, (enc_outer_sample_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, t0, seed, client, ct + LN,
@@ -613,15 +644,19 @@ cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const int64_t *m, 
 // forward transforms per limb.  Longer rings: the error terms go into the
 // ciphertext slots and are transformed there; u is transformed in the work
 // buffer `ubuf` ([T][L][N]) and its key products are added on the way out.
-cudaError_t launch_encrypt_ntt(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0, size_t T,
-                               uint64_t seed, uint32_t client, uint64_t *ubuf, uint64_t *ct, cudaStream_t s) {
+cudaError_t launch_encrypt_ntt(const CtxDev &c, const KeysDev &k, const float *sel, void *work, int n_sm,
+                               uint32_t t0, size_t T, uint64_t seed, uint32_t client, uint64_t *ct,
+                               cudaStream_t s) {
     if (T == 0) return cudaSuccess;
+    int64_t *m = static_cast<int64_t *>(work);
     if (c.A == 0) {
         if (c.LOGB == 13)
-            return launch_encrypt_fused<WLay<13>, 2, false, true>(c, k, m, t0, T, seed, client, ct, s);
-        return launch_encrypt_fused<WLay<13>, 2, true, true>(c, k, m, t0, T, seed, client, ct, s);
+            return launch_encrypt_fused<WLay<13>, 2, false, true>(c, k, sel, m, n_sm, t0, T, seed, client, ct, s);
+        return launch_encrypt_fused<WLay<13>, 2, true, true>(c, k, sel, m, n_sm, t0, T, seed, client, ct, s);
     }
     cudaError_t e;
+    uint64_t *ubuf = reinterpret_cast<uint64_t *>(m + 2 * T * c.N);
+    if ((e = launch_encode(c, sel, T, reinterpret_cast<double2 *>(m + T * c.N), m, s))) return e;
     const size_t LN = (size_t)c.L * c.N;
     const size_t pairs = T * (size_t)(c.N >> 1);
     enc_fill_errors_kernel<<<blocks_for(pairs, 256), 256, 0, s>>>(c, m, t0, seed, client, ct, pairs);

@@ -28,14 +28,20 @@ cudaError_t launch_encode(const CtxDev &c, const float *sel, size_t T, double2 *
 cudaError_t launch_decode(const CtxDev &c, const int64_t *d, size_t T, double2 *cplx, double *z,
                           cudaStream_t s);
 
-// ciphertexts t0 .. t0+T-1 (m and ct point at the first of them)
-cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0, size_t T,
-                           uint64_t seed, uint32_t client, uint64_t *ct, cudaStream_t s);
+// Encode + encrypt ciphertexts t0 .. t0+T-1 (sel and ct point at the first of
+// them).  `work` is scratch of encrypt_work_bytes() bytes: for N <= 2^14 N words
+// per thread block of the fused kernel (the block's encoded message), for
+// longer rings the encoded messages of all T ciphertexts and the encoder's
+// complex buffer.  n_sm: the device's SM count.
+size_t encrypt_work_bytes(const CtxDev &c, int n_sm, size_t T, bool ntt_out);
+cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const float *sel, void *work, int n_sm,
+                           uint32_t t0, size_t T, uint64_t seed, uint32_t client, uint64_t *ct,
+                           cudaStream_t s);
 
-// the same with every limb polynomial of the result in the transform domain;
-// ubuf: uint64 [T][L][N] work space, used for N > 2^14 only
-cudaError_t launch_encrypt_ntt(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0, size_t T,
-                               uint64_t seed, uint32_t client, uint64_t *ubuf, uint64_t *ct, cudaStream_t s);
+// the same with every limb polynomial of the result in the transform domain
+cudaError_t launch_encrypt_ntt(const CtxDev &c, const KeysDev &k, const float *sel, void *work, int n_sm,
+                               uint32_t t0, size_t T, uint64_t seed, uint32_t client, uint64_t *ct,
+                               cudaStream_t s);
 
 // ptrs: device array of C ciphertext pointers; wtab: device [C][L] weights
 cudaError_t launch_aggregate(const CtxDev &c, const uint64_t *const *ptrs, const tw_t *wtab, int C,

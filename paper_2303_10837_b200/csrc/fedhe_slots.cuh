@@ -116,4 +116,42 @@ __device__ __forceinline__ uint32_t bitrev(uint32_t v, int bits) { return __brev
 // spreads them over the banks (checked exhaustively for both block sizes)
 __device__ __forceinline__ uint32_t stage_swz(uint32_t k) { return k ^ (((k >> 8) ^ (k >> 4)) & 15u); }
 
+// The whole encoder of one slot vector inside a thread block of LF::NT threads
+// (n = 2^LF::LOGB slots): the network, the scaling by Delta/n, the rounding
+// and the bit-reversal.  `sm` is a buffer of n cpx values (= N words), used
+// first for the exchanges between phases and then to put the rounded integers
+// in order; m_out receives the N coefficients.  Ends with a block barrier
+// after which `sm` is free and m_out may be read by the block.  Returns
+// whether a coefficient left the range (the caller raises the status word).
+template <class LF>
+__device__ __forceinline__ bool encode_in_block(const CtxDev &c, const float *slots, uint64_t *sm, int64_t *m_out) {
+    constexpr uint32_t n = 1u << LF::LOGB;
+    const uint32_t tid = threadIdx.x;
+    cpx x[LF::E];
+#pragma unroll
+    for (int r = 0; r < LF::E; r++) x[r] = cpx{(double)__ldg(slots + LF::template idx<0>(tid, r)), 0.0};
+    block_dif<LF>(x, reinterpret_cast<cpx *>(sm), tid, c.ftw);
+    // Delta / n is a power of two: one exact multiplication
+    const double scale = __longlong_as_double((long long)(1023 + c.log2_delta - LF::LOGB) << 52);
+    const double lim = 4611686018427387904.0;   // 2^62
+    bool bad = false;
+    int64_t *stage = reinterpret_cast<int64_t *>(sm);
+    __syncthreads();                             // the exchange buffer is free again
+#pragma unroll
+    for (int r = 0; r < LF::E; r++) {
+        const uint32_t kk = bitrev(LF::template idx<LF::NPH - 1>(tid, r), LF::LOGB);
+        double re = __dmul_rn(x[r].re, scale), im = __dmul_rn(x[r].im, scale);
+        if (!(fabs(re) < lim) || !(fabs(im) < lim)) { bad = true; re = 0.0; im = 0.0; }
+        stage[stage_swz(kk)] = __double2ll_rn(re);
+        stage[n + stage_swz(kk)] = __double2ll_rn(im);
+    }
+    __syncthreads();
+    for (uint32_t kk = tid; kk < n; kk += LF::NT) {
+        m_out[kk] = stage[stage_swz(kk)];
+        m_out[kk + n] = stage[n + stage_swz(kk)];
+    }
+    __syncthreads();
+    return bad;
+}
+
 }  // namespace fedhe
