@@ -283,74 +283,65 @@ static int build_mask(he_ctx *ctx, const float *score, size_t P, size_t k, const
     if (P == 0) return HE_ERR_INVALID_ARG;
     if (P >= (1ull << 32)) return HE_ERR_SIZE;
     if (num_ranges > 64 || (num_ranges && !ranges_host)) return HE_ERR_INVALID_ARG;
-    for (size_t r = 0; r < num_ranges; r++)
+    size_t forced = 0;                       // upper bound of what the ranges add to the mask
+    for (size_t r = 0; r < num_ranges; r++) {
         if (ranges_host[2 * r] > ranges_host[2 * r + 1] || ranges_host[2 * r + 1] > P) return HE_ERR_INVALID_ARG;
+        forced += ranges_host[2 * r + 1] - ranges_host[2 * r];
+    }
     cudaStream_t st = as_stream(stream);
     const size_t nblocks = (P + MASK_BLOCK - 1) / MASK_BLOCK, nwords = (P + 31) / 32;
+    const size_t kmax = k + forced < P ? k + forced : P;
 
-    // scratch: histogram (2048) | totals (2) | blk_a (nblocks) | blk_b (nblocks) | ranges
-    // (it lives in the context's work space: no allocation, and no free that would wait for the device)
-    const size_t scratch_words = 2048 + 2 + 2 * nblocks + 4 * 64 + 2;
+    // Scratch in the context's work space (no allocation, and no free that would wait for the
+    // device): selection state (2) | totals (2) | three histograms (2048 each) | blk_a | blk_b | ranges
+    const size_t scratch_words = 4 + 3 * 2048 + 2 * nblocks + 4 * 64 + 2;
     {
         const int erc = ensure(&ctx->ws, &ctx->ws_bytes, scratch_words * sizeof(uint32_t));
         if (erc != HE_OK) return erc;
     }
     uint32_t *scratch = static_cast<uint32_t *>(ctx->ws);
-    uint32_t *hist = scratch, *totals = scratch + 2048, *blk_eq = totals + 2, *blk_sel = blk_eq + nblocks;
-    uint64_t *ranges_dev = reinterpret_cast<uint64_t *>(scratch + ((2048 + 2 + 2 * nblocks + 1) & ~(size_t)1));
+    SelectState *state = reinterpret_cast<SelectState *>(scratch);
+    uint32_t *totals = scratch + 2, *hist = scratch + 4, *blk_eq = hist + 3 * 2048, *blk_sel = blk_eq + nblocks;
+    uint64_t *ranges_dev = reinterpret_cast<uint64_t *>(scratch + ((4 + 3 * 2048 + 2 * nblocks + 1) & ~(size_t)1));
+    // The mask owns one allocation: bit mask | per-word prefix counts | index list (its size is
+    // known up to the overlap of the forced ranges with the top-k set and with each other).
+    uint32_t *bits = nullptr;
+    if (cudaMalloc(reinterpret_cast<void **>(&bits), (2 * nwords + (kmax ? kmax : 1)) * sizeof(uint32_t)) != cudaSuccess)
+        return HE_ERR_ALLOC;
+    uint32_t *wpre = bits + nwords, *idx = wpre + nwords;
     int rc = HE_OK;
     he_mask *m = nullptr;
-    uint32_t *bits = nullptr, *wpre = nullptr, *idx = nullptr;
     do {
 #define MCU(expr) if ((expr) != cudaSuccess) { rc = HE_ERR_CUDA; break; }
-        // radix select of the k-th largest key: 11 + 11 + 10 bits
-        uint32_t prefix = 0, need = (uint32_t)k;   // need = how many keys equal to tau are taken
-        uint32_t tau = 0;
-        if (k == 0) {
-            tau = 0xffffffffu;                       // nothing is above or equal
-            need = 0;
-        } else {
+        // Radix select of the k-th largest key, 11 + 11 + 10 bits, entirely on the device: the
+        // digit walk between two histogram passes is a one-block kernel, so nothing is read
+        // back before the end.
+        const SelectState init = {k ? 0u : 0xffffffffu, (uint32_t)k};      // k = 0: no key reaches the threshold
+        MCU(cudaMemcpyAsync(state, &init, sizeof(init), cudaMemcpyHostToDevice, st));
+        if (k) {
             static const int digits[3] = {11, 11, 10};
+            MCU(cudaMemsetAsync(hist, 0, 3 * 2048 * sizeof(uint32_t), st));
             int prefix_bits = 0;
-            std::vector<uint32_t> h(2048);
             bool fail = false;
-            for (int pass = 0; pass < 3; pass++) {
-                const int db = digits[pass];
-                if (cudaMemsetAsync(hist, 0, sizeof(uint32_t) << db, st) != cudaSuccess ||
-                    launch_key_histogram(score, P, prefix, prefix_bits, db, hist, st) != cudaSuccess ||
-                    cudaMemcpyAsync(h.data(), hist, sizeof(uint32_t) << db, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-                    cudaStreamSynchronize(st) != cudaSuccess) {
-                    fail = true;
-                    break;
-                }
-                // walk the digits from the largest down until `need` keys are covered
-                int b = (1 << db) - 1;
-                for (; b > 0; b--) {
-                    if (h[b] >= need) break;
-                    need -= h[b];
-                }
-                prefix = (prefix << db) | (uint32_t)b;
-                prefix_bits += db;
+            for (int pass = 0; pass < 3 && !fail; pass++) {
+                uint32_t *h = hist + pass * 2048;
+                fail = launch_key_histogram(score, P, state, prefix_bits, digits[pass], ctx->sm_count, h, st) != cudaSuccess ||
+                       launch_radix_pick(h, digits[pass], state, st) != cudaSuccess;
+                prefix_bits += digits[pass];
             }
             if (fail) { rc = HE_ERR_CUDA; break; }
-            tau = prefix;
         }
-        // bit mask and per-word prefix counts share one allocation
-        MCU(cudaMalloc(reinterpret_cast<void **>(&bits), 2 * nwords * sizeof(uint32_t)));
-        wpre = bits + nwords;
         if (num_ranges)
             MCU(cudaMemcpyAsync(ranges_dev, ranges_host, 2 * num_ranges * sizeof(uint64_t), cudaMemcpyHostToDevice, st));
-        MCU(launch_mask_count_eq(score, P, tau, blk_eq, st));
+        MCU(launch_mask_count_eq(score, P, state, blk_eq, st));
         MCU(launch_scan(blk_eq, nblocks, totals, st));
-        MCU(launch_mask_select(score, P, tau, need, ranges_dev, (uint32_t)num_ranges, blk_eq, bits, blk_sel, st));
+        MCU(launch_mask_select(score, P, state, ranges_dev, (uint32_t)num_ranges, blk_eq, bits, blk_sel, st));
         MCU(launch_scan(blk_sel, nblocks, totals + 1, st));
+        MCU(launch_mask_write(P, bits, blk_sel, wpre, idx, st));
         uint32_t ksel = 0;
         MCU(cudaMemcpyAsync(&ksel, totals + 1, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
-        MCU(cudaStreamSynchronize(st));
-        if (num_ranges == 0 && ksel != k) { rc = HE_ERR_CUDA; break; }     // cannot happen
-        MCU(cudaMalloc(reinterpret_cast<void **>(&idx), (ksel ? ksel : 1) * sizeof(uint32_t)));
-        MCU(launch_mask_write(P, bits, blk_sel, wpre, idx, st));
-        MCU(cudaStreamSynchronize(st));
+        MCU(cudaStreamSynchronize(st));                                      // the one wait of the call
+        if ((num_ranges == 0 && ksel != k) || ksel > kmax) { rc = HE_ERR_CUDA; break; }     // cannot happen
         m = new (std::nothrow) he_mask();
         if (!m) { rc = HE_ERR_ALLOC; break; }
         m->magic = MASK_MAGIC;
@@ -362,8 +353,8 @@ static int build_mask(he_ctx *ctx, const float *score, size_t P, size_t k, const
 #undef MCU
     } while (0);
     if (rc != HE_OK) {
-        if (bits) cudaFree(bits);
-        if (idx) cudaFree(idx);
+        cudaStreamSynchronize(st);           // nothing may still write the allocation
+        cudaFree(bits);
         return rc;
     }
     *out = m;
@@ -396,8 +387,7 @@ int he_mask_copy_indices(const he_mask *mask, uint32_t *out_dev, void *stream) {
 int he_mask_destroy(he_mask *mask) {
     if (!good(mask)) return HE_ERR_INVALID_ARG;
     cudaDeviceSynchronize();
-    cudaFree(mask->idx);
-    cudaFree(mask->bits);      // the prefix counts are the second half of this allocation
+    cudaFree(mask->bits);      // prefix counts and index list are parts of this allocation
     mask->magic = 0;
     delete mask;
     return HE_OK;
@@ -526,10 +516,12 @@ int he_plain_aggregate(he_ctx *ctx, const float *const *rests_host, const double
     std::vector<unsigned char> host(C * (sizeof(void *) + sizeof(double)));
     const float **ptrs = reinterpret_cast<const float **>(host.data());
     double *al = reinterpret_cast<double *>(host.data() + C * sizeof(void *));
+    bool aligned = true;
     for (int i = 0; i < C; i++) {
         if (!rests_host[i]) return HE_ERR_INVALID_ARG;
         ptrs[i] = rests_host[i];
         al[i] = alpha_host[i];
+        aligned = aligned && aligned16(rests_host[i]);
     }
     cudaStream_t st = as_stream(stream);
     // second half of the table buffer, so that it does not collide with a
@@ -537,7 +529,8 @@ int he_plain_aggregate(he_ctx *ctx, const float *const *rests_host, const double
     unsigned char *base = static_cast<unsigned char *>(ctx->tab) + HE_MAX_CLIENTS * (sizeof(void *) + HE_MAX_LIMBS * sizeof(tw_t));
     CU(cudaMemcpyAsync(base, host.data(), host.size(), cudaMemcpyHostToDevice, st));
     CU(launch_plain_aggregate(reinterpret_cast<const float *const *>(base),
-                              reinterpret_cast<const double *>(base + C * sizeof(void *)), C, len, out_dev, st));
+                              reinterpret_cast<const double *>(base + C * sizeof(void *)), C, len, out_dev, aligned,
+                              st));
     return HE_OK;
 }
 

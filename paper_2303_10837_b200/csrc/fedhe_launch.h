@@ -49,8 +49,9 @@ cudaError_t launch_aggregate(const CtxDev &c, const uint64_t *const *ptrs, const
 // transform-domain ciphertexts in and out; scratch: uint64 [T][2][L][N]
 cudaError_t launch_aggregate_ntt(const CtxDev &c, const uint64_t *const *ptrs, const tw_t *wtab, int C,
                                  size_t T, uint64_t *scratch, uint64_t *out, cudaStream_t s);
+// aligned16: every client's pointer is 16-byte aligned (the caller knows the host copies)
 cudaError_t launch_plain_aggregate(const float *const *ptrs, const double *alpha, int C, size_t len,
-                                   double *out, cudaStream_t s);
+                                   double *out, bool aligned16, cudaStream_t s);
 
 // scratch: uint64 [T][N]; on return it holds the centred integers as int64
 cudaError_t launch_decrypt(const CtxDev &c, const KeysDev &k, const uint64_t *ct, uint32_t level,
@@ -82,13 +83,18 @@ int ctx_workspace(he_ctx *ctx, size_t T, void **out);
 
 // mask construction (blocks of MASK_BLOCK consecutive parameters)
 constexpr uint32_t MASK_BLOCK = 1024;
-cudaError_t launch_key_histogram(const float *score, size_t P, uint32_t prefix, int prefix_bits,
-                                 int digit_bits, uint32_t *hist, cudaStream_t s);
-cudaError_t launch_mask_count_eq(const float *score, size_t P, uint32_t tau, uint32_t *blk_eq,
+// progress of the radix selection, in device memory: the key prefix found so far (tau after
+// the last step) and how many keys are still to be covered (after the last step: how many keys
+// equal to tau belong to the mask)
+struct SelectState { uint32_t prefix, need; };
+cudaError_t launch_key_histogram(const float *score, size_t P, const SelectState *state, int prefix_bits,
+                                 int digit_bits, int n_sm, uint32_t *hist, cudaStream_t s);
+cudaError_t launch_radix_pick(const uint32_t *hist, int digit_bits, SelectState *state, cudaStream_t s);
+cudaError_t launch_mask_count_eq(const float *score, size_t P, const SelectState *state, uint32_t *blk_eq,
                                  cudaStream_t s);
 // in-place exclusive scan of a[0..count); the grand total goes to *total
 cudaError_t launch_scan(uint32_t *a, size_t count, uint32_t *total, cudaStream_t s);
-cudaError_t launch_mask_select(const float *score, size_t P, uint32_t tau, uint32_t need,
+cudaError_t launch_mask_select(const float *score, size_t P, const SelectState *state,
                                const uint64_t *ranges, uint32_t nranges, const uint32_t *blk_eq_prefix,
                                uint32_t *bits, uint32_t *blk_sel, cudaStream_t s);
 cudaError_t launch_mask_write(size_t P, const uint32_t *bits, const uint32_t *blk_sel_prefix,

@@ -14,51 +14,6 @@ __device__ __forceinline__ uint32_t score_key(float s) {
     return ((b & 0x80000000u) || b > 0x7f800000u) ? 0u : b;
 }
 
-// histogram of the next `digit_bits` key bits among the keys whose leading
-// `prefix_bits` bits equal `prefix`
-__global__ void __launch_bounds__(512)
-key_histogram_kernel(const float *score, size_t P, uint32_t prefix, int prefix_bits, int digit_bits,
-                     uint32_t *hist) {
-    extern __shared__ uint32_t sh[];
-    const uint32_t bins = 1u << digit_bits;
-    for (uint32_t b = threadIdx.x; b < bins; b += blockDim.x) sh[b] = 0;
-    __syncthreads();
-    const int shift = 32 - prefix_bits - digit_bits;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < P; i += (size_t)gridDim.x * blockDim.x) {
-        const uint32_t key = score_key(__ldg(score + i));
-        if (prefix_bits == 0 || (key >> (32 - prefix_bits)) == prefix)
-            atomicAdd(&sh[(key >> shift) & (bins - 1u)], 1u);
-    }
-    __syncthreads();
-    for (uint32_t b = threadIdx.x; b < bins; b += blockDim.x)
-        if (sh[b]) atomicAdd(&hist[b], sh[b]);
-}
-
-cudaError_t launch_key_histogram(const float *score, size_t P, uint32_t prefix, int prefix_bits,
-                                 int digit_bits, uint32_t *hist, cudaStream_t s) {
-    unsigned grid = blocks_for(P, 512);
-    if (grid > 148 * 8) grid = 148 * 8;
-    if (grid == 0) grid = 1;
-    key_histogram_kernel<<<grid, 512, sizeof(uint32_t) << digit_bits, s>>>(score, P, prefix, prefix_bits,
-                                                                          digit_bits, hist);
-    return FEDHE_LAUNCHED();
-}
-
-// number of keys equal to tau in every block of MASK_BLOCK parameters
-__global__ void __launch_bounds__(MASK_BLOCK)
-mask_count_eq_kernel(const float *score, size_t P, uint32_t tau, uint32_t *blk_eq) {
-    const size_t i = (size_t)blockIdx.x * MASK_BLOCK + threadIdx.x;
-    const bool eq = i < P && score_key(__ldg(score + i)) == tau;
-    const int n = __syncthreads_count(eq);
-    if (threadIdx.x == 0) blk_eq[blockIdx.x] = (uint32_t)n;
-}
-
-cudaError_t launch_mask_count_eq(const float *score, size_t P, uint32_t tau, uint32_t *blk_eq,
-                                 cudaStream_t s) {
-    mask_count_eq_kernel<<<blocks_for(P, MASK_BLOCK), MASK_BLOCK, 0, s>>>(score, P, tau, blk_eq);
-    return FEDHE_LAUNCHED();
-}
-
 // exclusive prefix sum inside a block of 1024 threads; returns the block total
 __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t *warp_sums, uint32_t &total) {
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -87,20 +42,109 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t *w
     return res;
 }
 
-// single-block exclusive scan of an array (block totals: at most a few
-// hundred thousand entries)
+// histogram of the next `digit_bits` key bits among the keys whose leading
+// `prefix_bits` bits equal the prefix found so far (state->prefix)
+__global__ void __launch_bounds__(512)
+key_histogram_kernel(const float *score, size_t P, const SelectState *state, int prefix_bits, int digit_bits,
+                     uint32_t *hist) {
+    extern __shared__ uint32_t sh[];
+    const uint32_t bins = 1u << digit_bits;
+    const uint32_t prefix = prefix_bits ? state->prefix : 0u;
+    for (uint32_t b = threadIdx.x; b < bins; b += blockDim.x) sh[b] = 0;
+    __syncthreads();
+    const int shift = 32 - prefix_bits - digit_bits;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < P; i += (size_t)gridDim.x * blockDim.x) {
+        const uint32_t key = score_key(__ldg(score + i));
+        if (prefix_bits == 0 || (key >> (32 - prefix_bits)) == prefix)
+            atomicAdd(&sh[(key >> shift) & (bins - 1u)], 1u);
+    }
+    __syncthreads();
+    for (uint32_t b = threadIdx.x; b < bins; b += blockDim.x)
+        if (sh[b]) atomicAdd(&hist[b], sh[b]);
+}
+
+cudaError_t launch_key_histogram(const float *score, size_t P, const SelectState *state, int prefix_bits,
+                                 int digit_bits, int n_sm, uint32_t *hist, cudaStream_t s) {
+    unsigned grid = blocks_for(P, 512);
+    const unsigned resident = (unsigned)n_sm * 4u;       // four blocks of 512 threads fit one SM
+    if (grid > resident) grid = resident;
+    if (grid == 0) grid = 1;
+    key_histogram_kernel<<<grid, 512, sizeof(uint32_t) << digit_bits, s>>>(score, P, state, prefix_bits,
+                                                                          digit_bits, hist);
+    return FEDHE_LAUNCHED();
+}
+
+// One step of the radix selection on the device: walks the digits of a
+// histogram from the largest down until `need` keys are covered, appends the
+// digit found to the prefix and takes the keys above it off `need`.  One block;
+// after the last step prefix is the threshold key tau and need the number of
+// keys equal to tau that belong to the mask.
+__global__ void __launch_bounds__(1024)
+radix_pick_kernel(const uint32_t *hist, int digit_bits, SelectState *state) {
+    __shared__ uint32_t warp_sums[33];
+    const uint32_t bins = 1u << digit_bits;
+    const uint32_t need = state->need;
+    // thread t looks at digits b = bins - 1 - (2 t), bins - 2 - (2 t): descending order
+    const uint32_t per = bins / 1024u ? bins / 1024u : 1u;       // 2 for 11 bits, 1 for 10 bits
+    uint32_t h[2] = {0u, 0u}, mine = 0u;
+    for (uint32_t j = 0; j < per; j++) {
+        const uint32_t pos = threadIdx.x * per + j;              // position in descending order
+        h[j] = pos < bins ? hist[bins - 1u - pos] : 0u;
+        mine += h[j];
+    }
+    uint32_t tot;
+    uint32_t above = block_exclusive_scan(mine, warp_sums, tot);   // keys in digits above this thread's
+    __syncthreads();
+    for (uint32_t j = 0; j < per; j++) {
+        const uint32_t pos = threadIdx.x * per + j;
+        // the digit where the running count first reaches `need` (digit 0 if it never does)
+        if (pos < bins && above < need && (above + h[j] >= need || pos == bins - 1u)) {
+            state->prefix = (state->prefix << digit_bits) | (bins - 1u - pos);
+            state->need = need - above;
+        }
+        above += h[j];
+    }
+}
+
+cudaError_t launch_radix_pick(const uint32_t *hist, int digit_bits, SelectState *state, cudaStream_t s) {
+    radix_pick_kernel<<<1, 1024, 0, s>>>(hist, digit_bits, state);
+    return FEDHE_LAUNCHED();
+}
+
+// number of keys equal to tau in every block of MASK_BLOCK parameters
+__global__ void __launch_bounds__(MASK_BLOCK)
+mask_count_eq_kernel(const float *score, size_t P, const SelectState *state, uint32_t *blk_eq) {
+    const uint32_t tau = state->prefix;
+    const size_t i = (size_t)blockIdx.x * MASK_BLOCK + threadIdx.x;
+    const bool eq = i < P && score_key(__ldg(score + i)) == tau;
+    const int n = __syncthreads_count(eq);
+    if (threadIdx.x == 0) blk_eq[blockIdx.x] = (uint32_t)n;
+}
+
+cudaError_t launch_mask_count_eq(const float *score, size_t P, const SelectState *state, uint32_t *blk_eq,
+                                 cudaStream_t s) {
+    mask_count_eq_kernel<<<blocks_for(P, MASK_BLOCK), MASK_BLOCK, 0, s>>>(score, P, state, blk_eq);
+    return FEDHE_LAUNCHED();
+}
+
+// single-block exclusive scan of an array (block totals: about a hundred
+// thousand entries for the largest model): every thread sums a contiguous
+// chunk, the chunk sums are scanned across the block, and the thread writes
+// the running prefix back over its chunk
 __global__ void __launch_bounds__(1024) scan_kernel(uint32_t *a, size_t count, uint32_t *total_out) {
     __shared__ uint32_t warp_sums[33];
-    uint32_t carry = 0;
-    for (size_t base = 0; base < count; base += 1024) {
-        const size_t i = base + threadIdx.x;
-        const uint32_t v = i < count ? a[i] : 0u;
-        uint32_t tot;
-        const uint32_t ex = block_exclusive_scan(v, warp_sums, tot);
-        if (i < count) a[i] = carry + ex;
-        carry += tot;
+    const size_t per = (count + 1023) / 1024;
+    const size_t b = threadIdx.x * per, e = b + per < count ? b + per : count;
+    uint32_t sum = 0;
+    for (size_t i = b; i < e; i++) sum += a[i];
+    uint32_t tot;
+    uint32_t run = block_exclusive_scan(sum, warp_sums, tot);
+    for (size_t i = b; i < e; i++) {
+        const uint32_t v = a[i];
+        a[i] = run;
+        run += v;
     }
-    if (threadIdx.x == 0) *total_out = carry;
+    if (threadIdx.x == 0) *total_out = tot;
 }
 
 cudaError_t launch_scan(uint32_t *a, size_t count, uint32_t *total, cudaStream_t s) {
@@ -111,9 +155,10 @@ cudaError_t launch_scan(uint32_t *a, size_t count, uint32_t *total, cudaStream_t
 // membership bits: key > tau, or key == tau and fewer than `need` equal keys
 // at lower indices, or inside a forced index range
 __global__ void __launch_bounds__(MASK_BLOCK)
-mask_select_kernel(const float *score, size_t P, uint32_t tau, uint32_t need, const uint64_t *ranges,
+mask_select_kernel(const float *score, size_t P, const SelectState *state, const uint64_t *ranges,
                    uint32_t nranges, const uint32_t *blk_eq_prefix, uint32_t *bits, uint32_t *blk_sel) {
     __shared__ uint32_t warp_sums[33];
+    const uint32_t tau = state->prefix, need = state->need;
     const size_t i = (size_t)blockIdx.x * MASK_BLOCK + threadIdx.x;
     const uint32_t key = i < P ? score_key(__ldg(score + i)) : 0u;
     const bool eq = i < P && key == tau;
@@ -130,10 +175,10 @@ mask_select_kernel(const float *score, size_t P, uint32_t tau, uint32_t need, co
     if (threadIdx.x == 0) blk_sel[blockIdx.x] = (uint32_t)n;
 }
 
-cudaError_t launch_mask_select(const float *score, size_t P, uint32_t tau, uint32_t need,
+cudaError_t launch_mask_select(const float *score, size_t P, const SelectState *state,
                                const uint64_t *ranges, uint32_t nranges, const uint32_t *blk_eq_prefix,
                                uint32_t *bits, uint32_t *blk_sel, cudaStream_t s) {
-    mask_select_kernel<<<blocks_for(P, MASK_BLOCK), MASK_BLOCK, 0, s>>>(score, P, tau, need, ranges, nranges,
+    mask_select_kernel<<<blocks_for(P, MASK_BLOCK), MASK_BLOCK, 0, s>>>(score, P, state, ranges, nranges,
                                                                         blk_eq_prefix, bits, blk_sel);
     return FEDHE_LAUNCHED();
 }
@@ -162,97 +207,128 @@ cudaError_t launch_mask_write(size_t P, const uint32_t *bits, const uint32_t *bl
 // ===========================================================================
 // packing and merging
 // ===========================================================================
+//
+// These are single passes over the update, bound by HBM.  With a mask, a warp
+// takes PACK_WORDS consecutive words of the bit mask at a time and lane l the
+// parameter of bit l of each: loads and stores of a warp instruction are then
+// consecutive addresses (the compacted outputs as well, because the lanes'
+// positions are consecutive among the selected / unselected bits of the word),
+// and all of a thread's loads are issued before the first store.  Without a
+// mask the steps are copies with 16-byte accesses where the pointers allow.
 
-// one pass over the update: masked parameters go to their slot, the others to
-// the compacted remainder; the tail of the last ciphertext is zeroed.  A
-// thread takes four neighbouring parameters (one 16-byte load when the
-// pointers allow it; they always share one word of the bit mask).
+constexpr int PACK_WORDS = 8;       // mask words (256 parameters) per warp
+constexpr int COPY_VECS = 4;        // 16-byte vectors per thread of the copies
+
+// masked parameters go to their slot, the others to the compacted remainder
 __global__ void __launch_bounds__(256)
-pack_kernel(const uint32_t *bits, const uint32_t *wpre, const float *x, size_t P, size_t k, size_t padded,
-            float *sel, float *rest, bool vec) {
-    const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const size_t i0 = t * 4;
-    if (i0 < P) {
-        float v[4];
-        const uint32_t cnt = P - i0 < 4 ? (uint32_t)(P - i0) : 4u;
-        if (vec && cnt == 4) {
-            const float4 q = __ldg(reinterpret_cast<const float4 *>(x + i0));
-            v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
-        } else {
+pack_masked_kernel(const uint32_t *bits, const uint32_t *wpre, const float *x, size_t P, float *sel, float *rest) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const size_t warp = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const size_t word0 = warp * PACK_WORDS, nwords = (P + 31) >> 5;
+    if (word0 >= nwords) return;
+    float v[PACK_WORDS];
+    uint32_t w[PACK_WORDS], pre[PACK_WORDS];
 #pragma unroll
-            for (uint32_t j = 0; j < 4; j++) v[j] = j < cnt ? __ldg(x + i0 + j) : 0.0f;
-        }
-        if (bits == nullptr) {
-            if (vec && cnt == 4) {
-                *reinterpret_cast<float4 *>(sel + i0) = make_float4(v[0], v[1], v[2], v[3]);
-            } else {
-#pragma unroll
-                for (uint32_t j = 0; j < 4; j++)
-                    if (j < cnt) sel[i0 + j] = v[j];
-            }
-        } else {
-            const uint32_t w = bits[i0 >> 5], lane = (uint32_t)(i0 & 31);
-            size_t before = (size_t)wpre[i0 >> 5] + __popc(w & ((1u << lane) - 1u));
-#pragma unroll
-            for (uint32_t j = 0; j < 4; j++) {
-                if (j < cnt) {
-                    if ((w >> (lane + j)) & 1u) sel[before++] = v[j];
-                    else rest[i0 + j - before] = v[j];
-                }
-            }
-        }
+    for (int j = 0; j < PACK_WORDS; j++) {
+        const size_t word = word0 + j, i = (word << 5) + lane;
+        v[j] = i < P ? __ldg(x + i) : 0.0f;
+        w[j] = word < nwords ? __ldg(bits + word) : 0u;
+        pre[j] = word < nwords ? __ldg(wpre + word) : 0u;
     }
-    if (t < padded - k) sel[k + t] = 0.0f;
+#pragma unroll
+    for (int j = 0; j < PACK_WORDS; j++) {
+        const size_t i = ((word0 + j) << 5) + lane;
+        if (i >= P) continue;
+        const size_t before = (size_t)pre[j] + __popc(w[j] & ((1u << lane) - 1u));
+        if ((w[j] >> lane) & 1u) sel[before] = v[j];
+        else rest[i - before] = v[j];
+    }
+}
+
+// dst[i] = src[i] for i < count, dst[i] = 0 for count <= i < padded (T may be float or double)
+template <class T, class V>
+__global__ void __launch_bounds__(256)
+copy_pad_kernel(const T *src, size_t count, size_t padded, T *dst, bool vec) {
+    constexpr size_t per = sizeof(V) / sizeof(T);
+    const size_t base = (size_t)blockIdx.x * blockDim.x * COPY_VECS * per;
+    if (vec && base + (size_t)blockDim.x * COPY_VECS * per <= count) {
+        V t[COPY_VECS];
+#pragma unroll
+        for (int j = 0; j < COPY_VECS; j++)
+            t[j] = __ldg(reinterpret_cast<const V *>(src + base) + j * blockDim.x + threadIdx.x);
+#pragma unroll
+        for (int j = 0; j < COPY_VECS; j++)
+            reinterpret_cast<V *>(dst + base)[j * blockDim.x + threadIdx.x] = t[j];
+        return;
+    }
+    // ragged end of the input, unaligned pointers, and the zero padding
+    for (size_t i = base + threadIdx.x; i < base + (size_t)blockDim.x * COPY_VECS * per && i < padded; i += blockDim.x)
+        dst[i] = i < count ? src[i] : (T)0;
+}
+
+template <class T, class V>
+static cudaError_t launch_copy_pad(const T *src, size_t count, size_t padded, T *dst, cudaStream_t s) {
+    if (padded == 0) return cudaSuccess;
+    const bool vec = ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & (sizeof(V) - 1)) == 0;
+    const size_t per_block = 256 * COPY_VECS * (sizeof(V) / sizeof(T));
+    copy_pad_kernel<T, V><<<blocks_for(padded, (unsigned)per_block), 256, 0, s>>>(src, count, padded, dst, vec);
+    return FEDHE_LAUNCHED();
+}
+
+__global__ void __launch_bounds__(256) zero_tail_kernel(float *dst, size_t count) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < count) dst[i] = 0.0f;
 }
 
 cudaError_t launch_pack(const he_mask *mask, const float *x, size_t P, size_t k, size_t padded,
                         float *sel, float *rest, cudaStream_t s) {
-    const size_t quads = (P + 3) / 4;
-    size_t threads = quads > padded - k ? quads : padded - k;
-    if (threads == 0) return cudaSuccess;
-    const bool vec = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(sel)) & 15u) == 0;
-    pack_kernel<<<blocks_for(threads, 256), 256, 0, s>>>(mask ? mask->bits : nullptr, mask ? mask->wpre : nullptr,
-                                                          x, P, k, padded, sel, rest, vec);
-    return FEDHE_LAUNCHED();
+    if (!mask) return launch_copy_pad<float, float4>(x, P, padded, sel, s);     // k = P: a copy and the zero tail
+    if (P) {
+        const size_t warps = (((P + 31) >> 5) + PACK_WORDS - 1) / PACK_WORDS;
+        pack_masked_kernel<<<blocks_for(warps * 32, 256), 256, 0, s>>>(mask->bits, mask->wpre, x, P, sel, rest);
+        const cudaError_t e = FEDHE_LAUNCHED();
+        if (e) return e;
+    }
+    if (padded > k) {                                                            // tail of the last ciphertext
+        zero_tail_kernel<<<blocks_for(padded - k, 256), 256, 0, s>>>(sel + k, padded - k);
+        return FEDHE_LAUNCHED();
+    }
+    return cudaSuccess;
 }
 
-// the reverse: two neighbouring parameters per thread (one 16-byte store)
+// the reverse with a mask: w_glob[i] = z[r] for the r-th masked parameter, the remainder's
+// average in order elsewhere
 __global__ void __launch_bounds__(256)
-unpack_kernel(const uint32_t *bits, const uint32_t *wpre, const double *z, const double *rest_avg, size_t P,
-              double *w_glob, bool vec) {
-    const size_t i0 = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 2;
-    if (i0 >= P) return;
-    const bool two = i0 + 1 < P;
-    double a, b = 0.0;
-    if (bits == nullptr) {
-        if (vec && two) {
-            *reinterpret_cast<double2 *>(w_glob + i0) = *reinterpret_cast<const double2 *>(z + i0);
-            return;
+unpack_masked_kernel(const uint32_t *bits, const uint32_t *wpre, const double *z, const double *rest_avg, size_t P,
+                     double *w_glob) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const size_t warp = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const size_t word0 = warp * PACK_WORDS, nwords = (P + 31) >> 5;
+    if (word0 >= nwords) return;
+    double v[PACK_WORDS];
+#pragma unroll
+    for (int j = 0; j < PACK_WORDS; j++) {
+        const size_t word = word0 + j, i = (word << 5) + lane;
+        v[j] = 0.0;
+        if (i < P) {
+            const uint32_t w = __ldg(bits + word);
+            const size_t before = (size_t)__ldg(wpre + word) + __popc(w & ((1u << lane) - 1u));
+            v[j] = ((w >> lane) & 1u) ? __ldg(z + before) : __ldg(rest_avg + (i - before));
         }
-        a = z[i0];
-        if (two) b = z[i0 + 1];
-    } else {
-        const uint32_t w = bits[i0 >> 5], lane = (uint32_t)(i0 & 31);
-        size_t before = (size_t)wpre[i0 >> 5] + __popc(w & ((1u << lane) - 1u));
-        const bool s0 = (w >> lane) & 1u;
-        a = s0 ? z[before] : rest_avg[i0 - before];
-        before += s0 ? 1 : 0;
-        if (two) b = ((w >> (lane + 1)) & 1u) ? z[before] : rest_avg[i0 + 1 - before];
     }
-    if (vec && two) {
-        *reinterpret_cast<double2 *>(w_glob + i0) = make_double2(a, b);
-    } else {
-        w_glob[i0] = a;
-        if (two) w_glob[i0 + 1] = b;
+#pragma unroll
+    for (int j = 0; j < PACK_WORDS; j++) {
+        const size_t i = ((word0 + j) << 5) + lane;
+        if (i < P) w_glob[i] = v[j];
     }
 }
 
 cudaError_t launch_unpack(const he_mask *mask, const double *z, const double *rest_avg, size_t P,
                           double *w_glob, cudaStream_t s) {
     if (P == 0) return cudaSuccess;
-    const bool vec = ((reinterpret_cast<uintptr_t>(z) | reinterpret_cast<uintptr_t>(w_glob)) & 15u) == 0;
-    unpack_kernel<<<blocks_for((P + 1) / 2, 256), 256, 0, s>>>(mask ? mask->bits : nullptr,
-                                                               mask ? mask->wpre : nullptr, z, rest_avg, P, w_glob, vec);
+    if (!mask) return launch_copy_pad<double, double2>(z, P, P, w_glob, s);
+    const size_t warps = (((P + 31) >> 5) + PACK_WORDS - 1) / PACK_WORDS;
+    unpack_masked_kernel<<<blocks_for(warps * 32, 256), 256, 0, s>>>(mask->bits, mask->wpre, z, rest_avg, P, w_glob);
     return FEDHE_LAUNCHED();
 }
 

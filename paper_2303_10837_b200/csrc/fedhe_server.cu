@@ -176,40 +176,43 @@ cudaError_t launch_aggregate_ntt(const CtxDev &c, const uint64_t *const *ptrs, c
     return cudaSuccess;
 }
 
-// plaintext remainder: out = sum_i alpha_i * (double) rest_i, client order,
-// separate multiply and add; two neighbouring entries per thread (8-byte loads,
-// one 16-byte store) when every pointer allows it
+// out[k] = sum_i alpha_i * rest_i[k] in fp64, clients in order, separate
+// multiply and add.  A thread takes four neighbouring entries (one 16-byte
+// load per client, two 16-byte stores) when every pointer allows it, and the
+// loads of several clients are in flight at once.
 __global__ void __launch_bounds__(256)
-plain_aggregate_kernel(const float *const *ptrs, const double *alpha, int C, size_t len, double *out) {
-    const size_t g = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 2;
+plain_aggregate_kernel(const float *const *ptrs, const double *alpha, int C, size_t len, double *out, bool vec) {
+    const size_t g = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (g >= len) return;
-    bool vec = g + 1 < len && (reinterpret_cast<uintptr_t>(out) & 15u) == 0;
-    for (int cl = 0; cl < C && vec; cl++) vec = (reinterpret_cast<uintptr_t>(ptrs[cl]) & 7u) == 0;
-    double a = 0.0, b = 0.0;
-    if (vec) {
+    double a[4] = {0.0, 0.0, 0.0, 0.0};
+    if (vec && g + 4 <= len) {
+#pragma unroll 5
         for (int cl = 0; cl < C; cl++) {
-            const float2 v = __ldg(reinterpret_cast<const float2 *>(ptrs[cl] + g));
+            const float4 v = __ldg(reinterpret_cast<const float4 *>(ptrs[cl] + g));
             const double al = alpha[cl];
-            a = __dadd_rn(a, __dmul_rn(al, (double)v.x));
-            b = __dadd_rn(b, __dmul_rn(al, (double)v.y));
+            a[0] = __dadd_rn(a[0], __dmul_rn(al, (double)v.x));
+            a[1] = __dadd_rn(a[1], __dmul_rn(al, (double)v.y));
+            a[2] = __dadd_rn(a[2], __dmul_rn(al, (double)v.z));
+            a[3] = __dadd_rn(a[3], __dmul_rn(al, (double)v.w));
         }
-        *reinterpret_cast<double2 *>(out + g) = make_double2(a, b);
+        *reinterpret_cast<double2 *>(out + g) = make_double2(a[0], a[1]);
+        *reinterpret_cast<double2 *>(out + g + 2) = make_double2(a[2], a[3]);
         return;
     }
-    const bool two = g + 1 < len;
+    const uint32_t cnt = len - g < 4 ? (uint32_t)(len - g) : 4u;
     for (int cl = 0; cl < C; cl++) {
         const double al = alpha[cl];
-        a = __dadd_rn(a, __dmul_rn(al, (double)__ldg(ptrs[cl] + g)));
-        if (two) b = __dadd_rn(b, __dmul_rn(al, (double)__ldg(ptrs[cl] + g + 1)));
+        for (uint32_t j = 0; j < cnt; j++) a[j] = __dadd_rn(a[j], __dmul_rn(al, (double)__ldg(ptrs[cl] + g + j)));
     }
-    out[g] = a;
-    if (two) out[g + 1] = b;
+    for (uint32_t j = 0; j < cnt; j++) out[g + j] = a[j];
 }
 
+// aligned16: every client's pointer is 16-byte aligned
 cudaError_t launch_plain_aggregate(const float *const *ptrs, const double *alpha, int C, size_t len,
-                                   double *out, cudaStream_t s) {
+                                   double *out, bool aligned16, cudaStream_t s) {
     if (len == 0) return cudaSuccess;
-    plain_aggregate_kernel<<<blocks_for((len + 1) / 2, 256), 256, 0, s>>>(ptrs, alpha, C, len, out);
+    const bool vec = aligned16 && (reinterpret_cast<uintptr_t>(out) & 15u) == 0;
+    plain_aggregate_kernel<<<blocks_for((len + 3) / 4, 256), 256, 0, s>>>(ptrs, alpha, C, len, out, vec);
     return FEDHE_LAUNCHED();
 }
 
