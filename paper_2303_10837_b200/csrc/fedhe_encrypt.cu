@@ -1,4 +1,6 @@
 // Encryption kernels (part 3 of the kernels).
+#include <cooperative_groups.h>
+
 #include "fedhe_kernels.cuh"
 #include "fedhe_slots.cuh"
 
@@ -370,12 +372,261 @@ encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const f
     }
 }
 
-// Long rings (N = 2^15, 2^16), where a limb does not fit one SM: the ciphertext
-// buffer itself is the only work space and every pass over it does as much as
-// it can.  (1) draw u and run the outer forward stages into the c1 slots;
-// (2) block transforms of the c1 slots whose last phase writes both products
-// u^ pk0^ -> c0 and u^ pk1^ -> c1; (3) inverse block transforms of all slots;
-// (4) outer inverse stages fused with the error and message terms.
+// ===========================================================================
+// Long rings (N = 2^15, 2^16) on thread-block clusters: a limb of 256 or 512 KB
+// does not fit one SM's shared memory, but it fits the shared memories of a
+// cluster of CS = 2 or 4 thread blocks.  The limb is cut into ROWS = 2 CS
+// pieces of HB = 2^13 residues; block `rank` of the cluster holds pieces
+// 2 rank and 2 rank + 1, and each of its two groups of 512 threads transforms
+// one piece as a sub-block of the long transform on its own schedule (named
+// barriers), as in the two-group kernel above.  The log2 ROWS outer stages,
+// which pair elements of different pieces, are done where all pieces are at
+// hand:
+//   forward, on the way in: the input u is ternary, so an output of the outer
+//     stages is a signed sum of ROWS constants (one row of the outer butterfly
+//     network applied to unit vectors, computed once per unit), picked by the
+//     samples -- no multiplication;
+//   inverse, after the sub-transforms: block `rank` takes the columns
+//     [rank HB / CS, (rank + 1) HB / CS) of the ROWS x HB view, reads the
+//     elements of a column from the shared memories of all blocks of the
+//     cluster (distributed shared memory, plain loads), runs the outer stages
+//     with 1/N folded in, adds the error and message terms and writes the
+//     ciphertext.
+// HBM sees the encoded message and the ciphertext once (the second key
+// product waits in its final slot), instead of the six passes over the
+// ciphertext of the multi-kernel path below.  The cluster's blocks meet at a
+// cluster barrier before and after every read of each other's shared memory;
+// all of them run the same units, so every block reaches every barrier.
+// ===========================================================================
+
+namespace cg = cooperative_groups;
+
+template <class M, int CL>
+__device__ __forceinline__ void encrypt_unit_cluster(const LimbDev &lb, const tw_t *pk0, const tw_t *pk1, uint64_t *sm,
+                                                     uint64_t *consts, const int8_t *su, const int8_t *se,
+                                                     const int64_t *mt, uint64_t *cbase, size_t cstride,
+                                                     uint32_t rank, cg::cluster_group &cluster) {
+    using L = WLay<13>;
+    constexpr int V = 2;
+    using val = typename M::val;
+    constexpr uint32_t HB = 1u << 13, CS = 1u << CL, ROWS = 2 * CS, AO = CL + 1, COLS = HB / CS;
+    constexpr uint32_t GT = L::NT / V, RT = 2 * GT;            // threads per group, per block
+    const uint32_t tid = threadIdx.x, grp = tid / GT, gt = tid % GT;
+    const uint32_t row = 2 * rank + grp;                       // the piece this group transforms
+    uint64_t *smg = sm + grp * HB;
+    const GroupSync gsync = {1 + grp, GT};
+    const uint64_t q = lb.q;
+    // the message words of this block's columns will be wanted at the end of the first pass
+    for (uint32_t c2 = tid; c2 < COLS / 2; c2 += RT)
+#pragma unroll
+        for (uint32_t a = 0; a < ROWS; a++)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(mt + a * HB + rank * COLS + 2 * c2));
+    // row `row` of the outer forward stages applied to the unit vectors
+    if (gt < ROWS) {
+        const auto fo = LimbOf<M>::args(lb, true, 0, 0);
+        val x[ROWS], y[ROWS];
+#pragma unroll
+        for (uint32_t a = 0; a < ROWS; a++) {
+            x[a] = fo.m.small(a == gt ? 1 : 0);
+            y[a] = fo.m.small(0);
+        }
+        outer_forward<AO>(x, y, fo);
+        val r = x[0];
+#pragma unroll
+        for (uint32_t a = 1; a < ROWS; a++)
+            if (a == row) r = x[a];
+        consts[grp * ROWS + gt] = M::bits(fo.m.from_residue(fo.m.canon_wide(r)));       // in [0, q)
+    }
+    gsync();
+    {
+        const tw_t *p0 = pk0 + row * HB, *p1 = pk1 + row * HB;
+        uint64_t *c1 = cbase + cstride + row * HB;
+        const auto fa = LimbOf<M>::args(lb, true, AO, row);
+        const M &ar = fa.m;
+        val cst[ROWS];
+#pragma unroll
+        for (uint32_t k = 0; k < ROWS; k++) cst[k] = M::from_bits(consts[grp * ROWS + k]);
+        smem_ntt_forward<L, V>(
+            smg, gt, fa,
+            [&](uint32_t i) {
+                if constexpr (std::is_same<M, ModF64>::value) {
+                    double acc = 0.0;                                // |acc| < ROWS q
+#pragma unroll
+                    for (uint32_t k = 0; k < ROWS; k++) acc = f64_fma((double)su[bswz(k * HB + i)], cst[k], acc);
+                    return ROWS > 4 ? ar.settle(acc) : acc;
+                } else {
+                    uint64_t acc = 0;                                // below ROWS q
+#pragma unroll
+                    for (uint32_t k = 0; k < ROWS; k++) {
+                        const int b = su[bswz(k * HB + i)];
+                        acc += b == 0 ? 0 : (b > 0 ? cst[k] : q - cst[k]);
+                    }
+                    return ROWS > 4 ? csub_as<true>(acc, 2 * ar.q2) : acc;      // below 4q
+                }
+            },
+            [&](uint32_t p, val a, val b) {
+                const auto a0 = M::load_key(p1 + p), a1 = M::load_key(p1 + p + 1);
+                u64x2 v;
+                v.x = M::bits(ar.mul_key(a, a0));
+                v.y = M::bits(ar.mul_key(b, a1));
+                *reinterpret_cast<u64x2 *>(c1 + p) = v;      // parked until the second pass
+                const auto b0 = M::load_key(p0 + p), b1 = M::load_key(p0 + p + 1);
+                smg[wswz(p)] = M::bits(ar.mul_key(a, b0));
+                smg[wswz(p + 1)] = M::bits(ar.mul_key(b, b1));
+            },
+            gsync);
+    }
+    const uint64_t *piece[CS];                                   // the same buffer in every block of the cluster
+#pragma unroll
+    for (uint32_t a = 0; a < CS; a++) piece[a] = cluster.map_shared_rank(sm, a);
+#pragma unroll 1
+    for (int h = 0; h < 2; h++) {
+        uint64_t *cc = cbase + h * cstride;
+        const int8_t *seh = se + h * 2 * HB;
+        const auto ia = LimbOf<M>::args(lb, false, AO, row);
+        const auto ninv = LimbOf<M>::ninv(lb), wn = LimbOf<M>::wn(lb);
+        smem_ntt_inverse<L, V, false>(
+            smg, gt, ia, ninv, wn,
+            [&](uint32_t p) {
+                if (h == 0) return pair_of<val>{M::from_bits(smg[wswz(p)]), M::from_bits(smg[wswz(p + 1)])};
+                const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + row * HB + p);
+                return pair_of<val>{M::from_bits(t.x), M::from_bits(t.y)};
+            },
+            [&](uint32_t i, val v) { smg[wswz(i)] = M::bits(v); }, gsync);
+        cluster.sync();                                          // every piece is transformed and visible
+        const auto to = LimbOf<M>::args(lb, false, 0, 0);
+#pragma unroll 1
+        for (uint32_t c2 = tid; c2 < COLS / 2; c2 += RT) {
+            const uint32_t lc = 2 * c2, i = rank * COLS + lc;    // two neighbouring columns
+            val x[ROWS], y[ROWS];
+#pragma unroll
+            for (uint32_t a = 0; a < ROWS; a++) {
+                const uint64_t *src = piece[a >> 1] + (a & 1u) * HB;
+                x[a] = M::from_bits(src[wswz(i)]);
+                y[a] = M::from_bits(src[wswz(i + 1)]);
+            }
+            outer_inverse<AO>(x, y, to, ninv, wn);
+#pragma unroll
+            for (uint32_t a = 0; a < ROWS; a++) {
+                const int ex = seh[a * COLS + lc], ey = seh[a * COLS + lc + 1];
+                uint64_t ax, ay;
+                if (h == 0) {
+                    const longlong2 mm = __ldcg(reinterpret_cast<const longlong2 *>(mt + a * HB + i));
+                    ax = signed_residue(mm.x + (int64_t)ex, q, lb.mu);
+                    ay = signed_residue(mm.y + (int64_t)ey, q, lb.mu);
+                } else {
+                    ax = small_residue(ex, q);
+                    ay = small_residue(ey, q);
+                }
+                // streaming store: the finished ciphertext should not push the waiting products out of L2
+                __stcs(reinterpret_cast<ulonglong2 *>(cc + a * HB + i),
+                       make_ulonglong2(to.m.canon_add(x[a], ax), to.m.canon_add(y[a], ay)));
+            }
+        }
+        cluster.sync();                                          // nobody still reads this block's pieces
+    }
+}
+
+template <int CL>
+__global__ void __launch_bounds__(1024, 1)
+encrypt_cluster_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const int64_t *m, uint32_t t0,
+                       uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
+    extern __shared__ __align__(128) uint64_t sm[];
+    constexpr uint32_t HB = 1u << 13, CS = 1u << CL, ROWS = 2 * CS, N = ROWS * HB, COLS = HB / CS, RT = 1024;
+    int8_t *su = reinterpret_cast<int8_t *>(sm + 2 * HB);        // u, all N coefficients
+    int8_t *se = su + N;                                         // e0 then e1: this block's columns of every row
+    const uint32_t tid = threadIdx.x;
+    __shared__ GaussTables gt;
+    __shared__ uint64_t consts[2 * 8];
+    gauss_tables_init(gt, tid);
+    cg::cluster_group cluster = cg::this_cluster();
+    const uint32_t rank = cluster.block_rank();
+    const uint32_t cid = blockIdx.x / CS, nclusters = gridDim.x / CS;
+
+    // (ciphertext, limb) units in ciphertext-major order, dealt evenly to the clusters
+    const uint64_t units = (uint64_t)T * c.L;
+    const uint32_t u_begin = (uint32_t)(units * cid / nclusters);
+    const uint32_t u_end = (uint32_t)(units * (cid + 1) / nclusters);
+    const size_t cstride = (size_t)c.L * N;
+    uint32_t sampled = 0xffffffffu;
+    for (uint32_t unit = u_begin; unit < u_end; unit++) {
+        const uint32_t tl = unit / c.L, j = unit % c.L;
+        if (tl != sampled) {
+            sampled = tl;
+            const uint32_t t = t0 + tl;
+            __syncthreads();
+            for (uint32_t b = tid; b < N / 4; b += RT) {
+                u32x4 w = stream_block(seed, b, t, client, TAG_ENC_U);
+                char4 v = make_char4((signed char)ternary_from_word(w.x), (signed char)ternary_from_word(w.y),
+                                     (signed char)ternary_from_word(w.z), (signed char)ternary_from_word(w.w));
+                *reinterpret_cast<char4 *>(su + bswz(4 * b)) = v;
+            }
+            // the error terms of the coefficients this block finishes: columns [rank COLS, (rank + 1) COLS) of every row
+            for (uint32_t pp = tid; pp < HB; pp += RT) {
+                const uint32_t a = pp / (COLS / 2), lc = 2 * (pp % (COLS / 2));
+                const uint32_t coef = a * HB + rank * COLS + lc;         // even: one Philox block per pair
+                u32x4 w0 = stream_block(seed, coef >> 1, t, client, TAG_ENC_E0);
+                u32x4 w1 = stream_block(seed, coef >> 1, t, client, TAG_ENC_E1);
+                char2 e0 = make_char2((signed char)gauss_from_u64(gt, (uint64_t)w0.x | ((uint64_t)w0.y << 32)),
+                                      (signed char)gauss_from_u64(gt, (uint64_t)w0.z | ((uint64_t)w0.w << 32)));
+                char2 e1 = make_char2((signed char)gauss_from_u64(gt, (uint64_t)w1.x | ((uint64_t)w1.y << 32)),
+                                      (signed char)gauss_from_u64(gt, (uint64_t)w1.z | ((uint64_t)w1.w << 32)));
+                *reinterpret_cast<char2 *>(se + a * COLS + lc) = e0;
+                *reinterpret_cast<char2 *>(se + 2 * HB + a * COLS + lc) = e1;
+            }
+            __syncthreads();
+        }
+        const LimbDev &lb = c.limb[j];
+        uint64_t *cbase = ct + (((size_t)tl * 2 + 0) * c.L + j) * N;
+        FEDHE_FOR_ARITH_SEL(lb, (encrypt_unit_cluster<M_, CL>(lb, k.pk0_hat + (size_t)j * N, k.pk1_hat + (size_t)j * N, sm,
+                                                             consts, su, se, m + (size_t)tl * N, cbase, cstride, rank,
+                                                             cluster)));
+    }
+}
+
+// Launches the cluster kernel with as many clusters as the device holds at
+// once (74 pairs or 37 quadruples on 148 SMs); *launched is false, and nothing
+// was launched, when the device cannot hold such a cluster.
+template <int CL>
+static cudaError_t launch_encrypt_cluster(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0, size_t T,
+                                          uint64_t seed, uint32_t client, uint64_t *ct, cudaStream_t s,
+                                          bool *launched) {
+    constexpr unsigned CS = 1u << CL;
+    const size_t smem = ((size_t)8 << 14) + (size_t)c.N + ((size_t)2 << 14);
+    auto kern = encrypt_cluster_kernel<CL>;
+    *launched = false;
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = CS;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(CS, 1, 1);
+    cfg.blockDim = dim3(1024, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg) != cudaSuccess || clusters < 1) {
+        cudaGetLastError();                                      // reported by the caller
+        return cudaSuccess;
+    }
+    const size_t units = T * c.L;
+    if ((size_t)clusters > units) clusters = (int)units;
+    cfg.gridDim = dim3((unsigned)clusters * CS, 1, 1);
+    const uint32_t T32 = (uint32_t)T;
+    if ((e = cudaLaunchKernelEx(&cfg, kern, c, k, m, t0, seed, client, ct, T32))) return e;
+    *launched = true;
+    return FEDHE_LAUNCHED();
+}
+
+// Long rings, transform-domain wire format (the coefficient format runs on
+// clusters, above): the error terms go into the ciphertext slots and are
+// transformed there; u is drawn and run through the outer forward stages into a
+// work buffer, block-transformed, and its key products are added on the way out.
 
 template <class M, uint32_t A>
 __device__ __forceinline__ void enc_outer_sample_limb(const LimbDev &lb, const int (&u)[1u << A][2], uint64_t *p,
@@ -394,7 +645,7 @@ __device__ __forceinline__ void enc_outer_sample_limb(const LimbDev &lb, const i
         *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = u64x2{M::bits(x[a]), M::bits(y[a])};
 }
 
-// (1) one thread per pair of neighbouring columns of one ciphertext, all limbs;
+// one thread per pair of neighbouring columns of one ciphertext, all limbs: draws u and runs the outer forward stages;
 // the limbs of ciphertext tl go to dst + tl * ct_stride
 template <uint32_t A>
 __global__ void __launch_bounds__(256)
@@ -422,9 +673,10 @@ enc_outer_sample_kernel(const __grid_constant__ CtxDev c, uint32_t t0, uint64_t 
     }
 }
 
-// (2) one thread block per (ciphertext, limb, block): forward block transform of
-// the c1 slot, products with both halves of the public key on the way out
-template <class M, class L, int V, bool ACC>
+// one thread block per (ciphertext, limb, block): forward block transform of u
+// from `ubuf` ([T][L][N]); the products with both halves of the public key are
+// added to the canonical residues waiting in the ciphertext slots
+template <class M, class L, int V>
 __device__ __forceinline__ void enc_block_forward(const CtxDev &c, const LimbDev &lb, uint64_t *sm, uint32_t blk,
                                                   const tw_t *p0, const tw_t *p1, const uint64_t *u,
                                                   uint64_t *c0, uint64_t *c1) {
@@ -436,28 +688,17 @@ __device__ __forceinline__ void enc_block_forward(const CtxDev &c, const LimbDev
         [&](uint32_t p, val x, val y) {
             const auto a0 = M::load_key(p0 + p), a1 = M::load_key(p0 + p + 1);
             const auto b0 = M::load_key(p1 + p), b1 = M::load_key(p1 + p + 1);
-            u64x2 v0, v1;
-            if constexpr (ACC) {       // the slots hold canonical residues to add to
-                v0 = *reinterpret_cast<const u64x2 *>(c0 + p);
-                v1 = *reinterpret_cast<const u64x2 *>(c1 + p);
-                v0.x = ar.canon_add(ar.mul_key(x, a0), v0.x);
-                v0.y = ar.canon_add(ar.mul_key(y, a1), v0.y);
-                v1.x = ar.canon_add(ar.mul_key(x, b0), v1.x);
-                v1.y = ar.canon_add(ar.mul_key(y, b1), v1.y);
-            } else {
-                v0.x = ar.to_residue(ar.mul_key(x, a0));
-                v0.y = ar.to_residue(ar.mul_key(y, a1));
-                v1.x = ar.to_residue(ar.mul_key(x, b0));
-                v1.y = ar.to_residue(ar.mul_key(y, b1));
-            }
+            u64x2 v0 = *reinterpret_cast<const u64x2 *>(c0 + p), v1 = *reinterpret_cast<const u64x2 *>(c1 + p);
+            v0.x = ar.canon_add(ar.mul_key(x, a0), v0.x);
+            v0.y = ar.canon_add(ar.mul_key(y, a1), v0.y);
+            v1.x = ar.canon_add(ar.mul_key(x, b0), v1.x);
+            v1.y = ar.canon_add(ar.mul_key(y, b1), v1.y);
             *reinterpret_cast<u64x2 *>(c0 + p) = v0;
             *reinterpret_cast<u64x2 *>(c1 + p) = v1;
         });
 }
 
-// ACC = false: u comes from the c1 slot and the products replace both slots;
-// ACC = true: u comes from `ubuf` ([T][L][N]) and the products are added to the slots
-template <class L, int V, bool ACC>
+template <class L, int V>
 __global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
 enc_block_forward_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const uint64_t *ubuf, uint64_t *ct) {
     extern __shared__ __align__(128) uint64_t sm[];
@@ -470,9 +711,9 @@ enc_block_forward_kernel(const __grid_constant__ CtxDev c, const KeysDev k, cons
     const size_t off = ((size_t)blk << L::LOGB);
     uint64_t *c0 = ct + ((tl * 2 + 0) * c.L + j) * c.N + off;
     uint64_t *c1 = ct + ((tl * 2 + 1) * c.L + j) * c.N + off;
-    const uint64_t *u = ACC ? ubuf + (tl * c.L + j) * c.N + off : c1;
+    const uint64_t *u = ubuf + (tl * c.L + j) * c.N + off;
     const tw_t *p0 = k.pk0_hat + (size_t)j * c.N + off, *p1 = k.pk1_hat + (size_t)j * c.N + off;
-    FEDHE_FOR_ARITH(lb, (enc_block_forward<M_, L, V, ACC>(c, lb, sm, blk, p0, p1, u, c0, c1)));
+    FEDHE_FOR_ARITH(lb, (enc_block_forward<M_, L, V>(c, lb, sm, blk, p0, p1, u, c0, c1)));
 }
 
 // long rings, transform-domain format: residues of e0 + m into the c0 slots and
@@ -506,69 +747,6 @@ enc_fill_errors_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint3
     }
 }
 
-template <class M, uint32_t A>
-__device__ __forceinline__ void enc_outer_inverse_add_limb(const LimbDev &lb, uint64_t *p, uint32_t B,
-                                                           const int64_t (&add)[1u << A][2]) {
-    constexpr uint32_t rows = 1u << A;
-    const uint64_t q = lb.q;
-    const auto t = LimbOf<M>::args(lb, false, 0, 0);
-    typename M::val x[rows], y[rows];
-#pragma unroll
-    for (uint32_t a = 0; a < rows; a++) {
-        const u64x2 v = *reinterpret_cast<const u64x2 *>(p + (size_t)a * B);
-        x[a] = M::from_bits(v.x);
-        y[a] = M::from_bits(v.y);
-    }
-    outer_inverse<A>(x, y, t, LimbOf<M>::ninv(lb), LimbOf<M>::wn(lb));
-#pragma unroll
-    for (uint32_t a = 0; a < rows; a++) {
-        u64x2 o;
-        o.x = t.m.canon_add(x[a], signed_residue(add[a][0], q, lb.mu));
-        o.y = t.m.canon_add(y[a], signed_residue(add[a][1], q, lb.mu));
-        *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = o;
-    }
-}
-
-// (4) one thread per pair of neighbouring columns of one ciphertext: for each
-// component draws its error terms once (e0 + m, then e1), then finishes every limb
-template <uint32_t A>
-__global__ void __launch_bounds__(256, A == 3 ? 2 : 4)
-enc_outer_inverse_add_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint32_t t0, uint64_t seed,
-                             uint32_t client, uint64_t *ct, size_t total) {
-    __shared__ GaussTables gt;
-    gauss_tables_init(gt, threadIdx.x);
-    __syncthreads();
-    size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (g >= total) return;
-    const uint32_t B = 1u << c.LOGB, half = B >> 1;
-    constexpr uint32_t rows = 1u << A;
-    const uint32_t col = (uint32_t)(g % half) * 2;
-    const size_t tl = g / half;
-    const uint32_t t = t0 + (uint32_t)tl;
-#pragma unroll 1
-    for (uint32_t comp = 0; comp < 2; comp++) {
-        int64_t add[rows][2];                          // e0 + m, or e1
-#pragma unroll
-        for (uint32_t a = 0; a < rows; a++) {
-            const uint32_t i = a * B + col;           // one Philox block per pair of coefficients
-            const u32x4 w = stream_block(seed, i >> 1, t, client, comp == 0 ? TAG_ENC_E0 : TAG_ENC_E1);
-            add[a][0] = gauss_from_u64(gt, (uint64_t)w.x | ((uint64_t)w.y << 32));
-            add[a][1] = gauss_from_u64(gt, (uint64_t)w.z | ((uint64_t)w.w << 32));
-            if (comp == 0) {
-                const longlong2 mm = *reinterpret_cast<const longlong2 *>(m + tl * c.N + i);
-                add[a][0] += mm.x;
-                add[a][1] += mm.y;
-            }
-        }
-#pragma unroll 1
-        for (uint32_t j = 0; j < c.L; j++) {
-            const LimbDev &lb = c.limb[j];
-            uint64_t *p = ct + ((tl * 2 + comp) * c.L + j) * c.N + col;
-            FEDHE_FOR_ARITH(lb, (enc_outer_inverse_add_limb<M_, A>(lb, p, B, add)));
-        }
-    }
-}
-
 // shared memory of a block of the fused kernels: the limb and three one-byte sample arrays
 static size_t fused_smem(const CtxDev &c) { return ((size_t)c.N << 3) + 3 * (size_t)c.N; }
 
@@ -594,14 +772,13 @@ static cudaError_t launch_encrypt_fused(const CtxDev &c, const KeysDev &k, const
     return FEDHE_LAUNCHED();
 }
 
-// launches the block forward kernel of the long-ring paths
-template <bool ACC>
+// launches the block forward kernel of the long-ring transform-domain path
 static cudaError_t launch_enc_block_forward(const CtxDev &c, const KeysDev &k, const uint64_t *ubuf, size_t T,
                                             uint64_t *ct, cudaStream_t s) {
     using L = WLay<13>;                                 // long rings are cut into 2^13 blocks
     constexpr int V = 2;
     const size_t smem = sizeof(uint64_t) << L::LOGB;
-    auto kern = enc_block_forward_kernel<L, V, ACC>;
+    auto kern = enc_block_forward_kernel<L, V>;
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
     kern<<<(unsigned)((T * c.L) << c.A), L::NT / V, smem, s>>>(c, k, ubuf, ct);
@@ -627,16 +804,12 @@ cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const float *sel, 
     }
     cudaError_t e;
     if ((e = launch_encode(c, sel, T, reinterpret_cast<double2 *>(m + T * c.N), m, s))) return e;
-    const size_t cols = T * ((size_t)1 << (c.LOGB - 1));      // pairs of columns
-    const size_t LN = (size_t)c.L * c.N;
-    FEDHE_FOR_A(c, (enc_outer_sample_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, t0, seed, client, ct + LN,
-                                                                                     2 * LN, cols)));
-    if ((e = FEDHE_LAUNCHED())) return e;
-    if ((e = launch_enc_block_forward<false>(c, k, nullptr, T, ct, s))) return e;
-    if ((e = launch_ntt_inner(c, false, ct, 2 * T, LN, 0, c.L, s))) return e;
-    FEDHE_FOR_A(c, (enc_outer_inverse_add_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, m, t0, seed, client, ct,
-                                                                                          cols)));
-    return FEDHE_LAUNCHED();
+    // clusters of 2 (N = 2^15) or 4 (N = 2^16) thread blocks with up to 225 KB of shared memory each
+    bool launched = false;
+    if (c.logN == 15) e = launch_encrypt_cluster<1>(c, k, m, t0, T, seed, client, ct, s, &launched);
+    else e = launch_encrypt_cluster<2>(c, k, m, t0, T, seed, client, ct, s, &launched);
+    if (e) return e;
+    return launched ? cudaSuccess : cudaErrorLaunchOutOfResources;     // a device that cannot hold such a cluster
 }
 
 // Transform-domain wire format: the same ciphertext with every limb polynomial
@@ -666,7 +839,7 @@ cudaError_t launch_encrypt_ntt(const CtxDev &c, const KeysDev &k, const float *s
     FEDHE_FOR_A(c, (enc_outer_sample_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, t0, seed, client, ubuf, LN,
                                                                                      cols)));
     if ((e = FEDHE_LAUNCHED())) return e;
-    return launch_enc_block_forward<true>(c, k, ubuf, T, ct, s);
+    return launch_enc_block_forward(c, k, ubuf, T, ct, s);
 }
 
 }  // namespace fedhe
