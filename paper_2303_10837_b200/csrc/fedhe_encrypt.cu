@@ -373,9 +373,12 @@ encrypt_fused2_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const f
 }
 
 // ===========================================================================
-// Long rings (N = 2^15, 2^16) on thread-block clusters: a limb of 256 or 512 KB
-// does not fit one SM's shared memory, but it fits the shared memories of a
-// cluster of CS = 2 or 4 thread blocks.  The limb is cut into ROWS = 2 CS
+// Long rings on thread-block clusters: a limb of 256 KB (N = 2^15) does not fit
+// one SM's shared memory, but it fits the shared memories of a cluster of
+// CS = 2 thread blocks.  (The code is written for CS = 2^CL; with CS = 4, for
+// N = 2^16, the device holds only 33 clusters at once, 132 of its 148 SMs, and
+// the kernel measured 25 % slower than the multi-pass path, which N = 2^16
+// therefore keeps.)  The limb is cut into ROWS = 2 CS
 // pieces of HB = 2^13 residues; block `rank` of the cluster holds pieces
 // 2 rank and 2 rank + 1, and each of its two groups of 512 threads transforms
 // one piece as a sub-block of the long transform on its own schedule (named
@@ -623,10 +626,8 @@ static cudaError_t launch_encrypt_cluster(const CtxDev &c, const KeysDev &k, con
     return FEDHE_LAUNCHED();
 }
 
-// Long rings, transform-domain wire format (the coefficient format runs on
-// clusters, above): the error terms go into the ciphertext slots and are
-// transformed there; u is drawn and run through the outer forward stages into a
-// work buffer, block-transformed, and its key products are added on the way out.
+// Long rings without clusters (N = 2^16 in the coefficient format, both long rings in
+// the transform-domain format): kernels over the 2^A x 2^13 view of a limb.
 
 template <class M, uint32_t A>
 __device__ __forceinline__ void enc_outer_sample_limb(const LimbDev &lb, const int (&u)[1u << A][2], uint64_t *p,
@@ -673,10 +674,9 @@ enc_outer_sample_kernel(const __grid_constant__ CtxDev c, uint32_t t0, uint64_t 
     }
 }
 
-// one thread block per (ciphertext, limb, block): forward block transform of u
-// from `ubuf` ([T][L][N]); the products with both halves of the public key are
-// added to the canonical residues waiting in the ciphertext slots
-template <class M, class L, int V>
+// (2) one thread block per (ciphertext, limb, block): forward block transform of
+// the c1 slot, products with both halves of the public key on the way out
+template <class M, class L, int V, bool ACC>
 __device__ __forceinline__ void enc_block_forward(const CtxDev &c, const LimbDev &lb, uint64_t *sm, uint32_t blk,
                                                   const tw_t *p0, const tw_t *p1, const uint64_t *u,
                                                   uint64_t *c0, uint64_t *c1) {
@@ -688,17 +688,28 @@ __device__ __forceinline__ void enc_block_forward(const CtxDev &c, const LimbDev
         [&](uint32_t p, val x, val y) {
             const auto a0 = M::load_key(p0 + p), a1 = M::load_key(p0 + p + 1);
             const auto b0 = M::load_key(p1 + p), b1 = M::load_key(p1 + p + 1);
-            u64x2 v0 = *reinterpret_cast<const u64x2 *>(c0 + p), v1 = *reinterpret_cast<const u64x2 *>(c1 + p);
-            v0.x = ar.canon_add(ar.mul_key(x, a0), v0.x);
-            v0.y = ar.canon_add(ar.mul_key(y, a1), v0.y);
-            v1.x = ar.canon_add(ar.mul_key(x, b0), v1.x);
-            v1.y = ar.canon_add(ar.mul_key(y, b1), v1.y);
+            u64x2 v0, v1;
+            if constexpr (ACC) {       // the slots hold canonical residues to add to
+                v0 = *reinterpret_cast<const u64x2 *>(c0 + p);
+                v1 = *reinterpret_cast<const u64x2 *>(c1 + p);
+                v0.x = ar.canon_add(ar.mul_key(x, a0), v0.x);
+                v0.y = ar.canon_add(ar.mul_key(y, a1), v0.y);
+                v1.x = ar.canon_add(ar.mul_key(x, b0), v1.x);
+                v1.y = ar.canon_add(ar.mul_key(y, b1), v1.y);
+            } else {
+                v0.x = ar.to_residue(ar.mul_key(x, a0));
+                v0.y = ar.to_residue(ar.mul_key(y, a1));
+                v1.x = ar.to_residue(ar.mul_key(x, b0));
+                v1.y = ar.to_residue(ar.mul_key(y, b1));
+            }
             *reinterpret_cast<u64x2 *>(c0 + p) = v0;
             *reinterpret_cast<u64x2 *>(c1 + p) = v1;
         });
 }
 
-template <class L, int V>
+// ACC = false: u comes from the c1 slot and the products replace both slots;
+// ACC = true: u comes from `ubuf` ([T][L][N]) and the products are added to the slots
+template <class L, int V, bool ACC>
 __global__ void __launch_bounds__(L::NT / V, (L::NT / V) <= 512 ? 2 : 1)
 enc_block_forward_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const uint64_t *ubuf, uint64_t *ct) {
     extern __shared__ __align__(128) uint64_t sm[];
@@ -711,9 +722,9 @@ enc_block_forward_kernel(const __grid_constant__ CtxDev c, const KeysDev k, cons
     const size_t off = ((size_t)blk << L::LOGB);
     uint64_t *c0 = ct + ((tl * 2 + 0) * c.L + j) * c.N + off;
     uint64_t *c1 = ct + ((tl * 2 + 1) * c.L + j) * c.N + off;
-    const uint64_t *u = ubuf + (tl * c.L + j) * c.N + off;
+    const uint64_t *u = ACC ? ubuf + (tl * c.L + j) * c.N + off : c1;
     const tw_t *p0 = k.pk0_hat + (size_t)j * c.N + off, *p1 = k.pk1_hat + (size_t)j * c.N + off;
-    FEDHE_FOR_ARITH(lb, (enc_block_forward<M_, L, V>(c, lb, sm, blk, p0, p1, u, c0, c1)));
+    FEDHE_FOR_ARITH(lb, (enc_block_forward<M_, L, V, ACC>(c, lb, sm, blk, p0, p1, u, c0, c1)));
 }
 
 // long rings, transform-domain format: residues of e0 + m into the c0 slots and
@@ -747,6 +758,69 @@ enc_fill_errors_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint3
     }
 }
 
+template <class M, uint32_t A>
+__device__ __forceinline__ void enc_outer_inverse_add_limb(const LimbDev &lb, uint64_t *p, uint32_t B,
+                                                           const int64_t (&add)[1u << A][2]) {
+    constexpr uint32_t rows = 1u << A;
+    const uint64_t q = lb.q;
+    const auto t = LimbOf<M>::args(lb, false, 0, 0);
+    typename M::val x[rows], y[rows];
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++) {
+        const u64x2 v = *reinterpret_cast<const u64x2 *>(p + (size_t)a * B);
+        x[a] = M::from_bits(v.x);
+        y[a] = M::from_bits(v.y);
+    }
+    outer_inverse<A>(x, y, t, LimbOf<M>::ninv(lb), LimbOf<M>::wn(lb));
+#pragma unroll
+    for (uint32_t a = 0; a < rows; a++) {
+        u64x2 o;
+        o.x = t.m.canon_add(x[a], signed_residue(add[a][0], q, lb.mu));
+        o.y = t.m.canon_add(y[a], signed_residue(add[a][1], q, lb.mu));
+        *reinterpret_cast<u64x2 *>(p + (size_t)a * B) = o;
+    }
+}
+
+// (4) one thread per pair of neighbouring columns of one ciphertext: for each
+// component draws its error terms once (e0 + m, then e1), then finishes every limb
+template <uint32_t A>
+__global__ void __launch_bounds__(256, A == 3 ? 2 : 4)
+enc_outer_inverse_add_kernel(const __grid_constant__ CtxDev c, const int64_t *m, uint32_t t0, uint64_t seed,
+                             uint32_t client, uint64_t *ct, size_t total) {
+    __shared__ GaussTables gt;
+    gauss_tables_init(gt, threadIdx.x);
+    __syncthreads();
+    size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t B = 1u << c.LOGB, half = B >> 1;
+    constexpr uint32_t rows = 1u << A;
+    const uint32_t col = (uint32_t)(g % half) * 2;
+    const size_t tl = g / half;
+    const uint32_t t = t0 + (uint32_t)tl;
+#pragma unroll 1
+    for (uint32_t comp = 0; comp < 2; comp++) {
+        int64_t add[rows][2];                          // e0 + m, or e1
+#pragma unroll
+        for (uint32_t a = 0; a < rows; a++) {
+            const uint32_t i = a * B + col;           // one Philox block per pair of coefficients
+            const u32x4 w = stream_block(seed, i >> 1, t, client, comp == 0 ? TAG_ENC_E0 : TAG_ENC_E1);
+            add[a][0] = gauss_from_u64(gt, (uint64_t)w.x | ((uint64_t)w.y << 32));
+            add[a][1] = gauss_from_u64(gt, (uint64_t)w.z | ((uint64_t)w.w << 32));
+            if (comp == 0) {
+                const longlong2 mm = *reinterpret_cast<const longlong2 *>(m + tl * c.N + i);
+                add[a][0] += mm.x;
+                add[a][1] += mm.y;
+            }
+        }
+#pragma unroll 1
+        for (uint32_t j = 0; j < c.L; j++) {
+            const LimbDev &lb = c.limb[j];
+            uint64_t *p = ct + ((tl * 2 + comp) * c.L + j) * c.N + col;
+            FEDHE_FOR_ARITH(lb, (enc_outer_inverse_add_limb<M_, A>(lb, p, B, add)));
+        }
+    }
+}
+
 // shared memory of a block of the fused kernels: the limb and three one-byte sample arrays
 static size_t fused_smem(const CtxDev &c) { return ((size_t)c.N << 3) + 3 * (size_t)c.N; }
 
@@ -772,13 +846,14 @@ static cudaError_t launch_encrypt_fused(const CtxDev &c, const KeysDev &k, const
     return FEDHE_LAUNCHED();
 }
 
-// launches the block forward kernel of the long-ring transform-domain path
+// launches the block forward kernel of the long-ring paths
+template <bool ACC>
 static cudaError_t launch_enc_block_forward(const CtxDev &c, const KeysDev &k, const uint64_t *ubuf, size_t T,
                                             uint64_t *ct, cudaStream_t s) {
     using L = WLay<13>;                                 // long rings are cut into 2^13 blocks
     constexpr int V = 2;
     const size_t smem = sizeof(uint64_t) << L::LOGB;
-    auto kern = enc_block_forward_kernel<L, V>;
+    auto kern = enc_block_forward_kernel<L, V, ACC>;
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
     kern<<<(unsigned)((T * c.L) << c.A), L::NT / V, smem, s>>>(c, k, ubuf, ct);
@@ -804,12 +879,28 @@ cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const float *sel, 
     }
     cudaError_t e;
     if ((e = launch_encode(c, sel, T, reinterpret_cast<double2 *>(m + T * c.N), m, s))) return e;
-    // clusters of 2 (N = 2^15) or 4 (N = 2^16) thread blocks with up to 225 KB of shared memory each
-    bool launched = false;
-    if (c.logN == 15) e = launch_encrypt_cluster<1>(c, k, m, t0, T, seed, client, ct, s, &launched);
-    else e = launch_encrypt_cluster<2>(c, k, m, t0, T, seed, client, ct, s, &launched);
-    if (e) return e;
-    return launched ? cudaSuccess : cudaErrorLaunchOutOfResources;     // a device that cannot hold such a cluster
+    if (c.logN == 15) {
+        // N = 2^15: clusters of two thread blocks, 74 of them on 148 SMs
+        bool launched = false;
+        if ((e = launch_encrypt_cluster<1>(c, k, m, t0, T, seed, client, ct, s, &launched))) return e;
+        return launched ? cudaSuccess : cudaErrorLaunchOutOfResources;     // a device that cannot hold such a cluster
+    }
+    // N = 2^16 would need clusters of four blocks, of which the device holds only 33 at once
+    // (132 of its 148 SMs; measured 25 % slower than the passes below): the ciphertext buffer
+    // itself is the work space, and every pass over it does as much as it can.
+    // (1) draw u and run the outer forward stages into the c1 slots; (2) block transforms of the
+    // c1 slots whose last phase writes both products u^ pk0^ -> c0 and u^ pk1^ -> c1; (3) inverse
+    // block transforms of all slots; (4) outer inverse stages fused with the error and message terms.
+    const size_t cols = T * ((size_t)1 << (c.LOGB - 1));      // pairs of columns
+    const size_t LN = (size_t)c.L * c.N;
+    FEDHE_FOR_A(c, (enc_outer_sample_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, t0, seed, client, ct + LN,
+                                                                                     2 * LN, cols)));
+    if ((e = FEDHE_LAUNCHED())) return e;
+    if ((e = launch_enc_block_forward<false>(c, k, nullptr, T, ct, s))) return e;
+    if ((e = launch_ntt_inner(c, false, ct, 2 * T, LN, 0, c.L, s))) return e;
+    FEDHE_FOR_A(c, (enc_outer_inverse_add_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, m, t0, seed, client, ct,
+                                                                                          cols)));
+    return FEDHE_LAUNCHED();
 }
 
 // Transform-domain wire format: the same ciphertext with every limb polynomial
@@ -839,7 +930,7 @@ cudaError_t launch_encrypt_ntt(const CtxDev &c, const KeysDev &k, const float *s
     FEDHE_FOR_A(c, (enc_outer_sample_kernel<A_><<<blocks_for(cols, 256), 256, 0, s>>>(c, t0, seed, client, ubuf, LN,
                                                                                      cols)));
     if ((e = FEDHE_LAUNCHED())) return e;
-    return launch_enc_block_forward(c, k, ubuf, T, ct, s);
+    return launch_enc_block_forward<true>(c, k, ubuf, T, ct, s);
 }
 
 }  // namespace fedhe
