@@ -62,7 +62,8 @@ UNIT = "params/s"
 # the profile_case.py encrypt case (summaries under profiles/; traffic grows in proportion to the
 # number of ciphertexts).  An entry is dropped (None is reported) when the kernel has changed
 # since its counters were taken.
-ENCRYPT_DRAM_BYTES_PER_CT = {}
+ENCRYPT_DRAM_BYTES_PER_CT = {(16384, 4): 367.657984e6 / 296,       # encrypt_fused2_kernel, 296 ciphertexts
+                             (32768, 6): 505.139968e6 / 148}       # encrypt_cluster_kernel, 148 ciphertexts (without the encoder kernels)
 SLOTS_PER_SM_CLK = 64.0
 WIDE_COST = 2.5
 INT_SLOTS_PER_BUTTERFLY = 6 * WIDE_COST + 4
@@ -395,7 +396,7 @@ def measure(job, w, steps, warmup, with_cpu_baseline):
     kern_ms = max(enc_ms - encode_ms, 1e-6)
 
     # standalone transform: forward + inverse over a batch larger than L2
-    B = 256 if w.N <= 16384 else 64
+    B = 256
     polys = torch.from_numpy(si.random_residues(7, (B, w.L, w.N), w.primes).view(np.int64)).cuda()
     he.he_ntt_forward(g, polys)
     he.he_ntt_inverse(g, polys)
@@ -462,6 +463,15 @@ def measure(job, w, steps, warmup, with_cpu_baseline):
         # the encoder runs inside the kernel: (n/2) log2 n complex butterflies of 10 double-precision operations
         slots_per_ct += (n // 2) * (n.bit_length() - 1) * ENCODE_SLOTS_PER_BUTTERFLY
     achieved = slots_per_ct * per_launch / (kern_ms * 1e-3) / 1e12
+    # Everything else the method makes the kernel compute on the same pipe, per ciphertext:
+    # Philox4x32-10 (ten rounds of two 32x32->64 products for each of the N/4 + N/2 + N/2 blocks behind
+    # u, e0, e1), the two products with the public key per coefficient and limb, and the factor 1/N
+    # (one more product per butterfly of the last stage of both inverse transforms).
+    ints = sum(1 for q in w.primes if q >= F64_PRIME_LIMIT)
+    f64s = w.L - ints
+    per_product = ints * INT_SLOTS_PER_BUTTERFLY + f64s * 6.0
+    extra_per_ct = 1.25 * w.N * 20 * WIDE_COST + (2 * w.N + w.N) * per_product
+    achieved_all = (slots_per_ct + (0 if transform else extra_per_ct)) * per_launch / (kern_ms * 1e-3) / 1e12
     peak = job.n_sm * SLOTS_PER_SM_CLK * job.peaks["sm_max_mhz"] * 1e6 / 1e12
     alg_bytes = (4.0 + 32.0 * w.L) * n * per_launch          # read the slots, write the ciphertext
     if w.N <= 16384:
@@ -473,6 +483,7 @@ def measure(job, w, steps, warmup, with_cpu_baseline):
         "bound": "alu", "achieved": achieved, "peak": peak,
         "unit": "T slots/s (integer-multiply / double-precision pipe)",
         "frac": achieved / peak,
+        "frac_all_required_work": achieved_all / peak,
         "traffic": ENCRYPT_DRAM_BYTES_PER_CT.get((w.N, w.L), None) and ENCRYPT_DRAM_BYTES_PER_CT[(w.N, w.L)] * per_launch,
         "algorithmic_bytes": alg_bytes,
         "ms_per_launch": kern_ms, "launches_per_step": w.clients, "kernels_per_he_encrypt": int(launches_per_encrypt),
