@@ -419,11 +419,6 @@ __device__ __forceinline__ void encrypt_unit_cluster(const LimbDev &lb, const tw
     uint64_t *smg = sm + grp * HB;
     const GroupSync gsync = {1 + grp, GT};
     const uint64_t q = lb.q;
-    // the message words of this block's columns will be wanted at the end of the first pass
-    for (uint32_t c2 = tid; c2 < COLS / 2; c2 += RT)
-#pragma unroll
-        for (uint32_t a = 0; a < ROWS; a++)
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(mt + a * HB + rank * COLS + 2 * c2));
     // row `row` of the outer forward stages applied to the unit vectors
     if (gt < ROWS) {
         const auto fo = LimbOf<M>::args(lb, true, 0, 0);
@@ -532,8 +527,10 @@ __device__ __forceinline__ void encrypt_unit_cluster(const LimbDev &lb, const tw
 
 template <int CL>
 __global__ void __launch_bounds__(1024, 1)
-encrypt_cluster_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const int64_t *m, uint32_t t0,
-                       uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
+encrypt_cluster_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const float *sel, int64_t *mscr,
+                       uint32_t t0, uint64_t seed, uint32_t client, uint64_t *ct, uint32_t T) {
+    using LF = Lay<14 - CL, 3>;                                  // this block's share of the slot transform
+    static_assert(CL == 1, "the encoder is split over a cluster of two blocks");
     extern __shared__ __align__(128) uint64_t sm[];
     constexpr uint32_t HB = 1u << 13, CS = 1u << CL, ROWS = 2 * CS, N = ROWS * HB, COLS = HB / CS, RT = 1024;
     int8_t *su = reinterpret_cast<int8_t *>(sm + 2 * HB);        // u, all N coefficients
@@ -551,6 +548,7 @@ encrypt_cluster_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const 
     const uint32_t u_begin = (uint32_t)(units * cid / nclusters);
     const uint32_t u_end = (uint32_t)(units * (cid + 1) / nclusters);
     const size_t cstride = (size_t)c.L * N;
+    int64_t *mcl = mscr + (size_t)cid * N;                        // this cluster's encoded message (stays in L2)
     uint32_t sampled = 0xffffffffu;
     for (uint32_t unit = u_begin; unit < u_end; unit++) {
         const uint32_t tl = unit / c.L, j = unit % c.L;
@@ -577,13 +575,33 @@ encrypt_cluster_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const 
                 *reinterpret_cast<char2 *>(se + a * COLS + lc) = e0;
                 *reinterpret_cast<char2 *>(se + 2 * HB + a * COLS + lc) = e1;
             }
-            __syncthreads();
+            // The ciphertext's message.  The slot transform of n = N/2 values is split over the
+            // two blocks: the first stage pairs slot i with slot i + n/2, and each block computes
+            // its own half of that stage straight from the slots (real inputs, no exchange), then
+            // runs the remaining stages on its half in the limb buffer.  Block `rank` produces the
+            // coefficients of parity `rank`; both write to the cluster's scratch.
+            {
+                constexpr uint32_t half = N / 4;                 // n / 2
+                const float *slots = sel + (size_t)tl * (N / 2);
+                const double2 *ftw = c.ftw;
+                const bool bad = encode_block_in_place<LF>(
+                    c,
+                    [&](uint32_t i) {
+                        const cpx U = cpx{(double)__ldg(slots + i), 0.0}, V = cpx{(double)__ldg(slots + i + half), 0.0};
+                        if (rank == 0) return cadd_rn(U, V);
+                        cpx w = load_ftw(ftw, half + i);
+                        w.im = -w.im;
+                        return cmul_rn(csub_rn(U, V), w);
+                    },
+                    sm, mcl, 1, rank);
+                if (bad) atomicOr(c.status, 1);
+            }
+            cluster.sync();                                      // both halves of the message are written
         }
         const LimbDev &lb = c.limb[j];
         uint64_t *cbase = ct + (((size_t)tl * 2 + 0) * c.L + j) * N;
         FEDHE_FOR_ARITH_SEL(lb, (encrypt_unit_cluster<M_, CL>(lb, k.pk0_hat + (size_t)j * N, k.pk1_hat + (size_t)j * N, sm,
-                                                             consts, su, se, m + (size_t)tl * N, cbase, cstride, rank,
-                                                             cluster)));
+                                                             consts, su, se, mcl, cbase, cstride, rank, cluster)));
     }
 }
 
@@ -591,9 +609,9 @@ encrypt_cluster_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const 
 // once (74 pairs or 37 quadruples on 148 SMs); *launched is false, and nothing
 // was launched, when the device cannot hold such a cluster.
 template <int CL>
-static cudaError_t launch_encrypt_cluster(const CtxDev &c, const KeysDev &k, const int64_t *m, uint32_t t0, size_t T,
-                                          uint64_t seed, uint32_t client, uint64_t *ct, cudaStream_t s,
-                                          bool *launched) {
+static cudaError_t launch_encrypt_cluster(const CtxDev &c, const KeysDev &k, const float *sel, int64_t *mscr,
+                                          size_t max_clusters, uint32_t t0, size_t T, uint64_t seed, uint32_t client,
+                                          uint64_t *ct, cudaStream_t s, bool *launched) {
     constexpr unsigned CS = 1u << CL;
     const size_t smem = ((size_t)8 << 14) + (size_t)c.N + ((size_t)2 << 14);
     auto kern = encrypt_cluster_kernel<CL>;
@@ -619,9 +637,10 @@ static cudaError_t launch_encrypt_cluster(const CtxDev &c, const KeysDev &k, con
     }
     const size_t units = T * c.L;
     if ((size_t)clusters > units) clusters = (int)units;
+    if ((size_t)clusters > max_clusters) clusters = (int)max_clusters;     // the message scratch has room for so many
     cfg.gridDim = dim3((unsigned)clusters * CS, 1, 1);
     const uint32_t T32 = (uint32_t)T;
-    if ((e = cudaLaunchKernelEx(&cfg, kern, c, k, m, t0, seed, client, ct, T32))) return e;
+    if ((e = cudaLaunchKernelEx(&cfg, kern, c, k, sel, mscr, t0, seed, client, ct, T32))) return e;
     *launched = true;
     return FEDHE_LAUNCHED();
 }
@@ -862,6 +881,7 @@ static cudaError_t launch_enc_block_forward(const CtxDev &c, const KeysDev &k, c
 
 size_t encrypt_work_bytes(const CtxDev &c, int n_sm, size_t T, bool ntt_out) {
     if (c.A == 0) return encrypt_fused_blocks(c, n_sm) * c.N * sizeof(int64_t);
+    if (c.logN == 15 && !ntt_out) return (size_t)(n_sm / 2) * c.N * sizeof(int64_t);      // N words per cluster of two blocks
     // long rings: the encoded messages and the encoder's complex buffer; the
     // transform-domain format transforms u in a buffer of its own
     return (2 * T * c.N + (ntt_out ? T * (size_t)c.L * c.N : 0)) * sizeof(uint64_t);
@@ -878,13 +898,14 @@ cudaError_t launch_encrypt(const CtxDev &c, const KeysDev &k, const float *sel, 
         return launch_encrypt_fused<WLay<13>, 2, true, false>(c, k, sel, m, n_sm, t0, T, seed, client, ct, s);
     }
     cudaError_t e;
-    if ((e = launch_encode(c, sel, T, reinterpret_cast<double2 *>(m + T * c.N), m, s))) return e;
     if (c.logN == 15) {
-        // N = 2^15: clusters of two thread blocks, 74 of them on 148 SMs
+        // N = 2^15: clusters of two thread blocks, 74 of them on 148 SMs, encoder inside
         bool launched = false;
-        if ((e = launch_encrypt_cluster<1>(c, k, m, t0, T, seed, client, ct, s, &launched))) return e;
+        if ((e = launch_encrypt_cluster<1>(c, k, sel, m, (size_t)(n_sm / 2), t0, T, seed, client, ct, s, &launched)))
+            return e;
         return launched ? cudaSuccess : cudaErrorLaunchOutOfResources;     // a device that cannot hold such a cluster
     }
+    if ((e = launch_encode(c, sel, T, reinterpret_cast<double2 *>(m + T * c.N), m, s))) return e;
     // N = 2^16 would need clusters of four blocks, of which the device holds only 33 at once
     // (132 of its 148 SMs; measured 25 % slower than the passes below): the ciphertext buffer
     // itself is the work space, and every pass over it does as much as it can.

@@ -116,23 +116,29 @@ __device__ __forceinline__ uint32_t bitrev(uint32_t v, int bits) { return __brev
 // spreads them over the banks (checked exhaustively for both block sizes)
 __device__ __forceinline__ uint32_t stage_swz(uint32_t k) { return k ^ (((k >> 8) ^ (k >> 4)) & 15u); }
 
-// The whole encoder of one slot vector inside a thread block of LF::NT threads
-// (n = 2^LF::LOGB slots): the network, the scaling by Delta/n, the rounding
-// and the bit-reversal.  `sm` is a buffer of n cpx values (= N words), used
-// first for the exchanges between phases and then to put the rounded integers
-// in order; m_out receives the N coefficients.  Ends with a block barrier
-// after which `sm` is free and m_out may be read by the block.  Returns
-// whether a coefficient left the range (the caller raises the status word).
-template <class LF>
-__device__ __forceinline__ bool encode_in_block(const CtxDev &c, const float *slots, uint64_t *sm, int64_t *m_out) {
-    constexpr uint32_t n = 1u << LF::LOGB;
-    const uint32_t tid = threadIdx.x;
+// The encoder of one block of 2^LF::LOGB slots inside a thread block of LF::NT
+// threads: the network, the scaling by Delta/n, the rounding and the
+// bit-reversal.  `in(i)` gives the complex value at position i of the block as
+// it enters the block's stages (the slot itself when the block is the whole
+// vector, the output of the earlier stages otherwise); `sm` is a buffer of
+// 2^LF::LOGB cpx values, used first for the exchanges between phases and then
+// to put the rounded integers in order; coefficient kk of the block (kk its
+// bit-reversed position) goes to m_out[(kk << A) | rb] and its imaginary
+// partner to m_out[((kk << A) | rb) + n], where the whole vector has
+// n = 2^(LF::LOGB + A) slots and rb is the bit-reversed block number.  Ends with
+// a block barrier after which `sm` is free and m_out may be read by the block.
+// Returns whether a coefficient left the range (the caller raises the status word).
+template <class LF, class In>
+__device__ __forceinline__ bool encode_block_in_place(const CtxDev &c, const In &in, uint64_t *sm, int64_t *m_out,
+                                                      uint32_t A, uint32_t rb) {
+    constexpr uint32_t NB = 1u << LF::LOGB;
+    const uint32_t tid = threadIdx.x, n = NB << A;
     cpx x[LF::E];
 #pragma unroll
-    for (int r = 0; r < LF::E; r++) x[r] = cpx{(double)__ldg(slots + LF::template idx<0>(tid, r)), 0.0};
+    for (int r = 0; r < LF::E; r++) x[r] = in(LF::template idx<0>(tid, r));
     block_dif<LF>(x, reinterpret_cast<cpx *>(sm), tid, c.ftw);
     // Delta / n is a power of two: one exact multiplication
-    const double scale = __longlong_as_double((long long)(1023 + c.log2_delta - LF::LOGB) << 52);
+    const double scale = __longlong_as_double((long long)(1023 + c.log2_delta - (int)(LF::LOGB + A)) << 52);
     const double lim = 4611686018427387904.0;   // 2^62
     bool bad = false;
     int64_t *stage = reinterpret_cast<int64_t *>(sm);
@@ -143,15 +149,22 @@ __device__ __forceinline__ bool encode_in_block(const CtxDev &c, const float *sl
         double re = __dmul_rn(x[r].re, scale), im = __dmul_rn(x[r].im, scale);
         if (!(fabs(re) < lim) || !(fabs(im) < lim)) { bad = true; re = 0.0; im = 0.0; }
         stage[stage_swz(kk)] = __double2ll_rn(re);
-        stage[n + stage_swz(kk)] = __double2ll_rn(im);
+        stage[NB + stage_swz(kk)] = __double2ll_rn(im);
     }
     __syncthreads();
-    for (uint32_t kk = tid; kk < n; kk += LF::NT) {
-        m_out[kk] = stage[stage_swz(kk)];
-        m_out[kk + n] = stage[n + stage_swz(kk)];
+    for (uint32_t kk = tid; kk < NB; kk += LF::NT) {
+        const uint32_t k = (kk << A) | rb;
+        m_out[k] = stage[stage_swz(kk)];
+        m_out[k + n] = stage[NB + stage_swz(kk)];
     }
     __syncthreads();
     return bad;
+}
+
+// the whole encoder of one slot vector of 2^LF::LOGB slots
+template <class LF>
+__device__ __forceinline__ bool encode_in_block(const CtxDev &c, const float *slots, uint64_t *sm, int64_t *m_out) {
+    return encode_block_in_place<LF>(c, [&](uint32_t i) { return cpx{(double)__ldg(slots + i), 0.0}; }, sm, m_out, 0, 0);
 }
 
 }  // namespace fedhe

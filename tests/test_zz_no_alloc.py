@@ -35,12 +35,17 @@ def test_noalloc_decrypt_matches_decrypt_twice_in_a_row():
     he.he_decrypt_noalloc(g, keys, aggs[1], outs[0])
     torch.cuda.synchronize()
     free_before, _ = torch.cuda.mem_get_info()
+    stats_before = torch.cuda.memory_stats()
     # back to back on one stream: the second call reuses the array the first one filled
     he.he_decrypt_noalloc(g, keys, aggs[0], outs[0])
     he.he_decrypt_noalloc(g, keys, aggs[1], outs[1])
     torch.cuda.synchronize()
     free_after, _ = torch.cuda.mem_get_info()
     assert free_after == free_before                 # nothing was allocated on the device
+    # the free-memory figure is device-wide; torch's own allocator must not have moved either
+    stats_after = torch.cuda.memory_stats()
+    for key in ("num_alloc_retries", "allocation.all.allocated", "segment.all.allocated"):
+        assert stats_after.get(key, 0) == stats_before.get(key, 0), key
     for got, ref in zip(outs, want):
         assert float((got - ref).abs().max()) <= DECODE_TOL
     assert float((outs[0] - outs[1]).abs().max()) > 1e-4      # the two results really differ
