@@ -63,7 +63,7 @@ UNIT = "params/s"
 # number of ciphertexts).  An entry is dropped (None is reported) when the kernel has changed
 # since its counters were taken.
 ENCRYPT_DRAM_BYTES_PER_CT = {(16384, 4): 367.657984e6 / 296,       # encrypt_fused2_kernel, 296 ciphertexts
-                             (32768, 6): 505.139968e6 / 148}       # encrypt_cluster_kernel, 148 ciphertexts (without the encoder kernels)
+                             (32768, 6): 478.102528e6 / 148}       # encrypt_cluster_kernel, 148 ciphertexts
 SLOTS_PER_SM_CLK = 64.0
 WIDE_COST = 2.5
 INT_SLOTS_PER_BUTTERFLY = 6 * WIDE_COST + 4
@@ -308,7 +308,10 @@ def measure(job, w, steps, warmup, with_cpu_baseline):
         sels, rests = [], []
         for i in range(w.clients):
             if by_index and mask is None:           # full encryption: the rank's slots are a slice of x
-                sel, rest = he.he_pack(g, None, xs[i][sb:se])
+                if se > sb:
+                    sel, rest = he.he_pack(g, None, xs[i][sb:se])
+                else:                               # more ranks than ciphertexts: nothing for this one
+                    sel, rest = torch.empty(0, dtype=torch.float32, device="cuda"), None
             else:
                 sel, rest = he.he_pack(g, mask, xs[i])
                 sel = sel[tb * n:te * n]
@@ -423,16 +426,17 @@ def measure(job, w, steps, warmup, with_cpu_baseline):
             Pe = se - sb
         else:
             xh, Pe = xs_host, w.P
+        host_out = torch.empty(max(Pe, 1), dtype=torch.float64).pin_memory()[:Pe]
         if Pe:
-            host_out = torch.empty(Pe, dtype=torch.float64).pin_memory()
             he.he_round_host(g, keys, mask, xh, alpha, enc_seed, host_out)          # allocates its buffers
-            job.barrier()
-            e2e_steps = max(1, min(steps, 3))
-            t0 = time.perf_counter()
-            for _ in range(e2e_steps):
-                he.he_round_host(g, keys, mask, xh, alpha, enc_seed, host_out)
-            torch.cuda.synchronize()
-            e2e_secs = time.perf_counter() - t0
+        job.barrier()                                   # every rank, also one without work
+        e2e_steps = max(1, min(steps, 3))
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps if Pe else 0):
+            he.he_round_host(g, keys, mask, xh, alpha, enc_seed, host_out)
+        torch.cuda.synchronize()
+        e2e_secs = time.perf_counter() - t0
+        if Pe:
             ref = want[sb:se] if by_index else want
             if not float((host_out.cuda() - ref).abs().max()) <= 1e-6:
                 raise SystemExit("bench: host round differs from plaintext FedAvg")
@@ -442,8 +446,10 @@ def measure(job, w, steps, warmup, with_cpu_baseline):
     mine = float(w.P) if not by_index else float((se - sb) + (re - rb))
     units, job_secs = reduce_job(mine * steps, secs, world, "cuda")
     e2e_line = None
+    if not by_index or mask is None:                # the same on every rank: every rank joins the reduction
+        mine_e2e = e2e if e2e is not None else (0.0, 0.0, 0, 0, 0)
+        eu, es = reduce_job(mine_e2e[0], mine_e2e[1], world, "cuda")
     if e2e is not None:
-        eu, es = reduce_job(e2e[0], e2e[1], world, "cuda")
         e2e_line = {"value": eu / es, "unit": UNIT, "h2d_bytes_per_step": e2e[3], "d2h_bytes_per_step": e2e[4],
                     "steps": e2e[2]}
         if by_index:
@@ -484,7 +490,8 @@ def measure(job, w, steps, warmup, with_cpu_baseline):
         "unit": "T slots/s (integer-multiply / double-precision pipe)",
         "frac": achieved / peak,
         "frac_all_required_work": achieved_all / peak,
-        "traffic": ENCRYPT_DRAM_BYTES_PER_CT.get((w.N, w.L), None) and ENCRYPT_DRAM_BYTES_PER_CT[(w.N, w.L)] * per_launch,
+        "traffic": (ENCRYPT_DRAM_BYTES_PER_CT[(w.N, w.L)] * per_launch
+                    if (w.N, w.L) in ENCRYPT_DRAM_BYTES_PER_CT and not transform else None),
         "algorithmic_bytes": alg_bytes,
         "ms_per_launch": kern_ms, "launches_per_step": w.clients, "kernels_per_he_encrypt": int(launches_per_encrypt),
         "butterflies_per_launch": butterflies,
