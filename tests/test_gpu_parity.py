@@ -491,6 +491,45 @@ def test_host_round_refuses_bad_arguments_before_queueing(he):
     assert np.abs(host.numpy() - want).max() <= FEDAVG_TOL
 
 
+def test_index_partition_reproduces_the_whole_round(he):
+    """The multi-GPU partition (contiguous ciphertext indices and remainder entries per rank, context,
+    keys and mask replicated), played by one GPU one rank after the other: the ranks' ciphertexts,
+    aggregates, decoded slots and plaintext averages, put side by side, are the single run's, bit for bit."""
+    from paper_2303_10837_b200.sharding import shard_range, slot_range
+    w = si.Workload("partition", 16384, si.PRIMES_N16384, 40, 3, 7 * 8192 + 123, 0.01, ratio=0.6, seed=9,
+                    key_seed=91, enc_seed=92)                      # 5 ciphertexts, the last one ragged
+    g, _ = contexts(he, w.N, w.primes, w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    xs, alpha = [dev_f32(x) for x in si.client_updates(w)], si.client_weights(w)
+    mask = he.he_select_mask(g, dev_f32(si.sensitivity_scores(w)), w.k)
+    packed = [he.he_pack(g, mask, x) for x in xs]
+    cts = [he.he_encrypt(g, keys, sel, w.enc_seed, i) for i, (sel, _) in enumerate(packed)]
+    agg = he.he_weighted_aggregate(g, cts, alpha)
+    z = he.he_decrypt(g, keys, agg)
+    ravg = he.he_plain_aggregate(g, [rest for _, rest in packed], alpha)
+    whole = he.he_unpack(g, mask, z, ravg, w.P)
+    world = 3
+    z_parts, r_parts = [], []
+    for rank in range(world):
+        tb, te, sb, se = slot_range(w.T, w.n, w.k, rank, world)
+        rb, re = shard_range(w.P - w.k, rank, world)
+        mine = []
+        for i, (sel, _) in enumerate(packed):
+            ct = torch.empty((te - tb, 2, w.L, w.N), dtype=torch.int64, device="cuda")
+            he.he_encrypt_range(g, keys, sel[tb * w.n:te * w.n], tb, te - tb, w.enc_seed, i, ct)
+            assert torch.equal(ct, cts[i][tb:te])
+            mine.append(ct)
+        a = he.he_weighted_aggregate(g, mine, alpha)
+        assert torch.equal(a, agg[tb:te])
+        z_parts.append(he.he_decrypt(g, keys, a)[: se - sb])
+        r_parts.append(he.he_plain_aggregate(g, [rest[rb:re] for _, rest in packed], alpha))
+    zf = torch.cat(z_parts)
+    assert zf.numel() == w.k and torch.equal(zf, z[: w.k])
+    assert torch.equal(torch.cat(r_parts), ravg)
+    pad = torch.zeros(w.T * w.n - w.k, dtype=torch.float64, device="cuda")
+    assert torch.equal(he.he_unpack(g, mask, torch.cat([zf, pad]), torch.cat(r_parts), w.P), whole)
+
+
 def test_runs_are_deterministic(he):
     """Bit-identical outputs on repeated runs (a race would show up here)."""
     w = si.scaled(si.RESNET18, 5 * 8192, clients=2)
