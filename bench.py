@@ -222,9 +222,12 @@ def run_reference(args, w):
 def config_dict(w, note):
     return {"workload": w.name, "N": w.N, "slots": w.n, "limbs": w.L, "log2_delta": w.log2_delta,
             "clients": w.clients, "params": w.P, "encrypted_params": w.k, "ciphertexts_per_client": w.T,
-            "l2": "inputs larger than L2 (%.1f GB of ciphertexts per step%s)"
-                  % (w.clients * w.T * 2 * w.L * w.N * 8 / 1e9,
-                     ", streamed in chunks of ciphertext indices" if w.clients * w.T * 2 * w.L * w.N * 8 > 40e9 else ""),
+            "l2": ("inputs larger than L2 (%.1f GB of ciphertexts per step%s)"
+                   % (w.clients * w.T * 2 * w.L * w.N * 8 / 1e9,
+                      ", streamed in chunks of ciphertext indices" if w.clients * w.T * 2 * w.L * w.N * 8 > 40e9 else "")
+                   if w.clients * w.T * 2 * w.L * w.N * 8 > 126e6 else
+                   "the small case: %.0f MB of ciphertexts per step fit the L2 and are not flushed between steps"
+                   % (w.clients * w.T * 2 * w.L * w.N * 8 / 1e6)),
             "note": note}
 
 
