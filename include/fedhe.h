@@ -275,14 +275,18 @@ int he_ntt_inverse(he_ctx *ctx, uint64_t *polys_dev, size_t B, void *stream);
  * the merged global model back.
  *   xs: host array of C host pointers float[P]; alpha: host double[C];
  *   mask: NULL = full encryption; w_glob: host double[P].
- * Synchronous; allocates its device buffers through the context.  Uploads of
- * the next client and (with full encryption) downloads of a finished chunk
- * run on a second stream beside the arithmetic; they overlap it only when xs
- * and w_glob are page-locked (pinned) host memory, pageable memory is
- * correct but serialises.  With full encryption parts of w_glob are written
+ * Synchronous; allocates its device buffers through the context.  Uploads and
+ * downloads run on two streams of their own beside the arithmetic: with full
+ * encryption the slots of the next chunk of ciphertext indices (a contiguous
+ * piece of every update) go up while the current chunk is computed, and the
+ * decoded slots of a finished chunk go home while the next is computed; with
+ * a mask the whole update of the next client goes up while the current one is
+ * packed and encrypted.  They overlap the arithmetic only when xs and w_glob
+ * are page-locked (pinned) host memory; pageable memory is correct but
+ * serialises.  With full encryption parts of w_glob are written
  * before the call returns; after an error return its contents are unspecified.
  * Bad arguments (a NULL xs[i], a weight outside [0, 1]) are refused before
- * anything is queued.  On every return, error or not, both streams have been
+ * anything is queued.  On every return, error or not, all streams have been
  * waited for: no copy is still reading xs or writing w_glob. */
 int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const float *const *xs_host,
                   const double *alpha_host, int C, size_t P, uint64_t enc_seed, double *w_glob_host,

@@ -165,6 +165,7 @@ int he_ctx_destroy(he_ctx *ctx) {
     if (ctx->tab) cudaFree(ctx->tab);
     if (ctx->round_buf) cudaFree(ctx->round_buf);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+    if (ctx->down_stream) cudaStreamDestroy(ctx->down_stream);
     for (int i = 0; i < 2; i++) {
         if (ctx->ev_ready[i]) cudaEventDestroy(ctx->ev_ready[i]);
         if (ctx->ev_free[i]) cudaEventDestroy(ctx->ev_free[i]);
@@ -691,19 +692,144 @@ int he_threshold_combine(he_ctx *ctx, const uint64_t *ct_dev, uint32_t level, co
 // whole round from host memory
 // ---------------------------------------------------------------------------
 
-// The queued part of he_round_host; every argument has been validated.
+static int round_host_streams(he_ctx *ctx) {
+    if (ctx->copy_stream) return HE_OK;
+    CU(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+    CU(cudaStreamCreateWithFlags(&ctx->down_stream, cudaStreamNonBlocking));
+    for (int i = 0; i < 2; i++) {
+        CU(cudaEventCreateWithFlags(&ctx->ev_ready[i], cudaEventDisableTiming));
+        CU(cudaEventCreateWithFlags(&ctx->ev_free[i], cudaEventDisableTiming));
+    }
+    CU(cudaEventCreateWithFlags(&ctx->ev_chunk, cudaEventDisableTiming));
+    return HE_OK;
+}
+
+// The queued part of he_round_host with full encryption (no mask): the packed
+// slots of a chunk of ciphertext indices are a contiguous piece of every
+// client's update, so each chunk's pieces go straight from the host into the
+// slot buffers (no staging copy of the whole update, no pack kernel), on the
+// upload stream, one chunk ahead of the arithmetic; the decoded slots of a
+// chunk go home on the download stream while the next chunk is computed.
+// Chunks start at one wave of thread blocks, so that little is uploaded before
+// the first kernel can start, and double up to about 8 GiB of ciphertexts.
+static int round_host_full(he_ctx *ctx, const he_keys *keys, const float *const *xs_host, const double *alpha_host,
+                           int C, size_t P, uint64_t enc_seed, double *w_glob_host, void *stream) {
+    const CtxDev &d = ctx->dev;
+    const size_t n = d.N / 2, T = he_num_ct(ctx, P);
+    const size_t ctw = 2 * (size_t)d.L * d.N, aggw = 2 * (size_t)(d.L - 1) * d.N;
+    const size_t sm = (size_t)ctx->sm_count;
+    size_t cap = ((size_t)8 << 30) / (C * ctw * sizeof(uint64_t));
+    if (cap > sm) cap -= cap % sm;
+    if (cap < 1) cap = 1;
+    std::vector<size_t> sizes;
+    for (size_t done = 0, cur = sm < cap ? sm : cap; done < T;) {
+        size_t tc = T - done < cur ? T - done : cur;
+        if (T - done - tc < sm / 2) tc = T - done;          // no sliver at the end
+        if (tc > cap && cap >= sm) tc = cap;
+        sizes.push_back(tc);
+        done += tc;
+        cur = 2 * cur < cap ? 2 * cur : cap;
+    }
+    // the download of the last chunk's slots is not hidden behind anything: keep that chunk to one wave
+    if (sizes.size() > 1 && sizes.back() >= 2 * sm) {
+        sizes.back() -= sm;
+        sizes.push_back(sm);
+    }
+    size_t Tmax = 0;
+    for (size_t v : sizes) Tmax = v > Tmax ? v : Tmax;
+    auto align = [](size_t b) { return (b + 255) & ~(size_t)255; };
+    const size_t b_sel = align(Tmax * n * sizeof(float)), b_cts = align(C * Tmax * ctw * sizeof(uint64_t)),
+                 b_agg = align(Tmax * aggw * sizeof(uint64_t)), b_z = align(T * n * sizeof(double));
+    int rc = ensure(&ctx->round_buf, &ctx->round_bytes, 2 * C * b_sel + b_cts + b_agg + b_z);
+    if (rc != HE_OK) return rc;
+    {
+        size_t need = encrypt_work_bytes(d, ctx->sm_count, Tmax, false);
+        if (d.A > 0 && work_bytes(ctx, Tmax) > need) need = work_bytes(ctx, Tmax);
+        rc = ensure(&ctx->ws, &ctx->ws_bytes, need);
+    }
+    if (rc != HE_OK) return rc;
+    if ((rc = round_host_streams(ctx)) != HE_OK) return rc;
+    unsigned char *p = static_cast<unsigned char *>(ctx->round_buf);
+    unsigned char *selbuf[2];
+    selbuf[0] = p; p += C * b_sel;
+    selbuf[1] = p; p += C * b_sel;
+    uint64_t *cts = reinterpret_cast<uint64_t *>(p); p += b_cts;
+    uint64_t *agg = reinterpret_cast<uint64_t *>(p); p += b_agg;
+    double *z = reinterpret_cast<double *>(p);
+    cudaStream_t st = as_stream(stream);
+    CU(cudaEventRecord(ctx->ev_free[0], st));       // earlier work on `st` may still use the buffers
+    CU(cudaEventRecord(ctx->ev_free[1], st));
+
+    // one client's slots of the chunk [t0, t0 + tc) into the slot buffers of parity b
+    auto upload_client = [&](int b, int i, size_t t0, size_t tc) -> int {
+        const size_t first = t0 * n, want = tc * n, have = P - first < want ? P - first : want;
+        float *dst = reinterpret_cast<float *>(selbuf[b] + (size_t)i * b_sel);
+        CU(cudaMemcpyAsync(dst, xs_host[i] + first, have * sizeof(float), cudaMemcpyHostToDevice, ctx->copy_stream));
+        if (have < want)                             // the ragged tail of the last ciphertext
+            CU(cudaMemsetAsync(dst + have, 0, (want - have) * sizeof(float), ctx->copy_stream));
+        return HE_OK;
+    };
+    auto upload = [&](size_t c, size_t t0, size_t tc) -> int {
+        const int b = (int)(c & 1);
+        CU(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_free[b], 0));
+        for (int i = 0; i < C; i++) {
+            const int urc = upload_client(b, i, t0, tc);
+            if (urc != HE_OK) return urc;
+        }
+        CU(cudaEventRecord(ctx->ev_ready[b], ctx->copy_stream));
+        return HE_OK;
+    };
+    std::vector<const uint64_t *> cptr(C);
+    size_t t0 = 0;
+    for (size_t c = 0; c < sizes.size(); c++) {
+        const size_t tc = sizes[c];
+        const int b = (int)(c & 1);
+        if (c == 0) CU(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_free[b], 0));
+        else CU(cudaStreamWaitEvent(st, ctx->ev_ready[b], 0));
+        for (int i = 0; i < C; i++) {
+            if (c == 0) {
+                // the first chunk client by client: a client's encryption starts as soon as its own
+                // slots have arrived (a wait takes the event's latest record at the time of the call)
+                if ((rc = upload_client(b, i, t0, tc)) != HE_OK) return rc;
+                CU(cudaEventRecord(ctx->ev_ready[b], ctx->copy_stream));
+                CU(cudaStreamWaitEvent(st, ctx->ev_ready[b], 0));
+            }
+            uint64_t *ci = cts + (size_t)i * Tmax * ctw;
+            rc = he_encrypt_range(ctx, keys, reinterpret_cast<const float *>(selbuf[b] + (size_t)i * b_sel), t0, tc,
+                                  enc_seed, (uint32_t)i, ci, stream);
+            if (rc != HE_OK) return rc;
+            cptr[i] = ci;
+        }
+        CU(cudaEventRecord(ctx->ev_free[b], st));   // the slot buffers of this parity may be refilled
+        // the next chunk's slots go up while this chunk is computed
+        if (c + 1 < sizes.size() && (rc = upload(c + 1, t0 + tc, sizes[c + 1])) != HE_OK) return rc;
+        rc = he_weighted_aggregate(ctx, cptr.data(), alpha_host, C, tc, agg, stream);
+        if (rc != HE_OK) return rc;
+        rc = he_decrypt(ctx, keys, agg, tc, z + t0 * n, stream);
+        if (rc != HE_OK) return rc;
+        const size_t first = t0 * n, count = P - first < tc * n ? P - first : tc * n;
+        CU(cudaEventRecord(ctx->ev_chunk, st));
+        CU(cudaStreamWaitEvent(ctx->down_stream, ctx->ev_chunk, 0));
+        CU(cudaMemcpyAsync(w_glob_host + first, z + first, count * sizeof(double), cudaMemcpyDeviceToHost,
+                           ctx->down_stream));
+        t0 += tc;
+    }
+    return HE_OK;                                    // the caller waits for the streams
+}
+
+// The queued part of he_round_host with a mask; every argument has been validated.
 static int round_host_queued(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const float *const *xs_host,
                              const double *alpha_host, int C, size_t P, size_t k, uint64_t enc_seed,
                              double *w_glob_host, void *stream) {
     const CtxDev &d = ctx->dev;
     const size_t n = d.N / 2, T = he_num_ct(ctx, k), padded = T * n, restlen = P - k;
     const size_t ctw = 2 * (size_t)d.L * d.N, aggw = 2 * (size_t)(d.L - 1) * d.N;
+    // The mask gathers from anywhere in an update, so every client's whole
+    // update is uploaded (two staging buffers on the upload stream: the upload of
+    // client i+1 overlaps the packing and first encryption of client i).
     // Ciphertext indices are processed in chunks that keep all clients'
     // ciphertexts of a chunk within about 8 GiB; a chunk is a whole number of
-    // waves of one thread block per SM.  When there is enough work the first
-    // chunk takes half of it, so that encrypting a client's share of it
-    // outlasts the upload of the next client's update, and the rest goes in two
-    // chunks, so that the download of a chunk's result hides behind the next.
+    // waves of one thread block per SM.
     const size_t sm = (size_t)ctx->sm_count;
     auto whole_waves = [&](size_t want, size_t cap) {
         size_t v = want < cap ? want : cap;
@@ -742,70 +868,35 @@ static int round_host_queued(he_ctx *ctx, const he_keys *keys, const he_mask *ma
     double *out = reinterpret_cast<double *>(p);
     cudaStream_t st = as_stream(stream);
 
-    if (!ctx->copy_stream) {
-        CU(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
-        for (int i = 0; i < 2; i++) {
-            CU(cudaEventCreateWithFlags(&ctx->ev_ready[i], cudaEventDisableTiming));
-            CU(cudaEventCreateWithFlags(&ctx->ev_free[i], cudaEventDisableTiming));
-        }
-        CU(cudaEventCreateWithFlags(&ctx->ev_chunk, cudaEventDisableTiming));
-    }
-    // The upload of client i+1 (copy stream, two staging buffers) overlaps
-    // the packing of client i and the encryption of its first chunk.
+    if ((rc = round_host_streams(ctx)) != HE_OK) return rc;
     CU(cudaEventRecord(ctx->ev_free[0], st));       // earlier work on `st` may still use the buffers
     CU(cudaEventRecord(ctx->ev_free[1], st));
     std::vector<const uint64_t *> cptr(C);
     for (size_t t0 = 0, step = Tc; t0 < T || t0 == 0; t0 += step, step = Tc_rest) {
         const size_t tc = T - t0 < step ? T - t0 : step;
         for (int i = 0; i < C; i++) {
-            // With full encryption the first client's update is uploaded in two pieces so
-            // that its first chunk can be encrypted while the rest is still on its way
-            // (every later upload hides behind the arithmetic of the client before).
-            size_t head = P;
             const int b = i & 1;
             if (t0 == 0) {
-                if (!mask && i == 0 && Tc < T) head = Tc * n;
                 CU(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_free[b], 0));
-                CU(cudaMemcpyAsync(x[b], xs_host[i], head * sizeof(float), cudaMemcpyHostToDevice, ctx->copy_stream));
+                CU(cudaMemcpyAsync(x[b], xs_host[i], P * sizeof(float), cudaMemcpyHostToDevice, ctx->copy_stream));
                 CU(cudaEventRecord(ctx->ev_ready[b], ctx->copy_stream));
-                if (head < P) {
-                    CU(cudaMemcpyAsync(x[b] + head, xs_host[i] + head, (P - head) * sizeof(float),
-                                       cudaMemcpyHostToDevice, ctx->copy_stream));
-                    CU(cudaEventRecord(ctx->ev_chunk, ctx->copy_stream));
-                }
                 CU(cudaStreamWaitEvent(st, ctx->ev_ready[b], 0));
-                rc = he_pack(ctx, mask, x[b], head, sel[i], restlen ? rest[i] : nullptr, stream);
+                rc = he_pack(ctx, mask, x[b], P, sel[i], restlen ? rest[i] : nullptr, stream);
                 if (rc != HE_OK) return rc;
-                if (head == P) CU(cudaEventRecord(ctx->ev_free[b], st));
+                CU(cudaEventRecord(ctx->ev_free[b], st));
             }
             if (tc == 0) continue;
             uint64_t *ci = cts + (size_t)i * Tc * ctw;
             rc = he_encrypt_range(ctx, keys, sel[i] + t0 * n, t0, tc, enc_seed, (uint32_t)i, ci, stream);
             if (rc != HE_OK) return rc;
             cptr[i] = ci;
-            if (t0 == 0 && head < P) {          // the rest of the first client's slots
-                CU(cudaStreamWaitEvent(st, ctx->ev_chunk, 0));
-                rc = he_pack(ctx, nullptr, x[b] + head, P - head, sel[i] + head, nullptr, stream);
-                if (rc != HE_OK) return rc;
-                CU(cudaEventRecord(ctx->ev_free[b], st));
-            }
         }
         if (tc == 0) break;
         rc = he_weighted_aggregate(ctx, cptr.data(), alpha_host, C, tc, agg, stream);
         if (rc != HE_OK) return rc;
         rc = he_decrypt(ctx, keys, agg, tc, z + t0 * n, stream);
         if (rc != HE_OK) return rc;
-        if (!mask) {
-            // full encryption: the decoded slots are the result, in order; send this
-            // chunk's part home on the copy stream while the next chunk is computed
-            const size_t first = t0 * n, count = P - first < tc * n ? P - first : tc * n;
-            CU(cudaEventRecord(ctx->ev_chunk, st));
-            CU(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_chunk, 0));
-            CU(cudaMemcpyAsync(w_glob_host + first, z + first, count * sizeof(double), cudaMemcpyDeviceToHost,
-                               ctx->copy_stream));
-        }
     }
-    if (!mask) return HE_OK;                        // the caller waits for both streams
     if (restlen) {
         std::vector<const float *> rptr(rest.begin(), rest.end());
         rc = he_plain_aggregate(ctx, rptr.data(), alpha_host, C, restlen, ravg, stream);
@@ -833,13 +924,15 @@ int he_round_host(he_ctx *ctx, const he_keys *keys, const he_mask *mask, const f
         if (!xs_host[i]) return HE_ERR_INVALID_ARG;
         if (!(alpha_host[i] >= 0.0) || !(alpha_host[i] <= 1.0)) return HE_ERR_INVALID_ARG;
     }
-    const int rc = round_host_queued(ctx, keys, mask, xs_host, alpha_host, C, P, k, enc_seed, w_glob_host, stream);
+    const int rc = mask ? round_host_queued(ctx, keys, mask, xs_host, alpha_host, C, P, k, enc_seed, w_glob_host, stream)
+                        : round_host_full(ctx, keys, xs_host, alpha_host, C, P, enc_seed, w_glob_host, stream);
     // Success or not, nothing may still be reading xs or writing w_glob when the
     // call returns: wait for both streams (on an error path their status is ignored).
     cudaError_t e0 = ctx->copy_stream ? cudaStreamSynchronize(ctx->copy_stream) : cudaSuccess;
     cudaError_t e1 = cudaStreamSynchronize(as_stream(stream));
+    cudaError_t e2 = ctx->down_stream ? cudaStreamSynchronize(ctx->down_stream) : cudaSuccess;
     if (rc != HE_OK) return rc;
-    return (e0 == cudaSuccess && e1 == cudaSuccess) ? HE_OK : HE_ERR_CUDA;
+    return (e0 == cudaSuccess && e1 == cudaSuccess && e2 == cudaSuccess) ? HE_OK : HE_ERR_CUDA;
 }
 
 }  // extern "C"

@@ -82,6 +82,7 @@ struct he_ctx {
     size_t round_bytes = 0;
     int sm_count = 0;
     cudaStream_t copy_stream = nullptr;   // uploads of he_round_host, overlapped with compute
+    cudaStream_t down_stream = nullptr;   // downloads of he_round_host (PCIe carries both directions at once)
     cudaEvent_t ev_ready[2] = {nullptr, nullptr}, ev_free[2] = {nullptr, nullptr};
     cudaEvent_t ev_chunk = nullptr;       // a chunk's result is ready for download
 };
