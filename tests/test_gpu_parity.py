@@ -366,6 +366,23 @@ def test_host_round_in_several_chunks(he):
     assert np.abs(out - want).max() <= FEDAVG_TOL
 
 
+@pytest.mark.parametrize("P,clients", [(1, 1), (4096, 2), (148 * 4096, 1), (449 * 4096 + 17, 3), (30 * 4096 - 1, 5)])
+def test_host_round_sizes(he, P, clients):
+    """The host-buffer entry point on one context after the other of several sizes (one slot, exactly
+    one ciphertext, exactly one wave, several chunks with a ragged tail, more clients): the same bits
+    as the device calls, whatever the chunk schedule."""
+    w = si.scaled(si.TINY, P, clients=clients, name="host-%d-%d" % (P, clients))
+    g = he.he_ctx_create(w.N, list(w.primes), w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    xs, alpha = si.client_updates(w), si.client_weights(w)
+    out = run_round_gpu(he, g, keys, None, xs, alpha, w)
+    for _ in range(2):                                  # the second call reuses the buffers of the first
+        host = torch.full((w.P,), np.nan, dtype=torch.float64).pin_memory()
+        he.he_round_host(g, keys, None, [torch.from_numpy(x).pin_memory() for x in xs], alpha, w.enc_seed, host)
+        assert np.array_equal(host.numpy(), out)
+    assert he.he_ctx_status(g) == he.HE_OK
+
+
 def test_selective_round_with_mask(he):
     """Config 3 shape at reduced size: top-10 % encrypted, the rest averaged in plaintext."""
     w = si.scaled(si.RESNET50_TOP10, 300_000, clients=4)
