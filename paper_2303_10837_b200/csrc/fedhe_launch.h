@@ -82,7 +82,7 @@ cudaError_t launch_threshold_combine(const CtxDev &c, const uint64_t *ct, uint32
 int ctx_workspace(he_ctx *ctx, size_t T, void **out);
 
 // mask construction (blocks of MASK_BLOCK consecutive parameters)
-constexpr uint32_t MASK_BLOCK = 1024;
+constexpr uint32_t MASK_BLOCK = 4096;
 // progress of the radix selection, in device memory: the key prefix found so far (tau after
 // the last step) and how many keys are still to be covered (after the last step: how many keys
 // equal to tau belong to the mask)

@@ -14,7 +14,7 @@ __device__ __forceinline__ uint32_t score_key(float s) {
     return ((b & 0x80000000u) || b > 0x7f800000u) ? 0u : b;
 }
 
-// exclusive prefix sum inside a block of 1024 threads; returns the block total
+// exclusive prefix sum over the threads of a block (any whole number of warps up to 32); the block total goes to `total`
 __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t *warp_sums, uint32_t &total) {
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t inc = v;
@@ -26,7 +26,7 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t *w
     if (lane == 31) warp_sums[warp] = inc;
     __syncthreads();
     if (warp == 0) {
-        uint32_t w = warp_sums[lane], winc = w;
+        uint32_t w = lane < ((blockDim.x + 31u) >> 5) ? warp_sums[lane] : 0u, winc = w;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
             const uint32_t o = __shfl_up_sync(0xffffffffu, winc, d);
@@ -111,19 +111,38 @@ cudaError_t launch_radix_pick(const uint32_t *hist, int digit_bits, SelectState 
     return FEDHE_LAUNCHED();
 }
 
-// number of keys equal to tau in every block of MASK_BLOCK parameters
-__global__ void __launch_bounds__(MASK_BLOCK)
-mask_count_eq_kernel(const float *score, size_t P, const SelectState *state, uint32_t *blk_eq) {
+// Keys of the four neighbouring parameters a thread takes (one 16-byte load
+// where the pointer allows and all four exist; key 0 beyond the end).
+__device__ __forceinline__ void load_keys4(const float *score, size_t P, size_t i0, bool vec, uint32_t (&key)[4]) {
+    if (vec && i0 + 4 <= P) {
+        const float4 v = __ldg(reinterpret_cast<const float4 *>(score + i0));
+        key[0] = score_key(v.x); key[1] = score_key(v.y); key[2] = score_key(v.z); key[3] = score_key(v.w);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; j++) key[j] = i0 + j < P ? score_key(__ldg(score + i0 + j)) : 0u;
+    }
+}
+
+// number of keys equal to tau in every block of MASK_BLOCK parameters (four per thread)
+__global__ void __launch_bounds__(MASK_BLOCK / 4)
+mask_count_eq_kernel(const float *score, size_t P, const SelectState *state, uint32_t *blk_eq, bool vec) {
+    __shared__ uint32_t warp_sums[33];
     const uint32_t tau = state->prefix;
-    const size_t i = (size_t)blockIdx.x * MASK_BLOCK + threadIdx.x;
-    const bool eq = i < P && score_key(__ldg(score + i)) == tau;
-    const int n = __syncthreads_count(eq);
-    if (threadIdx.x == 0) blk_eq[blockIdx.x] = (uint32_t)n;
+    const size_t i0 = (size_t)blockIdx.x * MASK_BLOCK + 4 * threadIdx.x;
+    uint32_t key[4];
+    load_keys4(score, P, i0, vec, key);
+    uint32_t cnt = 0;
+#pragma unroll
+    for (int j = 0; j < 4; j++) cnt += (i0 + j < P && key[j] == tau) ? 1u : 0u;
+    uint32_t tot;
+    block_exclusive_scan(cnt, warp_sums, tot);
+    if (threadIdx.x == 0) blk_eq[blockIdx.x] = tot;
 }
 
 cudaError_t launch_mask_count_eq(const float *score, size_t P, const SelectState *state, uint32_t *blk_eq,
                                  cudaStream_t s) {
-    mask_count_eq_kernel<<<blocks_for(P, MASK_BLOCK), MASK_BLOCK, 0, s>>>(score, P, state, blk_eq);
+    const bool vec = (reinterpret_cast<uintptr_t>(score) & 15u) == 0;
+    mask_count_eq_kernel<<<blocks_for(P, MASK_BLOCK), MASK_BLOCK / 4, 0, s>>>(score, P, state, blk_eq, vec);
     return FEDHE_LAUNCHED();
 }
 
@@ -153,54 +172,77 @@ cudaError_t launch_scan(uint32_t *a, size_t count, uint32_t *total, cudaStream_t
 }
 
 // membership bits: key > tau, or key == tau and fewer than `need` equal keys
-// at lower indices, or inside a forced index range
-__global__ void __launch_bounds__(MASK_BLOCK)
+// at lower indices, or inside a forced index range.  A thread takes four
+// neighbouring parameters; eight neighbouring lanes put their four bits
+// together into one word of the bit mask.
+__global__ void __launch_bounds__(MASK_BLOCK / 4)
 mask_select_kernel(const float *score, size_t P, const SelectState *state, const uint64_t *ranges,
-                   uint32_t nranges, const uint32_t *blk_eq_prefix, uint32_t *bits, uint32_t *blk_sel) {
+                   uint32_t nranges, const uint32_t *blk_eq_prefix, uint32_t *bits, uint32_t *blk_sel, bool vec) {
     __shared__ uint32_t warp_sums[33];
     const uint32_t tau = state->prefix, need = state->need;
-    const size_t i = (size_t)blockIdx.x * MASK_BLOCK + threadIdx.x;
-    const uint32_t key = i < P ? score_key(__ldg(score + i)) : 0u;
-    const bool eq = i < P && key == tau;
+    const size_t i0 = (size_t)blockIdx.x * MASK_BLOCK + 4 * threadIdx.x;
+    uint32_t key[4];
+    load_keys4(score, P, i0, vec, key);
+    uint32_t eqs = 0;
+#pragma unroll
+    for (int j = 0; j < 4; j++) eqs += (i0 + j < P && key[j] == tau) ? 1u : 0u;
     uint32_t tot;
-    const uint32_t eq_before = blk_eq_prefix[blockIdx.x] + block_exclusive_scan(eq ? 1u : 0u, warp_sums, tot);
-    bool sel = i < P && (key > tau || (eq && eq_before < need));
-    if (i < P && !sel) {
-        for (uint32_t r = 0; r < nranges; r++)
-            if (i >= ranges[2 * r] && i < ranges[2 * r + 1]) sel = true;
+    uint32_t eq_before = blk_eq_prefix[blockIdx.x] + block_exclusive_scan(eqs, warp_sums, tot);
+    uint32_t nibble = 0, cnt = 0;
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+        const size_t i = i0 + j;
+        if (i >= P) continue;
+        const bool eq = key[j] == tau;
+        bool sel = key[j] > tau || (eq && eq_before < need);
+        eq_before += eq ? 1u : 0u;
+        if (!sel)
+            for (uint32_t r = 0; r < nranges; r++)
+                if (i >= ranges[2 * r] && i < ranges[2 * r + 1]) sel = true;
+        nibble |= sel ? (1u << j) : 0u;
+        cnt += sel ? 1u : 0u;
     }
-    const uint32_t word = __ballot_sync(0xffffffffu, sel);
-    if ((threadIdx.x & 31) == 0 && i < P) bits[i >> 5] = word;
-    const int n = __syncthreads_count(sel);
-    if (threadIdx.x == 0) blk_sel[blockIdx.x] = (uint32_t)n;
+    const uint32_t lane = threadIdx.x & 31u;
+    uint32_t word = nibble << (4u * (lane & 7u));
+    word |= __shfl_xor_sync(0xffffffffu, word, 1);
+    word |= __shfl_xor_sync(0xffffffffu, word, 2);
+    word |= __shfl_xor_sync(0xffffffffu, word, 4);
+    if ((lane & 7u) == 0 && i0 < P) bits[i0 >> 5] = word;
+    block_exclusive_scan(cnt, warp_sums, tot);
+    if (threadIdx.x == 0) blk_sel[blockIdx.x] = tot;
 }
 
 cudaError_t launch_mask_select(const float *score, size_t P, const SelectState *state,
                                const uint64_t *ranges, uint32_t nranges, const uint32_t *blk_eq_prefix,
                                uint32_t *bits, uint32_t *blk_sel, cudaStream_t s) {
-    mask_select_kernel<<<blocks_for(P, MASK_BLOCK), MASK_BLOCK, 0, s>>>(score, P, state, ranges, nranges,
-                                                                        blk_eq_prefix, bits, blk_sel);
+    const bool vec = (reinterpret_cast<uintptr_t>(score) & 15u) == 0;
+    mask_select_kernel<<<blocks_for(P, MASK_BLOCK), MASK_BLOCK / 4, 0, s>>>(score, P, state, ranges, nranges,
+                                                                            blk_eq_prefix, bits, blk_sel, vec);
     return FEDHE_LAUNCHED();
 }
 
-// per-word prefix counts and the ascending index list
-__global__ void __launch_bounds__(MASK_BLOCK)
+// per-word prefix counts and the ascending index list: a thread takes one word
+// of the bit mask (32 parameters), a block the MASK_BLOCK / 32 words of one
+// counted block
+__global__ void __launch_bounds__(MASK_BLOCK / 32)
 mask_write_kernel(size_t P, const uint32_t *bits, const uint32_t *blk_sel_prefix, uint32_t *wpre,
                   uint32_t *idx) {
     __shared__ uint32_t warp_sums[33];
-    const size_t i = (size_t)blockIdx.x * MASK_BLOCK + threadIdx.x;
-    const uint32_t lane = threadIdx.x & 31;
-    const uint32_t word = i < P ? bits[i >> 5] : 0u;      // same for the whole warp
-    const bool sel = i < P && ((word >> lane) & 1u);
+    const size_t word = (size_t)blockIdx.x * (MASK_BLOCK / 32) + threadIdx.x, nwords = (P + 31) >> 5;
+    uint32_t w = word < nwords ? bits[word] : 0u;
     uint32_t tot;
-    const uint32_t before = blk_sel_prefix[blockIdx.x] + block_exclusive_scan(sel ? 1u : 0u, warp_sums, tot);
-    if (lane == 0 && i < P) wpre[i >> 5] = before;
-    if (sel) idx[before] = (uint32_t)i;
+    uint32_t before = blk_sel_prefix[blockIdx.x] + block_exclusive_scan((uint32_t)__popc(w), warp_sums, tot);
+    if (word < nwords) wpre[word] = before;
+    const uint32_t base = (uint32_t)(word << 5);
+    while (w) {
+        idx[before++] = base + (uint32_t)(__ffs((int)w) - 1);
+        w &= w - 1u;
+    }
 }
 
 cudaError_t launch_mask_write(size_t P, const uint32_t *bits, const uint32_t *blk_sel_prefix,
                               uint32_t *wpre, uint32_t *idx, cudaStream_t s) {
-    mask_write_kernel<<<blocks_for(P, MASK_BLOCK), MASK_BLOCK, 0, s>>>(P, bits, blk_sel_prefix, wpre, idx);
+    mask_write_kernel<<<blocks_for(P, MASK_BLOCK), MASK_BLOCK / 32, 0, s>>>(P, bits, blk_sel_prefix, wpre, idx);
     return FEDHE_LAUNCHED();
 }
 
