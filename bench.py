@@ -485,8 +485,10 @@ def measure(job, w, steps, warmup, with_cpu_baseline):
     alg_bytes = (4.0 + 32.0 * w.L) * n * per_launch          # read the slots, write the ciphertext
     if w.N <= 16384:
         kname = "encrypt_fused2_kernel" if w.N == 16384 else "encrypt_fused_kernel"
+    elif launches_per_encrypt == 1:
+        kname = "encrypt_cluster_kernel"                     # one limb per pair of thread blocks (N = 32768)
     else:
-        kname = "the kernels of he_encrypt on a long ring (N > 16384), timed as one call"
+        kname = "the %d kernels of he_encrypt on this ring, timed as one call" % launches_per_encrypt
     roofline = {
         "kernel": kname,
         "bound": "alu", "achieved": achieved, "peak": peak,

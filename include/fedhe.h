@@ -115,7 +115,10 @@ int he_keys_export(he_ctx *ctx, const he_keys *keys, uint64_t *pk_dev, int8_t *s
  * sensitivity score.  key(score) = its fp32 bit pattern if the sign bit is
  * clear and it is not NaN, else 0; order by key descending, index ascending;
  * the first k form the mask.  score: dev float[P], P < 2^32, 0 <= k <= P.
- * Synchronous (the result sizes are needed on the host). */
+ * Synchronous (the result sizes are needed on the host).  The mask's device
+ * buffers come from a per-device memory pool that the library creates on
+ * first use and keeps until the process ends; he_mask_destroy returns them
+ * to the pool, which holds at most 256 MiB of unused memory. */
 int he_select_mask(he_ctx *ctx, const float *score_dev, size_t P, size_t k, he_mask **out, void *stream);
 /* Variant for the paper's empirical selection recipe (the top-p most
  * sensitive parameters as well as whole layers, e.g. the first and last):

@@ -3,6 +3,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -277,6 +278,31 @@ int he_keys_export(he_ctx *ctx, const he_keys *keys, uint64_t *pk_dev, int8_t *s
 // mask
 // ---------------------------------------------------------------------------
 
+// Masks are made and dropped once per round, and a plain device allocation costs more than the
+// kernels of the selection.  Their buffers therefore come from one memory pool per device, made
+// on first use and kept for the life of the process; the pool hands freed buffers out again and
+// gives back to the driver only what it holds beyond MASK_POOL_KEEP bytes.
+static constexpr uint64_t MASK_POOL_KEEP = 256ull << 20;
+static cudaMemPool_t mask_pool(int device) {
+    static std::mutex mu;
+    static cudaMemPool_t pools[64] = {};
+    if (device < 0 || device >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!pools[device]) {
+        cudaMemPoolProps props = {};
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = device;
+        cudaMemPool_t pool = nullptr;
+        if (cudaMemPoolCreate(&pool, &props) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        uint64_t keep = MASK_POOL_KEEP;
+        cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+        pools[device] = pool;
+    }
+    return pools[device];
+}
+
 static int build_mask(he_ctx *ctx, const float *score, size_t P, size_t k, const uint64_t *ranges_host,
                       size_t num_ranges, he_mask **out, void *stream) {
     if (!good(ctx) || !out || (!score && P) || k > P) return HE_ERR_INVALID_ARG;
@@ -307,8 +333,13 @@ static int build_mask(he_ctx *ctx, const float *score, size_t P, size_t k, const
     // The mask owns one allocation: bit mask | per-word prefix counts | index list (its size is
     // known up to the overlap of the forced ranges with the top-k set and with each other).
     uint32_t *bits = nullptr;
-    if (cudaMalloc(reinterpret_cast<void **>(&bits), (2 * nwords + (kmax ? kmax : 1)) * sizeof(uint32_t)) != cudaSuccess)
+    cudaMemPool_t pool = mask_pool(ctx->device);
+    if (!pool) return HE_ERR_CUDA;
+    if (cudaMallocFromPoolAsync(reinterpret_cast<void **>(&bits), (2 * nwords + (kmax ? kmax : 1)) * sizeof(uint32_t),
+                                pool, st) != cudaSuccess) {
+        cudaGetLastError();
         return HE_ERR_ALLOC;
+    }
     uint32_t *wpre = bits + nwords, *idx = wpre + nwords;
     int rc = HE_OK;
     he_mask *m = nullptr;
@@ -355,7 +386,7 @@ static int build_mask(he_ctx *ctx, const float *score, size_t P, size_t k, const
     } while (0);
     if (rc != HE_OK) {
         cudaStreamSynchronize(st);           // nothing may still write the allocation
-        cudaFree(bits);
+        cudaFreeAsync(bits, st);
         return rc;
     }
     *out = m;
@@ -388,7 +419,7 @@ int he_mask_copy_indices(const he_mask *mask, uint32_t *out_dev, void *stream) {
 int he_mask_destroy(he_mask *mask) {
     if (!good(mask)) return HE_ERR_INVALID_ARG;
     cudaDeviceSynchronize();
-    cudaFree(mask->bits);      // prefix counts and index list are parts of this allocation
+    cudaFreeAsync(mask->bits, nullptr);      // back to the pool; prefix counts and index list are parts of this allocation
     mask->magic = 0;
     delete mask;
     return HE_OK;
