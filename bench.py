@@ -267,8 +267,19 @@ def measure(job, w, steps, warmup, with_cpu_baseline):
     by_index = world > 1 and args.shard == "index"
     transform = args.format == "transform"
 
-    g = he.he_ctx_create(w.N, list(w.primes), w.log2_delta)
-    keys = he.he_keygen(g, w.key_seed)
+    # one-off steps (not part of a round): timed on the host around a device synchronisation
+    one_off = {}
+
+    def timed(name, fn):
+        torch.cuda.synchronize()
+        t_start = time.perf_counter()
+        r = fn()
+        torch.cuda.synchronize()
+        one_off[name] = 1e3 * (time.perf_counter() - t_start)
+        return r
+
+    g = timed("ctx_create", lambda: he.he_ctx_create(w.N, list(w.primes), w.log2_delta))
+    keys = timed("keygen", lambda: he.he_keygen(g, w.key_seed))
     alpha = si.client_weights(w)
     T, n = w.T, w.n
     # what this rank works on: everything (one GPU, or one batch per rank), or its range of one round
@@ -290,7 +301,9 @@ def measure(job, w, steps, warmup, with_cpu_baseline):
     xs = [x.cuda() for x in xs_host]
     mask, idx = None, None
     if w.k < w.P:
-        mask = he.he_select_mask(g, torch.from_numpy(si.sensitivity_scores(w)).cuda(), w.k)
+        scores = torch.from_numpy(si.sensitivity_scores(w)).cuda()
+        mask = timed("select_mask", lambda: he.he_select_mask(g, scores, w.k))
+        del scores
         idx = he.he_mask_indices(mask).long()
     # ciphertext indices are streamed in chunks when all clients' ciphertexts of this rank exceed 40 GB
     ct_bytes = 8 * 2 * w.L * w.N
@@ -526,6 +539,10 @@ def measure(job, w, steps, warmup, with_cpu_baseline):
         "gpu_launches": int(launches),
         "roofline": roofline,
         "max_abs_err_vs_fedavg": err,
+        # encrypted parameters / time of one client's he_encrypt calls (this rank's share when the round is cut)
+        "param_encryptions_per_s": float(se - sb) / (enc_ms * 1e-3) if enc_ms > 0 else None,
+        # not part of a round: once per task (context, keys) and once per mask (first round)
+        "one_off_ms": {k_: round(v_, 3) for k_, v_ in one_off.items()},
     }
     if with_cpu_baseline:
         cpu_ct = min(w.T, 768)
