@@ -22,8 +22,10 @@ indices [T r / N, T (r+1) / N) and the same share of the plaintext remainder,
 with context, keys and mask replicated and no collective on the path
 (``--gather`` adds the one all-gather of the decoded pieces, for when one
 place needs the whole model); fixed total work, "scaling": "strong".
-``--shard batch``: every rank runs its own full round ("weak").  The job time
-is the maximum over ranks either way.
+``--shard batch``: every rank runs its own full round ("weak").  ``--shard
+client``: the clients are spread over the ranks, whose weighted sums meet in
+one reduce-scatter (the layout of a server that receives different clients on
+different GPUs).  The job time is the maximum over ranks in every mode.
 """
 from __future__ import annotations
 
@@ -556,8 +558,94 @@ def measure(job, w, steps, warmup, with_cpu_baseline):
     return fields
 
 
+def measure_client_layout(job, w, steps, warmup):
+    """The round with the clients spread over the ranks (`--shard client`): rank r encrypts the
+    clients [C r / N, C (r+1) / N) on every ciphertext index and forms their weighted sum on all
+    limbs; one reduce-scatter of 64-bit words sums over the clients and leaves rank r the
+    ciphertext indices [T r / N, T (r+1) / N), which it rescales and decrypts.  The one layout with
+    an exchange step on the path; wired to full encryption without chunked streaming."""
+    import paper_2303_10837_b200 as he
+    from paper_2303_10837_b200.sharding import scatter_sum, shard_range, slot_range
+    torch = job.torch
+    rank, world = job.rank, job.world
+    if w.k < w.P:
+        raise SystemExit("bench: --shard client is wired to full encryption")
+    g = he.he_ctx_create(w.N, list(w.primes), w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    alpha = si.client_weights(w)
+    T, n = w.T, w.n
+    cb, ce = shard_range(w.clients, rank, world)
+    tb, te, sb, se = slot_range(T, n, w.k, rank, world)
+    ct_bytes = 8 * 2 * w.L * w.N
+    if (ce - cb + 2) * T * ct_bytes > 100e9:
+        raise SystemExit("bench: --shard client keeps all ciphertexts of a rank's clients resident; this workload needs more ranks")
+    xs = []
+    for i in range(w.clients):
+        rng = np.random.default_rng([w.seed, 1000 + i, 0])
+        x = rng.standard_normal(w.P, dtype=np.float32)
+        x *= np.float32(w.std)
+        xs.append(torch.from_numpy(x).cuda())
+    cts = [torch.empty((T, 2, w.L, w.N), dtype=torch.int64, device="cuda") for _ in range(cb, ce)]
+    partial = torch.zeros((T, 2, w.L, w.N), dtype=torch.int64, device="cuda")
+    agg = torch.empty((te - tb, 2, w.L - 1, w.N), dtype=torch.int64, device="cuda")
+    z = torch.empty((te - tb) * n, dtype=torch.float64, device="cuda")
+    he.he_ctx_reserve(g, T * n)
+
+    def step():
+        for j, i in enumerate(range(cb, ce)):
+            sel, _ = he.he_pack(g, None, xs[i])
+            he.he_encrypt(g, keys, sel, w.enc_seed, i, out=cts[j])
+        if ce > cb:
+            he.he_weighted_partial(g, cts, alpha[cb:ce], out=partial)
+        mine = scatter_sum(partial, rank, world)
+        if te > tb:
+            he.he_rescale_partial_sum(g, mine, world, out=agg)
+            he.he_decrypt(g, keys, agg, out=z)
+
+    for _ in range(warmup):
+        step()
+    job.barrier()
+    sampler = ClockSampler(job.local)
+    sampler.start()
+    launches0 = he.he_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(steps):
+        step()
+    ev1.record()
+    job.barrier()
+    launches = he.he_launch_count() - launches0
+    secs = ev0.elapsed_time(ev1) * 1e-3
+    clocks = sampler.stop()
+    want = sum(float(a) * x.double() for a, x in zip(alpha, xs))
+    err = float((z[: se - sb] - want[sb:se]).abs().max()) if se > sb else 0.0
+    if not err <= 1e-6 or he.he_ctx_status(g) != he.HE_OK:
+        raise SystemExit("bench: aggregate differs from plaintext FedAvg by %g" % err)
+    units, job_secs = reduce_job(float(se - sb) * steps, secs, world, "cuda")
+    if rank != 0:
+        return None
+    note = ("clients spread over %d ranks (rank r: clients [C r / N, C (r+1) / N)); one reduce-scatter of the "
+            "clients' weighted sums (%.1f MB of 64-bit words per rank and step), then every rank rescales and decrypts "
+            "its ciphertext indices" % (world, T * ct_bytes / 1e6))
+    return {"value": units / job_secs, "unit": UNIT, "ms_per_step": 1e3 * job_secs / steps, "steps": steps,
+            "warmup": warmup, "config": dict(config_dict(w, note), format="coefficient"),
+            "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"] or job.peaks["sm_max_mhz"],
+                       "reasons": clocks["reasons"], "samples": clocks["samples"]},
+            "e2e": None, "gpu_launches": int(launches), "roofline": None, "max_abs_err_vs_fedavg": err}
+
+
 def run_ours(args, w, extras):
     job = Job(args)
+    if args.shard == "client":
+        main = measure_client_layout(job, w, args.steps, args.warmup)
+        if job.rank == 0:
+            line = {"metric": METRIC, "n_gpus": job.world, "higher_is_better": True, "scaling": "strong",
+                    "vs_baseline": None, "dtype": "u64 (limbs below 2^46: exact f64)", "data": "synthetic"}
+            line.update(main)
+            print(json.dumps(line), flush=True)
+        if job.world > 1:
+            job.dist.destroy_process_group()
+        return
     main = measure(job, w, args.steps, args.warmup, with_cpu_baseline=(job.world == 1))
     others = {}
     for name, ew in extras:
@@ -592,9 +680,10 @@ def main():
     ap.add_argument("--also", default=None,
                     help="comma-separated further workloads reported under `workloads` (default: resnet50-top10,bert-100 "
                          "on one GPU when --workload is left at its default; 'none' for none)")
-    ap.add_argument("--shard", choices=["index", "batch"], default="index",
-                    help="N > 1: cut one round over the ranks by ciphertext index (strong scaling) or run one full "
-                         "batch per rank (weak scaling)")
+    ap.add_argument("--shard", choices=["index", "batch", "client"], default="index",
+                    help="N > 1: cut one round over the ranks by ciphertext index (strong scaling), run one full "
+                         "batch per rank (weak scaling), or spread the clients over the ranks with one "
+                         "reduce-scatter of their weighted sums (client; also runs on one GPU)")
     ap.add_argument("--gather", action="store_true",
                     help="with --shard index: all-gather the decoded pieces so that every rank holds the whole model")
     ap.add_argument("--format", choices=["coefficient", "transform"], default="coefficient",

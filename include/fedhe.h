@@ -171,6 +171,25 @@ int he_encrypt_range(he_ctx *ctx, const he_keys *keys, const float *sel_dev, siz
 int he_weighted_aggregate(he_ctx *ctx, const uint64_t *const *cts_host, const double *alpha_host,
                           int C, size_t T, uint64_t *agg_dev, void *stream);
 
+/* The same server step in two halves, for a server whose clients' ciphertexts
+ * sit on several GPUs (Algorithm 1's aggregation is a sum over clients, so it
+ * splits over any partition of them).  he_weighted_partial gives
+ *   partial = sum over the C given clients of W_i ct_i mod q_j
+ * on all L limbs, canonical residues, dev uint64 [T][2][L][N], no rescale;
+ * alpha are the clients' weights of the WHOLE round (normalised over all
+ * clients, not over this subset).  The caller adds the partial sums of all
+ * subsets word by word as plain 64-bit integers (e.g. a reduce-scatter with a
+ * sum over uint64/int64) -- at most floor(2^64 / max_j q_j) of them, 16 for
+ * 60-bit primes -- and he_rescale_partial_sum reduces that sum modulo every
+ * q_j and applies the rescale:  agg, dev uint64 [T][2][L-1][N], is then word
+ * for word what he_weighted_aggregate gives on all clients at once.
+ * `parts` is the number of partial sums that were added (HE_ERR_SIZE if that
+ * many could overflow 64 bits). */
+int he_weighted_partial(he_ctx *ctx, const uint64_t *const *cts_host, const double *alpha_host, int C, size_t T,
+                        uint64_t *partial_dev, void *stream);
+int he_rescale_partial_sum(he_ctx *ctx, const uint64_t *sum_dev, uint32_t parts, size_t T, uint64_t *agg_dev,
+                           void *stream);
+
 /* Plaintext part  sum_i a_i ((1-M) (.) W_i): out[k] = sum_i alpha_i * rest_i[k]
  * in fp64, client order, separate multiply and add.
  *   rests: host array of C dev pointers float[len]; out: dev double[len]. */

@@ -70,6 +70,8 @@ _SIGS = {
     "he_encrypt": (C.c_int, [_vp, _vp, _vp, _sz, _u64, _u32, _vp, _vp]),
     "he_encrypt_range": (C.c_int, [_vp, _vp, _vp, _sz, _sz, _u64, _u32, _vp, _vp]),
     "he_weighted_aggregate": (C.c_int, [_vp, _vp, _vp, C.c_int, _sz, _vp, _vp]),
+    "he_weighted_partial": (C.c_int, [_vp, _vp, _vp, C.c_int, _sz, _vp, _vp]),
+    "he_rescale_partial_sum": (C.c_int, [_vp, _vp, _u32, _sz, _vp, _vp]),
     "he_encrypt_ntt": (C.c_int, [_vp, _vp, _vp, _sz, _u64, _u32, _vp, _vp]),
     "he_weighted_aggregate_ntt": (C.c_int, [_vp, _vp, _vp, C.c_int, _sz, _vp, _vp]),
     "he_decrypt_level_ntt": (C.c_int, [_vp, _vp, _vp, _u32, _sz, _vp, _vp]),
@@ -328,6 +330,36 @@ def he_weighted_aggregate(ctx: Ctx, cts: List[torch.Tensor], alpha: Sequence[flo
     al = (C.c_double * Cn)(*[float(a) for a in alpha])
     _check(_lib.he_weighted_aggregate(ctx.handle, C.cast(ptrs, _vp), C.cast(al, _vp), Cn, T,
                                       _dev(out, torch.int64), _stream()), "he_weighted_aggregate")
+    return out
+
+
+def he_weighted_partial(ctx: Ctx, cts: List[torch.Tensor], alpha: Sequence[float],
+                        out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Weighted sum of a subset of the clients on all L limbs, no rescale: int64 [T][2][L][N]."""
+    _same_len(cts, alpha, "he_weighted_partial cts and alpha")
+    Cn = len(cts)
+    T = _ct_count(ctx, cts[0], ctx.L, "he_weighted_partial cts[0]")
+    for i, c in enumerate(cts):
+        _sized(c, T * 2 * ctx.L * ctx.N, "he_weighted_partial cts[%d]" % i, exact=True)
+    if out is None:
+        out = torch.empty((T, 2, ctx.L, ctx.N), dtype=torch.int64, device="cuda")
+    _sized(out, T * 2 * ctx.L * ctx.N, "he_weighted_partial out")
+    ptrs = (_vp * Cn)(*[_dev(c, torch.int64) for c in cts])
+    al = (C.c_double * Cn)(*[float(a) for a in alpha])
+    _check(_lib.he_weighted_partial(ctx.handle, C.cast(ptrs, _vp), C.cast(al, _vp), Cn, T,
+                                    _dev(out, torch.int64), _stream()), "he_weighted_partial")
+    return out
+
+
+def he_rescale_partial_sum(ctx: Ctx, summed: torch.Tensor, parts: int,
+                           out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Rescale of the word-by-word sum of `parts` results of he_weighted_partial."""
+    T = _ct_count(ctx, summed, ctx.L, "he_rescale_partial_sum summed")
+    if out is None:
+        out = torch.empty((T, 2, ctx.L - 1, ctx.N), dtype=torch.int64, device="cuda")
+    _sized(out, T * 2 * (ctx.L - 1) * ctx.N, "he_rescale_partial_sum out")
+    _check(_lib.he_rescale_partial_sum(ctx.handle, _dev(summed, torch.int64), int(parts), T,
+                                       _dev(out, torch.int64), _stream()), "he_rescale_partial_sum")
     return out
 
 

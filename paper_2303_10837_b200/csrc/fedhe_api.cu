@@ -490,8 +490,10 @@ int he_encrypt(he_ctx *ctx, const he_keys *keys, const float *sel_dev, size_t k,
     return he_encrypt_range(ctx, keys, sel_dev, 0, he_num_ct(ctx, k), seed, client_id, ct_dev, stream);
 }
 
+enum AggMode { AGG_RESCALE, AGG_NTT, AGG_PARTIAL };
+
 static int weighted_aggregate(he_ctx *ctx, const uint64_t *const *cts_host, const double *alpha_host, int C,
-                              size_t T, bool ntt, uint64_t *agg_dev, void *stream) {
+                              size_t T, AggMode mode, uint64_t *agg_dev, void *stream) {
     if (!good(ctx) || !cts_host || !alpha_host || C < 1) return HE_ERR_INVALID_ARG;
     if (C > HE_MAX_CLIENTS) return HE_ERR_SIZE;
     if (T && (!agg_dev || !aligned16(agg_dev))) return HE_ERR_INVALID_ARG;
@@ -519,10 +521,12 @@ static int weighted_aggregate(he_ctx *ctx, const uint64_t *const *cts_host, cons
     CU(cudaMemcpyAsync(ctx->tab, host.data(), host.size(), cudaMemcpyHostToDevice, st));
     const uint64_t *const *dptrs = static_cast<const uint64_t *const *>(ctx->tab);
     const tw_t *dw = reinterpret_cast<const tw_t *>(static_cast<unsigned char *>(ctx->tab) + C * sizeof(void *));
-    if (ntt) {
+    if (mode == AGG_NTT) {
         int rc = ensure(&ctx->ws, &ctx->ws_bytes, 2 * T * (size_t)L * d.N * sizeof(uint64_t));
         if (rc != HE_OK) return rc;
         CU(launch_aggregate_ntt(d, dptrs, dw, C, T, static_cast<uint64_t *>(ctx->ws), agg_dev, st));
+    } else if (mode == AGG_PARTIAL) {
+        CU(launch_aggregate_partial(d, dptrs, dw, C, T, agg_dev, st));
     } else {
         CU(launch_aggregate(d, dptrs, dw, C, T, agg_dev, st));
     }
@@ -531,12 +535,30 @@ static int weighted_aggregate(he_ctx *ctx, const uint64_t *const *cts_host, cons
 
 int he_weighted_aggregate(he_ctx *ctx, const uint64_t *const *cts_host, const double *alpha_host, int C,
                           size_t T, uint64_t *agg_dev, void *stream) {
-    return weighted_aggregate(ctx, cts_host, alpha_host, C, T, false, agg_dev, stream);
+    return weighted_aggregate(ctx, cts_host, alpha_host, C, T, AGG_RESCALE, agg_dev, stream);
+}
+
+int he_weighted_partial(he_ctx *ctx, const uint64_t *const *cts_host, const double *alpha_host, int C, size_t T,
+                        uint64_t *partial_dev, void *stream) {
+    return weighted_aggregate(ctx, cts_host, alpha_host, C, T, AGG_PARTIAL, partial_dev, stream);
+}
+
+int he_rescale_partial_sum(he_ctx *ctx, const uint64_t *sum_dev, uint32_t parts, size_t T, uint64_t *agg_dev,
+                           void *stream) {
+    if (!good(ctx) || parts < 1) return HE_ERR_INVALID_ARG;
+    // the caller added `parts` canonical partial sums word by word: that must fit 64 bits
+    uint64_t qmax = 0;
+    for (uint32_t j = 0; j < ctx->dev.L; j++) qmax = ctx->dev.limb[j].q > qmax ? ctx->dev.limb[j].q : qmax;
+    if (parts > UINT64_MAX / qmax) return HE_ERR_SIZE;
+    if (T == 0) return HE_OK;
+    if (!sum_dev || !agg_dev || !aligned16(sum_dev) || !aligned16(agg_dev)) return HE_ERR_INVALID_ARG;
+    CU(launch_rescale_partial_sum(ctx->dev, sum_dev, T, agg_dev, as_stream(stream)));
+    return HE_OK;
 }
 
 int he_weighted_aggregate_ntt(he_ctx *ctx, const uint64_t *const *cts_host, const double *alpha_host, int C,
                               size_t T, uint64_t *agg_dev, void *stream) {
-    return weighted_aggregate(ctx, cts_host, alpha_host, C, T, true, agg_dev, stream);
+    return weighted_aggregate(ctx, cts_host, alpha_host, C, T, AGG_NTT, agg_dev, stream);
 }
 
 int he_plain_aggregate(he_ctx *ctx, const float *const *rests_host, const double *alpha_host, int C,

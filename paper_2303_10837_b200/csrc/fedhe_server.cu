@@ -99,7 +99,8 @@ cudaError_t launch_aggregate(const CtxDev &c, const uint64_t *const *ptrs, const
 // ---------------------------------------------------------------------------
 
 // acc_j = sum_i W_i ct_i for all limbs: limbs below the last go to `out`
-// ([T][2][L-1][N]), the last limb to `last` ([T][2][N])
+// ([T][2][L-1][N]), the last limb to `last` ([T][2][N]); with `last` null all L
+// limbs go to `out` ([T][2][L][N]): the partial sum of a subset of the clients
 __global__ void __launch_bounds__(256)
 aggregate_sum_kernel(const __grid_constant__ CtxDev c, const uint64_t *const *ptrs, const tw_t *wtab, int C,
                      uint64_t *out, uint64_t *last, size_t total) {
@@ -118,9 +119,61 @@ aggregate_sum_kernel(const __grid_constant__ CtxDev c, const uint64_t *const *pt
     for (uint32_t j = 0; j < L; j++) {
         u64x2 o;
         weighted_sum_pair(sp, sw, C, L, j, (tc * L + j) * c.N + i, c.limb[j].q, o.x, o.y);
-        uint64_t *dst = j + 1 < L ? out + (tc * (L - 1) + j) * c.N + i : last + tc * c.N + i;
+        uint64_t *dst = !last ? out + (tc * L + j) * c.N + i
+                              : (j + 1 < L ? out + (tc * (L - 1) + j) * c.N + i : last + tc * c.N + i);
         *reinterpret_cast<u64x2 *>(dst) = o;
     }
+}
+
+// Rescale of a sum of partial sums ([T][2][L][N]; every word a sum of canonical
+// residues that did not overflow 64 bits): reduce, then as in the fused kernel.
+__global__ void __launch_bounds__(256)
+rescale_partial_sum_kernel(const __grid_constant__ CtxDev c, const uint64_t *sum, uint64_t *out, size_t total) {
+    const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const uint32_t L = c.L, pairs = c.N >> 1;
+    const uint32_t i = (uint32_t)(g % pairs) * 2;
+    const size_t tc = g / pairs;
+    const LimbDev &ll = c.limb[L - 1];
+    const uint64_t ql = ll.q;
+    const ulonglong2 rl = __ldg(reinterpret_cast<const ulonglong2 *>(sum + (tc * L + (L - 1)) * c.N + i));
+    const uint64_t rx = barrett64(rl.x, ql, ll.mu), ry = barrett64(rl.y, ql, ll.mu);
+    const bool negx = rx > ql / 2, negy = ry > ql / 2;
+    const uint64_t mx = negx ? ql - rx : rx, my = negy ? ql - ry : ry;
+    for (uint32_t j = 0; j + 1 < L; j++) {
+        const LimbDev &lb = c.limb[j];
+        const uint64_t q = lb.q;
+        const ulonglong2 a = __ldg(reinterpret_cast<const ulonglong2 *>(sum + (tc * L + j) * c.N + i));
+        const uint64_t ax = barrett64(a.x, q, lb.mu), ay = barrett64(a.y, q, lb.mu);
+        const uint64_t sx = barrett64(mx, q, lb.mu), sy = barrett64(my, q, lb.mu);
+        const uint64_t dx = negx ? addmod(ax, sx, q) : submod(ax, sx, q);
+        const uint64_t dy = negy ? addmod(ay, sy, q) : submod(ay, sy, q);
+        ulonglong2 o;
+        o.x = shoup(dx, lb.qlinv.w, lb.qlinv.wp, q);
+        o.y = shoup(dy, lb.qlinv.w, lb.qlinv.wp, q);
+        *reinterpret_cast<ulonglong2 *>(out + (tc * (L - 1) + j) * c.N + i) = o;
+    }
+}
+
+cudaError_t launch_aggregate_partial(const CtxDev &c, const uint64_t *const *ptrs, const tw_t *wtab, int C,
+                                     size_t T, uint64_t *out, cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    const size_t smem = (size_t)C * c.L * sizeof(tw_t) + (size_t)C * sizeof(void *);
+    cudaError_t e;
+    if (smem > 48 * 1024 &&
+        (e = cudaFuncSetAttribute(aggregate_sum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)))
+        return e;
+    const size_t pairs = T * 2 * (c.N >> 1);
+    aggregate_sum_kernel<<<blocks_for(pairs, 256), 256, smem, s>>>(c, ptrs, wtab, C, out, nullptr, pairs);
+    return FEDHE_LAUNCHED();
+}
+
+cudaError_t launch_rescale_partial_sum(const CtxDev &c, const uint64_t *sum, size_t T, uint64_t *out,
+                                       cudaStream_t s) {
+    if (T == 0) return cudaSuccess;
+    const size_t pairs = T * 2 * (c.N >> 1);
+    rescale_partial_sum_kernel<<<blocks_for(pairs, 256), 256, 0, s>>>(c, sum, out, pairs);
+    return FEDHE_LAUNCHED();
 }
 
 // residues modulo every remaining prime of the centred last-limb coefficients

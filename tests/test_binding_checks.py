@@ -55,6 +55,12 @@ def test_aggregate_sizes(ctx):
     refused(lambda: he.he_weighted_aggregate(ctx, [ct(4, L - 1), ct(4, L - 1)], [0.5, 0.5]))    # wrong level
     refused(lambda: he.he_weighted_aggregate(ctx, good, [0.5, 0.5], out=ct(3, L - 1)))          # out too short
     refused(lambda: he.he_weighted_aggregate_ntt(ctx, [ct(4), ct(3)], [0.5, 0.5]))
+    refused(lambda: he.he_weighted_partial(ctx, [ct(4), ct(3)], [0.5, 0.5]))                     # a shorter client
+    refused(lambda: he.he_weighted_partial(ctx, good, [0.5, 0.5], out=ct(4, L - 1)))              # partial sums keep all limbs
+    refused(lambda: he.he_rescale_partial_sum(ctx, ct(4, L - 1), 2))                              # not a sum on all limbs
+    refused(lambda: he.he_rescale_partial_sum(ctx, ct(4), 2, out=ct(3, L - 1)))
+    reaches_device_check(lambda: he.he_weighted_partial(ctx, good, [0.5, 0.5], out=ct(4)))
+    reaches_device_check(lambda: he.he_rescale_partial_sum(ctx, ct(4), 2, out=ct(4, L - 1)))
     refused(lambda: he.he_plain_aggregate(ctx, [torch.zeros(10), torch.zeros(9)], [0.5, 0.5]))
     refused(lambda: he.he_plain_aggregate(ctx, [torch.zeros(10)], [0.5, 0.5]))
     reaches_device_check(lambda: he.he_weighted_aggregate(ctx, good, [0.5, 0.5], out=ct(4, L - 1)))

@@ -508,6 +508,47 @@ def test_host_round_refuses_bad_arguments_before_queueing(he):
     assert np.abs(host.numpy() - want).max() <= FEDAVG_TOL
 
 
+@pytest.mark.parametrize("N,primes,ld", [(8192, si.PRIMES_N8192, 40), (16384, si.PRIMES_N16384, 40),
+                                         (32768, si.PRIMES_N32768, 45)],
+                         ids=["n8192", "n16384", "n32768"])
+def test_client_partition_reproduces_the_whole_aggregate(he, N, primes, ld):
+    """The server step in two halves (clients spread over GPUs): the partial weighted sums of
+    three groups of clients equal the oracle's, and their word-by-word sum, rescaled, equals both
+    the one-call aggregate and the oracle's rescale, bit for bit."""
+    w = si.Workload("client-groups", N, primes, ld, 5, 2 * (N // 2) + 11, 0.01, ratio=1.0, seed=31,
+                    key_seed=311, enc_seed=312, weights="uniform")
+    g, o = contexts(he, w.N, w.primes, w.log2_delta)
+    keys = he.he_keygen(g, w.key_seed)
+    xs, alpha = si.client_updates(w), si.client_weights(w)
+    cts = [he.he_encrypt(g, keys, he.he_pack(g, None, dev_f32(x))[0], w.enc_seed, i) for i, x in enumerate(xs)]
+    cts_o = [to_host_u64(c) for c in cts]                 # ciphertext parity is covered above
+    W = o.weights(alpha)
+    groups = [(0, 1), (1, 4), (4, 5)]
+    parts = []
+    for b, e in groups:
+        part = he.he_weighted_partial(g, cts[b:e], alpha[b:e])
+        assert np.array_equal(to_host_u64(part), o.weighted_sum(cts_o[b:e], W[b:e])), (b, e)
+        parts.append(part)
+    summed = parts[0] + parts[1] + parts[2]               # 64-bit words, as a reduce-scatter would add them
+    agg = he.he_rescale_partial_sum(g, summed, len(parts))
+    whole = he.he_weighted_aggregate(g, cts, alpha)
+    assert torch.equal(agg, whole)
+    assert np.array_equal(to_host_u64(agg), o.rescale(o.weighted_sum(cts_o, W)))
+    # a single part is the one-call aggregate as well
+    assert torch.equal(he.he_rescale_partial_sum(g, he.he_weighted_partial(g, cts, alpha), 1), whole)
+    # seventeen sums of residues of a 60-bit prime could overflow 64 bits
+    with pytest.raises(he.HeError) as ei:
+        he.he_rescale_partial_sum(g, summed, 17)
+    assert ei.value.code == he.HE_ERR_SIZE
+    with pytest.raises(he.HeError) as ei:
+        he.he_rescale_partial_sum(g, summed, 0)
+    assert ei.value.code == he.HE_ERR_INVALID_ARG
+    z = he.he_decrypt(g, keys, agg).cpu().numpy()
+    want = sum(a * x.astype(np.float64) for a, x in zip(alpha, xs))
+    assert np.abs(z[: w.P] - want).max() <= FEDAVG_TOL
+    assert he.he_ctx_status(g) == he.HE_OK
+
+
 def test_index_partition_reproduces_the_whole_round(he):
     """The multi-GPU partition (contiguous ciphertext indices and remainder entries per rank, context,
     keys and mask replicated), played by one GPU one rank after the other: the ranks' ciphertexts,
