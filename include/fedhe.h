@@ -189,6 +189,17 @@ int he_weighted_partial(he_ctx *ctx, const uint64_t *const *cts_host, const doub
                         uint64_t *partial_dev, void *stream);
 int he_rescale_partial_sum(he_ctx *ctx, const uint64_t *sum_dev, uint32_t parts, size_t T, uint64_t *agg_dev,
                            void *stream);
+/* The same without a separate addition: parts is a host array of P dev
+ * pointers, each a result of he_weighted_partial for the same T ciphertext
+ * indices (uint64 [T][2][L][N]); the kernel adds them while it reads.  The
+ * buffers are read with plain loads only, so they may be peer-mapped memory
+ * that he_weighted_partial calls on other GPUs wrote into (each GPU calls
+ * he_weighted_partial once per owner, on that owner's range of ciphertext
+ * indices, with partial_dev inside the owner's buffer); the caller orders
+ * those writes before this call.  1 <= P <= min(HE_MAX_CLIENTS,
+ * floor(2^64 / max_j q_j)). */
+int he_rescale_partial_parts(he_ctx *ctx, const uint64_t *const *parts_host, int P, size_t T, uint64_t *agg_dev,
+                             void *stream);
 
 /* Plaintext part  sum_i a_i ((1-M) (.) W_i): out[k] = sum_i alpha_i * rest_i[k]
  * in fp64, client order, separate multiply and add.

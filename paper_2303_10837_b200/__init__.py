@@ -72,6 +72,7 @@ _SIGS = {
     "he_weighted_aggregate": (C.c_int, [_vp, _vp, _vp, C.c_int, _sz, _vp, _vp]),
     "he_weighted_partial": (C.c_int, [_vp, _vp, _vp, C.c_int, _sz, _vp, _vp]),
     "he_rescale_partial_sum": (C.c_int, [_vp, _vp, _u32, _sz, _vp, _vp]),
+    "he_rescale_partial_parts": (C.c_int, [_vp, _vp, C.c_int, _sz, _vp, _vp]),
     "he_encrypt_ntt": (C.c_int, [_vp, _vp, _vp, _sz, _u64, _u32, _vp, _vp]),
     "he_weighted_aggregate_ntt": (C.c_int, [_vp, _vp, _vp, C.c_int, _sz, _vp, _vp]),
     "he_decrypt_level_ntt": (C.c_int, [_vp, _vp, _vp, _u32, _sz, _vp, _vp]),
@@ -360,6 +361,22 @@ def he_rescale_partial_sum(ctx: Ctx, summed: torch.Tensor, parts: int,
     _sized(out, T * 2 * (ctx.L - 1) * ctx.N, "he_rescale_partial_sum out")
     _check(_lib.he_rescale_partial_sum(ctx.handle, _dev(summed, torch.int64), int(parts), T,
                                        _dev(out, torch.int64), _stream()), "he_rescale_partial_sum")
+    return out
+
+
+def he_rescale_partial_parts(ctx: Ctx, parts: List[torch.Tensor], out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Rescale of the sum of several results of he_weighted_partial, added by the kernel itself."""
+    if len(parts) < 1:
+        raise HeError(HE_ERR_INVALID_ARG, "he_rescale_partial_parts: no parts")
+    T = _ct_count(ctx, parts[0], ctx.L, "he_rescale_partial_parts parts[0]")
+    for i, p in enumerate(parts):
+        _sized(p, T * 2 * ctx.L * ctx.N, "he_rescale_partial_parts parts[%d]" % i, exact=True)
+    if out is None:
+        out = torch.empty((T, 2, ctx.L - 1, ctx.N), dtype=torch.int64, device="cuda")
+    _sized(out, T * 2 * (ctx.L - 1) * ctx.N, "he_rescale_partial_parts out")
+    ptrs = (_vp * len(parts))(*[_dev(p, torch.int64) for p in parts])
+    _check(_lib.he_rescale_partial_parts(ctx.handle, C.cast(ptrs, _vp), len(parts), T,
+                                         _dev(out, torch.int64), _stream()), "he_rescale_partial_parts")
     return out
 
 

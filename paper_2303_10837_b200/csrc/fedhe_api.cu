@@ -543,17 +543,33 @@ int he_weighted_partial(he_ctx *ctx, const uint64_t *const *cts_host, const doub
     return weighted_aggregate(ctx, cts_host, alpha_host, C, T, AGG_PARTIAL, partial_dev, stream);
 }
 
-int he_rescale_partial_sum(he_ctx *ctx, const uint64_t *sum_dev, uint32_t parts, size_t T, uint64_t *agg_dev,
-                           void *stream) {
-    if (!good(ctx) || parts < 1) return HE_ERR_INVALID_ARG;
-    // the caller added `parts` canonical partial sums word by word: that must fit 64 bits
+// `added`: how many canonical partial sums every word of the buffers may hold in total
+static int rescale_partial(he_ctx *ctx, const uint64_t *const *parts_host, int P, uint64_t added, size_t T,
+                           uint64_t *agg_dev, void *stream) {
+    if (!good(ctx) || !parts_host || P < 1 || added < 1) return HE_ERR_INVALID_ARG;
+    if (P > HE_MAX_CLIENTS) return HE_ERR_SIZE;
     uint64_t qmax = 0;
     for (uint32_t j = 0; j < ctx->dev.L; j++) qmax = ctx->dev.limb[j].q > qmax ? ctx->dev.limb[j].q : qmax;
-    if (parts > UINT64_MAX / qmax) return HE_ERR_SIZE;
+    if (added > UINT64_MAX / qmax) return HE_ERR_SIZE;         // the 64-bit sums could wrap
     if (T == 0) return HE_OK;
-    if (!sum_dev || !agg_dev || !aligned16(sum_dev) || !aligned16(agg_dev)) return HE_ERR_INVALID_ARG;
-    CU(launch_rescale_partial_sum(ctx->dev, sum_dev, T, agg_dev, as_stream(stream)));
+    if (!agg_dev || !aligned16(agg_dev)) return HE_ERR_INVALID_ARG;
+    for (int p = 0; p < P; p++)
+        if (!parts_host[p] || !aligned16(parts_host[p])) return HE_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    CU(cudaMemcpyAsync(ctx->tab, parts_host, P * sizeof(void *), cudaMemcpyHostToDevice, st));
+    CU(launch_rescale_partial_sum(ctx->dev, static_cast<const uint64_t *const *>(ctx->tab), P, T, agg_dev, st));
     return HE_OK;
+}
+
+int he_rescale_partial_sum(he_ctx *ctx, const uint64_t *sum_dev, uint32_t parts, size_t T, uint64_t *agg_dev,
+                           void *stream) {
+    const uint64_t *one[1] = {sum_dev};
+    return rescale_partial(ctx, one, 1, parts, T, agg_dev, stream);
+}
+
+int he_rescale_partial_parts(he_ctx *ctx, const uint64_t *const *parts_host, int P, size_t T, uint64_t *agg_dev,
+                             void *stream) {
+    return rescale_partial(ctx, parts_host, P, P < 1 ? 1 : (uint64_t)P, T, agg_dev, stream);
 }
 
 int he_weighted_aggregate_ntt(he_ctx *ctx, const uint64_t *const *cts_host, const double *alpha_host, int C,

@@ -53,8 +53,8 @@ cudaError_t launch_aggregate_ntt(const CtxDev &c, const uint64_t *const *ptrs, c
 // the clients' weighted sum on all L limbs without the rescale, and the rescale of a sum of such sums
 cudaError_t launch_aggregate_partial(const CtxDev &c, const uint64_t *const *ptrs, const tw_t *wtab, int C,
                                      size_t T, uint64_t *out, cudaStream_t s);
-cudaError_t launch_rescale_partial_sum(const CtxDev &c, const uint64_t *sum, size_t T, uint64_t *out,
-                                       cudaStream_t s);
+cudaError_t launch_rescale_partial_sum(const CtxDev &c, const uint64_t *const *parts, int P, size_t T,
+                                       uint64_t *out, cudaStream_t s);
 cudaError_t launch_plain_aggregate(const float *const *ptrs, const double *alpha, int C, size_t len,
                                    double *out, bool aligned16, cudaStream_t s);
 

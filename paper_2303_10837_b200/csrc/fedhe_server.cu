@@ -125,25 +125,39 @@ aggregate_sum_kernel(const __grid_constant__ CtxDev c, const uint64_t *const *pt
     }
 }
 
-// Rescale of a sum of partial sums ([T][2][L][N]; every word a sum of canonical
-// residues that did not overflow 64 bits): reduce, then as in the fused kernel.
+// Rescale of a sum of partial sums.  `parts` names P buffers uint64 [T][2][L][N]
+// whose words are added here (P = 1: the caller has added them already); every
+// word is a sum of canonical residues that does not overflow 64 bits.  Reduce,
+// then as in the fused kernel.  The buffers are read with plain loads, so they
+// may be peer memory that other GPUs' he_weighted_partial calls wrote into.
 __global__ void __launch_bounds__(256)
-rescale_partial_sum_kernel(const __grid_constant__ CtxDev c, const uint64_t *sum, uint64_t *out, size_t total) {
+rescale_partial_sum_kernel(const __grid_constant__ CtxDev c, const uint64_t *const *parts, int P, uint64_t *out,
+                           size_t total) {
     const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= total) return;
     const uint32_t L = c.L, pairs = c.N >> 1;
     const uint32_t i = (uint32_t)(g % pairs) * 2;
     const size_t tc = g / pairs;
+    auto summed = [&](uint32_t j) {
+        const size_t off = (tc * L + j) * c.N + i;
+        ulonglong2 a = *reinterpret_cast<const ulonglong2 *>(parts[0] + off);
+        for (int p = 1; p < P; p++) {
+            const ulonglong2 b = *reinterpret_cast<const ulonglong2 *>(parts[p] + off);
+            a.x += b.x;
+            a.y += b.y;
+        }
+        return a;
+    };
     const LimbDev &ll = c.limb[L - 1];
     const uint64_t ql = ll.q;
-    const ulonglong2 rl = __ldg(reinterpret_cast<const ulonglong2 *>(sum + (tc * L + (L - 1)) * c.N + i));
+    const ulonglong2 rl = summed(L - 1);
     const uint64_t rx = barrett64(rl.x, ql, ll.mu), ry = barrett64(rl.y, ql, ll.mu);
     const bool negx = rx > ql / 2, negy = ry > ql / 2;
     const uint64_t mx = negx ? ql - rx : rx, my = negy ? ql - ry : ry;
     for (uint32_t j = 0; j + 1 < L; j++) {
         const LimbDev &lb = c.limb[j];
         const uint64_t q = lb.q;
-        const ulonglong2 a = __ldg(reinterpret_cast<const ulonglong2 *>(sum + (tc * L + j) * c.N + i));
+        const ulonglong2 a = summed(j);
         const uint64_t ax = barrett64(a.x, q, lb.mu), ay = barrett64(a.y, q, lb.mu);
         const uint64_t sx = barrett64(mx, q, lb.mu), sy = barrett64(my, q, lb.mu);
         const uint64_t dx = negx ? addmod(ax, sx, q) : submod(ax, sx, q);
@@ -168,11 +182,11 @@ cudaError_t launch_aggregate_partial(const CtxDev &c, const uint64_t *const *ptr
     return FEDHE_LAUNCHED();
 }
 
-cudaError_t launch_rescale_partial_sum(const CtxDev &c, const uint64_t *sum, size_t T, uint64_t *out,
-                                       cudaStream_t s) {
+cudaError_t launch_rescale_partial_sum(const CtxDev &c, const uint64_t *const *parts, int P, size_t T,
+                                       uint64_t *out, cudaStream_t s) {
     if (T == 0) return cudaSuccess;
     const size_t pairs = T * 2 * (c.N >> 1);
-    rescale_partial_sum_kernel<<<blocks_for(pairs, 256), 256, 0, s>>>(c, sum, out, pairs);
+    rescale_partial_sum_kernel<<<blocks_for(pairs, 256), 256, 0, s>>>(c, parts, P, out, pairs);
     return FEDHE_LAUNCHED();
 }
 

@@ -59,6 +59,9 @@ def test_aggregate_sizes(ctx):
     refused(lambda: he.he_weighted_partial(ctx, good, [0.5, 0.5], out=ct(4, L - 1)))              # partial sums keep all limbs
     refused(lambda: he.he_rescale_partial_sum(ctx, ct(4, L - 1), 2))                              # not a sum on all limbs
     refused(lambda: he.he_rescale_partial_sum(ctx, ct(4), 2, out=ct(3, L - 1)))
+    refused(lambda: he.he_rescale_partial_parts(ctx, [ct(4), ct(3)]))
+    refused(lambda: he.he_rescale_partial_parts(ctx, []))
+    reaches_device_check(lambda: he.he_rescale_partial_parts(ctx, [ct(4), ct(4)], out=ct(4, L - 1)))
     reaches_device_check(lambda: he.he_weighted_partial(ctx, good, [0.5, 0.5], out=ct(4)))
     reaches_device_check(lambda: he.he_rescale_partial_sum(ctx, ct(4), 2, out=ct(4, L - 1)))
     refused(lambda: he.he_plain_aggregate(ctx, [torch.zeros(10), torch.zeros(9)], [0.5, 0.5]))

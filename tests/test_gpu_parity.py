@@ -534,6 +534,7 @@ def test_client_partition_reproduces_the_whole_aggregate(he, N, primes, ld):
     whole = he.he_weighted_aggregate(g, cts, alpha)
     assert torch.equal(agg, whole)
     assert np.array_equal(to_host_u64(agg), o.rescale(o.weighted_sum(cts_o, W)))
+    assert torch.equal(he.he_rescale_partial_parts(g, parts), whole)       # added by the kernel itself
     # a single part is the one-call aggregate as well
     assert torch.equal(he.he_rescale_partial_sum(g, he.he_weighted_partial(g, cts, alpha), 1), whole)
     # seventeen sums of residues of a 60-bit prime could overflow 64 bits
