@@ -192,17 +192,21 @@ __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0
         const auto fa = LimbOf<M>::args(lb, true, 1, grp);
         const M &ar = fa.m;
         const auto w0 = M::load(fa.tw + 1);                // twiddle of the stage that pairs the halves
-        auto src = [&](uint32_t i) {
+        // sample of element i = base | reg: the swizzle of the sample arrays only involves index
+        // bits below the first phase's register bits, so it is taken of base once
+        auto src2 = [&](uint32_t base, uint32_t reg) {
             // u is ternary: the twiddle product is 0, w or -w
-            const int b = su[bswz(i + H)];
+            const int8_t *sb = su + bswz(base);
+            const int b = sb[reg + H];
             if constexpr (std::is_same<M, ModF64>::value) {
-                return f64_fma(grp == 0 ? (double)b : (double)-b, w0, (double)su[bswz(i)]);
+                return f64_fma(grp == 0 ? (double)b : (double)-b, w0, (double)sb[reg]);
             } else {
-                const uint64_t u = small_residue(su[bswz(i)], q);
+                const uint64_t u = small_residue(sb[reg], q);
                 const uint64_t v = b == 0 ? 0 : (b > 0 ? w0.w : q - w0.w);
                 return grp == 0 ? u + v : u - v + ar.q2;
             }
         };
+        auto src = [&](uint32_t i) { return src2(i, 0u); };
         if constexpr (NTT_OUT) {
             // transform-domain output: three passes over one copy of the forward code: u
             // (both products wait in their final slots), then e0 + m and e1, whose pairing
@@ -249,17 +253,18 @@ __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0
             __syncthreads();
             return;
         }
-        auto dst = [&](uint32_t p, val a, val b) {
+        auto dst = [&](uint32_t p, val a, val b, uint64_t *wa, uint64_t *wb) {
             const auto a0 = M::load_key(p1 + p), a1 = M::load_key(p1 + p + 1);
             u64x2 v;
             v.x = M::bits(ar.mul_key(a, a0));
             v.y = M::bits(ar.mul_key(b, a1));
             *reinterpret_cast<u64x2 *>(c1 + p) = v;      // parked until the second pass
             const auto b0 = M::load_key(p0 + p), b1 = M::load_key(p0 + p + 1);
-            smg[wswz(p)] = M::bits(ar.mul_key(a, b0));
-            smg[wswz(p + 1)] = M::bits(ar.mul_key(b, b1));
+            *wa = M::bits(ar.mul_key(a, b0));            // words wswz(p), wswz(p + 1) of this group's half
+            *wb = M::bits(ar.mul_key(b, b1));
         };
-        smem_ntt_forward<L, V>(smg, gt, fa, src, dst, gsync);
+        static_assert(L::reg_bit(0, 0) >= 10, "the sample swizzle stays clear of the first phase's register bits");
+        smem_ntt_forward<L, V>(smg, gt, fa, src2, dst, gsync);
     }
 #pragma unroll 1
     for (int h = 0; h < 2; h++) {
@@ -268,43 +273,56 @@ __device__ __forceinline__ void encrypt_unit2(const LimbDev &lb, const tw_t *pk0
         const auto ia = LimbOf<M>::args(lb, false, 1, grp);
         const M &ar = ia.m;
         const auto ninv = LimbOf<M>::ninv(lb), wn = LimbOf<M>::wn(lb);
-        auto isrc = [&](uint32_t p) {
-            if (h == 0) return pair_of<val>{M::from_bits(smg[wswz(p)]), M::from_bits(smg[wswz(p + 1)])};
+        auto isrc = [&](uint32_t p, const uint64_t *wa, const uint64_t *wb) {
+            if (h == 0) return pair_of<val>{M::from_bits(*wa), M::from_bits(*wb)};
             const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + grp * H + p);
             return pair_of<val>{M::from_bits(t.x), M::from_bits(t.y)};
         };
-        auto idst = [&](uint32_t i, val v) { smg[wswz(i)] = M::bits(v); };
+        auto idst = [&](uint32_t, val v, uint64_t *wv) { *wv = M::bits(v); };
         smem_ntt_inverse<L, V, false>(smg, gt, ia, ninv, wn, isrc, idst, gsync);
         __syncthreads();
         // last stage across the halves with 1/N folded in, then the error / message terms; the
         // message words of four rounds are requested before the first of them is used
         constexpr uint32_t ROUNDS = H / RT, AHEAD = ROUNDS < 4 ? ROUNDS : 4;
+        // element tid + r RT = tid ^ r RT sits at word wswz(tid) ^ wswz(r RT): a constant XOR into
+        // the low nibble and a constant offset above it
+        const uint32_t w_tid = word_address(sm, wswz(tid));
+        auto word_of_round = [&](uint32_t r) {
+            const uint32_t c = wswz(r * RT);
+            const uint32_t a = (w_tid ^ ((c & 15u) << 3)) + ((c & ~15u) << 3);
+            return reinterpret_cast<const uint64_t *>(__cvta_shared_to_generic((size_t)a));
+        };
+        // (the byte swizzle involves index bits 7..9 only: of tid, not of the round)
+        static_assert(RT % 1024 == 0, "a round advances the index above the swizzled bits");
+        const int8_t *se_tid = se + bswz(tid);
+        const int64_t *mt_tid = mt + tid;
+        uint64_t *cc_tid = cc + tid;
 #pragma unroll
         for (uint32_t k0 = 0; k0 < ROUNDS; k0 += AHEAD) {
             int64_t m_lo[AHEAD], m_hi[AHEAD];
             if (h == 0) {
 #pragma unroll
                 for (uint32_t k = 0; k < AHEAD; k++) {
-                    const uint32_t e = tid + (k0 + k) * RT;
-                    m_lo[k] = __ldcg(mt + e);
-                    m_hi[k] = __ldcg(mt + e + H);
+                    m_lo[k] = __ldcg(mt_tid + (k0 + k) * RT);
+                    m_hi[k] = __ldcg(mt_tid + (k0 + k) * RT + H);
                 }
             }
 #pragma unroll
             for (uint32_t k = 0; k < AHEAD; k++) {
-                const uint32_t e = tid + (k0 + k) * RT;
-                val lo = M::from_bits(sm[wswz(e)]), hi = M::from_bits(sm[H + wswz(e)]);
+                const uint32_t er = (k0 + k) * RT;             // element tid + er
+                const uint64_t *wl = word_of_round(k0 + k);
+                val lo = M::from_bits(wl[0]), hi = M::from_bits(wl[H]);
                 ar.inv_scaled(lo, hi, ninv, wn);
                 uint64_t add_lo, add_hi;
                 if (h == 0) {
-                    add_lo = signed_residue(m_lo[k] + (int64_t)se[bswz(e)], q, lb.mu);
-                    add_hi = signed_residue(m_hi[k] + (int64_t)se[bswz(e + H)], q, lb.mu);
+                    add_lo = signed_residue(m_lo[k] + (int64_t)se_tid[er], q, lb.mu);
+                    add_hi = signed_residue(m_hi[k] + (int64_t)se_tid[er + H], q, lb.mu);
                 } else {
-                    add_lo = small_residue(se[bswz(e)], q);
-                    add_hi = small_residue(se[bswz(e + H)], q);
+                    add_lo = small_residue(se_tid[er], q);
+                    add_hi = small_residue(se_tid[er + H], q);
                 }
-                cc[e] = ar.canon_add(lo, add_lo);
-                cc[e + H] = ar.canon_add(hi, add_hi);
+                cc_tid[er] = ar.canon_add(lo, add_lo);
+                cc_tid[er + H] = ar.canon_add(hi, add_hi);
             }
         }
         __syncthreads();

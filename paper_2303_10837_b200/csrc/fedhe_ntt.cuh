@@ -14,6 +14,8 @@
 // the twiddle index.
 #pragma once
 
+#include <type_traits>
+
 #include "fedhe_device.cuh"
 
 namespace fedhe {
@@ -496,13 +498,26 @@ __device__ __forceinline__ void forward_phases(uint64_t *sm, uint32_t warp, uint
         typename M::val x[L::E];
 #pragma unroll
         for (int r = 0; r < L::E; r++) {
-            if constexpr (P == 0) x[r] = src(base | L::template reg<P>(r));
-            else x[r] = M::from_bits(*reg_word<L, P>(a0, r));
+            if constexpr (P == 0) {
+                // a source may take the index in two parts, base (zero at the register bits, the
+                // same for all E calls) and the register's constant, to hoist what depends on base
+                if constexpr (std::is_invocable<Src, uint32_t, uint32_t>::value) x[r] = src(base, L::template reg<P>(r));
+                else x[r] = src(base | L::template reg<P>(r));
+            } else {
+                x[r] = M::from_bits(*reg_word<L, P>(a0, r));
+            }
         }
         fwd_phase<L, P>(x, base, a);
         if constexpr (P == LAST) {
 #pragma unroll
-            for (int r = 0; r < L::E; r += 2) dst(base | L::template reg<P>(r), x[r], x[r + 1]);
+            for (int r = 0; r < L::E; r += 2) {
+                // a sink that keeps the pair in this buffer may take the two words' addresses
+                // (one logic operation each) instead of swizzling the index itself
+                if constexpr (std::is_invocable<Dst, uint32_t, typename M::val, typename M::val, uint64_t *, uint64_t *>::value)
+                    dst(base | L::template reg<P>(r), x[r], x[r + 1], reg_word<L, P>(a0, r), reg_word<L, P>(a0, r + 1));
+                else
+                    dst(base | L::template reg<P>(r), x[r], x[r + 1]);
+            }
         } else {
 #pragma unroll
             for (int r = 0; r < L::E; r++) *reg_word<L, P>(a0, r) = M::bits(x[r]);
@@ -536,9 +551,15 @@ __device__ __forceinline__ void inverse_phases(uint64_t *sm, uint32_t warp, uint
         if constexpr (P == LAST) {
 #pragma unroll
             for (int r = 0; r < L::E; r += 2) {
-                const auto t = src(base | L::template reg<P>(r));
-                x[r] = t.x;
-                x[r + 1] = t.y;
+                if constexpr (std::is_invocable<Src, uint32_t, const uint64_t *, const uint64_t *>::value) {
+                    const auto t = src(base | L::template reg<P>(r), reg_word<L, P>(a0, r), reg_word<L, P>(a0, r + 1));
+                    x[r] = t.x;
+                    x[r + 1] = t.y;
+                } else {
+                    const auto t = src(base | L::template reg<P>(r));
+                    x[r] = t.x;
+                    x[r + 1] = t.y;
+                }
             }
         } else {
 #pragma unroll
@@ -552,7 +573,12 @@ __device__ __forceinline__ void inverse_phases(uint64_t *sm, uint32_t warp, uint
         }
         if constexpr (P == 0) {
 #pragma unroll
-            for (int r = 0; r < L::E; r++) dst(base | L::template reg<P>(r), x[r]);
+            for (int r = 0; r < L::E; r++) {
+                if constexpr (std::is_invocable<Dst, uint32_t, typename M::val, uint64_t *>::value)
+                    dst(base | L::template reg<P>(r), x[r], reg_word<L, P>(a0, r));
+                else
+                    dst(base | L::template reg<P>(r), x[r]);
+            }
         } else {
 #pragma unroll
             for (int r = 0; r < L::E; r++) *reg_word<L, P>(a0, r) = M::bits(x[r]);
