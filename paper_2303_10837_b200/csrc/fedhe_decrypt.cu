@@ -106,10 +106,10 @@ decrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const ui
         const NttArgs fa = LimbOf<ModInt>::args(lb, true, 0, 0);   // limb 0 carries the message
         smem_ntt_forward<L, V>(
             sm, tid, fa, [&](uint32_t i) { return c1[i]; },
-            [&](uint32_t p, uint64_t a, uint64_t b) {
+            [&](uint32_t p, uint64_t a, uint64_t b, uint64_t *wa, uint64_t *wb) {
                 const tw_t s0 = load_tw(k.s_hat + p), s1 = load_tw(k.s_hat + p + 1);
-                sm[wswz(p)] = shoup_lazy(a, s0.w, s0.wp, q);
-                sm[wswz(p + 1)] = shoup_lazy(b, s1.w, s1.wp, q);
+                *wa = shoup_lazy(a, s0.w, s0.wp, q);         // words wswz(p), wswz(p + 1)
+                *wb = shoup_lazy(b, s1.w, s1.wp, q);
             });
     }
     int64_t *d = reinterpret_cast<int64_t *>(sm);
@@ -117,19 +117,19 @@ decrypt_fused_kernel(const __grid_constant__ CtxDev c, const KeysDev k, const ui
         const NttArgs ia = LimbOf<ModInt>::args(lb, false, 0, 0);
         smem_ntt_inverse<L, V, true>(
             sm, tid, ia, lb.ninv, lb.wn,
-            [&](uint32_t p) {
+            [&](uint32_t p, const uint64_t *wa, const uint64_t *wb) {
                 if constexpr (NTT_IN) {
                     const u64x2 a = *reinterpret_cast<const u64x2 *>(c0 + p), b = *reinterpret_cast<const u64x2 *>(c1 + p);
                     const tw_t s0 = load_tw(k.s_hat + p), s1 = load_tw(k.s_hat + p + 1);
                     return u64x2{csub(a.x + shoup_lazy(b.x, s0.w, s0.wp, q), q2),
                                  csub(a.y + shoup_lazy(b.y, s1.w, s1.wp, q), q2)};
                 } else {
-                    return u64x2{sm[wswz(p)], sm[wswz(p + 1)]};
+                    return u64x2{*wa, *wb};
                 }
             },
-            [&](uint32_t i, uint64_t v) {
+            [&](uint32_t i, uint64_t v, uint64_t *wv) {
                 const uint64_t r = NTT_IN ? csub(v, q) : addmod(csub(v, q), c0[i], q);
-                d[wswz(i)] = r > q / 2 ? -(int64_t)(q - r) : (int64_t)r;
+                *reinterpret_cast<int64_t *>(wv) = r > q / 2 ? -(int64_t)(q - r) : (int64_t)r;     // d[wswz(i)]
             });
     }
     __syncthreads();

@@ -70,17 +70,18 @@ __device__ __forceinline__ void encrypt_unit(const LimbDev &lb, const tw_t *p0, 
         uint64_t *c1 = cbase + cstride;
         const auto fa = LimbOf<M>::args(lb, true, 0, 0);
         const M &ar = fa.m;
+        static_assert(L::reg_bit(0, 0) >= 10, "the sample swizzle stays clear of the first phase's register bits");
         smem_ntt_forward<L, V>(
-            sm, tid, fa, [&](uint32_t i) { return ar.small(su[bswz(i)]); },
-            [&](uint32_t p, val a, val b) {
+            sm, tid, fa, [&](uint32_t base, uint32_t reg) { return ar.small((su + bswz(base))[reg]); },
+            [&](uint32_t p, val a, val b, uint64_t *wa, uint64_t *wb) {
                 const auto a0 = M::load_key(p1 + p), a1 = M::load_key(p1 + p + 1);
                 u64x2 v;
                 v.x = M::bits(ar.mul_key(a, a0));
                 v.y = M::bits(ar.mul_key(b, a1));
                 *reinterpret_cast<u64x2 *>(c1 + p) = v;
                 const auto b0 = M::load_key(p0 + p), b1 = M::load_key(p0 + p + 1);
-                sm[wswz(p)] = M::bits(ar.mul_key(a, b0));
-                sm[wswz(p + 1)] = M::bits(ar.mul_key(b, b1));
+                *wa = M::bits(ar.mul_key(a, b0));            // words wswz(p), wswz(p + 1)
+                *wb = M::bits(ar.mul_key(b, b1));
             });
     }
 #pragma unroll 1
@@ -91,8 +92,8 @@ __device__ __forceinline__ void encrypt_unit(const LimbDev &lb, const tw_t *p0, 
         const M &ar = ia.m;
         smem_ntt_inverse<L, V, true>(
             sm, tid, ia, LimbOf<M>::ninv(lb), LimbOf<M>::wn(lb),
-            [&](uint32_t p) {
-                if (h == 0) return pair_of<val>{M::from_bits(sm[wswz(p)]), M::from_bits(sm[wswz(p + 1)])};
+            [&](uint32_t p, const uint64_t *wa, const uint64_t *wb) {
+                if (h == 0) return pair_of<val>{M::from_bits(*wa), M::from_bits(*wb)};
                 const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + p);
                 return pair_of<val>{M::from_bits(t.x), M::from_bits(t.y)};
             },
@@ -464,31 +465,33 @@ __device__ __forceinline__ void encrypt_unit_cluster(const LimbDev &lb, const tw
         for (uint32_t k = 0; k < ROWS; k++) cst[k] = M::from_bits(consts[grp * ROWS + k]);
         smem_ntt_forward<L, V>(
             smg, gt, fa,
-            [&](uint32_t i) {
+            // element base | reg of the piece: the sample swizzle (index bits 7..9) is taken of base once
+            [&](uint32_t base, uint32_t reg) {
+                const int8_t *sb = su + bswz(base) + reg;
                 if constexpr (std::is_same<M, ModF64>::value) {
                     double acc = 0.0;                                // |acc| < ROWS q
 #pragma unroll
-                    for (uint32_t k = 0; k < ROWS; k++) acc = f64_fma((double)su[bswz(k * HB + i)], cst[k], acc);
+                    for (uint32_t k = 0; k < ROWS; k++) acc = f64_fma((double)sb[k * HB], cst[k], acc);
                     return ROWS > 4 ? ar.settle(acc) : acc;
                 } else {
                     uint64_t acc = 0;                                // below ROWS q
 #pragma unroll
                     for (uint32_t k = 0; k < ROWS; k++) {
-                        const int b = su[bswz(k * HB + i)];
+                        const int b = sb[k * HB];
                         acc += b == 0 ? 0 : (b > 0 ? cst[k] : q - cst[k]);
                     }
                     return ROWS > 4 ? csub_as<true>(acc, 2 * ar.q2) : acc;      // below 4q
                 }
             },
-            [&](uint32_t p, val a, val b) {
+            [&](uint32_t p, val a, val b, uint64_t *wa, uint64_t *wb) {
                 const auto a0 = M::load_key(p1 + p), a1 = M::load_key(p1 + p + 1);
                 u64x2 v;
                 v.x = M::bits(ar.mul_key(a, a0));
                 v.y = M::bits(ar.mul_key(b, a1));
                 *reinterpret_cast<u64x2 *>(c1 + p) = v;      // parked until the second pass
                 const auto b0 = M::load_key(p0 + p), b1 = M::load_key(p0 + p + 1);
-                smg[wswz(p)] = M::bits(ar.mul_key(a, b0));
-                smg[wswz(p + 1)] = M::bits(ar.mul_key(b, b1));
+                *wa = M::bits(ar.mul_key(a, b0));            // words wswz(p), wswz(p + 1) of this group's piece
+                *wb = M::bits(ar.mul_key(b, b1));
             },
             gsync);
     }
@@ -503,12 +506,12 @@ __device__ __forceinline__ void encrypt_unit_cluster(const LimbDev &lb, const tw
         const auto ninv = LimbOf<M>::ninv(lb), wn = LimbOf<M>::wn(lb);
         smem_ntt_inverse<L, V, false>(
             smg, gt, ia, ninv, wn,
-            [&](uint32_t p) {
-                if (h == 0) return pair_of<val>{M::from_bits(smg[wswz(p)]), M::from_bits(smg[wswz(p + 1)])};
+            [&](uint32_t p, const uint64_t *wa, const uint64_t *wb) {
+                if (h == 0) return pair_of<val>{M::from_bits(*wa), M::from_bits(*wb)};
                 const u64x2 t = *reinterpret_cast<const u64x2 *>(cc + row * HB + p);
                 return pair_of<val>{M::from_bits(t.x), M::from_bits(t.y)};
             },
-            [&](uint32_t i, val v) { smg[wswz(i)] = M::bits(v); }, gsync);
+            [&](uint32_t, val v, uint64_t *wv) { *wv = M::bits(v); }, gsync);
         cluster.sync();                                          // every piece is transformed and visible
         const auto to = LimbOf<M>::args(lb, false, 0, 0);
 #pragma unroll 1
