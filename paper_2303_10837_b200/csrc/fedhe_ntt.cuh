@@ -372,7 +372,7 @@ HD void fwd_stage(typename M::val (&x)[L::E], uint32_t base, const NttArgsT<M> &
             if (r & (1 << bit)) continue;
             // registers that agree above the pair bit share one twiddle; the
             // compiler merges the equal loads of an unrolled group
-            a.m.fwd(x[r], x[r | (1 << bit)], last_twiddle<L, I>(base | L::template reg<P>(r), a));
+            a.m.fwd(x[r], x[r | (1 << bit)], last_twiddle<L, I>(base + L::template reg<P>(r), a));
         }
     }
 }
@@ -393,7 +393,7 @@ HD void inv_stage(typename M::val (&x)[L::E], uint32_t base, const NttArgsT<M> &
 #pragma unroll
         for (int r = 0; r < L::E; r++) {
             if (r & (1 << bit)) continue;
-            a.m.inv(x[r], x[r | (1 << bit)], last_twiddle<L, I>(base | L::template reg<P>(r), a));
+            a.m.inv(x[r], x[r | (1 << bit)], last_twiddle<L, I>(base + L::template reg<P>(r), a));
         }
     }
 }
@@ -502,7 +502,7 @@ __device__ __forceinline__ void forward_phases(uint64_t *sm, uint32_t warp, uint
                 // a source may take the index in two parts, base (zero at the register bits, the
                 // same for all E calls) and the register's constant, to hoist what depends on base
                 if constexpr (std::is_invocable<Src, uint32_t, uint32_t>::value) x[r] = src(base, L::template reg<P>(r));
-                else x[r] = src(base | L::template reg<P>(r));
+                else x[r] = src(base + L::template reg<P>(r));
             } else {
                 x[r] = M::from_bits(*reg_word<L, P>(a0, r));
             }
@@ -514,9 +514,9 @@ __device__ __forceinline__ void forward_phases(uint64_t *sm, uint32_t warp, uint
                 // a sink that keeps the pair in this buffer may take the two words' addresses
                 // (one logic operation each) instead of swizzling the index itself
                 if constexpr (std::is_invocable<Dst, uint32_t, typename M::val, typename M::val, uint64_t *, uint64_t *>::value)
-                    dst(base | L::template reg<P>(r), x[r], x[r + 1], reg_word<L, P>(a0, r), reg_word<L, P>(a0, r + 1));
+                    dst(base + L::template reg<P>(r), x[r], x[r + 1], reg_word<L, P>(a0, r), reg_word<L, P>(a0, r + 1));
                 else
-                    dst(base | L::template reg<P>(r), x[r], x[r + 1]);
+                    dst(base + L::template reg<P>(r), x[r], x[r + 1]);
             }
         } else {
 #pragma unroll
@@ -552,11 +552,11 @@ __device__ __forceinline__ void inverse_phases(uint64_t *sm, uint32_t warp, uint
 #pragma unroll
             for (int r = 0; r < L::E; r += 2) {
                 if constexpr (std::is_invocable<Src, uint32_t, const uint64_t *, const uint64_t *>::value) {
-                    const auto t = src(base | L::template reg<P>(r), reg_word<L, P>(a0, r), reg_word<L, P>(a0, r + 1));
+                    const auto t = src(base + L::template reg<P>(r), reg_word<L, P>(a0, r), reg_word<L, P>(a0, r + 1));
                     x[r] = t.x;
                     x[r + 1] = t.y;
                 } else {
-                    const auto t = src(base | L::template reg<P>(r));
+                    const auto t = src(base + L::template reg<P>(r));
                     x[r] = t.x;
                     x[r + 1] = t.y;
                 }
@@ -575,9 +575,9 @@ __device__ __forceinline__ void inverse_phases(uint64_t *sm, uint32_t warp, uint
 #pragma unroll
             for (int r = 0; r < L::E; r++) {
                 if constexpr (std::is_invocable<Dst, uint32_t, typename M::val, uint64_t *>::value)
-                    dst(base | L::template reg<P>(r), x[r], reg_word<L, P>(a0, r));
+                    dst(base + L::template reg<P>(r), x[r], reg_word<L, P>(a0, r));
                 else
-                    dst(base | L::template reg<P>(r), x[r]);
+                    dst(base + L::template reg<P>(r), x[r]);
             }
         } else {
 #pragma unroll
