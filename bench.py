@@ -420,8 +420,9 @@ def measure(job, w, steps, warmup, with_cpu_baseline):
     kern_ms = max(enc_ms - encode_ms, 1e-6)
 
     # standalone transform: forward + inverse over a batch larger than L2
-    B = 256
-    polys = torch.from_numpy(si.random_residues(7, (B, w.L, w.N), w.primes).view(np.int64)).cuda()
+    # (1024 polynomials: 256 seeded ones, repeated on the device; 0.5 to 1.6 GB)
+    B = 1024
+    polys = torch.from_numpy(si.random_residues(7, (B // 4, w.L, w.N), w.primes).view(np.int64)).cuda().repeat(4, 1, 1)
     he.he_ntt_forward(g, polys)
     he.he_ntt_inverse(g, polys)
     torch.cuda.synchronize()
