@@ -41,6 +41,48 @@ __device__ __forceinline__ void weighted_sum_pair(const uint64_t *const *sp, con
     ay = csub(ay, q);
 }
 
+// The same sum for a limb whose prime is below 2^46, in the exact double-precision arithmetic of
+// the transforms: a product costs the shared multiply / double-precision pipe 6 slots instead of
+// about 19, which matters because this pass keeps that pipe two thirds busy beside HBM.  Every
+// product has magnitude at most 3q/4 and the running sum is brought back below q after every 32
+// clients, so it stays below 25 q < 2^51 and every addition is exact.
+__device__ __forceinline__ void weighted_sum_pair_f64(const uint64_t *const *sp, const tw_t *sw, int C, uint32_t L,
+                                                      uint32_t j, size_t off, double q, double qi, uint64_t &ax,
+                                                      uint64_t &ay) {
+    double sx = 0.0, sy = 0.0;
+    int cl = 0;
+    for (; cl + 4 <= C; cl += 4) {
+        ulonglong2 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; u++) v[u] = __ldg(reinterpret_cast<const ulonglong2 *>(sp[cl + u] + off));
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+            const double w = f64_from_u64(sw[(cl + u) * L + j].w);
+            sx = f64_add(sx, f64_mulmod(f64_from_u64(v[u].x), w, q, qi));
+            sy = f64_add(sy, f64_mulmod(f64_from_u64(v[u].y), w, q, qi));
+        }
+        if ((cl & 31) == 28) {
+            sx = f64_reduce(sx, q, qi);
+            sy = f64_reduce(sy, q, qi);
+        }
+    }
+    for (; cl < C; cl++) {
+        const ulonglong2 v = __ldg(reinterpret_cast<const ulonglong2 *>(sp[cl] + off));
+        const double w = f64_from_u64(sw[cl * L + j].w);
+        sx = f64_add(sx, f64_mulmod(f64_from_u64(v.x), w, q, qi));
+        sy = f64_add(sy, f64_mulmod(f64_from_u64(v.y), w, q, qi));
+    }
+    ax = f64_canonical(f64_reduce(sx, q, qi), q);
+    ay = f64_canonical(f64_reduce(sy, q, qi), q);
+}
+
+// a limb's sum in whichever arithmetic its prime allows
+__device__ __forceinline__ void weighted_sum_limb(const LimbDev &lb, const uint64_t *const *sp, const tw_t *sw, int C,
+                                                  uint32_t L, uint32_t j, size_t off, uint64_t &ax, uint64_t &ay) {
+    if (lb.fwd_d) weighted_sum_pair_f64(sp, sw, C, L, j, off, lb.qd, lb.qi, ax, ay);
+    else weighted_sum_pair(sp, sw, C, L, j, off, lb.q, ax, ay);
+}
+
 __global__ void __launch_bounds__(256)
 aggregate_rescale_kernel(const __grid_constant__ CtxDev c, const uint64_t *const *ptrs, const tw_t *wtab,
                          int C, uint64_t *out, size_t total) {
@@ -58,14 +100,14 @@ aggregate_rescale_kernel(const __grid_constant__ CtxDev c, const uint64_t *const
     const size_t tc = g / pairs;                 // t * 2 + component
     const uint64_t ql = c.limb[L - 1].q;
     uint64_t rx, ry;
-    weighted_sum_pair(sp, sw, C, L, L - 1, (tc * L + (L - 1)) * c.N + i, ql, rx, ry);
+    weighted_sum_limb(c.limb[L - 1], sp, sw, C, L, L - 1, (tc * L + (L - 1)) * c.N + i, rx, ry);
     const bool negx = rx > ql / 2, negy = ry > ql / 2;
     const uint64_t mx = negx ? ql - rx : rx, my = negy ? ql - ry : ry;   // |centred remainder|
     for (uint32_t j = 0; j + 1 < L; j++) {
         const LimbDev &lb = c.limb[j];
         const uint64_t q = lb.q;
         uint64_t ax, ay;
-        weighted_sum_pair(sp, sw, C, L, j, (tc * L + j) * c.N + i, q, ax, ay);
+        weighted_sum_limb(lb, sp, sw, C, L, j, (tc * L + j) * c.N + i, ax, ay);
         const uint64_t sx = barrett64(mx, q, lb.mu), sy = barrett64(my, q, lb.mu);
         // acc - r: subtracting a negative remainder adds its magnitude
         const uint64_t dx = negx ? addmod(ax, sx, q) : submod(ax, sx, q);
@@ -118,7 +160,7 @@ aggregate_sum_kernel(const __grid_constant__ CtxDev c, const uint64_t *const *pt
     const size_t tc = g / pairs;
     for (uint32_t j = 0; j < L; j++) {
         u64x2 o;
-        weighted_sum_pair(sp, sw, C, L, j, (tc * L + j) * c.N + i, c.limb[j].q, o.x, o.y);
+        weighted_sum_limb(c.limb[j], sp, sw, C, L, j, (tc * L + j) * c.N + i, o.x, o.y);
         uint64_t *dst = !last ? out + (tc * L + j) * c.N + i
                               : (j + 1 < L ? out + (tc * (L - 1) + j) * c.N + i : last + tc * c.N + i);
         *reinterpret_cast<u64x2 *>(dst) = o;

@@ -508,6 +508,36 @@ def test_host_round_refuses_bad_arguments_before_queueing(he):
     assert np.abs(host.numpy() - want).max() <= FEDAVG_TOL
 
 
+@pytest.mark.parametrize("primes,C", [((si.PRIMES_SWEEP[0], si.PRIMES_SWEEP_45[0], si.PRIMES_SWEEP_45[1]), 70),
+                                      (si.PRIMES_SWEEP_45[:3], 131), (si.PRIMES_N8192, 37),
+                                      ((si.PRIMES_SWEEP_45[0], si.PRIMES_SWEEP[0], si.PRIMES_SWEEP[1]), 5)],
+                         ids=["f64-last-70", "all-f64-131", "mixed-37", "int-last-5"])
+def test_weighted_aggregate_many_clients_bit_exact(he, primes, C):
+    """The server's sum on arbitrary residues (all-maximal ones among them) for client counts beyond
+    one unrolled group and beyond the interval at which the sums in doubles are reduced, with the
+    dropped prime in either arithmetic; also in two halves."""
+    N, T = 8192, 2
+    g, o = contexts(he, N, primes, 30)
+    rng = np.random.default_rng(77)
+    cts_o = []
+    for i in range(C):
+        ct = si.random_residues(100 + i, (T, 2, len(primes), N), primes)
+        if i % 9 == 0:
+            for j, q in enumerate(primes):
+                ct[0, :, j, : N // 2] = q - 1
+        cts_o.append(ct)
+    alpha = rng.random(C)
+    alpha /= alpha.sum()
+    cts = [to_dev_u64(c) for c in cts_o]
+    W = o.weights(alpha)
+    want = o.rescale(o.weighted_sum(cts_o, W))
+    assert np.array_equal(to_host_u64(he.he_weighted_aggregate(g, cts, alpha)), want)
+    half = C // 2 + 1
+    parts = [he.he_weighted_partial(g, cts[:half], alpha[:half]), he.he_weighted_partial(g, cts[half:], alpha[half:])]
+    assert np.array_equal(to_host_u64(parts[0]), o.weighted_sum(cts_o[:half], W[:half]))
+    assert np.array_equal(to_host_u64(he.he_rescale_partial_parts(g, parts)), want)
+
+
 @pytest.mark.parametrize("N,primes,ld", [(8192, si.PRIMES_N8192, 40), (16384, si.PRIMES_N16384, 40),
                                          (32768, si.PRIMES_N32768, 45)],
                          ids=["n8192", "n16384", "n32768"])
