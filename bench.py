@@ -64,8 +64,8 @@ UNIT = "params/s"
 # the profile_case.py encrypt case (summaries under profiles/; traffic grows in proportion to the
 # number of ciphertexts).  An entry is dropped (None is reported) when the kernel has changed
 # since its counters were taken.
-ENCRYPT_DRAM_BYTES_PER_CT = {(16384, 4): 367.520256e6 / 296,       # encrypt_fused2_kernel, 296 ciphertexts
-                             (32768, 6): 479.387392e6 / 148}       # encrypt_cluster_kernel, 148 ciphertexts
+ENCRYPT_DRAM_BYTES_PER_CT = {(16384, 4): 372.248832e6 / 296,       # encrypt_fused2_kernel, 296 ciphertexts
+                             (32768, 6): 478.248704e6 / 148}       # encrypt_cluster_kernel, 148 ciphertexts
 SLOTS_PER_SM_CLK = 64.0
 WIDE_COST = 2.5
 INT_SLOTS_PER_BUTTERFLY = 6 * WIDE_COST + 4
