@@ -33,6 +33,10 @@ template<int MODE> __global__ void k(uint64_t* out, int iters, uint32_t seed) {
       if (MODE==2) b[i] = __umul64hi(b[i], m64) + 1;       // 64-bit mulhi
       if (MODE==3) b[i] = b[i]*m64 + 1;                    // 64-bit mullo
       if (MODE==4) a[i] = (a[i] + m) ^ (a[i]>>3);          // IADD/LOP/SHF
+      if (MODE==9) a[i] = __umulhi(a[i], m) + 12345u;      // IMAD.HI 32
+      if (MODE==10) { const uint32_t lo = a[i]*m, hi = __umulhi(a[i], m); a[i] = lo ^ hi; }   // both halves as two narrow multiplies
+      if (MODE==11) { const uint64_t p = (uint64_t)a[i]*m; a[i] = (uint32_t)p ^ (uint32_t)(p >> 32); }   // both halves as one wide multiply
+      if (MODE==12) { double r; asm("cvt.rni.f64.f64 %0, %1;" : "=d"(r) : "d"(d[i])); d[i] = r + dm; }   // round to integer + DADD
       if (MODE==6) d[i] = __fma_rn(d[i], dm, dc);          // DFMA
       if (MODE==7) {                                        // exact modular product in doubles (6 operations)
         const double y = d[i], w = 123456789012.0;
@@ -60,4 +64,5 @@ template<int MODE> int run(const char* name, double ops_per_iter) {
 }
 int main(){ int sms; cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, 0); int clk; cudaDeviceGetAttribute(&clk, cudaDevAttrClockRate, 0); printf("SMs %d clock attr %d kHz\n", sms, clk);
   run<0>("imad.lo32",1); run<1>("imad.wide",1); run<2>("umul64hi",1); run<3>("mul.lo.u64",1); run<4>("iadd+lop+shf (3 ops)",3); run<5>("shoup lazy modmul",1);
+  run<9>("imad.hi32",1); run<10>("mul.lo + mul.hi pair",1); run<11>("mul.wide, both halves",1); run<12>("cvt.rni.f64 + dadd",1);
   run<6>("dfma",1); run<7>("f64 modmul (6 dp ops)",1); run<8>("imad.lo32 + dfma, alternate warps",1); return 0; }
